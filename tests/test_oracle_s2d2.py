@@ -1,0 +1,149 @@
+"""Pins the oracle's decode loop: the 2L verifier pass against L literal
+single-row passes, block size 1 against greedy AR decoding, the incrementally
+committed K/V against a literal end-of-block causal pass, and the behaviour
+the algorithms fix (progress every step, stop at first rejection, resampled
+token differs from the rejected proposal)."""
+import numpy as np
+import pytest
+
+from oracle import model as M
+from oracle import s2d2 as S
+from oracle.accept import logsumexp
+from s2d2_inputs import generate_prompts, generate_weights, get_config
+
+
+def test_verifier_rows_equal_literal_single_position_passes(tiny_f32):
+    """MASK-copy row i of the 2L pass conditions on the prefix and the drafted
+    tokens to its left and keeps position i masked: identical to a pass of
+    prefix ++ x̂_<i ++ [MASK] read at its last row."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = [5, 9, 2, 44, 17, 3, 8]
+    n = len(prompt)
+    _, kv = M.forward(W, cfg, prompt, np.arange(n), M.causal_mask(n), need_logits=[])
+    cache = M.append_kv(None, kv, np.arange(n))
+    xhat = [11, 4, 30, 7]
+    L = len(xhat)
+    vt, vp, vm = S.verify_pass_rows(xhat, list(range(n, n + L)), cfg.mask_id)
+    # the mask is [[A, 0], [A<, I]]
+    assert vm[:L, :L].tolist() == np.tril(np.ones((L, L), bool)).tolist()
+    assert not vm[:L, L:].any()
+    assert vm[L:, :L].tolist() == np.tril(np.ones((L, L), bool), -1).tolist()
+    assert vm[L:, L:].tolist() == np.eye(L, dtype=bool).tolist()
+    got, _ = M.forward(W, cfg, vt, vp, vm, cache, need_logits=list(range(L, 2 * L)))
+    for i in range(L):
+        seq = prompt + xhat[:i] + [cfg.mask_id]
+        lit, _ = M.forward(W, cfg, seq, np.arange(len(seq)), M.causal_mask(len(seq)))
+        np.testing.assert_allclose(got[i], lit[-1], rtol=1e-9, atol=1e-11)
+
+
+def test_block_size_one_is_greedy_autoregressive(tiny_f32):
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=4)[0][:9]
+    seq = S.SequenceOracle(W, cfg, block_size=1, seed=1, seq_stream=0, keep_logits=True)
+    out = seq.generate(prompt, 10)
+    assert out == S.greedy_ar_decode(W, cfg, prompt, 10)
+    for st in seq.trace:
+        # drafter row and verifier row are the same computation: ratio 1, never rejects
+        assert st.result.n_accepted == 1 and st.result.first_reject == -1
+        assert abs(st.result.a[0] - 1.0) < 1e-9
+        np.testing.assert_allclose(st.verify_logits, st.draft_logits[:1], rtol=1e-9, atol=1e-11)
+    assert seq.n_verify_passes == 10
+
+
+@pytest.mark.parametrize("B", [4, 8])
+def test_loop_invariants_and_cache_is_causal(tiny_f32, B):
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=5)[1][:6]
+    seq = S.SequenceOracle(W, cfg, block_size=B, seed=1, seq_stream=2, keep_logits=True)
+    out = seq.generate(prompt, 24)
+    assert len(out) == 24 and all(0 <= t < cfg.vocab for t in out)
+    n_rej = 0
+    for st in seq.trace:
+        assert st.verified and len(st.committed) >= 1          # progress every step
+        r = st.result
+        assert st.span == list(range(st.j, st.j + len(st.span)))
+        if r.first_reject >= 0:
+            n_rej += 1
+            assert r.first_reject == r.n_accepted
+            assert len(st.committed) == r.n_accepted + 1
+            assert r.resampled != st.xhat[r.first_reject]      # residual is zero at the rejected proposal
+            assert st.u_accept[r.first_reject] >= r.a[r.first_reject]
+        else:
+            assert r.n_accepted == len(st.span)
+        for k in range(r.n_accepted):
+            assert st.u_accept[k] < r.a[k]
+    assert n_rej >= 1                                           # the run exercises the rejection path
+    # the cache holds exactly the K/V a single causal pass over the committed tokens gives
+    full = list(prompt) + out
+    _, kv = M.forward(W, cfg, full, np.arange(len(full)), M.causal_mask(len(full)), need_logits=[])
+    assert seq.n_c <= len(full)
+    for l in range(cfg.n_layers):
+        np.testing.assert_allclose(seq.cache[l][0], kv[l][0][: seq.n_c], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(seq.cache[l][1], kv[l][1][: seq.n_c], rtol=1e-9, atol=1e-12)
+
+
+def test_committed_kv_equals_literal_end_of_block_pass(tiny_f32):
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = [1, 2, 3, 4, 5]
+    B = 4
+    seq = S.SequenceOracle(W, cfg, block_size=B, seed=3, seq_stream=0)
+    seq.prefill(prompt)
+    cache0 = seq.cache
+    while len(seq.tokens) < len(prompt) + B:
+        seq.step()
+    block = seq.tokens[len(prompt):]
+    lit = S.literal_block_kv(W, cfg, block, len(prompt), cache0)
+    have = seq.n_c - len(prompt)                 # block tokens already cached (a pending tail may remain)
+    assert 0 < have <= B
+    for l in range(cfg.n_layers):
+        np.testing.assert_allclose(seq.cache[l][0][len(prompt):], lit[l][0][:have], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(seq.cache[l][1][len(prompt):], lit[l][1][:have], rtol=1e-9, atol=1e-12)
+
+
+def test_confidence_branch_is_the_bd3_sampler(tiny_f32):
+    """Never verifying reduces SampleBlock to confidence-threshold decoding:
+    tau = 1 commits exactly the most confident masked position per step."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    seq = S.SequenceOracle(W, cfg, block_size=4, seed=1, seq_stream=0, route=lambda st: False, tau_conf=1.0)
+    seq.generate([7, 8, 9], 8)
+    assert seq.n_verify_passes == 0 and seq.n_draft_passes == 8
+    for st in seq.trace:
+        assert len(st.committed) == 1
+        best = max(range(len(st.masked)), key=lambda k: (st.d[k], -k))
+        assert st.committed == [st.masked[best]]
+    # a low threshold commits every masked position at once
+    seq2 = S.SequenceOracle(W, cfg, block_size=4, seed=1, seq_stream=0, route=lambda st: False, tau_conf=0.0)
+    seq2.generate([7, 8, 9], 8)
+    assert seq2.n_draft_passes == 2
+
+
+def test_mixed_routing_handles_non_contiguous_commits(tiny_f32):
+    """Alternate verification and the confidence branch so that known tokens
+    appear to the right of masked ones; the span is then the first masked run only."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    flip = {"n": 0}
+
+    def route(st):
+        flip["n"] += 1
+        return flip["n"] % 2 == 0
+    seq = S.SequenceOracle(W, cfg, block_size=8, seed=2, seq_stream=1, route=route, tau_conf=1.0)
+    out = seq.generate([3, 1, 4, 1, 5], 16)
+    assert len(out) == 16
+    assert any(len(st.span) < len(st.masked) for st in seq.trace if st.verified)
+    full = [3, 1, 4, 1, 5] + out
+    _, kv = M.forward(W, cfg, full, np.arange(len(full)), M.causal_mask(len(full)), need_logits=[])
+    np.testing.assert_allclose(seq.cache[0][0], kv[0][0][: seq.n_c], rtol=1e-9, atol=1e-12)
+
+
+def test_sequences_are_independent_of_their_stream_only_through_uniforms(tiny_f32):
+    wl, W = tiny_f32
+    cfg = wl.model
+    a = S.SequenceOracle(W, cfg, 4, seed=1, seq_stream=0).generate([1, 2, 3], 8)
+    b = S.SequenceOracle(W, cfg, 4, seed=1, seq_stream=0).generate([1, 2, 3], 8)
+    assert a == b
