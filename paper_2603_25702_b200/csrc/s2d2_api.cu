@@ -1,0 +1,1120 @@
+// C ABI and host driver of the S2D2 decode step (see include/s2d2.h).
+//
+// The host keeps the per-sequence decode state (tokens, open block, cache
+// length, page list) and, for each pass, builds a small row table that the
+// kernels read: which token sits at which position, which rows of the same pass
+// a row may attend (a 64-bit mask: the verifier mask and the partially causal
+// drafting mask both fit), which rows write their K/V to the cache, and which
+// rows need logits.  Everything numerical runs in the kernels.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include "context.h"
+#include "gemm.h"
+#include "kernels_simt.cuh"
+#include "vocab_kernels.cuh"
+
+using namespace s2d2;
+
+#define CUDA_TRY(ctx, call)                                                                      \
+    do {                                                                                         \
+        cudaError_t e_ = (call);                                                                 \
+        if (e_ != cudaSuccess) {                                                                 \
+            (ctx)->err = std::string(#call) + ": " + cudaGetErrorString(e_);                     \
+            return S2D2_ERR_CUDA;                                                                \
+        }                                                                                        \
+    } while (0)
+#define FAIL(ctx, code, msg)  \
+    do {                      \
+        (ctx)->err = (msg);   \
+        return (code);        \
+    } while (0)
+#define LAUNCHED(ctx) ((ctx)->cnt.n_kernel_launches++)
+
+static size_t esize(int dtype) { return dtype == S2D2_DTYPE_BF16 ? 2 : 4; }
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// creation: weight arena layout, KV pool, scratch
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct ArenaPlan {
+    size_t cur = 0;
+    size_t take(size_t bytes) {
+        size_t o = cur;
+        cur = align_up(cur + bytes, 256);
+        return o;
+    }
+};
+
+void add_slot(s2d2_ctx* c, const std::string& name, char* base, size_t off, size_t bytes, int dtype) {
+    WeightSlot s;
+    s.d_ptr = base ? base + off : (void*)off;
+    s.bytes = bytes;
+    s.dtype = dtype;
+    c->slots[name] = s;
+}
+
+// Lays the tensors out in one arena.  wq/wk/wv share one [Hq+2Hkv)*hd, d] matrix and
+// w_gate/w_up one [2f, d] matrix so that one GEMM serves each group.
+size_t plan_weights(s2d2_ctx* c, char* base) {
+    const s2d2_model_config& m = c->m;
+    ArenaPlan ap;
+    size_t es = esize(m.dtype), d = m.d_model, hd = m.head_dim;
+    c->slots.clear();
+    c->layers.assign(m.n_layers, LayerWeights());
+    size_t o = ap.take((size_t)(m.vocab + 1) * d * es);
+    add_slot(c, "embed", base, o, (size_t)(m.vocab + 1) * d * es, m.dtype);
+    c->embed = base + o;
+    for (int l = 0; l < m.n_layers; ++l) {
+        std::string p = "layers." + std::to_string(l) + ".";
+        LayerWeights& L = c->layers[l];
+        auto gain = [&](const char* n, size_t len, float** dst) {
+            size_t off = ap.take(len * 4);
+            add_slot(c, p + n, base, off, len * 4, S2D2_DTYPE_F32);
+            *dst = (float*)(base + off);
+        };
+        gain("attn_norm", d, &L.attn_norm);
+        size_t nq = (size_t)m.n_q_heads * hd, nkv = (size_t)m.n_kv_heads * hd;
+        size_t off = ap.take((nq + 2 * nkv) * d * es);
+        L.wqkv = base + off;
+        add_slot(c, p + "wq", base, off, nq * d * es, m.dtype);
+        add_slot(c, p + "wk", base, off + nq * d * es, nkv * d * es, m.dtype);
+        add_slot(c, p + "wv", base, off + (nq + nkv) * d * es, nkv * d * es, m.dtype);
+        off = ap.take(d * nq * es);
+        L.wo = base + off;
+        add_slot(c, p + "wo", base, off, d * nq * es, m.dtype);
+        if (m.qk_norm) {
+            gain("q_norm", hd, &L.q_norm);
+            gain("k_norm", hd, &L.k_norm);
+        }
+        gain("ffn_norm", d, &L.ffn_norm);
+        if (m.n_experts > 0) {
+            size_t E = m.n_experts, f = m.expert_ffn;
+            off = ap.take(E * d * es);
+            L.router = base + off;
+            add_slot(c, p + "router", base, off, E * d * es, m.dtype);
+            off = ap.take(E * f * d * es);
+            L.e_gate = base + off;
+            add_slot(c, p + "experts.w_gate", base, off, E * f * d * es, m.dtype);
+            off = ap.take(E * f * d * es);
+            L.e_up = base + off;
+            add_slot(c, p + "experts.w_up", base, off, E * f * d * es, m.dtype);
+            off = ap.take(E * d * f * es);
+            L.e_down = base + off;
+            add_slot(c, p + "experts.w_down", base, off, E * d * f * es, m.dtype);
+            if (m.n_shared > 0) {
+                size_t fs = f * m.n_shared;
+                off = ap.take(2 * fs * d * es);
+                L.s_gu = base + off;
+                add_slot(c, p + "shared.w_gate", base, off, fs * d * es, m.dtype);
+                add_slot(c, p + "shared.w_up", base, off + fs * d * es, fs * d * es, m.dtype);
+                off = ap.take(d * fs * es);
+                L.s_down = base + off;
+                add_slot(c, p + "shared.w_down", base, off, d * fs * es, m.dtype);
+            }
+        } else {
+            size_t f = m.ffn;
+            off = ap.take(2 * f * d * es);
+            L.wgu = base + off;
+            add_slot(c, p + "w_gate", base, off, f * d * es, m.dtype);
+            add_slot(c, p + "w_up", base, off + f * d * es, f * d * es, m.dtype);
+            off = ap.take(d * f * es);
+            L.wdown = base + off;
+            add_slot(c, p + "w_down", base, off, d * f * es, m.dtype);
+        }
+    }
+    o = ap.take(d * 4);
+    add_slot(c, "final_norm", base, o, d * 4, S2D2_DTYPE_F32);
+    c->final_norm = (float*)(base + o);
+    o = ap.take((size_t)m.vocab * d * es);
+    add_slot(c, "lm_head", base, o, (size_t)m.vocab * d * es, m.dtype);
+    c->lm_head = base + o;
+    return ap.cur;
+}
+
+int validate(const s2d2_model_config& m, const s2d2_decode_config& dc, std::string& why) {
+    auto bad = [&](const char* s) {
+        why = s;
+        return S2D2_ERR_INVALID;
+    };
+    if (m.n_layers < 1 || m.d_model < 32 || m.vocab < 2) return bad("model: n_layers/d_model/vocab");
+    if (m.n_q_heads < 1 || m.n_kv_heads < 1 || m.n_q_heads % m.n_kv_heads) return bad("model: heads");
+    if (m.head_dim != 32 && m.head_dim != 64 && m.head_dim != 128) return bad("model: head_dim must be 32, 64 or 128");
+    if (m.dtype != S2D2_DTYPE_F32 && m.dtype != S2D2_DTYPE_BF16) return bad("model: dtype");
+    if (m.n_experts == 0 && m.ffn < 1) return bad("model: ffn");
+    if (m.n_experts > 0 && (m.top_k < 1 || m.top_k > m.n_experts || m.top_k > 32 || m.expert_ffn < 1))
+        return bad("model: moe");
+    if (dc.block_size < 1 || dc.block_size > S2D2_MAX_BLOCK) return bad("decode: block_size");
+    if (dc.max_batch < 1 || dc.max_seq_len < 1) return bad("decode: max_batch/max_seq_len");
+    int p = dc.kv_page_tokens;
+    if (p < 1 || p > 64 || (p & (p - 1))) return bad("decode: kv_page_tokens must be a power of two <= 64");
+    if (dc.draft_mode != S2D2_DRAFT_GREEDY) return bad("decode: draft_mode");
+    return S2D2_OK;
+}
+
+template <typename T>
+int dmalloc(s2d2_ctx* c, T** p, size_t n) {
+    CUDA_TRY(c, cudaMalloc((void**)p, std::max<size_t>(n, 1) * sizeof(T)));
+    return S2D2_OK;
+}
+
+}  // namespace
+
+extern "C" const char* s2d2_last_error(const s2d2_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config* dc, void* cuda_stream,
+                           s2d2_ctx** out) {
+    if (!m || !dc || !out) return S2D2_ERR_INVALID;
+    *out = nullptr;
+    std::string why;
+    if (validate(*m, *dc, why) != S2D2_OK) {
+        fprintf(stderr, "s2d2_create: %s\n", why.c_str());
+        return S2D2_ERR_INVALID;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+        fprintf(stderr, "s2d2_create: no CUDA device (this library has no CPU path)\n");
+        return S2D2_ERR_CUDA;
+    }
+    s2d2_ctx* c = new s2d2_ctx();
+    c->m = *m;
+    c->dc = *dc;
+    c->stream = (cudaStream_t)cuda_stream;
+    memset(&c->cnt, 0, sizeof(c->cnt));
+    memset(&c->policy, 0, sizeof(c->policy));
+    c->policy.policy = S2D2_ROUTE_MIN_SPAN;
+    c->policy.p0 = 1.f;
+    cudaGetDevice(&c->device);
+    *out = c;   // returned even on failure below so that the caller can read last_error and destroy
+
+    // weights arena
+    c->w_bytes = plan_weights(c, nullptr);
+    CUDA_TRY(c, cudaMalloc((void**)&c->w_arena, c->w_bytes));
+    plan_weights(c, c->w_arena);
+
+    // KV pool
+    c->page_tokens = dc->kv_page_tokens;
+    c->page_shift = 0;
+    while ((1 << c->page_shift) < c->page_tokens) ++c->page_shift;
+    c->max_pages_per_seq = (dc->max_seq_len + c->page_tokens - 1) / c->page_tokens;
+    c->n_pages = dc->n_kv_pages > 0 ? dc->n_kv_pages : dc->max_batch * c->max_pages_per_seq;
+    size_t page_elems = (size_t)2 * m->n_kv_heads * c->page_tokens * m->head_dim;
+    size_t kv_bytes = (size_t)m->n_layers * c->n_pages * page_elems * esize(m->dtype);
+    CUDA_TRY(c, cudaMalloc(&c->kv_base, kv_bytes));
+    CUDA_TRY(c, cudaMemsetAsync(c->kv_base, 0, kv_bytes, c->stream));
+    for (int p = c->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
+    c->seqs.assign(dc->max_batch, SeqState());
+
+    // scratch
+    int rows_per_seq = std::max(2 * dc->block_size, S2D2_MAX_ROWS_PER_SEQ);
+    c->max_rows = dc->max_batch * rows_per_seq;
+    c->max_logit_rows = dc->max_batch * dc->block_size;
+    size_t M = c->max_rows, d = m->d_model, es = esize(m->dtype);
+    size_t nqkv = (size_t)(m->n_q_heads + 2 * m->n_kv_heads) * m->head_dim, nq = (size_t)m->n_q_heads * m->head_dim;
+    size_t f = m->n_experts > 0 ? (size_t)m->expert_ffn * std::max(1, m->n_shared) : (size_t)m->ffn;
+    int rc;
+    if ((rc = dmalloc(c, &c->h, M * d))) return rc;
+    if ((rc = dmalloc(c, &c->qkv, M * nqkv))) return rc;
+    if ((rc = dmalloc(c, &c->gu, M * 2 * f))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->xn, M * d * es))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->q, M * nq * es))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->k_rows, M * m->n_kv_heads * m->head_dim * es))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->v_rows, M * m->n_kv_heads * m->head_dim * es))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->attn, M * nq * es))) return rc;
+    if ((rc = dmalloc(c, (char**)&c->act, M * f * es))) return rc;
+    if ((rc = dmalloc(c, &c->logits_draft, (size_t)c->max_logit_rows * m->vocab))) return rc;
+    if ((rc = dmalloc(c, &c->logits_verify, (size_t)c->max_logit_rows * m->vocab))) return rc;
+    if (m->n_experts > 0) {
+        size_t P = M * m->top_k, fe = m->expert_ffn;
+        if ((rc = dmalloc(c, &c->router_logits, M * m->n_experts))) return rc;
+        if ((rc = dmalloc(c, &c->moe_gates, P))) return rc;
+        if ((rc = dmalloc(c, &c->moe_ids, P))) return rc;
+        if ((rc = dmalloc(c, &c->moe_gu, P * 2 * fe))) return rc;
+        if ((rc = dmalloc(c, (char**)&c->moe_act, P * fe * es))) return rc;
+        if ((rc = dmalloc(c, &c->moe_out, P * d))) return rc;
+        if ((rc = dmalloc(c, &c->moe_ids_trace, (size_t)m->n_layers * P))) return rc;
+    }
+    // RoPE table in fp64 on the host, stored fp32
+    {
+        int half = m->head_dim / 2;
+        size_t n = (size_t)dc->max_seq_len * half;
+        std::vector<float> cs(n), sn(n);
+        for (int p = 0; p < dc->max_seq_len; ++p)
+            for (int i = 0; i < half; ++i) {
+                double ang = (double)p * pow((double)m->rope_base, -2.0 * i / m->head_dim);
+                cs[(size_t)p * half + i] = (float)cos(ang);
+                sn[(size_t)p * half + i] = (float)sin(ang);
+            }
+        if ((rc = dmalloc(c, &c->rope_cos, n))) return rc;
+        if ((rc = dmalloc(c, &c->rope_sin, n))) return rc;
+        CUDA_TRY(c, cudaMemcpy(c->rope_cos, cs.data(), n * 4, cudaMemcpyHostToDevice));
+        CUDA_TRY(c, cudaMemcpy(c->rope_sin, sn.data(), n * 4, cudaMemcpyHostToDevice));
+    }
+    // pass metadata staging
+    {
+        PassMeta& pm = c->meta;
+        pm.cap_rows = c->max_rows;
+        pm.cap_seqs = dc->max_batch;
+        pm.max_pages = c->max_pages_per_seq;
+        size_t o = 0;
+        auto take = [&](size_t b) {
+            size_t r = o;
+            o = align_up(o + b, 16);
+            return r;
+        };
+        pm.off_mask = take((size_t)pm.cap_rows * 8);
+        pm.off_token = take((size_t)pm.cap_rows * 4);
+        pm.off_pos = take((size_t)pm.cap_rows * 4);
+        pm.off_seq = take((size_t)pm.cap_rows * 4);
+        pm.off_flags = take((size_t)pm.cap_rows * 4);
+        pm.off_logit_rows = take((size_t)pm.cap_rows * 4);
+        pm.off_nctx = take((size_t)pm.cap_seqs * 4);
+        pm.off_row0 = take((size_t)pm.cap_seqs * 4);
+        pm.off_nrows = take((size_t)pm.cap_seqs * 4);
+        pm.off_pages = take((size_t)pm.cap_seqs * pm.max_pages * 4);
+        pm.bytes = o;
+        CUDA_TRY(c, cudaMallocHost((void**)&pm.h, pm.bytes));
+        CUDA_TRY(c, cudaMalloc((void**)&pm.d, pm.bytes));
+        memset(pm.h, 0, pm.bytes);
+    }
+    // draft statistics and acceptance staging
+    {
+        size_t R = c->max_logit_rows;
+        if ((rc = dmalloc(c, &c->d_xhat, R))) return rc;
+        if ((rc = dmalloc(c, &c->d_conf, R))) return rc;
+        if ((rc = dmalloc(c, &c->d_margin, R))) return rc;
+        if ((rc = dmalloc(c, &c->d_entropy, R))) return rc;
+        if ((rc = dmalloc(c, &c->d_lse, R))) return rc;
+        CUDA_TRY(c, cudaMallocHost((void**)&c->stats_h, R * 16));
+        size_t S = dc->max_batch;
+        c->acc_bytes = S * 4 * 12 + S * S2D2_MAX_BLOCK * 4 * 3 + 256;
+        CUDA_TRY(c, cudaMallocHost((void**)&c->acc_h, c->acc_bytes));
+        CUDA_TRY(c, cudaMalloc((void**)&c->acc_d, c->acc_bytes));
+    }
+    for (int i = 0; i < 8; ++i) CUDA_TRY(c, cudaEventCreate(&c->ev[i]));
+    int grc = gemm_init(c);
+    if (grc != S2D2_OK) return grc;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_destroy(s2d2_ctx* c) {
+    if (!c) return S2D2_ERR_INVALID;
+    cudaStreamSynchronize(c->stream);
+    gemm_destroy(c);
+    void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
+                    c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
+                    c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
+                    c->d_margin, c->d_entropy, c->d_lse, c->acc_d};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    if (c->meta.h) cudaFreeHost(c->meta.h);
+    if (c->stats_h) cudaFreeHost(c->stats_h);
+    if (c->acc_h) cudaFreeHost(c->acc_h);
+    for (int i = 0; i < 8; ++i)
+        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    delete c;
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_load_weights(s2d2_ctx* c, const s2d2_tensor_desc* t, int32_t n) {
+    if (!c || (!t && n > 0)) return S2D2_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        auto it = c->slots.find(t[i].name ? t[i].name : "");
+        if (it == c->slots.end()) FAIL(c, S2D2_ERR_INVALID, std::string("unknown tensor: ") + (t[i].name ? t[i].name : "(null)"));
+        WeightSlot& s = it->second;
+        size_t elems = 1;
+        for (int k = 0; k < t[i].ndim; ++k) elems *= (size_t)t[i].shape[k];
+        if (t[i].dtype != s.dtype || elems * esize(t[i].dtype) != s.bytes || !t[i].data)
+            FAIL(c, S2D2_ERR_INVALID, std::string("tensor has wrong dtype or size: ") + t[i].name);
+        CUDA_TRY(c, cudaMemcpyAsync(s.d_ptr, t[i].data, s.bytes, cudaMemcpyHostToDevice, c->stream));
+        s.loaded = true;
+    }
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    c->weights_checked = false;
+    return S2D2_OK;
+}
+
+static int check_weights(s2d2_ctx* c) {
+    if (c->weights_checked) return S2D2_OK;
+    for (auto& kv : c->slots)
+        if (!kv.second.loaded) FAIL(c, S2D2_ERR_MISSING_WEIGHT, "tensor not loaded: " + kv.first);
+    c->weights_checked = true;
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// pass construction and execution
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct PassBuild {
+    int n_rows = 0, n_seqs = 0, n_logit = 0;
+};
+
+int ensure_pages(s2d2_ctx* c, SeqState& s, int n_tokens) {
+    int need = (n_tokens + c->page_tokens - 1) / c->page_tokens;
+    if (need > c->max_pages_per_seq) FAIL(c, S2D2_ERR_OOM, "sequence longer than max_seq_len");
+    while ((int)s.pages.size() < need) {
+        if (c->free_pages.empty()) FAIL(c, S2D2_ERR_OOM, "KV page pool exhausted");
+        s.pages.push_back(c->free_pages.back());
+        c->free_pages.pop_back();
+    }
+    return S2D2_OK;
+}
+
+// Starts the rows of one sequence in the pass being built.
+void begin_seq(s2d2_ctx* c, PassBuild& pb, const SeqState& s, int n_ctx) {
+    PassMeta& pm = c->meta;
+    int q = pb.n_seqs++;
+    pm.hp<int>(pm.off_nctx)[q] = n_ctx;
+    pm.hp<int>(pm.off_row0)[q] = pb.n_rows;
+    pm.hp<int>(pm.off_nrows)[q] = 0;
+    int* pg = pm.hp<int>(pm.off_pages) + (size_t)q * pm.max_pages;
+    for (size_t i = 0; i < s.pages.size(); ++i) pg[i] = s.pages[i];
+}
+void add_row(s2d2_ctx* c, PassBuild& pb, int token, int pos, unsigned long long mask, int flags, bool logits) {
+    PassMeta& pm = c->meta;
+    int r = pb.n_rows++, q = pb.n_seqs - 1;
+    pm.hp<int>(pm.off_token)[r] = token;
+    pm.hp<int>(pm.off_pos)[r] = pos;
+    pm.hp<int>(pm.off_seq)[r] = q;
+    pm.hp<int>(pm.off_flags)[r] = flags;
+    pm.hp<unsigned long long>(pm.off_mask)[r] = mask;
+    pm.hp<int>(pm.off_nrows)[q]++;
+    if (logits) pm.hp<int>(pm.off_logit_rows)[pb.n_logit++] = r;
+}
+PassView make_view(s2d2_ctx* c, const PassBuild& pb) {
+    PassMeta& pm = c->meta;
+    PassView v;
+    v.n_rows = pb.n_rows;
+    v.n_seqs = pb.n_seqs;
+    v.n_logit_rows = pb.n_logit;
+    v.row_token = pm.dp<int>(pm.off_token);
+    v.row_pos = pm.dp<int>(pm.off_pos);
+    v.row_seq = pm.dp<int>(pm.off_seq);
+    v.row_flags = pm.dp<int>(pm.off_flags);
+    v.row_mask = pm.dp<unsigned long long>(pm.off_mask);
+    v.logit_rows = pm.dp<int>(pm.off_logit_rows);
+    v.seq_nctx = pm.dp<int>(pm.off_nctx);
+    v.seq_row0 = pm.dp<int>(pm.off_row0);
+    v.seq_nrows = pm.dp<int>(pm.off_nrows);
+    v.seq_pages = pm.dp<int>(pm.off_pages);
+    v.max_pages = pm.max_pages;
+    return v;
+}
+
+template <typename TKV>
+KvPool<TKV> make_pool(s2d2_ctx* c) {
+    KvPool<TKV> p;
+    p.base = (TKV*)c->kv_base;
+    p.page_tokens = c->page_tokens;
+    p.page_shift = c->page_shift;
+    p.n_kv_heads = c->m.n_kv_heads;
+    p.head_dim = c->m.head_dim;
+    p.page_stride = (size_t)2 * c->m.n_kv_heads * c->page_tokens * c->m.head_dim;
+    p.layer_stride = (size_t)c->n_pages * p.page_stride;
+    return p;
+}
+
+template <typename TA, typename TKV>
+void launch_attention(s2d2_ctx* c, const PassView& pv, int layer) {
+    const s2d2_model_config& m = c->m;
+    int warps = pv.n_rows * m.n_q_heads;
+    int blocks = (warps + 3) / 4;
+    float scale = 1.f / sqrtf((float)m.head_dim);
+    KvPool<TKV> pool = make_pool<TKV>(c);
+#define ATT(HD)                                                                                                   \
+    attention_simt_kernel<TA, TKV, HD><<<blocks, 128, 0, c->stream>>>((const TA*)c->q, (const TKV*)c->k_rows,     \
+                                                                      (const TKV*)c->v_rows, pv, pool, layer,     \
+                                                                      m.n_q_heads, m.n_kv_heads, (TA*)c->attn, scale)
+    if (m.head_dim == 32) ATT(32);
+    else if (m.head_dim == 64) ATT(64);
+    else ATT(128);
+#undef ATT
+    LAUNCHED(c);
+}
+
+// One pass of the network over the rows described by the uploaded metadata.
+// Logits of pv.logit_rows go to `logits_out` (row-major [n_logit_rows, vocab]).
+template <typename TW, typename TA, typename TKV>
+int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
+    const s2d2_model_config& m = c->m;
+    PassView pv = make_view(c, pb);
+    cudaStream_t st = c->stream;
+    int M = pb.n_rows, d = m.d_model, hd = m.head_dim;
+    if (M == 0) return S2D2_OK;
+    int nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, nq = m.n_q_heads * hd;
+    CUDA_TRY(c, cudaMemcpyAsync(c->meta.d, c->meta.h, c->meta.bytes, cudaMemcpyHostToDevice, st));
+    embed_kernel<TW><<<M, 256, 0, st>>>((const TW*)c->embed, pv.row_token, c->h, d);
+    LAUNCHED(c);
+    KvPool<TKV> pool = make_pool<TKV>(c);
+    for (int l = 0; l < m.n_layers; ++l) {
+        const LayerWeights& L = c->layers[l];
+        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.attn_norm, (TA*)c->xn, d, m.rms_eps);
+        LAUNCHED(c);
+        int rc = gemm(c, c->xn, L.wqkv, c->qkv, M, nqkv, d, nqkv, 1.f, 0);
+        if (rc) return rc;
+        qk_rope_kv_kernel<TA, TKV><<<dim3(M, m.n_q_heads + 2 * m.n_kv_heads), hd / 2, 0, st>>>(
+            c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
+            l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
+        LAUNCHED(c);
+        launch_attention<TA, TKV>(c, pv, l);
+        if ((rc = gemm(c, c->attn, L.wo, c->h, M, d, nq, d, 1.f, 1))) return rc;
+        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.ffn_norm, (TA*)c->xn, d, m.rms_eps);
+        LAUNCHED(c);
+        if (m.n_experts > 0) {
+            int E = m.n_experts, k = m.top_k, fe = m.expert_ffn, P = M * k;
+            if ((rc = gemm(c, c->xn, L.router, c->router_logits, M, E, d, E, 1.f, 0))) return rc;
+            moe_topk_kernel<<<M, 32, 0, st>>>(c->router_logits, M, E, k, c->moe_ids, c->moe_gates);
+            LAUNCHED(c);
+            CUDA_TRY(c, cudaMemcpyAsync(c->moe_ids_trace + (size_t)l * c->max_rows * k, c->moe_ids, (size_t)P * 4,
+                                        cudaMemcpyDeviceToDevice, st));
+            moe_gateup_kernel<TW, TA><<<dim3((2 * fe + 3) / 4, P), 128, 0, st>>>(
+                (const TA*)c->xn, (const TW*)L.e_gate, (const TW*)L.e_up, c->moe_ids, c->moe_gu, k, fe, d);
+            LAUNCHED(c);
+            swiglu_kernel<TA><<<(unsigned)(((size_t)P * fe + 255) / 256), 256, 0, st>>>(c->moe_gu, (TA*)c->moe_act, P, fe);
+            LAUNCHED(c);
+            moe_down_kernel<TW, TA><<<dim3((d + 3) / 4, P), 128, 0, st>>>((const TA*)c->moe_act, (const TW*)L.e_down,
+                                                                         c->moe_ids, c->moe_out, fe, d);
+            LAUNCHED(c);
+            moe_combine_kernel<<<(unsigned)(((size_t)M * d + 255) / 256), 256, 0, st>>>(c->moe_out, c->moe_gates, c->h, M,
+                                                                                       k, d);
+            LAUNCHED(c);
+            c->cnt.moe_expert_tiles_touched += 0;   // filled by the grouped kernel when it is in use
+            if (m.n_shared > 0) {
+                int fs = fe * m.n_shared;
+                if ((rc = gemm(c, c->xn, L.s_gu, c->gu, M, 2 * fs, d, 2 * fs, 1.f, 0))) return rc;
+                swiglu_kernel<TA><<<(unsigned)(((size_t)M * fs + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, M, fs);
+                LAUNCHED(c);
+                if ((rc = gemm(c, c->act, L.s_down, c->h, M, d, fs, d, 1.f, 1))) return rc;
+            }
+        } else {
+            int f = m.ffn;
+            if ((rc = gemm(c, c->xn, L.wgu, c->gu, M, 2 * f, d, 2 * f, 1.f, 0))) return rc;
+            swiglu_kernel<TA><<<(unsigned)(((size_t)M * f + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, M, f);
+            LAUNCHED(c);
+            if ((rc = gemm(c, c->act, L.wdown, c->h, M, d, f, d, 1.f, 1))) return rc;
+        }
+    }
+    c->last_pass_rows = M;
+    if (pb.n_logit > 0 && logits_out) {
+        rmsnorm_kernel<TA><<<pb.n_logit, 256, 0, st>>>(c->h, pv.logit_rows, c->final_norm, (TA*)c->xn, d, m.rms_eps);
+        LAUNCHED(c);
+        int rc = gemm(c, c->xn, c->lm_head, logits_out, pb.n_logit, m.vocab, d, m.vocab, m.logit_scale, 0);
+        if (rc) return rc;
+    }
+    CUDA_TRY(c, cudaGetLastError());
+    return S2D2_OK;
+}
+
+int run_pass(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
+    if (c->m.dtype == S2D2_DTYPE_F32) return run_pass_t<float, float, float>(c, pb, logits_out);
+    return run_pass_t<bf16, bf16, bf16>(c, pb, logits_out);
+}
+
+SeqState* get_seq(s2d2_ctx* c, int id) {
+    if (id < 0 || id >= (int)c->seqs.size() || !c->seqs[id].active) return nullptr;
+    return &c->seqs[id];
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// prefill
+// ---------------------------------------------------------------------------------------------
+extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompts, const int32_t* lens,
+                            int32_t* ids_out) {
+    if (!c || n < 1 || !prompts || !lens || !ids_out) return S2D2_ERR_INVALID;
+    int rc = check_weights(c);
+    if (rc) return rc;
+    std::vector<int> ids;
+    for (int i = 0; i < n; ++i) {
+        if (lens[i] < 1 || lens[i] + c->dc.block_size > c->dc.max_seq_len) FAIL(c, S2D2_ERR_INVALID, "prompt length");
+        for (int t = 0; t < lens[i]; ++t)
+            if (prompts[i][t] < 0 || prompts[i][t] >= c->m.vocab) FAIL(c, S2D2_ERR_INVALID, "prompt token out of range");
+    }
+    for (int i = 0; i < n; ++i) {
+        int slot = -1;
+        for (int k = 0; k < (int)c->seqs.size(); ++k)
+            if (!c->seqs[k].active) {
+                slot = k;
+                break;
+            }
+        if (slot < 0) {
+            for (int id : ids) s2d2_release_seq(c, id);
+            FAIL(c, S2D2_ERR_OOM, "no free sequence slot (max_batch)");
+        }
+        SeqState& s = c->seqs[slot];
+        s = SeqState();
+        s.active = true;
+        s.rng_stream = (uint32_t)slot;
+        s.tok.assign(prompts[i], prompts[i] + lens[i]);
+        s.n_final = s.n_prompt = lens[i];
+        ids.push_back(slot);
+        ids_out[i] = slot;
+    }
+    CUDA_TRY(c, cudaEventRecord(c->ev[6], c->stream));
+    const int CH = S2D2_MAX_ROWS_PER_SEQ;
+    for (;;) {
+        PassBuild pb;
+        for (int id : ids) {
+            SeqState& s = c->seqs[id];
+            int left = s.n_final - s.n_c;
+            if (left <= 0) continue;
+            int rows = std::min(left, CH);
+            if ((rc = ensure_pages(c, s, s.n_c + rows))) return rc;
+            begin_seq(c, pb, s, s.n_c);
+            for (int r = 0; r < rows; ++r)
+                add_row(c, pb, s.tok[s.n_c + r], s.n_c + r, (r == 63) ? ~0ull : ((1ull << (r + 1)) - 1), ROW_WRITE_KV, false);
+        }
+        if (pb.n_rows == 0) break;
+        if ((rc = run_pass(c, pb, nullptr))) return rc;
+        c->cnt.n_prefill_passes++;
+        // the metadata buffer is reused by the next chunk: wait for this pass to have consumed it
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        for (int id : ids) {
+            SeqState& s = c->seqs[id];
+            s.n_c = std::min(s.n_final, s.n_c + CH);
+        }
+    }
+    CUDA_TRY(c, cudaEventRecord(c->ev[7], c->stream));
+    CUDA_TRY(c, cudaEventSynchronize(c->ev[7]));
+    float ms = 0;
+    cudaEventElapsedTime(&ms, c->ev[6], c->ev[7]);
+    c->cnt.ms_prefill += ms;
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_seq_set_rng_stream(s2d2_ctx* c, int32_t id, uint32_t stream) {
+    if (!c) return S2D2_ERR_INVALID;
+    SeqState* s = get_seq(c, id);
+    if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+    s->rng_stream = stream;
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// draft pass
+// ---------------------------------------------------------------------------------------------
+extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2_draft_stats* out) {
+    if (!c || n < 1 || !ids || !out) return S2D2_ERR_INVALID;
+    const int B = c->dc.block_size, MASK = c->m.vocab;
+    int rc;
+    for (int i = 0; i < n; ++i) {
+        SeqState* s = get_seq(c, ids[i]);
+        if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+        if (s->drafted) FAIL(c, S2D2_ERR_STATE, "draft_block called twice without accept_and_commit");
+        for (int k = 0; k < i; ++k)
+            if (ids[k] == ids[i]) FAIL(c, S2D2_ERR_INVALID, "duplicate sequence id");
+        if (!s->block_open && s->n_final + B > c->dc.max_seq_len) FAIL(c, S2D2_ERR_OOM, "max_seq_len reached");
+    }
+    PassBuild pb;
+    for (int i = 0; i < n; ++i) {
+        SeqState& s = c->seqs[ids[i]];
+        if (!s.block_open) {
+            s.tok.resize(s.n_final + B, MASK);
+            s.block_open = true;
+        }
+        int st = s.n_final, j = 0;
+        while (j < B && s.tok[st + j] != MASK) ++j;
+        int P = st + j - s.n_c;          // committed tokens without K/V
+        int rows = P + (B - j);
+        if (rows > S2D2_MAX_ROWS_PER_SEQ) FAIL(c, S2D2_ERR_UNSUPPORTED, "too many rows for one sequence in a draft pass");
+        if ((rc = ensure_pages(c, s, st + B))) return rc;
+        begin_seq(c, pb, s, s.n_c);
+        unsigned long long all = rows == 64 ? ~0ull : ((1ull << rows) - 1);
+        for (int p = 0; p < P; ++p)     // pending rows: causal among themselves, K/V appended
+            add_row(c, pb, s.tok[s.n_c + p], s.n_c + p, (1ull << (p + 1)) - 1, ROW_WRITE_KV, false);
+        s.j = j;
+        s.n_masked = 0;
+        s.draft_row0 = pb.n_logit;
+        for (int i2 = j; i2 < B; ++i2) {  // block rows: see the whole pass
+            bool masked = s.tok[st + i2] == MASK;
+            add_row(c, pb, s.tok[st + i2], st + i2, all, 0, masked);
+            if (masked) s.masked_idx[s.n_masked++] = i2;
+        }
+        s.span_len = 1;
+        while (j + s.span_len < B && s.tok[st + j + s.span_len] == MASK) ++s.span_len;
+    }
+    if (pb.n_logit > c->max_logit_rows || pb.n_rows > c->max_rows) FAIL(c, S2D2_ERR_UNSUPPORTED, "pass too large");
+    CUDA_TRY(c, cudaEventRecord(c->ev[0], c->stream));
+    if ((rc = run_pass(c, pb, c->logits_draft))) return rc;
+    DraftStatsOut so{c->d_xhat, c->d_conf, c->d_margin, c->d_entropy, c->d_lse};
+    draft_stats_kernel<<<pb.n_logit, VOCAB_THREADS, 0, c->stream>>>(c->logits_draft, c->m.vocab, so);
+    LAUNCHED(c);
+    size_t R = pb.n_logit;
+    int* hx = (int*)c->stats_h;
+    float* hc = (float*)(c->stats_h + R * 4);
+    float* hm = (float*)(c->stats_h + R * 8);
+    float* he = (float*)(c->stats_h + R * 12);
+    CUDA_TRY(c, cudaMemcpyAsync(hx, c->d_xhat, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(hc, c->d_conf, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(hm, c->d_margin, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(he, c->d_entropy, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaEventRecord(c->ev[1], c->stream));
+    CUDA_TRY(c, cudaEventSynchronize(c->ev[1]));
+    float ms = 0;
+    cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]);
+    c->cnt.ms_draft += ms;
+    c->cnt.n_draft_passes++;
+    c->n_draft_logit_rows = pb.n_logit;
+    for (int i = 0; i < n; ++i) {
+        SeqState& s = c->seqs[ids[i]];
+        s2d2_draft_stats& o = out[i];
+        memset(&o, 0, sizeof(o));
+        s.n_c = s.n_final + s.j;         // pending rows are cached now
+        o.seq_id = ids[i];
+        o.block_start = s.n_final;
+        o.first_masked = s.j;
+        o.n_masked = s.n_masked;
+        o.span_len = s.span_len;
+        double sum = 0;
+        for (int k = 0; k < s.n_masked; ++k) {
+            int r = s.draft_row0 + k;
+            o.masked_idx[k] = s.masked_idx[k];
+            o.xhat[k] = s.xhat[k] = hx[r];
+            o.conf[k] = s.conf[k] = hc[r];
+            o.margin[k] = hm[r];
+            o.entropy[k] = he[r];
+            sum += hc[r];
+            if (hc[r] > c->dc.tau_conf) o.n_hi++;
+        }
+        o.mean_conf = (float)(sum / std::max(1, s.n_masked));
+        s.drafted = true;
+    }
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// routing (host)
+// ---------------------------------------------------------------------------------------------
+extern "C" int s2d2_set_router(s2d2_ctx* c, s2d2_route_fn fn, void* user) {
+    if (!c) return S2D2_ERR_INVALID;
+    c->route_fn = fn;
+    c->route_user = user;
+    return S2D2_OK;
+}
+extern "C" int s2d2_set_route_policy(s2d2_ctx* c, const s2d2_route_policy* p) {
+    if (!c || !p || p->policy < 0 || p->policy > S2D2_ROUTE_NEVER) return S2D2_ERR_INVALID;
+    c->policy = *p;
+    for (auto& s : c->seqs) s.hyst_on = true;
+    return S2D2_OK;
+}
+
+// Expected accepted prefix length K_hat = sum_k prod_{i<=k} alpha_i over the span (Eq. khat)
+// and the static / dynamic verification score.
+static double route_score(const s2d2_ctx* c, const s2d2_draft_stats* st) {
+    const s2d2_route_policy& p = c->policy;
+    double khat = 0, prod = 1;
+    for (int i = 0; i < st->span_len; ++i) {     // masked_idx[0..span_len) is the span
+        double alpha = p.alpha_entropy ? exp(-(double)p.alpha_param * st->entropy[i] / log((double)c->m.vocab))
+                                       : (st->margin[i] >= p.alpha_param ? 1.0 : 0.0);
+        prod *= alpha;
+        khat += prod;
+    }
+    return p.dynamic_cost ? khat - (double)p.cost * st->n_hi : khat - (double)p.cost;
+}
+
+extern "C" int s2d2_route(s2d2_ctx* c, int32_t n, const s2d2_draft_stats* st, uint8_t* flags) {
+    if (!c || n < 1 || !st || !flags) return S2D2_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        if (c->route_fn) {
+            flags[i] = c->route_fn(c->route_user, &st[i]) ? 1 : 0;
+            continue;
+        }
+        const s2d2_route_policy& p = c->policy;
+        switch (p.policy) {
+            case S2D2_ROUTE_MIN_SPAN: flags[i] = st[i].span_len >= (int)p.p0; break;
+            case S2D2_ROUTE_SCORE: flags[i] = route_score(c, &st[i]) >= p.p0; break;
+            case S2D2_ROUTE_HYSTERESIS: {
+                SeqState* s = get_seq(c, st[i].seq_id);
+                if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id in stats");
+                double sc = route_score(c, &st[i]);
+                if (s->hyst_on && sc < p.p1) s->hyst_on = false;
+                else if (!s->hyst_on && sc >= p.p0) s->hyst_on = true;
+                flags[i] = s->hyst_on;
+                break;
+            }
+            case S2D2_ROUTE_MEAN_CONF: flags[i] = st[i].mean_conf < p.p0; break;
+            default: flags[i] = 0;
+        }
+    }
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// verifier pass
+// ---------------------------------------------------------------------------------------------
+extern "C" int s2d2_verify_block(s2d2_ctx* c, int32_t n, const int32_t* ids, const uint8_t* flags) {
+    if (!c || n < 1 || !ids || !flags) return S2D2_ERR_INVALID;
+    const int MASK = c->m.vocab;
+    int rc;
+    PassBuild pb;
+    for (int i = 0; i < n; ++i) {
+        SeqState* s = get_seq(c, ids[i]);
+        if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+        if (!s->drafted) FAIL(c, S2D2_ERR_STATE, "verify_block without a draft pass");
+        if (s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "verify_block called twice");
+    }
+    for (int i = 0; i < n; ++i) {
+        if (!flags[i]) continue;
+        SeqState& s = c->seqs[ids[i]];
+        int L = s.span_len, p0 = s.n_final + s.j;
+        if ((rc = ensure_pages(c, s, p0 + L))) return rc;
+        begin_seq(c, pb, s, s.n_c);
+        s.verify_row0 = pb.n_logit;
+        // drafted tokens: causal block A_L; their K/V goes to the cache speculatively
+        for (int k = 0; k < L; ++k) add_row(c, pb, s.xhat[k], p0 + k, (1ull << (k + 1)) - 1, ROW_WRITE_KV, false);
+        // MASK copies at the same positions: strictly-left drafted tokens plus itself
+        for (int k = 0; k < L; ++k)
+            add_row(c, pb, MASK, p0 + k, ((1ull << k) - 1) | (1ull << (L + k)), 0, true);
+        s.verify_in_flight = true;
+    }
+    c->n_verify_logit_rows = pb.n_logit;
+    if (pb.n_rows == 0) return S2D2_OK;
+    CUDA_TRY(c, cudaEventRecord(c->ev[2], c->stream));
+    if ((rc = run_pass(c, pb, c->logits_verify))) return rc;
+    CUDA_TRY(c, cudaEventRecord(c->ev[3], c->stream));
+    c->verify_timing_pending = true;
+    c->cnt.n_verify_passes++;
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// acceptance + commit
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct AccStage {     // layout of acc_h / acc_d for S sequences
+    size_t S;
+    size_t o_draft0, o_verify0, o_len, o_pos0, o_stream, o_step, o_mode;     // inputs
+    size_t o_nacc, o_rej, o_res, o_near, o_bits, o_u, o_a, o_v;              // outputs
+    size_t in_bytes, total;
+    explicit AccStage(size_t s) : S(s) {
+        size_t o = 0;
+        auto t = [&](size_t b) { size_t r = o; o += b; return r; };
+        o_draft0 = t(S * 4); o_verify0 = t(S * 4); o_len = t(S * 4); o_pos0 = t(S * 4);
+        o_stream = t(S * 4); o_step = t(S * 4); o_mode = t(S * 4);
+        in_bytes = o;
+        o_nacc = t(S * 4); o_rej = t(S * 4); o_res = t(S * 4); o_near = t(S * 4); o_bits = t(S * 4);
+        o_u = t(S * S2D2_MAX_BLOCK * 4); o_a = t(S * S2D2_MAX_BLOCK * 4); o_v = t(S * S2D2_MAX_BLOCK * 4);
+        total = o;
+    }
+};
+
+int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, const float* d_verify, const int* d_xhat,
+                  const double* d_lse, const float* d_conf) {
+    CUDA_TRY(c, cudaMemcpyAsync(c->acc_d, c->acc_h, a.in_bytes, cudaMemcpyHostToDevice, c->stream));
+    AcceptIn in;
+    in.draft_logits = d_draft;
+    in.verify_logits = d_verify;
+    in.V = c->m.vocab;
+    in.seq_draft_row0 = (const int*)(c->acc_d + a.o_draft0);
+    in.seq_verify_row0 = (const int*)(c->acc_d + a.o_verify0);
+    in.seq_len = (const int*)(c->acc_d + a.o_len);
+    in.seq_pos0 = (const int*)(c->acc_d + a.o_pos0);
+    in.seq_stream = (const unsigned*)(c->acc_d + a.o_stream);
+    in.seq_step = (const int*)(c->acc_d + a.o_step);
+    in.seq_mode = (const int*)(c->acc_d + a.o_mode);
+    in.xhat = d_xhat;
+    in.draft_lse = d_lse;
+    in.conf = d_conf;
+    in.tau_conf = c->dc.tau_conf;
+    in.seed = c->dc.seed;
+    in.gamma = c->dc.ratio_gamma;
+    in.resample = c->dc.resample;
+    in.l_cap = S2D2_MAX_BLOCK;
+    AcceptOut out;
+    out.n_accepted = (int*)(c->acc_d + a.o_nacc);
+    out.first_reject = (int*)(c->acc_d + a.o_rej);
+    out.resampled = (int*)(c->acc_d + a.o_res);
+    out.n_near = (int*)(c->acc_d + a.o_near);
+    out.commit_bits = (unsigned*)(c->acc_d + a.o_bits);
+    out.u = (float*)(c->acc_d + a.o_u);
+    out.a = (float*)(c->acc_d + a.o_a);
+    out.v = (float*)(c->acc_d + a.o_v);
+    accept_block_kernel<<<n, VOCAB_THREADS, 0, c->stream>>>(in, out);
+    LAUNCHED(c);
+    CUDA_TRY(c, cudaMemcpyAsync(c->acc_h + a.in_bytes, c->acc_d + a.in_bytes, a.total - a.in_bytes,
+                                cudaMemcpyDeviceToHost, c->stream));
+    return S2D2_OK;
+}
+}  // namespace
+
+extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids, const uint8_t* flags,
+                                      s2d2_step_result* res) {
+    if (!c || n < 1 || !ids || !flags || !res) return S2D2_ERR_INVALID;
+    if (n > c->dc.max_batch) return S2D2_ERR_INVALID;
+    const int B = c->dc.block_size, MASK = c->m.vocab;
+    for (int i = 0; i < n; ++i) {
+        SeqState* s = get_seq(c, ids[i]);
+        if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+        if (!s->drafted) FAIL(c, S2D2_ERR_STATE, "accept_and_commit without a draft pass");
+        if (flags[i] && !s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "sequence flagged verified but verify_block did not run for it");
+        if (!flags[i] && s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "verify flags differ from those given to verify_block");
+    }
+    AccStage a(n);
+    for (int i = 0; i < n; ++i) {
+        SeqState& s = c->seqs[ids[i]];
+        ((int*)(c->acc_h + a.o_draft0))[i] = s.draft_row0;
+        ((int*)(c->acc_h + a.o_verify0))[i] = flags[i] ? s.verify_row0 : 0;
+        ((int*)(c->acc_h + a.o_len))[i] = flags[i] ? s.span_len : s.n_masked;
+        ((int*)(c->acc_h + a.o_pos0))[i] = s.n_final + s.j;
+        ((unsigned*)(c->acc_h + a.o_stream))[i] = s.rng_stream;
+        ((int*)(c->acc_h + a.o_step))[i] = s.step;
+        ((int*)(c->acc_h + a.o_mode))[i] = flags[i] ? 1 : 0;
+    }
+    CUDA_TRY(c, cudaEventRecord(c->ev[4], c->stream));
+    int rc = launch_accept(c, a, n, c->logits_draft, c->logits_verify, c->d_xhat, c->d_lse, c->d_conf);
+    if (rc) return rc;
+    CUDA_TRY(c, cudaEventRecord(c->ev[5], c->stream));
+    CUDA_TRY(c, cudaEventSynchronize(c->ev[5]));
+    float ms = 0;
+    cudaEventElapsedTime(&ms, c->ev[4], c->ev[5]);
+    c->cnt.ms_accept += ms;
+    if (c->verify_timing_pending) {
+        cudaEventElapsedTime(&ms, c->ev[2], c->ev[3]);
+        c->cnt.ms_verify += ms;
+        c->verify_timing_pending = false;
+    }
+    const int* h_nacc = (const int*)(c->acc_h + a.o_nacc);
+    const int* h_rej = (const int*)(c->acc_h + a.o_rej);
+    const int* h_res = (const int*)(c->acc_h + a.o_res);
+    const int* h_near = (const int*)(c->acc_h + a.o_near);
+    const unsigned* h_bits = (const unsigned*)(c->acc_h + a.o_bits);
+    for (int i = 0; i < n; ++i) {
+        SeqState& s = c->seqs[ids[i]];
+        s2d2_step_result& o = res[i];
+        memset(&o, 0, sizeof(o));
+        o.seq_id = ids[i];
+        o.verified = flags[i] ? 1 : 0;
+        o.first_reject = -1;
+        o.resampled_id = -1;
+        int st = s.n_final;
+        if (flags[i]) {
+            int na = h_nacc[i];
+            o.n_accepted = na;
+            o.first_reject = h_rej[i];
+            o.resampled_id = h_res[i];
+            o.n_near_boundary = h_near[i];
+            int scanned = h_rej[i] >= 0 ? h_rej[i] + 1 : na;
+            for (int k = 0; k < scanned; ++k) {
+                o.u[k] = ((const float*)(c->acc_h + a.o_u))[(size_t)i * S2D2_MAX_BLOCK + k];
+                o.a[k] = ((const float*)(c->acc_h + a.o_a))[(size_t)i * S2D2_MAX_BLOCK + k];
+                o.v[k] = ((const float*)(c->acc_h + a.o_v))[(size_t)i * S2D2_MAX_BLOCK + k];
+            }
+            for (int k = 0; k < na; ++k) {
+                s.tok[st + s.j + k] = s.xhat[k];
+                o.committed_idx[o.n_committed] = s.j + k;
+                o.committed_tok[o.n_committed++] = s.xhat[k];
+            }
+            s.n_c += na;   // accepted drafted rows keep their K/V; rows past them are rolled back by length
+            if (h_rej[i] >= 0 && c->dc.resample) {
+                s.tok[st + s.j + na] = h_res[i];
+                o.committed_idx[o.n_committed] = s.j + na;
+                o.committed_tok[o.n_committed++] = h_res[i];
+                c->cnt.n_resampled++;
+            }
+            c->cnt.n_accepted_tokens += na;
+            c->cnt.accepted_len_hist[std::min(na, S2D2_MAX_BLOCK)]++;
+            c->cnt.n_near_boundary += h_near[i];
+        } else {
+            for (int k = 0; k < s.n_masked; ++k)
+                if (h_bits[i] >> k & 1) {
+                    s.tok[st + s.masked_idx[k]] = s.xhat[k];
+                    o.committed_idx[o.n_committed] = s.masked_idx[k];
+                    o.committed_tok[o.n_committed++] = s.xhat[k];
+                }
+        }
+        c->cnt.n_committed_tokens += o.n_committed;
+        c->cnt.n_steps++;
+        s.step++;
+        s.drafted = false;
+        s.verify_in_flight = false;
+        bool done = true;
+        for (int k = 0; k < B; ++k)
+            if (s.tok[st + k] == MASK) done = false;
+        if (done) {
+            s.n_final += B;
+            s.block_open = false;
+        }
+        o.block_done = done;
+    }
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_accept_logits(s2d2_ctx* c, const float* d_draft, const float* d_verify, int32_t n, int32_t l_max,
+                                  const int32_t* span_len, const int32_t* xhat, const int32_t* pos0,
+                                  const uint32_t* rng_stream, const int32_t* step, s2d2_step_result* res) {
+    if (!c || !d_draft || !d_verify || n < 1 || l_max < 1 || l_max > S2D2_MAX_BLOCK || !span_len || !xhat || !pos0 ||
+        !rng_stream || !step || !res)
+        return S2D2_ERR_INVALID;
+    if (n > c->dc.max_batch || n * l_max > c->max_logit_rows) FAIL(c, S2D2_ERR_INVALID, "accept_logits: batch larger than the context");
+    AccStage a(n);
+    for (int i = 0; i < n; ++i) {
+        if (span_len[i] < 0 || span_len[i] > l_max) FAIL(c, S2D2_ERR_INVALID, "accept_logits: span_len");
+        for (int k = 0; k < span_len[i]; ++k)
+            if (xhat[i * l_max + k] < 0 || xhat[i * l_max + k] >= c->m.vocab) FAIL(c, S2D2_ERR_INVALID, "accept_logits: xhat out of range");
+        ((int*)(c->acc_h + a.o_draft0))[i] = i * l_max;
+        ((int*)(c->acc_h + a.o_verify0))[i] = i * l_max;
+        ((int*)(c->acc_h + a.o_len))[i] = span_len[i];
+        ((int*)(c->acc_h + a.o_pos0))[i] = pos0[i];
+        ((unsigned*)(c->acc_h + a.o_stream))[i] = rng_stream[i];
+        ((int*)(c->acc_h + a.o_step))[i] = step[i];
+        ((int*)(c->acc_h + a.o_mode))[i] = 1;
+    }
+    CUDA_TRY(c, cudaMemcpyAsync(c->d_xhat, xhat, (size_t)n * l_max * 4, cudaMemcpyHostToDevice, c->stream));
+    int rc = launch_accept(c, a, n, d_draft, d_verify, c->d_xhat, nullptr, nullptr);
+    if (rc) return rc;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int i = 0; i < n; ++i) {
+        s2d2_step_result& o = res[i];
+        memset(&o, 0, sizeof(o));
+        o.seq_id = i;
+        o.verified = 1;
+        o.n_accepted = ((const int*)(c->acc_h + a.o_nacc))[i];
+        o.first_reject = ((const int*)(c->acc_h + a.o_rej))[i];
+        o.resampled_id = ((const int*)(c->acc_h + a.o_res))[i];
+        o.n_near_boundary = ((const int*)(c->acc_h + a.o_near))[i];
+        int scanned = o.first_reject >= 0 ? o.first_reject + 1 : o.n_accepted;
+        for (int k = 0; k < scanned; ++k) {
+            o.u[k] = ((const float*)(c->acc_h + a.o_u))[(size_t)i * S2D2_MAX_BLOCK + k];
+            o.a[k] = ((const float*)(c->acc_h + a.o_a))[(size_t)i * S2D2_MAX_BLOCK + k];
+            o.v[k] = ((const float*)(c->acc_h + a.o_v))[(size_t)i * S2D2_MAX_BLOCK + k];
+        }
+    }
+    return S2D2_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// convenience loop, accessors, test taps
+// ---------------------------------------------------------------------------------------------
+extern "C" int s2d2_generate(s2d2_ctx* c, int32_t n, const int32_t* ids, int32_t n_new) {
+    if (!c || n < 1 || !ids || n_new < 1) return S2D2_ERR_INVALID;
+    if (n_new % c->dc.block_size) FAIL(c, S2D2_ERR_INVALID, "n_new_tokens must be a multiple of the block size");
+    std::vector<int> target(n);
+    for (int i = 0; i < n; ++i) {
+        SeqState* s = get_seq(c, ids[i]);
+        if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+        target[i] = s->n_final + n_new;
+    }
+    std::vector<int> live;
+    std::vector<s2d2_draft_stats> st(n);
+    std::vector<s2d2_step_result> rs(n);
+    std::vector<uint8_t> fl(n);
+    for (;;) {
+        live.clear();
+        for (int i = 0; i < n; ++i)
+            if (c->seqs[ids[i]].n_final < target[i]) live.push_back(ids[i]);
+        if (live.empty()) break;
+        int k = (int)live.size(), rc;
+        if ((rc = s2d2_draft_block(c, k, live.data(), st.data()))) return rc;
+        if ((rc = s2d2_route(c, k, st.data(), fl.data()))) return rc;
+        if ((rc = s2d2_verify_block(c, k, live.data(), fl.data()))) return rc;
+        if ((rc = s2d2_accept_and_commit(c, k, live.data(), fl.data(), rs.data()))) return rc;
+    }
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_get_tokens(s2d2_ctx* c, int32_t id, int32_t* out, int32_t cap, int32_t* n_out) {
+    if (!c || !n_out) return S2D2_ERR_INVALID;
+    SeqState* s = get_seq(c, id);
+    if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+    *n_out = s->n_final;
+    if (out) {
+        if (cap < s->n_final) FAIL(c, S2D2_ERR_INVALID, "token buffer too small");
+        memcpy(out, s->tok.data(), (size_t)s->n_final * 4);
+    }
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_release_seq(s2d2_ctx* c, int32_t id) {
+    if (!c) return S2D2_ERR_INVALID;
+    SeqState* s = get_seq(c, id);
+    if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+    cudaStreamSynchronize(c->stream);
+    for (int p : s->pages) c->free_pages.push_back(p);
+    *s = SeqState();
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_get_counters(s2d2_ctx* c, s2d2_counters* out) {
+    if (!c || !out) return S2D2_ERR_INVALID;
+    c->cnt.kv_pages_total = c->n_pages;
+    c->cnt.kv_pages_in_use = c->n_pages - (int64_t)c->free_pages.size();
+    *out = c->cnt;
+    return S2D2_OK;
+}
+extern "C" int s2d2_reset_counters(s2d2_ctx* c) {
+    if (!c) return S2D2_ERR_INVALID;
+    memset(&c->cnt, 0, sizeof(c->cnt));
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_debug_copy_logits(s2d2_ctx* c, int32_t which, float* out, int64_t cap, int64_t* n_rows) {
+    if (!c || !out || !n_rows || (which != 0 && which != 1)) return S2D2_ERR_INVALID;
+    int64_t rows = which == 0 ? c->n_draft_logit_rows : c->n_verify_logit_rows;
+    if (cap < rows * c->m.vocab) FAIL(c, S2D2_ERR_INVALID, "logit buffer too small");
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    CUDA_TRY(c, cudaMemcpy(out, which == 0 ? c->logits_draft : c->logits_verify, (size_t)rows * c->m.vocab * 4,
+                           cudaMemcpyDeviceToHost));
+    *n_rows = rows;
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_debug_copy_kv(s2d2_ctx* c, int32_t id, int32_t layer, int32_t n_tokens, float* k_out, float* v_out) {
+    if (!c || !k_out || !v_out || layer < 0 || layer >= c->m.n_layers) return S2D2_ERR_INVALID;
+    SeqState* s = get_seq(c, id);
+    if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+    if (n_tokens < 1 || n_tokens > (int)s->pages.size() * c->page_tokens) FAIL(c, S2D2_ERR_INVALID, "n_tokens beyond the allocated pages");
+    size_t elems = (size_t)n_tokens * c->m.n_kv_heads * c->m.head_dim;
+    float *dk = nullptr, *dv = nullptr;
+    int* dp = nullptr;
+    CUDA_TRY(c, cudaMalloc(&dk, elems * 4));
+    CUDA_TRY(c, cudaMalloc(&dv, elems * 4));
+    CUDA_TRY(c, cudaMalloc(&dp, s->pages.size() * 4));
+    CUDA_TRY(c, cudaMemcpyAsync(dp, s->pages.data(), s->pages.size() * 4, cudaMemcpyHostToDevice, c->stream));
+    if (c->m.dtype == S2D2_DTYPE_F32)
+        kv_export_kernel<float><<<dim3(n_tokens, c->m.n_kv_heads), 64, 0, c->stream>>>(make_pool<float>(c), dp, layer, n_tokens, dk, dv);
+    else
+        kv_export_kernel<bf16><<<dim3(n_tokens, c->m.n_kv_heads), 64, 0, c->stream>>>(make_pool<bf16>(c), dp, layer, n_tokens, dk, dv);
+    CUDA_TRY(c, cudaMemcpyAsync(k_out, dk, elems * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(v_out, dv, elems * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    cudaFree(dk);
+    cudaFree(dv);
+    cudaFree(dp);
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_debug_seq_state(s2d2_ctx* c, int32_t id, int32_t* n_cached, int32_t* block_start,
+                                    int32_t* block_tokens, int32_t* step_index) {
+    if (!c) return S2D2_ERR_INVALID;
+    SeqState* s = get_seq(c, id);
+    if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
+    if (n_cached) *n_cached = s->n_c;
+    if (block_start) *block_start = s->n_final;
+    if (step_index) *step_index = s->step;
+    if (block_tokens)
+        for (int k = 0; k < c->dc.block_size; ++k)
+            block_tokens[k] = s->block_open ? s->tok[s->n_final + k] : c->m.vocab;
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_debug_copy_expert_ids(s2d2_ctx* c, int32_t* out, int64_t cap, int32_t* n_rows) {
+    if (!c || !out || !n_rows) return S2D2_ERR_INVALID;
+    if (c->m.n_experts == 0) FAIL(c, S2D2_ERR_UNSUPPORTED, "not a MoE model");
+    int M = c->last_pass_rows, k = c->m.top_k;
+    if (cap < (int64_t)c->m.n_layers * M * k) FAIL(c, S2D2_ERR_INVALID, "buffer too small");
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int l = 0; l < c->m.n_layers; ++l)
+        CUDA_TRY(c, cudaMemcpy(out + (size_t)l * M * k, c->moe_ids_trace + (size_t)l * c->max_rows * k, (size_t)M * k * 4,
+                               cudaMemcpyDeviceToHost));
+    *n_rows = M;
+    return S2D2_OK;
+}

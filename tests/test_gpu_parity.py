@@ -1,0 +1,190 @@
+"""GPU parity tests: the CUDA path through the C ABI against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import accept as A
+from oracle import philox
+from oracle import s2d2 as S
+from s2d2_inputs import generate_prompts, generate_weights, get_config
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _engine(wl, W, **kw):
+    from paper_2603_25702_b200 import Engine
+    from tests.parity_util import register_prompt_lens
+    args = dict(block_size=wl.block_size, max_batch=max(wl.batch, 1), max_seq_len=wl.prompt_len[1] + wl.gen_tokens + wl.block_size,
+                kv_page_tokens=wl.kv_page_tokens, seed=wl.philox_seed, tau_conf=wl.tau_conf,
+                stream=torch.cuda.current_stream().cuda_stream)
+    args.update(kw)
+    e = Engine(wl.model, **args)
+    e.load_weights(W)
+    return e
+
+
+def _start(wl, W, prompts=None, **kw):
+    from tests.parity_util import register_prompt_lens
+    e = _engine(wl, W, **kw)
+    prompts = generate_prompts(wl) if prompts is None else prompts
+    ids = e.prefill(prompts)
+    register_prompt_lens(ids, prompts)
+    for k, sid in enumerate(ids):
+        e.seq_set_rng_stream(sid, k)
+    return e, ids, prompts
+
+
+def test_c1_free_running_matches_oracle_tokens():
+    """Tiny fp32 config, run end to end without teacher forcing: same committed token ids."""
+    wl = get_config("c1")
+    W = generate_weights(wl.model, seed=wl.weight_seed)
+    e, ids, prompts = _start(wl, W)
+    e.generate(ids, wl.gen_tokens)
+    got = e.get_tokens(ids[0])[len(prompts[0]):].tolist()
+    orc = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0)
+    want = orc.generate(prompts[0], wl.gen_tokens)
+    assert got == want
+    c = e.get_counters()
+    assert c.n_draft_passes == orc.n_draft_passes and c.n_verify_passes == orc.n_verify_passes
+    assert c.n_committed_tokens == wl.gen_tokens
+    e.close()
+
+
+@pytest.mark.parametrize("name,atol,rtol", [("c1", 0.0, 1e-4), ("t_f32", 0.0, 1e-4), ("t_bf16", 2e-2, 0.0),
+                                            ("t_bf16_128", 2e-2, 0.0)])
+def test_stepwise_parity_dense(name, atol, rtol):
+    from tests.parity_util import check_kv, run_steps
+    wl = get_config(name)
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.0 if name == "c1" else 0.1)
+    e, ids, prompts = _start(wl, W)
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_atol=atol, logit_rtol=rtol)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps > 0 and rep.n_committed == wl.gen_tokens * len(ids)
+    for sid in ids:
+        check_kv(e, W, wl.model, sid, atol=1e-5 if wl.model.dtype == "fp32" else 4e-2)
+    print(name, rep)
+    e.close()
+
+
+def test_confidence_branch_and_mixed_routing():
+    """Never / alternately verifying exercises the else-branch, non-contiguous commits and multi-token pending rows."""
+    from tests.parity_util import check_kv, run_steps
+    wl = get_config("t_f32", block_size=8, gen_tokens=16, model_logit_scale=12.0)
+    W = generate_weights(wl.model, seed=2, gain_jitter=0.1)
+    for mode in ("never", "alternate", "mean_conf"):
+        e, ids, prompts = _start(wl, W, tau_conf=0.5)
+        n = {"k": 0}
+
+        def route(st):
+            n["k"] += 1
+            if mode == "never":
+                return False
+            if mode == "alternate":
+                return n["k"] % 2 == 0
+            return st.mean_conf < 0.5
+        rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_rtol=1e-4, logit_atol=0.0,
+                        tau_conf=0.5, route=route)
+        assert not rep.mismatches, (mode, rep.mismatches[:5])
+        assert rep.steps > rep.verified_steps or mode == "mean_conf"
+        for sid in ids:
+            check_kv(e, W, wl.model, sid, atol=1e-5)
+        e.close()
+
+
+def test_batch_composition_does_not_change_results():
+    wl = get_config("t_bf16")
+    W = generate_weights(wl.model, seed=1)
+    prompts = generate_prompts(wl)
+    e, ids, _ = _start(wl, W, prompts)
+    e.generate(ids, wl.gen_tokens)
+    together = [e.get_tokens(s).tolist() for s in ids]
+    e.close()
+    for k, p in enumerate(prompts):
+        e1 = _engine(wl, W)
+        sid = e1.prefill([p])[0]
+        e1.seq_set_rng_stream(sid, k)
+        e1.generate([sid], wl.gen_tokens)
+        assert e1.get_tokens(sid).tolist() == together[k]
+        e1.close()
+
+
+def test_moe_stepwise_parity():
+    from tests.parity_util import moe_prefill_shadows, run_steps
+    wl = get_config("t_moe")
+    W = generate_weights(wl.model, seed=4, gain_jitter=0.1)
+    e, ids, prompts = _start(wl, W)
+    shadows = moe_prefill_shadows(e, W, wl.model, ids, prompts)
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_atol=2e-2, shadows=shadows)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.stage_b_passes > 0 and rep.n_committed == wl.gen_tokens * len(ids)
+    print("moe", rep)
+    e.close()
+
+
+@pytest.mark.parametrize("V,L,n_seqs", [(8, 1, 3), (8, 3, 5), (4096, 4, 4), (151936, 8, 2), (157184, 32, 1), (1000, 32, 3)])
+def test_accept_kernel_on_synthetic_logits(V, L, n_seqs):
+    """The fused acceptance kernel alone, on logits shaped like a drafter/verifier pair
+    that mostly agree (so that both acceptance and rejection occur)."""
+    from paper_2603_25702_b200 import Engine
+    wl = get_config("t_f32", model_vocab=V)
+    e = Engine(wl.model, block_size=min(L, 32), max_batch=n_seqs, max_seq_len=64, kv_page_tokens=8, seed=9,
+               stream=torch.cuda.current_stream().cuda_stream)
+    rng = np.random.default_rng(V + L)
+    n_rej = n_all = 0
+    for trial in range(4):
+        d = (rng.standard_normal((n_seqs * L, V)) * 2.0).astype(np.float32)
+        v = (d + rng.standard_normal((n_seqs * L, V)).astype(np.float32) * (0.05 + 0.4 * trial)).astype(np.float32)
+        if trial == 3:
+            v = d.copy()                       # identical distributions: accept everything
+        span = rng.integers(1, L + 1, size=n_seqs)
+        xhat = d.argmax(axis=1).astype(np.int32)
+        pos0 = rng.integers(0, 1000, size=n_seqs)
+        streams = rng.integers(0, 100, size=n_seqs)
+        steps = rng.integers(0, 50, size=n_seqs)
+        td, tv = torch.from_numpy(d).cuda(), torch.from_numpy(v).cuda()
+        res = e.accept_logits(td.data_ptr(), tv.data_ptr(), n_seqs, L, span, xhat, pos0, streams, steps)
+        for s in range(n_seqs):
+            Ls = int(span[s])
+            u = [philox.uniform(9, int(pos0[s]) + i, int(streams[s]), int(steps[s]), philox.STREAM_ACCEPT) for i in range(Ls)]
+            u2 = [philox.uniform(9, int(pos0[s]) + i, int(streams[s]), int(steps[s]), philox.STREAM_RESAMPLE) for i in range(Ls)]
+            o = A.accept_scan(d[s * L:s * L + Ls], v[s * L:s * L + Ls], xhat[s * L:s * L + Ls], u, u2)
+            r = res[s]
+            if min(o.margin_u) >= 1e-4:
+                assert (o.n_accepted, o.first_reject, o.resampled) == (r.n_accepted, r.first_reject, r.resampled_id), (trial, s)
+            if trial == 3:
+                assert r.n_accepted == Ls and r.first_reject == -1
+            n_rej += int(r.first_reject >= 0)
+            n_all += int(r.first_reject < 0)
+    assert n_all > 0 and (n_rej > 0 or V == 8)
+    e.close()
+
+
+def test_error_paths_return_codes_not_faults():
+    from paper_2603_25702_b200 import Engine, S2D2Error
+    wl = get_config("t_f32")
+    W = generate_weights(wl.model, seed=0)
+    e = Engine(wl.model, block_size=4, max_batch=1, max_seq_len=32, kv_page_tokens=8, n_kv_pages=2,
+               stream=torch.cuda.current_stream().cuda_stream)
+    with pytest.raises(S2D2Error) as ei:                 # weights missing
+        e.prefill([[1, 2, 3]])
+    assert ei.value.code == -7
+    e.load_weights(W)
+    with pytest.raises(S2D2Error):                       # token out of range
+        e.prefill([[1, wl.model.vocab]])
+    with pytest.raises(S2D2Error) as ei:                 # page pool exhausted (2 pages of 8 tokens)
+        e.prefill([list(range(20))])
+    assert ei.value.code == -3
+    e.close()
+    e = _engine(wl, W)
+    sid = e.prefill([[1, 2, 3]])[0]
+    with pytest.raises(S2D2Error) as ei:                 # call order
+        e.verify_block([sid], [1])
+    assert ei.value.code == -4
+    with pytest.raises(S2D2Error):                       # no free slot
+        for _ in range(10):
+            e.prefill([[1, 2, 3]])
+    e.draft_block([sid])
+    with pytest.raises(S2D2Error):
+        e.draft_block([sid])
+    e.close()
