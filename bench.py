@@ -1,0 +1,280 @@
+#!/usr/bin/env python
+"""Benchmark of the S2D2 decode step (draft -> route -> verify -> accept/commit).
+
+One "step" is one pass of the whole hot path over the workload's batch.  The
+metric is committed tokens per second.  ``value`` is device time (CUDA events on
+the library's stream, weights / KV cache / logits resident in HBM); ``e2e`` is the
+wall clock of the same steps through the public C-ABI calls, which take host
+arrays and copy the per-step row tables host->device from pinned memory and the
+statistics / results device->host.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl reference]
+
+N > 1 (under torchrun): independent replicas, one per GPU, no collective on the
+data path ("weak" scaling: every rank decodes its own batch).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from s2d2_inputs import generate_prompts, generate_weights, get_config, weight_shapes  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+        sm, mx, reasons = [], 0.0, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1]))
+                mx = max(mx, float(r[2]))
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_decode_steps(wl, W, n_steps: int, prompt_len: int = 8):
+    """Times the oracle, as it stands, on decode steps of the same model and block size
+    (bounded sample: a short prompt, since an fp64 prefill of the full prompt takes hours)."""
+    from oracle.s2d2 import SequenceOracle
+    rng = np.random.default_rng(0)
+    prompt = rng.integers(0, wl.model.vocab, size=prompt_len).tolist()
+    seq = SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0)
+    seq.prefill(prompt)
+    times, toks = [], []
+    for _ in range(n_steps):
+        t0 = time.perf_counter()
+        st = seq.step()
+        times.append(time.perf_counter() - t0)
+        toks.append(len(st.committed))
+    return times, toks
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle on the host cores of the box."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    W = generate_weights(wl.model, seed=wl.weight_seed)
+    t0 = time.perf_counter()
+    times, toks = oracle_decode_steps(wl, W, 1)                     # first step doubles as the size probe
+    per_step = times[0]
+    budget = 150.0
+    total = args.warmup + args.steps
+    k_eff = args.steps if per_step * total <= budget else max(1, int(budget / per_step) - min(args.warmup, 1))
+    w_eff = args.warmup if k_eff == args.steps else min(args.warmup, 1)
+    times, toks = oracle_decode_steps(wl, W, w_eff + k_eff)
+    t, n = sum(times[w_eff:]), sum(toks[w_eff:])
+    value = n * wl.batch / t          # sequences are independent: a batch is `batch` such runs
+    sample = (f"{k_eff} decode steps (draft+verify+accept, block {wl.block_size}) of one sequence after an 8-token prompt, "
+              f"full model shape; batch-{wl.batch} throughput = {wl.batch} x one sequence")
+    line = {"impl": "reference", "metric": "committed_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": k_eff, "steps_requested": args.steps, "warmup": w_eff, "ms_per_step": 1e3 * t / k_eff,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "model": wl.model.name, "batch": wl.batch, "block_size": wl.block_size},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "wall_s": time.perf_counter() - t0}
+    print(json.dumps(line))
+
+
+def model_pass_bytes(m):
+    """Weight bytes one pass of the network streams (every matrix once, [MASK]/embedding rows excluded)."""
+    es = 2 if m.dtype == "bf16" else 4
+    total = 0
+    for name, shape, kind in weight_shapes(m):
+        if name == "embed" or "experts." in name:
+            continue
+        total += int(np.prod(shape)) * (es if kind == "matrix" else 4)
+    return total
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--workload", default="c4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-steps", type=int, default=6)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = get_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2603_25702_b200 import Engine
+    from paper_2603_25702_b200.build import build
+    build()
+    m, B = wl.model, wl.block_size
+    total_steps = args.warmup + args.steps + args.profile_steps + 2
+    max_seq = wl.prompt_len[1] + total_steps * B + 2 * B
+    t_setup = time.perf_counter()
+    W = generate_weights(m, seed=wl.weight_seed)
+    prompts = generate_prompts(wl, seed=wl.prompt_seed + rank)
+    eng = Engine(m, block_size=B, max_batch=wl.batch, max_seq_len=max_seq, kv_page_tokens=wl.kv_page_tokens,
+                 seed=wl.philox_seed, tau_conf=wl.tau_conf, stream=torch.cuda.current_stream().cuda_stream)
+    eng.load_weights(W)
+    if wl.route == "mean_conf":
+        from paper_2603_25702_b200 import RoutePolicy
+        eng.set_route_policy(RoutePolicy(RoutePolicy.MEAN_CONF, wl.tau_route, 0, 0, 0, 0, 0))
+    ids = eng.prefill(prompts)
+    c0 = eng.get_counters()
+    setup_s = time.perf_counter() - t_setup
+
+    def step():
+        st = eng.draft_block(ids)
+        fl = eng.route(st)
+        eng.verify_block(ids, fl)
+        return eng.accept_and_commit(ids, fl)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    eng.reset_counters()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ev0.record()
+    committed = 0
+    ctx_lens = []
+    for _ in range(args.steps):
+        res = step()
+        committed += sum(r.n_committed for r in res)
+    ev1.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    dev_ms = ev0.elapsed_time(ev1)
+    cnt = eng.get_counters()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([dev_ms, wall], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        n = torch.tensor([committed], device="cuda", dtype=torch.float64)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        dev_ms, wall, committed = float(t[0]), float(t[1]), int(n[0])
+
+    # per-kernel roofline: GEMM launches bracketed by event pairs on the library's stream
+    eng.set_profiling(True)
+    for _ in range(args.profile_steps):
+        step()
+    prof = eng.get_gemm_profile()
+    eng.set_profiling(False)
+    peak, peak_kind = measured_peaks()
+    achieved = prof["bytes"] / (prof["ms"] * 1e-3) / 1e9 if prof["ms"] > 0 else 0.0
+    n_ctx = eng.debug_seq_state(ids[0])["n_cached"]
+
+    pass_bytes = model_pass_bytes(m)
+    verify_ms = cnt.ms_verify / max(1, cnt.n_verify_passes)
+    accept_ms = cnt.ms_accept / max(1, cnt.n_steps // max(1, wl.batch) or 1)
+    steps_done = args.steps
+    accept_ms = cnt.ms_accept / steps_done
+    draft_ms = cnt.ms_draft / max(1, cnt.n_draft_passes)
+    kv_bytes_tok = 2 * m.n_layers * m.n_kv_heads * m.head_dim * (2 if m.dtype == "bf16" else 4)
+    verify_step_bytes = pass_bytes + wl.batch * n_ctx * kv_bytes_tok
+    line = {
+        "metric": "committed_tokens_per_s", "value": committed / (dev_ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dev_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if m.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "model": m.name, "batch": wl.batch, "prompt_len": list(wl.prompt_len),
+                   "block_size": B, "kv_page_tokens": wl.kv_page_tokens, "route": wl.route,
+                   "context_at_end": n_ctx, "l2": "inputs larger than L2 (weights streamed every pass)",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "e2e": {"value": committed / wall, "unit": "tokens/s",
+                "h2d_bytes_per_step": cnt.h2d_bytes / args.steps, "d2h_bytes_per_step": cnt.d2h_bytes / args.steps},
+        "gpu_launches": int(cnt.n_kernel_launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "forward-pass GEMMs (weight streaming)", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "launches": prof["launches"], "avg_launch_us": 1e3 * prof["ms"] / max(1, prof["launches"])},
+        "verify_step": {"verify_us": 1e3 * verify_ms, "accept_us": 1e3 * accept_ms, "draft_us": 1e3 * draft_ms,
+                        "algorithmic_bytes": verify_step_bytes,
+                        "hbm_frac_of_measured": verify_step_bytes / ((verify_ms + accept_ms) * 1e-3) / 1e9 / peak,
+                        "hbm_frac_of_8TBs": verify_step_bytes / ((verify_ms + accept_ms) * 1e-3) / 1e9 / 8000.0},
+        "acceptance": {"mean_accepted_per_verify": cnt.n_accepted_tokens / max(1, cnt.n_verify_passes * wl.batch),
+                       "tokens_per_step": committed / args.steps / world, "resampled": int(cnt.n_resampled),
+                       "near_boundary": int(cnt.n_near_boundary)},
+        "setup_s": setup_s, "prefill_ms": c0.ms_prefill,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        times, toks = oracle_decode_steps(wl, W, 1)
+        line["cpu_baseline"] = {"value": sum(toks) * wl.batch / sum(times), "unit": "tokens/s", "cores": cores,
+                                "kind": "oracle",
+                                "sample": f"1 decode step (draft+verify+accept, block {B}) of one sequence after an 8-token "
+                                          f"prompt on the full model shape, x batch {wl.batch}; {sum(times):.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

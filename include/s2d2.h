@@ -128,6 +128,7 @@ typedef struct {
     double ms_draft, ms_verify, ms_accept, ms_prefill;  /* device time, CUDA events */
     int64_t kv_pages_in_use, kv_pages_total;
     int64_t moe_expert_tiles_touched;                   /* (layer, expert) pairs streamed */
+    int64_t h2d_bytes, d2h_bytes;                       /* host<->device copies made by the calls */
 } s2d2_counters;
 
 typedef struct s2d2_ctx s2d2_ctx;
@@ -210,6 +211,14 @@ int s2d2_get_tokens(s2d2_ctx* ctx, int32_t seq_id, int32_t* out, int32_t cap, in
 int s2d2_release_seq(s2d2_ctx* ctx, int32_t seq_id);
 int s2d2_get_counters(s2d2_ctx* ctx, s2d2_counters* out);
 int s2d2_reset_counters(s2d2_ctx* ctx);
+
+/* Kernel-level timing for roofline reports: while on, every GEMM launch of the
+ * forward pass is bracketed by a CUDA event pair on the context's stream.
+ * s2d2_get_gemm_profile synchronises and returns the launches, their summed
+ * device time and their summed algorithmic bytes (weight matrix read once +
+ * activations read + output written) since profiling was switched on. */
+int s2d2_set_profiling(s2d2_ctx* ctx, int32_t on);
+int s2d2_get_gemm_profile(s2d2_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_bytes);
 
 /* Stand-alone entry to the fused acceptance kernel on caller-supplied device
  * logits (Algorithm "SampleBlock for S2D2", ScoreFromLogits and the scan).

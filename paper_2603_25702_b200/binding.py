@@ -62,7 +62,7 @@ class Counters(C.Structure):
                                          "n_kernel_launches")] + \
                [("accepted_len_hist", C.c_int64 * (MAX_BLOCK + 1))] + \
                [(n, C.c_double) for n in ("ms_draft", "ms_verify", "ms_accept", "ms_prefill")] + \
-               [(n, C.c_int64) for n in ("kv_pages_in_use", "kv_pages_total", "moe_expert_tiles_touched")]
+               [(n, C.c_int64) for n in ("kv_pages_in_use", "kv_pages_total", "moe_expert_tiles_touched", "h2d_bytes", "d2h_bytes")]
 
 
 class RoutePolicy(C.Structure):
@@ -77,7 +77,7 @@ EXPORTS = [
     "s2d2_create", "s2d2_destroy", "s2d2_last_error", "s2d2_load_weights", "s2d2_prefill",
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
-    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_accept_logits", "s2d2_debug_copy_logits",
+    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
     "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_copy_expert_ids",
 ]
 
@@ -117,6 +117,8 @@ def load_library() -> C.CDLL:
     lib.s2d2_release_seq.argtypes = [C.c_void_p, C.c_int32]
     lib.s2d2_get_counters.argtypes = [C.c_void_p, C.POINTER(Counters)]
     lib.s2d2_reset_counters.argtypes = [C.c_void_p]
+    lib.s2d2_set_profiling.argtypes = [C.c_void_p, C.c_int32]
+    lib.s2d2_get_gemm_profile.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.s2d2_accept_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
                                        C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_uint32),
                                        C.POINTER(C.c_int32), C.POINTER(StepResult)]
@@ -265,6 +267,14 @@ class Engine:
 
     def reset_counters(self):
         self._check(self.lib.s2d2_reset_counters(self._h))
+
+    def set_profiling(self, on: bool):
+        self._check(self.lib.s2d2_set_profiling(self._h, int(on)))
+
+    def get_gemm_profile(self):
+        n, ms, b = C.c_int64(), C.c_double(), C.c_double()
+        self._check(self.lib.s2d2_get_gemm_profile(self._h, C.byref(n), C.byref(ms), C.byref(b)))
+        return {"launches": n.value, "ms": ms.value, "bytes": b.value}
 
     def accept_logits(self, d_draft_logits: int, d_verify_logits: int, n_seqs: int, l_max: int, span_len, xhat,
                       position0, rng_stream, step):

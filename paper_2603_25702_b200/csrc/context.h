@@ -121,4 +121,11 @@ struct s2d2_ctx {
     s2d2_counters cnt;
     cudaEvent_t ev[8];
     bool verify_timing_pending = false;
+    // per-GEMM profiling (off by default)
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_events;   // pairs
+    size_t prof_used = 0;
+    double prof_bytes = 0, prof_ms_done = 0;
+    int64_t prof_launches = 0;
+    void* gemm_state = nullptr;             // owned by gemm.cu
 };

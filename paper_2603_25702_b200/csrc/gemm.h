@@ -5,3 +5,7 @@ struct s2d2_ctx;
 int gemm_init(s2d2_ctx* c);
 void gemm_destroy(s2d2_ctx* c);
 int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate);
+// Profiling helpers: bracket a launch with an event pair while profiling is on.
+void gemm_prof_begin(s2d2_ctx* c);
+void gemm_prof_end(s2d2_ctx* c, double algorithmic_bytes);
+int gemm_prof_collect(s2d2_ctx* c);   // synchronises, folds finished pairs into the totals

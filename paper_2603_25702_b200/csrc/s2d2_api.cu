@@ -451,6 +451,7 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
     if (M == 0) return S2D2_OK;
     int nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, nq = m.n_q_heads * hd;
     CUDA_TRY(c, cudaMemcpyAsync(c->meta.d, c->meta.h, c->meta.bytes, cudaMemcpyHostToDevice, st));
+    c->cnt.h2d_bytes += c->meta.bytes;
     embed_kernel<TW><<<M, 256, 0, st>>>((const TW*)c->embed, pv.row_token, c->h, d);
     LAUNCHED(c);
     KvPool<TKV> pool = make_pool<TKV>(c);
@@ -657,6 +658,7 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     CUDA_TRY(c, cudaMemcpyAsync(hc, c->d_conf, R * 4, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(hm, c->d_margin, R * 4, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(he, c->d_entropy, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    c->cnt.d2h_bytes += R * 16;
     CUDA_TRY(c, cudaEventRecord(c->ev[1], c->stream));
     CUDA_TRY(c, cudaEventSynchronize(c->ev[1]));
     float ms = 0;
@@ -810,6 +812,8 @@ struct AccStage {     // layout of acc_h / acc_d for S sequences
 int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, const float* d_verify, const int* d_xhat,
                   const double* d_lse, const float* d_conf) {
     CUDA_TRY(c, cudaMemcpyAsync(c->acc_d, c->acc_h, a.in_bytes, cudaMemcpyHostToDevice, c->stream));
+    c->cnt.h2d_bytes += a.in_bytes;
+    c->cnt.d2h_bytes += a.total - a.in_bytes;
     AcceptIn in;
     in.draft_logits = d_draft;
     in.verify_logits = d_verify;
@@ -1053,6 +1057,27 @@ extern "C" int s2d2_get_counters(s2d2_ctx* c, s2d2_counters* out) {
 extern "C" int s2d2_reset_counters(s2d2_ctx* c) {
     if (!c) return S2D2_ERR_INVALID;
     memset(&c->cnt, 0, sizeof(c->cnt));
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_set_profiling(s2d2_ctx* c, int32_t on) {
+    if (!c) return S2D2_ERR_INVALID;
+    int rc = gemm_prof_collect(c);
+    if (rc) return rc;
+    if (on && !c->profiling) {
+        c->prof_bytes = c->prof_ms_done = 0;
+        c->prof_launches = 0;
+    }
+    c->profiling = on != 0;
+    return S2D2_OK;
+}
+extern "C" int s2d2_get_gemm_profile(s2d2_ctx* c, int64_t* n, double* ms, double* bytes) {
+    if (!c || !n || !ms || !bytes) return S2D2_ERR_INVALID;
+    int rc = gemm_prof_collect(c);
+    if (rc) return rc;
+    *n = c->prof_launches;
+    *ms = c->prof_ms_done;
+    *bytes = c->prof_bytes;
     return S2D2_OK;
 }
 

@@ -31,7 +31,7 @@ def test_struct_sizes_match_header():
     assert ctypes.sizeof(b.DecodeConfigC) == 11 * 4
     assert ctypes.sizeof(b.DraftStats) == 7 * 4 + 5 * 32 * 4
     assert ctypes.sizeof(b.StepResult) == 8 * 4 + 5 * 32 * 4
-    assert ctypes.sizeof(b.Counters) == 9 * 8 + 33 * 8 + 4 * 8 + 3 * 8
+    assert ctypes.sizeof(b.Counters) == 9 * 8 + 33 * 8 + 4 * 8 + 5 * 8
     assert ctypes.sizeof(b.RoutePolicy) == 7 * 4
 
 
