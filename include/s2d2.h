@@ -242,6 +242,11 @@ int s2d2_debug_copy_kv(s2d2_ctx* ctx, int32_t seq_id, int32_t layer, int32_t n_t
 /* Cache length (tokens whose K/V is committed) and open-block state. */
 int s2d2_debug_seq_state(s2d2_ctx* ctx, int32_t seq_id, int32_t* n_cached, int32_t* block_start,
                          int32_t* block_tokens /* [B], vocab = MASK, may be NULL */, int32_t* step_index);
+/* One GEMM of the forward pass on host data (test tap): y[M,N] = x[M,K] w[N,K]^T with
+ * x and w in the model's storage type (bf16 bit patterns or fp32), y fp32. Uses the
+ * same kernel selection as the forward pass. Allocates temporaries. */
+int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int32_t N, int32_t K, float* y);
+
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);
 

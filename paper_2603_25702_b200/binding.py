@@ -78,7 +78,7 @@ EXPORTS = [
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
     "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
-    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_copy_expert_ids",
+    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids",
 ]
 
 
@@ -125,6 +125,7 @@ def load_library() -> C.CDLL:
     lib.s2d2_debug_copy_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
     lib.s2d2_debug_copy_kv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.s2d2_debug_seq_state.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.s2d2_debug_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.s2d2_debug_copy_expert_ids.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int64, C.POINTER(C.c_int32)]
     _LIB = lib
     return lib
@@ -307,6 +308,15 @@ class Engine:
         self._check(self.lib.s2d2_debug_seq_state(self._h, seq_id, C.byref(nc), C.byref(bs),
                                                   blk.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(st)))
         return {"n_cached": nc.value, "block_start": bs.value, "block_tokens": blk.tolist(), "step": st.value}
+
+    def debug_gemm(self, x: np.ndarray, w: np.ndarray) -> np.ndarray:
+        """x [M, K], w [N, K] in the model's storage type (uint16 = bf16 bits, or float32)."""
+        x, w = np.ascontiguousarray(x), np.ascontiguousarray(w)
+        M, K = x.shape
+        N = w.shape[0]
+        y = np.empty((M, N), dtype=np.float32)
+        self._check(self.lib.s2d2_debug_gemm(self._h, x.ctypes.data, w.ctypes.data, M, N, K, y.ctypes.data))
+        return y
 
     def debug_copy_expert_ids(self, max_rows: int) -> np.ndarray:
         k, nl = self.model.top_k, self.model.n_layers

@@ -1,24 +1,172 @@
-// GEMM dispatch of the forward pass.
+// GEMM dispatch of the forward pass: bf16 models go to the tcgen05 weight-streaming
+// kernel (gemm_tc.cuh); the fp32 model, shapes the tensor-core kernel does not take
+// (K not a multiple of 64) and contexts created with use_tensor_cores = 0 go to the
+// SIMT kernel.
 #include "gemm.h"
 
+#include <cuda.h>
+
+#include <map>
+#include <tuple>
+
 #include "context.h"
+#include "gemm_tc.cuh"
 #include "kernels_simt.cuh"
 
 using namespace s2d2;
 
-int gemm_init(s2d2_ctx*) { return S2D2_OK; }
-void gemm_destroy(s2d2_ctx* c) {
-    for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
-    c->prof_events.clear();
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct GemmState {
+    EncodeTiledFn encode = nullptr;
+    bool tc_ok = false;
+    int n_sms = 148;
+    float* ws = nullptr;
+    size_t ws_floats = 0;
+    unsigned* tickets = nullptr;
+    size_t n_tickets = 0;
+    int max_smem = 0;
+    std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;   // (ptr, rows, K, box_rows)
+};
+
+GemmState* state(s2d2_ctx* c) { return (GemmState*)c->gemm_state; }
+
+// Tensor map of a row-major bf16 matrix [rows, K]: boxes of box_rows x 64 elements, 128-byte swizzle,
+// zero fill outside the matrix.
+const CUtensorMap* get_map(s2d2_ctx* c, const void* ptr, int rows, int K, int box_rows) {
+    GemmState* g = state(c);
+    auto key = std::make_tuple(ptr, rows, K, box_rows);
+    auto it = g->maps.find(key);
+    if (it != g->maps.end()) return &it->second;
+    CUtensorMap m;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)tc::BLOCK_K, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        c->err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+        return nullptr;
+    }
+    return &(g->maps[key] = m);
 }
 
 template <typename TW, typename TX>
-static void gemm_simt(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
-                      int accumulate) {
+void gemm_simt(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
+               int accumulate) {
     constexpr int ROWS = 8;
     dim3 grid((N + 3) / 4, (M + ROWS - 1) / ROWS);
     gemm_simt_kernel<TW, TX, ROWS><<<grid, 128, 0, c->stream>>>((const TX*)X, (const TW*)W, Y, M, N, K, ldy, scale, accumulate);
     c->cnt.n_kernel_launches++;
+}
+
+int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
+            int accumulate) {
+    GemmState* g = state(c);
+    tc::GemmParams p;
+    p.Y = Y;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.ldy = ldy;
+    p.scale = scale;
+    p.accumulate = accumulate;
+    p.kb_total = K / tc::BLOCK_K;
+    p.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
+    p.m_tiles = (M + 255) / 256;
+    int per = (M + p.m_tiles - 1) / p.m_tiles;
+    p.T = std::min(256, (per + 15) / 16 * 16);
+    p.m_tiles = (M + p.T - 1) / p.T;
+    // two CTAs per SM while the token tile is small, one otherwise
+    bool two = p.T <= 64;
+    size_t budget = two ? 100 * 1024 : 200 * 1024;
+    p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(p.T));
+    p.stages = std::max(2, std::min(p.stages, p.kb_total));
+    // K splits: fill the resident CTA slots; cost model in K-blocks per CTA plus a fixed set-up cost
+    int slots = g->n_sms * (two ? 2 : 1);
+    int tiles = p.n_tiles * p.m_tiles;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= 16 && s <= p.kb_total / 2 + (p.kb_total < 2 ? 1 : 0); ++s) {
+        if ((size_t)tiles * s * p.T * tc::BLOCK_N > g->ws_floats && s > 1) break;
+        if ((size_t)tiles > g->n_tickets && s > 1) break;
+        int waves = (tiles * s + slots - 1) / slots;
+        double cost = waves * ((double)(p.kb_total + s - 1) / s + 6.0) + (s > 1 ? 2.0 : 0.0);
+        if (cost < best_cost - 1e-9) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    p.splits = best;
+    p.ws = g->ws;
+    p.tickets = g->tickets;
+    p.status = c->d_status;
+    p.evict_first = (M <= 64);
+    const CUtensorMap* mw = get_map(c, W, N, K, tc::BLOCK_N);
+    const CUtensorMap* mx = get_map(c, X, M, K, p.T);
+    if (!mw || !mx) return S2D2_ERR_CUDA;
+    size_t smem = tc::smem_bytes(p.T, p.stages);
+    int grid = tiles * p.splits;
+    tc::gemm_tc_kernel<<<grid, tc::THREADS, smem, c->stream>>>(*mw, *mx, p);
+    c->cnt.n_kernel_launches++;
+    return S2D2_OK;
+}
+
+}  // namespace
+
+int gemm_init(s2d2_ctx* c) {
+    GemmState* g = new GemmState();
+    c->gemm_state = g;
+    if (c->m.dtype != S2D2_DTYPE_BF16 || !c->dc.use_tensor_cores) return S2D2_OK;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return S2D2_ERR_CUDA;
+    g->n_sms = prop.multiProcessorCount;
+    if (prop.major != 10) {
+        c->err = "the tensor-core kernels are built for sm_100a only";
+        return S2D2_ERR_UNSUPPORTED;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) {
+        c->err = "cuTensorMapEncodeTiled not available";
+        return S2D2_ERR_CUDA;
+    }
+    g->encode = (EncodeTiledFn)fn;
+    g->ws_floats = (size_t)16 << 20;          // 64 MiB of split-K partial tiles
+    g->n_tickets = 1 << 16;
+    if (cudaMalloc((void**)&g->ws, g->ws_floats * 4) != cudaSuccess) return S2D2_ERR_CUDA;
+    if (cudaMalloc((void**)&g->tickets, g->n_tickets * 4) != cudaSuccess) return S2D2_ERR_CUDA;
+    if (cudaMemset(g->tickets, 0, g->n_tickets * 4) != cudaSuccess) return S2D2_ERR_CUDA;
+    if (cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
+        c->err = "cannot raise the dynamic shared memory limit";
+        return S2D2_ERR_CUDA;
+    }
+    g->tc_ok = true;
+    return S2D2_OK;
+}
+
+void gemm_destroy(s2d2_ctx* c) {
+    for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
+    c->prof_events.clear();
+    GemmState* g = state(c);
+    if (!g) return;
+    if (g->ws) cudaFree(g->ws);
+    if (g->tickets) cudaFree(g->tickets);
+    delete g;
+    c->gemm_state = nullptr;
+}
+
+void gemm_forget(s2d2_ctx* c, const void* ptr) {
+    GemmState* g = state(c);
+    if (!g) return;
+    for (auto it = g->maps.begin(); it != g->maps.end();)
+        it = (std::get<0>(it->first) == ptr) ? g->maps.erase(it) : std::next(it);
 }
 
 void gemm_prof_begin(s2d2_ctx* c) {
@@ -58,7 +206,11 @@ int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int 
         double b;
         ~End() { gemm_prof_end(c, b); }
     } end{c, (double)N * K * es + (double)M * K * es + (double)M * N * 4 * (accumulate ? 2 : 1)};
-    if (c->m.dtype == S2D2_DTYPE_F32) gemm_simt<float, float>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
-    else gemm_simt<bf16, bf16>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
+    if (c->m.dtype == S2D2_DTYPE_F32) {
+        gemm_simt<float, float>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
+        return S2D2_OK;
+    }
+    if (state(c)->tc_ok && K % tc::BLOCK_K == 0) return gemm_tc(c, X, W, Y, M, N, K, ldy, scale, accumulate);
+    gemm_simt<bf16, bf16>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
     return S2D2_OK;
 }

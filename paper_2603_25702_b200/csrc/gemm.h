@@ -9,3 +9,5 @@ int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int 
 void gemm_prof_begin(s2d2_ctx* c);
 void gemm_prof_end(s2d2_ctx* c, double algorithmic_bytes);
 int gemm_prof_collect(s2d2_ctx* c);   // synchronises, folds finished pairs into the totals
+// Drops cached tensor maps of a buffer that is about to be freed.
+void gemm_forget(s2d2_ctx* c, const void* ptr);

@@ -1,0 +1,322 @@
+// Skinny weight-streaming GEMM on the 5th-generation tensor cores (sm_100a).
+//
+//   Y[m, n] (+)= scale * sum_k X[m, k] * W[n, k]      X bf16 [M, K], W bf16 [N, K], Y fp32
+//
+// The decode step multiplies a few token rows (M = block x batch, 4..512) by every
+// weight matrix of the network, so the weights are the stream and the tokens are
+// the small operand.  The roles are therefore swapped with respect to a square
+// GEMM: a tile of 128 weight rows is the MMA "M" operand (A, K-major, staged by
+// TMA with the 128-byte swizzle), the token rows are the MMA "N" operand
+// (B, K-major, T = 16..256 rows), and the fp32 accumulator D[128 x T] lives in
+// tensor memory.  One CTA owns one (weight tile, token tile, K split):
+//   warp 0 / lane 0   TMA producer: W and X K-blocks of 64 into a ring of stages
+//   warp 1 / lane 0   tcgen05.mma issuer, 4 MMAs (K = 16 each) per stage;
+//                     tcgen05.commit frees the stage and finally signals the epilogue
+//   warps 0..3        epilogue: tcgen05.ld of the 128 accumulator lanes, then either
+//                     the final store or, with split K, a partial tile to a workspace;
+//                     the last CTA to arrive for a tile (ticket counter) sums the
+//                     partials in split order, so the result does not depend on timing.
+// Two CTAs fit on one SM, so one CTA's set-up and epilogue overlap the other's stream.
+// Every wait on an mbarrier is bounded; on time-out the kernel raises a status word
+// that the host turns into S2D2_ERR_TIMEOUT, drains its copies and frees its TMEM.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace s2d2 {
+namespace tc {
+
+constexpr int BLOCK_N = 128;   // weight rows per tile (MMA M)
+constexpr int BLOCK_K = 64;    // bf16 elements per K-block = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int THREADS = 128;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;   // polls of try_wait before giving up
+
+struct GemmParams {
+    float* Y;
+    int M, N, K;
+    int ldy;
+    float scale;
+    int accumulate;      // Y += result
+    int T;               // token rows per tile (multiple of 16, <= 256)
+    int stages;
+    int splits;          // K splits per tile
+    int kb_total;        // K / 64
+    int n_tiles, m_tiles;
+    float* ws;           // split-K partial tiles [(tile * splits + split)][T][128]
+    unsigned* tickets;   // one counter per (n_tile, m_tile), zero between launches
+    int* status;         // device status word (0 = ok)
+    int evict_first;     // stream W with an evict-first L2 policy
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false on time-out or when another
+// role of the CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag = nullptr) {
+    uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (abort_flag && (it & 1023u) == 1023u && *abort_flag) return false;
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], "
+        "[%4], %5;" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive fp32 columns of this warp's 32 accumulator lanes.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
+// (64 bf16) written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);         // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                              // leading byte offset (ignored), bits [16,30)
+    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                              // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                              // layout: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = T.
+__host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int T) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T >> 3) << 17) | ((uint32_t)(BLOCK_N >> 4) << 24);
+}
+
+__host__ __device__ __forceinline__ size_t stage_bytes(int T) { return (size_t)BLOCK_N * 128 + (size_t)T * 128; }
+__host__ __device__ __forceinline__ size_t smem_bytes(int T, int stages) { return stages * stage_bytes(T) + 1024 + 256; }
+
+__global__ void __launch_bounds__(THREADS)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // tiles need 1024-byte alignment for the 128-byte swizzle
+    uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int S = p.stages, T = p.T;
+    const size_t sbytes = stage_bytes(T);
+    uint64_t* full = (uint64_t*)(tiles + S * sbytes);
+    uint64_t* empty = full + S;
+    uint64_t* acc_ready = empty + S;
+    uint32_t* tmem_slot = (uint32_t*)(acc_ready + 1);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    volatile int* issued = abort_flag + 1;
+    volatile int* consumed = issued + 1;
+    int* last_flag = (int*)(consumed + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // work item: blockIdx.x -> (n_tile, m_tile, split); the token tile varies fastest so that CTAs
+    // sharing a weight tile run together and the tile is fetched from DRAM once
+    int item = blockIdx.x;
+    const int m_tile = item % p.m_tiles;
+    item /= p.m_tiles;
+    const int split = item % p.splits;
+    const int n_tile = item / p.splits;
+    const int kb0 = (int)((long long)p.kb_total * split / p.splits);
+    const int kb1 = (int)((long long)p.kb_total * (split + 1) / p.splits);
+    const int n0 = n_tile * BLOCK_N, m0 = m_tile * T;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < T) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_ready, 1);
+        *abort_flag = 0;
+        *issued = 0;
+        *consumed = 0;
+        *last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+    }
+    if (warp == 0) {
+        tmem_alloc(tmem_slot, tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer ----------------
+        uint64_t policy = 0;
+        if (p.evict_first) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        for (int kb = kb0; kb < kb1; ++kb) {
+            int i = kb - kb0, s = i % S;
+            if (i >= S && !mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
+                *abort_flag = 1;
+                break;
+            }
+            if (*abort_flag) break;
+            uint8_t* a = tiles + s * sbytes;
+            uint8_t* b = a + BLOCK_N * 128;
+            mbar_expect_tx(&full[s], (uint32_t)sbytes);
+            if (p.evict_first) tma_load_2d_hint(a, &map_w, kb * BLOCK_K, n0, &full[s], policy);
+            else tma_load_2d(a, &map_w, kb * BLOCK_K, n0, &full[s]);
+            tma_load_2d(b, &map_x, kb * BLOCK_K, m0, &full[s]);
+            *issued = i + 1;
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer ----------------
+        const uint32_t idesc = instr_desc_bf16(T);
+        int i = 0;
+        for (int kb = kb0; kb < kb1; ++kb, ++i) {
+            int s = i % S;
+            if (!mbar_wait(&full[s], (i / S) & 1, abort_flag)) {
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
+            uint32_t a_addr = smem_u32(tiles + s * sbytes);
+            uint32_t b_addr = a_addr + BLOCK_N * 128;
+            uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                // stepping 16 elements (32 bytes) along K inside the swizzled row: +2 in the address field
+                umma_bf16(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&empty[s]);   // arrives when the MMAs that read this stage are done
+            *consumed = i + 1;
+        }
+        umma_commit(acc_ready);       // arrives when every MMA issued above is done
+    }
+    __syncwarp();
+    // ---------------- epilogue: all four warps ----------------
+    bool ok = mbar_wait(acc_ready, 0);
+    if (!ok) *abort_flag = 1;
+    tc_fence_after();
+    __syncthreads();
+    const bool aborted = *abort_flag != 0;
+    if (aborted) {
+        if (threadIdx.x == 0) {
+            atomicExch(p.status, 1);
+            // both roles have stopped: wait (bounded) for copies already issued into this CTA's
+            // shared memory before the CTA may exit
+            for (int i = *consumed; i < *issued; ++i) mbar_wait(&full[i % S], (i / S) & 1);
+        }
+    } else {
+        const int n_local = warp * 32 + lane;
+        const int n = n0 + n_local;
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const int m_hi = min(T, p.M - m0);
+        if (p.splits == 1) {
+            for (int c = 0; c < T; c += 16) {
+                float v[16];
+                tmem_ld16(taddr + c, v);      // executed by the whole warp even past m_hi (aligned instruction)
+                if (n < p.N) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        int m = c + j;
+                        if (m < m_hi) {
+                            float* y = p.Y + (size_t)(m0 + m) * p.ldy + n;
+                            *y = p.accumulate ? (*y + p.scale * v[j]) : p.scale * v[j];
+                        }
+                    }
+                }
+            }
+        } else {
+            const int tile = n_tile * p.m_tiles + m_tile;
+            float* mine = p.ws + ((size_t)tile * p.splits + split) * (size_t)T * BLOCK_N;
+            for (int c = 0; c < T; c += 16) {
+                float v[16];
+                tmem_ld16(taddr + c, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (c + j < m_hi) mine[(size_t)(c + j) * BLOCK_N + n_local] = v[j];
+            }
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned t = atomicAdd(&p.tickets[tile], 1u);
+                *last_flag = (t == (unsigned)p.splits - 1);
+            }
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                const float* base = p.ws + (size_t)tile * p.splits * (size_t)T * BLOCK_N;
+                if (n < p.N) {
+                    for (int m = 0; m < m_hi; ++m) {
+                        float acc = 0.f;
+                        for (int s = 0; s < p.splits; ++s) acc += __ldcg(base + ((size_t)s * T + m) * BLOCK_N + n_local);
+                        float* y = p.Y + (size_t)(m0 + m) * p.ldy + n;
+                        *y = p.accumulate ? (*y + p.scale * acc) : p.scale * acc;
+                    }
+                }
+                if (threadIdx.x == 0) p.tickets[tile] = 0;   // ready for the next launch
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+}
+
+}  // namespace tc
+}  // namespace s2d2

@@ -297,6 +297,10 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
         CUDA_TRY(c, cudaMalloc((void**)&c->acc_d, c->acc_bytes));
     }
     for (int i = 0; i < 8; ++i) CUDA_TRY(c, cudaEventCreate(&c->ev[i]));
+    CUDA_TRY(c, cudaMalloc((void**)&c->d_status, 4));
+    CUDA_TRY(c, cudaMemset(c->d_status, 0, 4));
+    CUDA_TRY(c, cudaMallocHost((void**)&c->h_status, 4));
+    *c->h_status = 0;
     int grc = gemm_init(c);
     if (grc != S2D2_OK) return grc;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
@@ -310,12 +314,13 @@ extern "C" int s2d2_destroy(s2d2_ctx* c) {
     void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
                     c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
-                    c->d_margin, c->d_entropy, c->d_lse, c->acc_d};
+                    c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->meta.h) cudaFreeHost(c->meta.h);
     if (c->stats_h) cudaFreeHost(c->stats_h);
     if (c->acc_h) cudaFreeHost(c->acc_h);
+    if (c->h_status) cudaFreeHost(c->h_status);
     for (int i = 0; i < 8; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
@@ -338,6 +343,18 @@ extern "C" int s2d2_load_weights(s2d2_ctx* c, const s2d2_tensor_desc* t, int32_t
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     c->weights_checked = false;
     return S2D2_OK;
+}
+
+// The device status word travels back with the results of every synchronous call.
+static int enqueue_status_read(s2d2_ctx* c) {
+    CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, 4, cudaMemcpyDeviceToHost, c->stream));
+    return S2D2_OK;
+}
+static int check_status(s2d2_ctx* c) {
+    if (*c->h_status == 0) return S2D2_OK;
+    *c->h_status = 0;
+    cudaMemsetAsync(c->d_status, 0, 4, c->stream);
+    FAIL(c, S2D2_ERR_TIMEOUT, "a kernel gave up on a bounded wait (results of this call are invalid)");
 }
 
 static int check_weights(s2d2_ctx* c) {
@@ -584,8 +601,10 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
             s.n_c = std::min(s.n_final, s.n_c + CH);
         }
     }
+    if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[7], c->stream));
     CUDA_TRY(c, cudaEventSynchronize(c->ev[7]));
+    if ((rc = check_status(c))) return rc;
     float ms = 0;
     cudaEventElapsedTime(&ms, c->ev[6], c->ev[7]);
     c->cnt.ms_prefill += ms;
@@ -659,8 +678,10 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     CUDA_TRY(c, cudaMemcpyAsync(hm, c->d_margin, R * 4, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaMemcpyAsync(he, c->d_entropy, R * 4, cudaMemcpyDeviceToHost, c->stream));
     c->cnt.d2h_bytes += R * 16;
+    if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[1], c->stream));
     CUDA_TRY(c, cudaEventSynchronize(c->ev[1]));
+    if ((rc = check_status(c))) return rc;
     float ms = 0;
     cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]);
     c->cnt.ms_draft += ms;
@@ -876,8 +897,10 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
     CUDA_TRY(c, cudaEventRecord(c->ev[4], c->stream));
     int rc = launch_accept(c, a, n, c->logits_draft, c->logits_verify, c->d_xhat, c->d_lse, c->d_conf);
     if (rc) return rc;
+    if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[5], c->stream));
     CUDA_TRY(c, cudaEventSynchronize(c->ev[5]));
+    if ((rc = check_status(c))) return rc;
     float ms = 0;
     cudaEventElapsedTime(&ms, c->ev[4], c->ev[5]);
     c->cnt.ms_accept += ms;
@@ -1129,6 +1152,31 @@ extern "C" int s2d2_debug_seq_state(s2d2_ctx* c, int32_t id, int32_t* n_cached, 
         for (int k = 0; k < c->dc.block_size; ++k)
             block_tokens[k] = s->block_open ? s->tok[s->n_final + k] : c->m.vocab;
     return S2D2_OK;
+}
+
+extern "C" int s2d2_debug_gemm(s2d2_ctx* c, const void* x, const void* w, int32_t M, int32_t N, int32_t K, float* y) {
+    if (!c || !x || !w || !y || M < 1 || N < 1 || K < 1) return S2D2_ERR_INVALID;
+    size_t es = esize(c->m.dtype);
+    void *dx = nullptr, *dw = nullptr;
+    float* dy = nullptr;
+    CUDA_TRY(c, cudaMalloc(&dx, (size_t)M * K * es));
+    CUDA_TRY(c, cudaMalloc(&dw, (size_t)N * K * es));
+    CUDA_TRY(c, cudaMalloc((void**)&dy, (size_t)M * N * 4));
+    CUDA_TRY(c, cudaMemcpyAsync(dx, x, (size_t)M * K * es, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(dw, w, (size_t)N * K * es, cudaMemcpyHostToDevice, c->stream));
+    int rc = gemm(c, dx, dw, dy, M, N, K, N, 1.f, 0);
+    if (!rc) rc = enqueue_status_read(c);
+    if (!rc) {
+        CUDA_TRY(c, cudaMemcpyAsync(y, dy, (size_t)M * N * 4, cudaMemcpyDeviceToHost, c->stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        rc = check_status(c);
+    }
+    gemm_forget(c, dx);
+    gemm_forget(c, dw);
+    cudaFree(dx);
+    cudaFree(dw);
+    cudaFree(dy);
+    return rc;
 }
 
 extern "C" int s2d2_debug_copy_expert_ids(s2d2_ctx* c, int32_t* out, int64_t cap, int32_t* n_rows) {

@@ -1,0 +1,36 @@
+"""The tensor-core weight-streaming GEMM against a float64 matmul of the same bf16 inputs."""
+import numpy as np
+import pytest
+
+from s2d2_inputs import bf16_bits_to_f32, f32_to_bf16_bits, get_config
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def engine():
+    from paper_2603_25702_b200 import Engine
+    wl = get_config("t_bf16")
+    e = Engine(wl.model, block_size=4, max_batch=1, max_seq_len=64, kv_page_tokens=16,
+               stream=torch.cuda.current_stream().cuda_stream)
+    yield e
+    e.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 128, 64), (4, 256, 256), (8, 384, 128), (16, 128, 4096), (16, 6144, 4096),
+                                   (5, 200, 192), (33, 1000, 512), (64, 4096, 1024), (100, 640, 2048), (257, 300, 320),
+                                   (512, 1024, 512), (16, 151936, 256), (3, 64, 704)])
+def test_gemm_matches_float64(engine, M, N, K):
+    rng = np.random.default_rng(M * 1000003 + N * 101 + K)
+    x = f32_to_bf16_bits(rng.standard_normal((M, K)).astype(np.float32))
+    w = f32_to_bf16_bits((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
+    got = engine.debug_gemm(x, w)
+    want = bf16_bits_to_f32(x).astype(np.float64) @ bf16_bits_to_f32(w).astype(np.float64).T
+    err = np.abs(got - want).max()
+    # fp32 accumulation of exact bf16 products: error ~ K * eps_fp32 * |terms|
+    bound = 2e-6 * np.sqrt(K) * np.abs(want).max() + 1e-6
+    assert err <= bound, (err, bound)
+    # twice the same launch: bitwise identical (split-K partials are summed in a fixed order)
+    again = engine.debug_gemm(x, w)
+    assert np.array_equal(got, again)
