@@ -250,6 +250,32 @@ int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int3
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);
 
+/* y[M, N] = x[M, K] w[N, K]^T on device buffers, without any allocation.
+ * (The paper has no counterpart: this is a service entry for hosts that must not
+ * allocate.)  Some callers cannot call cudaMalloc: a serving process whose framework
+ * has already reserved the whole GPU for its own arena, so that any further driver
+ * allocation fails or fragments it, and latency-critical loops, because cudaMalloc
+ * and cudaFree synchronise the device and stall every stream.  This variant of the
+ * tensor-core split-K GEMM keeps its scratch (partial tiles, ticket counters, status
+ * word) in a fixed region that is part of the library image: S2D2_NOALLOC_WS_BYTES +
+ * 16 KiB of device memory, held by every GPU that loads the library until exit.
+ *   d_x  bf16 [M, K], d_w  bf16 [N, K], d_y  fp32 [M, N]: device pointers, row-major,
+ *   16-byte aligned, owned by the caller.  1 <= M <= 256, 1 <= N <= 1048576,
+ *   K a multiple of 64 with 64 <= K <= 65536; anything else returns S2D2_ERR_INVALID
+ *   (text from s2d2_noalloc_last_error()).  The K split is lowered until the partial
+ *   tiles fit the fixed scratch, so every shape inside these limits runs.
+ * The call is synchronous on `cuda_stream` (it reads back the status word) and calls
+ * no cudaMalloc, cudaFree or allocating library routine.  The first call on a device
+ * looks up the address of the scratch region and raises the kernel's shared-memory
+ * limit; make that first call before any stream capture begins.  All calls on a
+ * device share the one scratch region, which keeps the previous call's contents (the
+ * counters are cleared at the start of every call): two calls that overlap on the
+ * GPU, from different streams or threads, race and give wrong results. */
+#define S2D2_NOALLOC_WS_BYTES (8u << 20)
+int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d_y, int32_t M, int32_t N, int32_t K,
+                           void* cuda_stream);
+const char* s2d2_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

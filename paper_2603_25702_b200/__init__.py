@@ -7,6 +7,7 @@ from .binding import (  # noqa: F401
     RoutePolicy,
     S2D2Error,
     StepResult,
+    gemm_bf16_noalloc,
     library_path,
     load_library,
 )

@@ -79,6 +79,7 @@ EXPORTS = [
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
     "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
     "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids",
+    "s2d2_gemm_bf16_noalloc", "s2d2_noalloc_last_error",
 ]
 
 
@@ -97,10 +98,13 @@ def load_library() -> C.CDLL:
     lib = C.CDLL(path)
     lib.s2d2_last_error.restype = C.c_char_p
     lib.s2d2_last_error.argtypes = [C.c_void_p]
+    lib.s2d2_noalloc_last_error.restype = C.c_char_p
+    lib.s2d2_noalloc_last_error.argtypes = []
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name != "s2d2_last_error":
+        if name not in ("s2d2_last_error", "s2d2_noalloc_last_error"):
             fn.restype = C.c_int
+    lib.s2d2_gemm_bf16_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.s2d2_create.argtypes = [C.POINTER(ModelConfigC), C.POINTER(DecodeConfigC), C.c_void_p, C.POINTER(C.c_void_p)]
     lib.s2d2_destroy.argtypes = [C.c_void_p]
     lib.s2d2_load_weights.argtypes = [C.c_void_p, C.POINTER(TensorDesc), C.c_int32]
@@ -134,6 +138,17 @@ def load_library() -> C.CDLL:
 def _i32(a: Sequence[int]):
     arr = np.ascontiguousarray(a, dtype=np.int32)
     return arr, arr.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def gemm_bf16_noalloc(d_x: int, d_w: int, d_y: int, M: int, N: int, K: int, stream: int = 0) -> None:
+    """y[M, N] = x[M, K] w[N, K]^T on caller-owned device buffers (raw device pointers),
+    for hosts that must not allocate device memory: nothing is allocated, the scratch is a
+    fixed region inside the library.  Synchronous; calls that overlap on the GPU race on
+    that shared scratch.  Make the first call on a device outside any stream capture."""
+    lib = load_library()
+    rc = lib.s2d2_gemm_bf16_noalloc(C.c_void_p(d_x), C.c_void_p(d_w), C.c_void_p(d_y), M, N, K, C.c_void_p(stream))
+    if rc != 0:
+        raise S2D2Error(rc, lib.s2d2_noalloc_last_error().decode())
 
 
 class Engine:

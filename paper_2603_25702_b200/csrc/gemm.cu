@@ -214,3 +214,140 @@ int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int 
     gemm_simt<bf16, bf16>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
     return S2D2_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free GEMM entry (see s2d2_gemm_bf16_noalloc in the header).
+//
+// The scratch of the split-K kernel lives in file-scope device arrays.  In host code the
+// array names below are only handles: the device addresses come from cudaGetSymbolAddress,
+// looked up once per device with that device current, and are what the kernel receives.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t NOALLOC_WS_FLOATS = S2D2_NOALLOC_WS_BYTES / 4;
+constexpr int NOALLOC_TICKETS = 4096;
+constexpr int NOALLOC_MAX_DEVICES = 64;
+static __device__ __align__(256) float g_noalloc_ws[NOALLOC_WS_FLOATS];
+static __device__ __align__(256) unsigned g_noalloc_tickets[NOALLOC_TICKETS];
+static __device__ __align__(256) int g_noalloc_status[4];
+
+struct NoallocDevice {
+    bool ready = false;
+    float* ws = nullptr;
+    unsigned* tickets = nullptr;
+    int* status = nullptr;
+    int n_sms = 0;
+};
+NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+EncodeTiledFn g_noalloc_encode = nullptr;
+thread_local char g_noalloc_err[256] = "";
+
+int noalloc_fail(int code, const char* msg, cudaError_t e = cudaSuccess) {
+    if (e != cudaSuccess) snprintf(g_noalloc_err, sizeof(g_noalloc_err), "%s: %s", msg, cudaGetErrorString(e));
+    else snprintf(g_noalloc_err, sizeof(g_noalloc_err), "%s", msg);
+    return code;
+}
+
+int noalloc_map(CUtensorMap* m, const void* ptr, int rows, int K, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)tc::BLOCK_K, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_noalloc_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : (int)r;
+}
+}  // namespace
+
+extern "C" const char* s2d2_noalloc_last_error(void) { return g_noalloc_err; }
+
+extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d_y, int32_t M, int32_t N, int32_t K,
+                                      void* cuda_stream) {
+    g_noalloc_err[0] = 0;
+    if (!d_x || !d_w || !d_y) return noalloc_fail(S2D2_ERR_INVALID, "null pointer");
+    if (M < 1 || M > 256) return noalloc_fail(S2D2_ERR_INVALID, "M must be in 1..256");
+    if (N < 1 || N > (1 << 20)) return noalloc_fail(S2D2_ERR_INVALID, "N must be in 1..1048576");
+    if (K < 64 || K > 65536 || K % 64) return noalloc_fail(S2D2_ERR_INVALID, "K must be a multiple of 64 in 64..65536");
+    if (((uintptr_t)d_x | (uintptr_t)d_w | (uintptr_t)d_y) & 15) return noalloc_fail(S2D2_ERR_INVALID, "pointers must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return noalloc_fail(S2D2_ERR_CUDA, "cudaGetDevice", e);
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return noalloc_fail(S2D2_ERR_UNSUPPORTED, "device index too large");
+    NoallocDevice& nd = g_noalloc_dev[dev];
+    if (!nd.ready) {
+        // one-time set-up for this device (do this before any stream capture)
+        int major = 0;
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaDeviceGetAttribute", e);
+        if (major != 10) return noalloc_fail(S2D2_ERR_UNSUPPORTED, "built for sm_100a only");
+        if ((e = cudaDeviceGetAttribute(&nd.n_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaDeviceGetAttribute", e);
+        if (!g_noalloc_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            if ((e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q)) != cudaSuccess || !fn)
+                return noalloc_fail(S2D2_ERR_CUDA, "cuTensorMapEncodeTiled not available", e);
+            g_noalloc_encode = (EncodeTiledFn)fn;
+        }
+        if ((e = cudaGetSymbolAddress((void**)&nd.ws, g_noalloc_ws)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaGetSymbolAddress(ws)", e);
+        if ((e = cudaGetSymbolAddress((void**)&nd.tickets, g_noalloc_tickets)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaGetSymbolAddress(tickets)", e);
+        if ((e = cudaGetSymbolAddress((void**)&nd.status, g_noalloc_status)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaGetSymbolAddress(status)", e);
+        if ((e = cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024)) != cudaSuccess)
+            return noalloc_fail(S2D2_ERR_CUDA, "cudaFuncSetAttribute", e);
+        nd.ready = true;
+    }
+    tc::GemmParams p;
+    p.Y = d_y;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.ldy = N;
+    p.scale = 1.f;
+    p.accumulate = 0;
+    p.kb_total = K / tc::BLOCK_K;
+    p.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
+    p.T = (M + 15) / 16 * 16;
+    p.m_tiles = 1;
+    bool two = p.T <= 64;
+    size_t budget = two ? 100 * 1024 : 200 * 1024;
+    p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(p.T));
+    p.stages = std::max(2, std::min(p.stages, p.kb_total));
+    int slots = nd.n_sms * (two ? 2 : 1);
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= 16 && s <= std::max(1, p.kb_total / 2); ++s) {
+        // the partial tiles and the ticket counters must fit the fixed scratch
+        if (s > 1 && ((size_t)p.n_tiles * s * p.T * tc::BLOCK_N > NOALLOC_WS_FLOATS || p.n_tiles > NOALLOC_TICKETS)) break;
+        int waves = (p.n_tiles * s + slots - 1) / slots;
+        double cost = waves * ((double)(p.kb_total + s - 1) / s + 6.0) + (s > 1 ? 2.0 : 0.0);
+        if (cost < best_cost - 1e-9) {
+            best_cost = cost;
+            best = s;
+        }
+    }
+    p.splits = best;
+    p.ws = nd.ws;
+    p.tickets = nd.tickets;
+    p.status = nd.status;
+    p.evict_first = 0;
+    CUtensorMap mw, mx;
+    if (noalloc_map(&mw, d_w, N, K, tc::BLOCK_N) || noalloc_map(&mx, d_x, M, K, p.T))
+        return noalloc_fail(S2D2_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    // the scratch keeps whatever the previous call left: counters and status start from zero
+    if ((e = cudaMemsetAsync(nd.tickets, 0, NOALLOC_TICKETS * sizeof(unsigned), st)) != cudaSuccess)
+        return noalloc_fail(S2D2_ERR_CUDA, "cudaMemsetAsync", e);
+    if ((e = cudaMemsetAsync(nd.status, 0, sizeof(int), st)) != cudaSuccess)
+        return noalloc_fail(S2D2_ERR_CUDA, "cudaMemsetAsync", e);
+    tc::gemm_tc_kernel<<<p.n_tiles * p.splits, tc::THREADS, tc::smem_bytes(p.T, p.stages), st>>>(mw, mx, p);
+    if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(S2D2_ERR_CUDA, "kernel launch", e);
+    int status = 0;
+    if ((e = cudaMemcpyAsync(&status, nd.status, sizeof(int), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return noalloc_fail(S2D2_ERR_CUDA, "cudaMemcpyAsync", e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return noalloc_fail(S2D2_ERR_CUDA, "cudaStreamSynchronize", e);
+    if (status != 0) return noalloc_fail(S2D2_ERR_TIMEOUT, "a bounded wait inside the kernel ran out");
+    return S2D2_OK;
+}
