@@ -1,0 +1,148 @@
+// Attention dispatch: bf16 models with 16/32/64-token pages run the tensor-core kernel with
+// TMA-staged pages (attention_tc.cuh); everything else runs the plain SIMT kernel.
+#include "attention.h"
+
+#include <cuda.h>
+
+#include <algorithm>
+
+#include "attention_tc.cuh"
+#include "context.h"
+#include "gemm.h"
+#include "kernels_simt.cuh"
+
+using namespace s2d2;
+
+namespace {
+struct AttnState {
+    bool tc_ok = false;
+    CUtensorMap map_kv;
+    float* part_o = nullptr;
+    float* part_ml = nullptr;
+    size_t cap_items = 0;
+    int n_sms = 148;
+};
+AttnState* state(s2d2_ctx* c) { return (AttnState*)c->attn_state; }
+
+template <typename TKV>
+KvPool<TKV> make_pool(s2d2_ctx* c) {
+    KvPool<TKV> p;
+    p.base = (TKV*)c->kv_base;
+    p.page_tokens = c->page_tokens;
+    p.page_shift = c->page_shift;
+    p.n_kv_heads = c->m.n_kv_heads;
+    p.head_dim = c->m.head_dim;
+    p.page_stride = (size_t)2 * c->m.n_kv_heads * c->page_tokens * c->m.head_dim;
+    p.layer_stride = (size_t)c->n_pages * p.page_stride;
+    return p;
+}
+
+template <typename TA, typename TKV>
+void attention_simt(s2d2_ctx* c, const PassView& pv, int layer) {
+    const s2d2_model_config& m = c->m;
+    int warps = pv.n_rows * m.n_q_heads;
+    int blocks = (warps + 3) / 4;
+    float scale = 1.f / sqrtf((float)m.head_dim);
+    KvPool<TKV> pool = make_pool<TKV>(c);
+#define ATT(HD)                                                                                               \
+    attention_simt_kernel<TA, TKV, HD><<<blocks, 128, 0, c->stream>>>((const TA*)c->q, (const TKV*)c->k_rows, \
+                                                                      (const TKV*)c->v_rows, pv, pool, layer, \
+                                                                      m.n_q_heads, m.n_kv_heads, (TA*)c->attn, scale)
+    if (m.head_dim == 32) ATT(32);
+    else if (m.head_dim == 64) ATT(64);
+    else ATT(128);
+#undef ATT
+    c->cnt.n_kernel_launches++;
+}
+}  // namespace
+
+int attention_init(s2d2_ctx* c) {
+    AttnState* a = new AttnState();
+    c->attn_state = a;
+    const s2d2_model_config& m = c->m;
+    if (m.dtype != S2D2_DTYPE_BF16 || !gemm_tc_available(c)) return S2D2_OK;
+    if (!(m.head_dim == 64 || m.head_dim == 128) || c->page_tokens < 16) return S2D2_OK;
+    unsigned long long rows = (unsigned long long)m.n_layers * c->n_pages * 2 * m.n_kv_heads * c->page_tokens;
+    if (rows >= (1ull << 31)) return S2D2_OK;      // row coordinates are 32-bit
+    if (gemm_encode_map(c, &a->map_kv, c->kv_base, rows, m.head_dim, c->page_tokens) != 0) {
+        c->err = "cuTensorMapEncodeTiled failed for the KV pool";
+        return S2D2_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return S2D2_ERR_CUDA;
+    a->n_sms = prop.multiProcessorCount;
+    int group = m.n_q_heads / m.n_kv_heads;
+    size_t base_items = (size_t)c->dc.max_batch * m.n_kv_heads * ((S2D2_MAX_ROWS_PER_SEQ * group + att::QT - 1) / att::QT);
+    a->cap_items = std::max<size_t>(2048, base_items * 2);
+    if (cudaMalloc((void**)&a->part_o, a->cap_items * att::QT * m.head_dim * 4) != cudaSuccess) return S2D2_ERR_CUDA;
+    if (cudaMalloc((void**)&a->part_ml, a->cap_items * att::QT * 2 * 4) != cudaSuccess) return S2D2_ERR_CUDA;
+    cudaError_t e = m.head_dim == 128
+                        ? cudaFuncSetAttribute(att::attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)att::attn_smem_bytes(128))
+                        : cudaFuncSetAttribute(att::attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)att::attn_smem_bytes(64));
+    if (e != cudaSuccess) return S2D2_ERR_CUDA;
+    a->tc_ok = true;
+    return S2D2_OK;
+}
+
+void attention_destroy(s2d2_ctx* c) {
+    AttnState* a = state(c);
+    if (!a) return;
+    if (a->part_o) cudaFree(a->part_o);
+    if (a->part_ml) cudaFree(a->part_ml);
+    delete a;
+    c->attn_state = nullptr;
+}
+
+int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_rows) {
+    const s2d2_model_config& m = c->m;
+    AttnState* a = state(c);
+    if (m.dtype == S2D2_DTYPE_F32) {
+        attention_simt<float, float>(c, pv, layer);
+        return S2D2_OK;
+    }
+    if (!a->tc_ok) {
+        attention_simt<bf16, bf16>(c, pv, layer);
+        return S2D2_OK;
+    }
+    att::AttnParams p;
+    p.q = (const bf16*)c->q;
+    p.k_rows = (const bf16*)c->k_rows;
+    p.v_rows = (const bf16*)c->v_rows;
+    p.out = (bf16*)c->attn;
+    p.part_o = a->part_o;
+    p.part_ml = a->part_ml;
+    p.pv = pv;
+    p.layer = layer;
+    p.Hq = m.n_q_heads;
+    p.Hkv = m.n_kv_heads;
+    p.group = m.n_q_heads / m.n_kv_heads;
+    p.page_tokens = c->page_tokens;
+    p.page_shift = c->page_shift;
+    p.n_pages_pool = c->n_pages;
+    p.n_qtiles = std::max(1, (max_rows * p.group + att::QT - 1) / att::QT);
+    int max_pages = (max_ctx + c->page_tokens - 1) / c->page_tokens;
+    size_t base = (size_t)pv.n_seqs * m.n_kv_heads * p.n_qtiles;
+    // enough key splits to cover the SMs twice, bounded by the partial buffers
+    int want = (int)std::min<size_t>((2 * a->n_sms + base - 1) / base, a->cap_items / base - 1);
+    want = std::max(1, std::min(want, std::max(1, max_pages)));
+    p.pages_per_split = std::max(1, (max_pages + want - 1) / want);
+    p.n_cache_splits = (max_pages + p.pages_per_split - 1) / p.pages_per_split;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)m.head_dim);
+    p.status = c->d_status;
+    if (base * (p.n_cache_splits + 1) > a->cap_items) {
+        attention_simt<bf16, bf16>(c, pv, layer);
+        return S2D2_OK;
+    }
+    dim3 grid(p.n_cache_splits + 1, p.n_qtiles, pv.n_seqs * m.n_kv_heads);
+    if (m.head_dim == 128) {
+        att::attn_tc_kernel<128><<<grid, att::THREADS, att::attn_smem_bytes(128), c->stream>>>(a->map_kv, p);
+        att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);
+    } else {
+        att::attn_tc_kernel<64><<<grid, att::THREADS, att::attn_smem_bytes(64), c->stream>>>(a->map_kv, p);
+        att::attn_combine_kernel<64><<<dim3(pv.n_rows, m.n_q_heads), 64, 0, c->stream>>>(p);
+    }
+    c->cnt.n_kernel_launches += 2;
+    return S2D2_OK;
+}

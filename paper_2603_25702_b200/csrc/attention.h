@@ -1,0 +1,9 @@
+// Host side of the attention step of a pass.
+#pragma once
+#include "common.cuh"
+struct s2d2_ctx;
+int attention_init(s2d2_ctx* c);
+void attention_destroy(s2d2_ctx* c);
+// Attention of one layer over the rows of the pass; reads c->q / c->k_rows / c->v_rows and the KV
+// pool, writes c->attn.  max_ctx / max_rows: largest cached length and row count of a sequence.
+int attention(s2d2_ctx* c, const s2d2::PassView& pv, int layer, int max_ctx, int max_rows);

@@ -1,0 +1,342 @@
+// Two-mask prefix + block attention for bf16 models.
+//
+// Every row of a pass attends (1) the whole cached prefix of its sequence, read from
+// the paged KV pool, and (2) the rows of the same pass that its 64-bit mask allows
+// (the verifier mask [[A, 0], [A<, I]] and the partially causal drafting mask both
+// arrive as such masks).  Work is split over (sequence, kv head, tile of 64 query
+// vectors, key split): the query vectors of one kv head are the rows of the pass times
+// the GQA group, so one CTA serves a whole group with one read of K and V.
+//   * cache splits stream whole pages: K and V tiles of one (page, head) are fetched by
+//     TMA (2D tensor map over the pool, 128-byte swizzle) into a two-stage ring;
+//   * the last split handles the in-pass rows, copied with plain loads into the same
+//     swizzled layout, and applies the row masks.
+// Each warp owns 16 query vectors: S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in,
+// fp32 accumulate) with ldmatrix fragments; the online softmax is per thread quad with
+// warp shuffles.  Every split writes an unnormalised partial (max, sum, O) and
+// attn_combine_kernel merges them in split order.
+#pragma once
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace s2d2 {
+namespace att {
+
+constexpr int QT = 64;          // query vectors per CTA
+constexpr int THREADS = 128;
+constexpr int STAGES = 2;
+
+struct AttnParams {
+    const bf16* q;              // [M, Hq, HD]
+    const bf16* k_rows;         // [M, Hkv, HD] K of this pass's rows
+    const bf16* v_rows;
+    bf16* out;                  // [M, Hq*HD]
+    float* part_o;              // [items, QT, HD] unnormalised partial outputs
+    float* part_ml;             // [items, QT, 2]  (max in log2 units, sum)
+    PassView pv;
+    int layer, Hq, Hkv, group;
+    int page_tokens, page_shift;
+    int n_pages_pool;
+    int pages_per_split;
+    int n_cache_splits;         // grid.x = n_cache_splits + 1 (the last split is the in-pass part)
+    int n_qtiles;               // grid.y
+    float scale_log2;           // log2(e) / sqrt(HD)
+    int* status;
+};
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// Byte offset of 16-byte chunk c of row r in a tile of `rows` rows stored as 64-column halves
+// of 128-byte rows with the 128-byte swizzle (the layout TMA writes).
+__device__ __forceinline__ uint32_t sw_off(int r, int c, int rows) {
+    return (uint32_t)((c >> 3) * rows * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+template <int HD>
+__global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
+    constexpr int CH = HD / 8;          // 16-byte chunks per row
+    constexpr int KS = HD / 16;         // k-steps of Q K^T
+    constexpr int NT_O = HD / 8;        // n-tiles of the output
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int PT = p.page_tokens;                 // keys per tile (16, 32 or 64)
+    const int tile_bytes = 64 * HD * 2;           // room for 64 keys even when the page is smaller
+    uint8_t* q_s = base;                          // [QT][HD]
+    uint8_t* kv_s = base + QT * HD * 2;           // STAGES x (K tile, V tile)
+    uint64_t* full = (uint64_t*)(kv_s + STAGES * 2 * tile_bytes);
+
+    const int split = blockIdx.x, qt = blockIdx.y;
+    const int seq = blockIdx.z / p.Hkv, kvh = blockIdx.z % p.Hkv;
+    const int nrows = p.pv.seq_nrows[seq], row0 = p.pv.seq_row0[seq];
+    const int nq = nrows * p.group;
+    const int q0 = qt * QT;
+    if (q0 >= nq) return;
+    const int n_ctx = p.pv.seq_nctx[seq];
+    const bool in_pass = split == p.n_cache_splits;
+    const int n_pages = (n_ctx + PT - 1) >> p.page_shift;
+    const int pg0 = split * p.pages_per_split;
+    const int pg1 = in_pass ? 0 : min(n_pages, pg0 + p.pages_per_split);
+    const int n_tiles = in_pass ? 1 : max(0, pg1 - pg0);
+    const size_t item = ((size_t)blockIdx.z * p.n_qtiles + qt) * (p.n_cache_splits + 1) + split;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) tc::mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int* pages = p.pv.seq_pages + (size_t)seq * p.pv.max_pages;
+    auto issue = [&](int t) {   // thread 0: TMA of cache tile t of this split into stage t % STAGES
+        int s = t % STAGES;
+        int page = pages[pg0 + t];
+        uint8_t* kd = kv_s + (size_t)s * 2 * tile_bytes;
+        uint8_t* vd = kd + tile_bytes;
+        // row of the pool viewed as a 2D matrix [.., HD]: (((layer*n_pages + page)*2 + kv)*Hkv + head)*PT
+        long long rk = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 0) * p.Hkv + kvh) * PT;
+        long long rv = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 1) * p.Hkv + kvh) * PT;
+        tc::mbar_expect_tx(&full[s], (uint32_t)(2 * PT * HD * 2));
+#pragma unroll
+        for (int h = 0; h < HD / 64; ++h) {
+            tc::tma_load_2d(kd + h * PT * 128, &map_kv, h * 64, (int)rk, &full[s]);
+            tc::tma_load_2d(vd + h * PT * 128, &map_kv, h * 64, (int)rv, &full[s]);
+        }
+    };
+    if (!in_pass && threadIdx.x == 0)
+        for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
+
+    // ---- Q tile: global -> swizzled shared -> A fragments ----
+    for (int i = threadIdx.x; i < QT * CH; i += THREADS) {
+        int r = i / CH, c = i % CH;
+        int qv = q0 + r;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (qv < nq) {
+            int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
+            val = *reinterpret_cast<const uint4*>(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+        }
+        *reinterpret_cast<uint4*>(q_s + sw_off(r, c, QT)) = val;
+    }
+    if (in_pass) {
+        // K and V of this pass's rows of the sequence into stage 0 (rows past nrows are zero)
+        uint8_t* kd = kv_s;
+        uint8_t* vd = kd + tile_bytes;
+        for (int i = threadIdx.x; i < 64 * CH; i += THREADS) {
+            int r = i / CH, c = i % CH;
+            uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
+            if (r < nrows) {
+                size_t o = ((size_t)(row0 + r) * p.Hkv + kvh) * HD + c * 8;
+                kk = *reinterpret_cast<const uint4*>(p.k_rows + o);
+                vv = *reinterpret_cast<const uint4*>(p.v_rows + o);
+            }
+            *reinterpret_cast<uint4*>(kd + sw_off(r, c, 64)) = kk;
+            *reinterpret_cast<uint4*>(vd + sw_off(r, c, 64)) = vv;
+        }
+    }
+    __syncthreads();
+    uint32_t qf[KS][4];
+    {
+        const uint32_t qb = tc::smem_u32(q_s);
+        int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            int c = ks * 2 + (lane >> 4);
+            ldsm_x4(qb + sw_off(r, c, QT), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+        }
+    }
+    // masks of this thread's two query vectors (rows g and g + 8 of the warp's 16)
+    const int qa = q0 + warp * 16 + g, qb_ = qa + 8;
+    unsigned long long mask_a = 0, mask_b = 0;
+    if (in_pass) {
+        if (qa < nq) mask_a = p.pv.row_mask[row0 + qa / p.group];
+        if (qb_ < nq) mask_b = p.pv.row_mask[row0 + qb_ / p.group];
+    }
+
+    float o[NT_O][4];
+#pragma unroll
+    for (int i = 0; i < NT_O; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+    bool failed = false;
+
+    for (int t = 0; t < n_tiles; ++t) {
+        const int s = in_pass ? 0 : t % STAGES;
+        const int rows_t = in_pass ? 64 : PT;           // rows of the tile layout
+        const int keys = in_pass ? ((nrows + 15) & ~15) : PT;
+        // the wait is bounded; all threads agree on its outcome before going on
+        bool ok = in_pass || tc::mbar_wait(&full[s], (t / STAGES) & 1);
+        if (__syncthreads_or(!ok)) {
+            failed = true;
+            break;
+        }
+        const uint32_t kb = tc::smem_u32(kv_s + (size_t)s * 2 * tile_bytes);
+        const uint32_t vb = kb + tile_bytes;
+        // ---- S = Q K^T for `keys` keys (8 keys per n-tile) ----
+        float sc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+#pragma unroll
+        for (int np = 0; np < 4; ++np) {             // pairs of n-tiles = 16 keys
+            if (np * 16 < keys) {
+                int r = np * 16 + (lane & 7) + (lane >> 4) * 8;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    int c = ks * 2 + ((lane >> 3) & 1);
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4(kb + sw_off(r, c, rows_t), b0, b1, b2, b3);
+                    mma_bf16(sc[np * 2], qf[ks], b0, b1);
+                    mma_bf16(sc[np * 2 + 1], qf[ks], b2, b3);
+                }
+            }
+        }
+        // ---- mask, online softmax (log2 domain) ----
+        const int key0 = in_pass ? 0 : (pg0 + t) * PT;
+        float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                int col = nt * 8 + tq * 2 + (e & 1);
+                bool ok;
+                if (in_pass) ok = col < nrows && (((e < 2 ? mask_a : mask_b) >> col) & 1ull);
+                else ok = col < keys && key0 + col < n_ctx;
+                float v = ok ? sc[nt][e] * p.scale_log2 : -INFINITY;
+                sc[nt][e] = v;
+                if (e < 2) mx_a = fmaxf(mx_a, v);
+                else mx_b = fmaxf(mx_b, v);
+            }
+        }
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+        float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+        float ref_a = mn_a == -INFINITY ? 0.f : mn_a, ref_b = mn_b == -INFINITY ? 0.f : mn_b;
+        float corr_a = exp2f(m_a - ref_a), corr_b = exp2f(m_b - ref_b);
+        m_a = mn_a;
+        m_b = mn_b;
+        float sum_a = 0.f, sum_b = 0.f;
+        uint32_t pf[4][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            float p0 = exp2f(sc[nt][0] - ref_a), p1 = exp2f(sc[nt][1] - ref_a);
+            float p2 = exp2f(sc[nt][2] - ref_b), p3 = exp2f(sc[nt][3] - ref_b);
+            sum_a += p0 + p1;
+            sum_b += p2 + p3;
+            // C fragments of two adjacent key n-tiles are the A fragment of one 16-key k-step
+            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+        l_a = l_a * corr_a + sum_a;
+        l_b = l_b * corr_b + sum_b;
+#pragma unroll
+        for (int i = 0; i < NT_O; ++i) {
+            o[i][0] *= corr_a;
+            o[i][1] *= corr_a;
+            o[i][2] *= corr_b;
+            o[i][3] *= corr_b;
+        }
+        // ---- O += P V ----
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {             // 16 keys per k-step
+            if (kk * 16 < keys) {
+                int r = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+                for (int np = 0; np < NT_O / 2; ++np) {
+                    int c = np * 2 + (lane >> 4);
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(vb + sw_off(r, c, rows_t), b0, b1, b2, b3);
+                    mma_bf16(o[np * 2], pf[kk], b0, b1);
+                    mma_bf16(o[np * 2 + 1], pf[kk], b2, b3);
+                }
+            }
+        }
+        __syncthreads();   // every warp is done with stage s
+        if (!in_pass && threadIdx.x == 0 && t + STAGES < n_tiles) issue(t + STAGES);
+    }
+    if (failed) {   // uniform across the CTA
+        if (threadIdx.x == 0) {
+            atomicExch(p.status, 2);
+            // copies already issued target this CTA's shared memory: give them one more bounded
+            // wait before the CTA leaves
+            for (int s = 0; s < STAGES; ++s) tc::mbar_wait(&full[s], 0);
+        }
+        return;
+    }
+    // row sums across the quad
+    l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+    l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+    l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+    l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+    // ---- partial (max, sum, O) of this split ----
+    float* po = p.part_o + item * QT * HD;
+    float* pml = p.part_ml + item * QT * 2;
+    int ra = warp * 16 + g, rb = ra + 8;
+    if (tq == 0) {
+        pml[ra * 2] = m_a;
+        pml[ra * 2 + 1] = l_a;
+        pml[rb * 2] = m_b;
+        pml[rb * 2 + 1] = l_b;
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT_O; ++nt) {
+        int col = nt * 8 + tq * 2;
+        *reinterpret_cast<float2*>(po + (size_t)ra * HD + col) = make_float2(o[nt][0], o[nt][1]);
+        *reinterpret_cast<float2*>(po + (size_t)rb * HD + col) = make_float2(o[nt][2], o[nt][3]);
+    }
+}
+
+// Merges the partials of all splits of one query vector (fixed split order) and writes bf16.
+template <int HD>
+__global__ void attn_combine_kernel(AttnParams p) {
+    int r = blockIdx.x, hq = blockIdx.y;
+    int seq = p.pv.row_seq[r];
+    int kvh = hq / p.group;
+    int qv = (r - p.pv.seq_row0[seq]) * p.group + hq % p.group;
+    int qt = qv / QT, qi = qv % QT;
+    int n_splits = p.n_cache_splits + 1;
+    int n_ctx = p.pv.seq_nctx[seq];
+    int n_pages = (n_ctx + p.page_tokens - 1) >> p.page_shift;
+    size_t item0 = ((size_t)(seq * p.Hkv + kvh) * p.n_qtiles + qt) * n_splits;
+    float m = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) {
+        bool used = s == p.n_cache_splits || s * p.pages_per_split < n_pages;
+        if (used) m = fmaxf(m, p.part_ml[(item0 + s) * QT * 2 + qi * 2]);
+    }
+    for (int c = threadIdx.x; c < HD; c += blockDim.x) {
+        float acc = 0.f, l = 0.f;
+        for (int s = 0; s < n_splits; ++s) {
+            bool used = s == p.n_cache_splits || s * p.pages_per_split < n_pages;
+            if (!used) continue;
+            float ms = p.part_ml[(item0 + s) * QT * 2 + qi * 2];
+            if (ms == -INFINITY) continue;
+            float w = exp2f(ms - m);
+            l += w * p.part_ml[(item0 + s) * QT * 2 + qi * 2 + 1];
+            acc += w * p.part_o[((item0 + s) * QT + qi) * HD + c];
+        }
+        p.out[((size_t)r * p.Hq + hq) * HD + c] = __float2bfloat16_rn(acc / l);
+    }
+}
+
+__host__ __device__ inline size_t attn_smem_bytes(int HD) {
+    return (size_t)QT * HD * 2 + (size_t)STAGES * 2 * 64 * HD * 2 + 64 + 1024;
+}
+
+}  // namespace att
+}  // namespace s2d2

@@ -128,6 +128,7 @@ struct s2d2_ctx {
     double prof_bytes = 0, prof_ms_done = 0;
     int64_t prof_launches = 0;
     void* gemm_state = nullptr;             // owned by gemm.cu
+    void* attn_state = nullptr;             // owned by attention.cu
     int* d_status = nullptr;                // raised by a kernel whose bounded wait ran out
     int* h_status = nullptr;                // pinned mirror
 };

@@ -11,3 +11,7 @@ void gemm_prof_end(s2d2_ctx* c, double algorithmic_bytes);
 int gemm_prof_collect(s2d2_ctx* c);   // synchronises, folds finished pairs into the totals
 // Drops cached tensor maps of a buffer that is about to be freed.
 void gemm_forget(s2d2_ctx* c, const void* ptr);
+// 2D bf16 tensor map [rows, cols] with boxes of box_rows x 64 columns and the 128-byte swizzle.
+// `out` points to a CUtensorMap (128 bytes). Returns 0 on success.
+int gemm_encode_map(s2d2_ctx* c, void* out, const void* ptr, unsigned long long rows, int cols, int box_rows);
+bool gemm_tc_available(s2d2_ctx* c);

@@ -13,6 +13,7 @@
 #include <algorithm>
 
 #include "context.h"
+#include "attention.h"
 #include "gemm.h"
 #include "kernels_simt.cuh"
 #include "vocab_kernels.cuh"
@@ -303,6 +304,7 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
     *c->h_status = 0;
     int grc = gemm_init(c);
     if (grc != S2D2_OK) return grc;
+    if ((grc = attention_init(c)) != S2D2_OK) return grc;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     return S2D2_OK;
 }
@@ -310,6 +312,7 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
 extern "C" int s2d2_destroy(s2d2_ctx* c) {
     if (!c) return S2D2_ERR_INVALID;
     cudaStreamSynchronize(c->stream);
+    attention_destroy(c);
     gemm_destroy(c);
     void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
@@ -372,6 +375,7 @@ namespace {
 
 struct PassBuild {
     int n_rows = 0, n_seqs = 0, n_logit = 0;
+    int max_ctx = 0, max_rows = 0;     // over the sequences of the pass
 };
 
 int ensure_pages(s2d2_ctx* c, SeqState& s, int n_tokens) {
@@ -389,6 +393,7 @@ int ensure_pages(s2d2_ctx* c, SeqState& s, int n_tokens) {
 void begin_seq(s2d2_ctx* c, PassBuild& pb, const SeqState& s, int n_ctx) {
     PassMeta& pm = c->meta;
     int q = pb.n_seqs++;
+    pb.max_ctx = std::max(pb.max_ctx, n_ctx);
     pm.hp<int>(pm.off_nctx)[q] = n_ctx;
     pm.hp<int>(pm.off_row0)[q] = pb.n_rows;
     pm.hp<int>(pm.off_nrows)[q] = 0;
@@ -403,7 +408,7 @@ void add_row(s2d2_ctx* c, PassBuild& pb, int token, int pos, unsigned long long 
     pm.hp<int>(pm.off_seq)[r] = q;
     pm.hp<int>(pm.off_flags)[r] = flags;
     pm.hp<unsigned long long>(pm.off_mask)[r] = mask;
-    pm.hp<int>(pm.off_nrows)[q]++;
+    pb.max_rows = std::max(pb.max_rows, ++pm.hp<int>(pm.off_nrows)[q]);
     if (logits) pm.hp<int>(pm.off_logit_rows)[pb.n_logit++] = r;
 }
 PassView make_view(s2d2_ctx* c, const PassBuild& pb) {
@@ -439,24 +444,6 @@ KvPool<TKV> make_pool(s2d2_ctx* c) {
     return p;
 }
 
-template <typename TA, typename TKV>
-void launch_attention(s2d2_ctx* c, const PassView& pv, int layer) {
-    const s2d2_model_config& m = c->m;
-    int warps = pv.n_rows * m.n_q_heads;
-    int blocks = (warps + 3) / 4;
-    float scale = 1.f / sqrtf((float)m.head_dim);
-    KvPool<TKV> pool = make_pool<TKV>(c);
-#define ATT(HD)                                                                                                   \
-    attention_simt_kernel<TA, TKV, HD><<<blocks, 128, 0, c->stream>>>((const TA*)c->q, (const TKV*)c->k_rows,     \
-                                                                      (const TKV*)c->v_rows, pv, pool, layer,     \
-                                                                      m.n_q_heads, m.n_kv_heads, (TA*)c->attn, scale)
-    if (m.head_dim == 32) ATT(32);
-    else if (m.head_dim == 64) ATT(64);
-    else ATT(128);
-#undef ATT
-    LAUNCHED(c);
-}
-
 // One pass of the network over the rows described by the uploaded metadata.
 // Logits of pv.logit_rows go to `logits_out` (row-major [n_logit_rows, vocab]).
 template <typename TW, typename TA, typename TKV>
@@ -482,7 +469,7 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
             c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
             l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
         LAUNCHED(c);
-        launch_attention<TA, TKV>(c, pv, l);
+        if ((rc = attention(c, pv, l, pb.max_ctx, pb.max_rows))) return rc;
         if ((rc = gemm(c, c->attn, L.wo, c->h, M, d, nq, d, 1.f, 1))) return rc;
         rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.ffn_norm, (TA*)c->xn, d, m.rms_eps);
         LAUNCHED(c);
