@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libs2d2.so")
-SOURCES = ["s2d2_api.cu", "gemm.cu", "attention.cu"]
+SOURCES = ["s2d2_api.cu", "gemm.cu", "attention.cu", "pass.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

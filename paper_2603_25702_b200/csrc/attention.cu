@@ -95,17 +95,13 @@ void attention_destroy(s2d2_ctx* c) {
     c->attn_state = nullptr;
 }
 
-int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_rows) {
+// Geometry of the tensor-core attention for one pass (query tiles, key splits, partial buffers).
+// Returns false when the pass must take the plain kernel instead.
+bool attention_plan(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, int target_items, att::AttnParams* out,
+                    const void** map_kv) {
     const s2d2_model_config& m = c->m;
     AttnState* a = state(c);
-    if (m.dtype == S2D2_DTYPE_F32) {
-        attention_simt<float, float>(c, pv, layer);
-        return S2D2_OK;
-    }
-    if (!a->tc_ok) {
-        attention_simt<bf16, bf16>(c, pv, layer);
-        return S2D2_OK;
-    }
+    if (!a || !a->tc_ok) return false;
     att::AttnParams p;
     p.q = (const bf16*)c->q;
     p.k_rows = (const bf16*)c->k_rows;
@@ -114,7 +110,7 @@ int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_r
     p.part_o = a->part_o;
     p.part_ml = a->part_ml;
     p.pv = pv;
-    p.layer = layer;
+    p.layer = 0;
     p.Hq = m.n_q_heads;
     p.Hkv = m.n_kv_heads;
     p.group = m.n_q_heads / m.n_kv_heads;
@@ -124,17 +120,33 @@ int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_r
     p.n_qtiles = std::max(1, (max_rows * p.group + att::QT - 1) / att::QT);
     int max_pages = (max_ctx + c->page_tokens - 1) / c->page_tokens;
     size_t base = (size_t)pv.n_seqs * m.n_kv_heads * p.n_qtiles;
-    // enough key splits to cover the SMs twice, bounded by the partial buffers
-    int want = (int)std::min<size_t>((2 * a->n_sms + base - 1) / base, a->cap_items / base - 1);
+    // enough key splits to reach the wanted number of work items, bounded by the partial buffers
+    if (target_items <= 0) target_items = 2 * a->n_sms;
+    int want = (int)std::min<size_t>((target_items + base - 1) / base, a->cap_items / base - 1);
     want = std::max(1, std::min(want, std::max(1, max_pages)));
     p.pages_per_split = std::max(1, (max_pages + want - 1) / want);
     p.n_cache_splits = (max_pages + p.pages_per_split - 1) / p.pages_per_split;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)m.head_dim);
     p.status = c->d_status;
-    if (base * (p.n_cache_splits + 1) > a->cap_items) {
+    if (base * (p.n_cache_splits + 1) > a->cap_items) return false;
+    *out = p;
+    if (map_kv) *map_kv = &a->map_kv;
+    return true;
+}
+
+int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_rows) {
+    const s2d2_model_config& m = c->m;
+    AttnState* a = state(c);
+    if (m.dtype == S2D2_DTYPE_F32) {
+        attention_simt<float, float>(c, pv, layer);
+        return S2D2_OK;
+    }
+    att::AttnParams p;
+    if (!attention_plan(c, pv, max_ctx, max_rows, 0, &p, nullptr)) {
         attention_simt<bf16, bf16>(c, pv, layer);
         return S2D2_OK;
     }
+    p.layer = layer;
     dim3 grid(p.n_cache_splits + 1, p.n_qtiles, pv.n_seqs * m.n_kv_heads);
     if (m.head_dim == 128) {
         att::attn_tc_kernel<128><<<grid, att::THREADS, att::attn_smem_bytes(128), c->stream>>>(a->map_kv, p);

@@ -65,48 +65,66 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 // Byte offset of 16-byte chunk c of row r in a tile of `rows` rows stored as 64-column halves
 // of 128-byte rows with the 128-byte swizzle (the layout TMA writes).
+__host__ __device__ inline size_t attn_tiles_bytes(int HD) { return (size_t)QT * HD * 2 + (size_t)STAGES * 2 * 64 * HD * 2; }
 __device__ __forceinline__ uint32_t sw_off(int r, int c, int rows) {
     return (uint32_t)((c >> 3) * rows * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
+// Barrier over a group of `n` threads of the CTA (a whole CTA of 128 threads with id 0, or the
+// compute warps of a larger CTA with their own id).
+__device__ __forceinline__ void group_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ bool group_or(int id, int n, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(n)
+        : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ uint4 ldcg16(const void* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
+
+// One work item (sequence z / Hkv, kv head z % Hkv, query tile qt, key split) of the attention
+// step, run by a group of 128 threads (`tid` 0..127, barrier `bar_id`).  `base` is 1024-byte
+// aligned shared memory of attn_tiles_bytes(HD); `full` are STAGES mbarriers initialised once
+// by the caller and `ring_pos` counts the cache tiles this group has streamed through them so
+// far (it carries the barrier phase from one item to the next).  Activations are read with
+// L2-only loads: inside a persistent kernel they are rewritten by other CTAs between items.
+// Returns false when a bounded wait ran out (the status word is raised).
 template <int HD>
-__global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
+__device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
+                                          uint8_t* base, uint64_t* full, uint32_t& ring_pos, int tid, int bar_id) {
     constexpr int CH = HD / 8;          // 16-byte chunks per row
     constexpr int KS = HD / 16;         // k-steps of Q K^T
     constexpr int NT_O = HD / 8;        // n-tiles of the output
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int PT = p.page_tokens;                 // keys per tile (16, 32 or 64)
     const int tile_bytes = 64 * HD * 2;           // room for 64 keys even when the page is smaller
     uint8_t* q_s = base;                          // [QT][HD]
     uint8_t* kv_s = base + QT * HD * 2;           // STAGES x (K tile, V tile)
-    uint64_t* full = (uint64_t*)(kv_s + STAGES * 2 * tile_bytes);
 
-    const int split = blockIdx.x, qt = blockIdx.y;
-    const int seq = blockIdx.z / p.Hkv, kvh = blockIdx.z % p.Hkv;
+    const int seq = z / p.Hkv, kvh = z % p.Hkv;
     const int nrows = p.pv.seq_nrows[seq], row0 = p.pv.seq_row0[seq];
     const int nq = nrows * p.group;
     const int q0 = qt * QT;
-    if (q0 >= nq) return;
+    if (q0 >= nq) return true;
     const int n_ctx = p.pv.seq_nctx[seq];
     const bool in_pass = split == p.n_cache_splits;
     const int n_pages = (n_ctx + PT - 1) >> p.page_shift;
     const int pg0 = split * p.pages_per_split;
     const int pg1 = in_pass ? 0 : min(n_pages, pg0 + p.pages_per_split);
     const int n_tiles = in_pass ? 1 : max(0, pg1 - pg0);
-    const size_t item = ((size_t)blockIdx.z * p.n_qtiles + qt) * (p.n_cache_splits + 1) + split;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t item = ((size_t)z * p.n_qtiles + qt) * (p.n_cache_splits + 1) + split;
+    const int warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, tq = lane & 3;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) tc::mbar_init(&full[s], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
+    const uint32_t ring0 = ring_pos;
+    if (!in_pass) ring_pos += (uint32_t)n_tiles;
 
     const int* pages = p.pv.seq_pages + (size_t)seq * p.pv.max_pages;
     auto issue = [&](int t) {   // thread 0: TMA of cache tile t of this split into stage t % STAGES
-        int s = t % STAGES;
+        int s = (int)((ring0 + t) % STAGES);
         int page = pages[pg0 + t];
         uint8_t* kd = kv_s + (size_t)s * 2 * tile_bytes;
         uint8_t* vd = kd + tile_bytes;
@@ -116,21 +134,21 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
         tc::mbar_expect_tx(&full[s], (uint32_t)(2 * PT * HD * 2));
 #pragma unroll
         for (int h = 0; h < HD / 64; ++h) {
-            tc::tma_load_2d(kd + h * PT * 128, &map_kv, h * 64, (int)rk, &full[s]);
-            tc::tma_load_2d(vd + h * PT * 128, &map_kv, h * 64, (int)rv, &full[s]);
+            tc::tma_load_2d(kd + h * PT * 128, map_kv_ptr, h * 64, (int)rk, &full[s]);
+            tc::tma_load_2d(vd + h * PT * 128, map_kv_ptr, h * 64, (int)rv, &full[s]);
         }
     };
-    if (!in_pass && threadIdx.x == 0)
+    if (!in_pass && tid == 0)
         for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
 
     // ---- Q tile: global -> swizzled shared -> A fragments ----
-    for (int i = threadIdx.x; i < QT * CH; i += THREADS) {
+    for (int i = tid; i < QT * CH; i += THREADS) {
         int r = i / CH, c = i % CH;
         int qv = q0 + r;
         uint4 val = make_uint4(0, 0, 0, 0);
         if (qv < nq) {
             int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
-            val = *reinterpret_cast<const uint4*>(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+            val = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
         }
         *reinterpret_cast<uint4*>(q_s + sw_off(r, c, QT)) = val;
     }
@@ -138,19 +156,19 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
         // K and V of this pass's rows of the sequence into stage 0 (rows past nrows are zero)
         uint8_t* kd = kv_s;
         uint8_t* vd = kd + tile_bytes;
-        for (int i = threadIdx.x; i < 64 * CH; i += THREADS) {
+        for (int i = tid; i < 64 * CH; i += THREADS) {
             int r = i / CH, c = i % CH;
             uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
             if (r < nrows) {
                 size_t o = ((size_t)(row0 + r) * p.Hkv + kvh) * HD + c * 8;
-                kk = *reinterpret_cast<const uint4*>(p.k_rows + o);
-                vv = *reinterpret_cast<const uint4*>(p.v_rows + o);
+                kk = ldcg16(p.k_rows + o);
+                vv = ldcg16(p.v_rows + o);
             }
             *reinterpret_cast<uint4*>(kd + sw_off(r, c, 64)) = kk;
             *reinterpret_cast<uint4*>(vd + sw_off(r, c, 64)) = vv;
         }
     }
-    __syncthreads();
+    group_sync(bar_id, THREADS);
     uint32_t qf[KS][4];
     {
         const uint32_t qb = tc::smem_u32(q_s);
@@ -176,12 +194,12 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
     bool failed = false;
 
     for (int t = 0; t < n_tiles; ++t) {
-        const int s = in_pass ? 0 : t % STAGES;
+        const int s = in_pass ? 0 : (int)((ring0 + t) % STAGES);
         const int rows_t = in_pass ? 64 : PT;           // rows of the tile layout
         const int keys = in_pass ? ((nrows + 15) & ~15) : PT;
         // the wait is bounded; all threads agree on its outcome before going on
-        bool ok = in_pass || tc::mbar_wait(&full[s], (t / STAGES) & 1);
-        if (__syncthreads_or(!ok)) {
+        bool ok = in_pass || tc::mbar_wait(&full[s], ((ring0 + t) / STAGES) & 1);
+        if (group_or(bar_id, THREADS, !ok)) {
             failed = true;
             break;
         }
@@ -267,17 +285,12 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
                 }
             }
         }
-        __syncthreads();   // every warp is done with stage s
-        if (!in_pass && threadIdx.x == 0 && t + STAGES < n_tiles) issue(t + STAGES);
+        group_sync(bar_id, THREADS);   // every warp is done with stage s
+        if (!in_pass && tid == 0 && t + STAGES < n_tiles) issue(t + STAGES);
     }
-    if (failed) {   // uniform across the CTA
-        if (threadIdx.x == 0) {
-            atomicExch(p.status, 2);
-            // copies already issued target this CTA's shared memory: give them one more bounded
-            // wait before the CTA leaves
-            for (int s = 0; s < STAGES; ++s) tc::mbar_wait(&full[s], 0);
-        }
-        return;
+    if (failed) {   // uniform across the group
+        if (tid == 0) atomicExch(p.status, 2);
+        return false;
     }
     // row sums across the quad
     l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
@@ -299,6 +312,29 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
         int col = nt * 8 + tq * 2;
         *reinterpret_cast<float2*>(po + (size_t)ra * HD + col) = make_float2(o[nt][0], o[nt][1]);
         *reinterpret_cast<float2*>(po + (size_t)rb * HD + col) = make_float2(o[nt][2], o[nt][3]);
+    }
+    // the group's shared memory is reused by its next item, possibly by TMA after plain stores
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    group_sync(bar_id, THREADS);
+    return true;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* full = (uint64_t*)(base + attn_tiles_bytes(HD));
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) tc::mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t ring_pos = 0;
+    bool ok = attn_item<HD>(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, full, ring_pos, threadIdx.x, 0);
+    if (!ok && threadIdx.x == 0) {
+        // copies already issued target this CTA's shared memory: give them one more bounded wait
+        // before the CTA leaves
+        for (int s = 0; s < STAGES; ++s) tc::mbar_wait(&full[s], 0);
     }
 }
 
@@ -334,9 +370,7 @@ __global__ void attn_combine_kernel(AttnParams p) {
     }
 }
 
-__host__ __device__ inline size_t attn_smem_bytes(int HD) {
-    return (size_t)QT * HD * 2 + (size_t)STAGES * 2 * 64 * HD * 2 + 64 + 1024;
-}
+__host__ __device__ inline size_t attn_smem_bytes(int HD) { return attn_tiles_bytes(HD) + 64 + 1024; }
 
 }  // namespace att
 }  // namespace s2d2

@@ -129,6 +129,7 @@ struct s2d2_ctx {
     int64_t prof_launches = 0;
     void* gemm_state = nullptr;             // owned by gemm.cu
     void* attn_state = nullptr;             // owned by attention.cu
+    void* pass_state = nullptr;             // owned by pass.cu
     int* d_status = nullptr;                // raised by a kernel whose bounded wait ran out
     int* h_status = nullptr;                // pinned mirror
 };

@@ -70,7 +70,7 @@ __host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int T) {
 __host__ __device__ __forceinline__ size_t stage_bytes(int T) { return (size_t)BLOCK_N * 128 + (size_t)T * 128; }
 __host__ __device__ __forceinline__ size_t smem_bytes(int T, int stages) { return stages * stage_bytes(T) + 1024 + 256; }
 
-__global__ void __launch_bounds__(THREADS)
+static __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle

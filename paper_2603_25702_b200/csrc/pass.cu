@@ -1,0 +1,226 @@
+// Launch logic of the persistent pass kernel: tensor maps of every weight matrix and activation
+// buffer, split-K workspace sizing, eligibility, cooperative launch.
+#include "pass.h"
+
+#include <cuda.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "attention.h"
+#include "context.h"
+#include "gemm.h"
+#include "pass_kernel.cuh"
+
+using namespace s2d2;
+
+namespace {
+struct PassState {
+    bool ok = false;
+    int grid = 0;
+    int max_smem = 0;
+    int n_weight_maps = 0;
+    int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act
+    int map_kv = 0;
+    CUtensorMap* d_maps = nullptr;
+    pp::LayerGains* d_gains = nullptr;
+    float* ws = nullptr;
+    int max_segs = 0;
+    float *ssq_a = nullptr, *ssq_b = nullptr;
+    unsigned* barrier = nullptr;
+    double weight_bytes = 0;     // bytes of every matrix a pass streams (without the LM head)
+    double head_bytes = 0;
+};
+PassState* state(s2d2_ctx* c) { return (PassState*)c->pass_state; }
+
+template <int HD>
+cudaError_t prepare_kernel(PassState* s, int smem) {
+    cudaError_t e = cudaFuncSetAttribute(pp::pass_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pp::pass_kernel<HD>, pp::THREADS, smem);
+    if (e != cudaSuccess) return e;
+    return per_sm >= 1 ? cudaSuccess : cudaErrorCooperativeLaunchTooLarge;
+}
+int stages_for(const PassState* s, int T, int hd) {
+    long avail = (long)s->max_smem - 1024 - (long)att::attn_tiles_bytes(hd) - (long)pp::misc_bytes();
+    return (int)std::min<long>(12, avail / (long)pp::stage_bytes(T));
+}
+}  // namespace
+
+int pass_init(s2d2_ctx* c) {
+    PassState* s = new PassState();
+    c->pass_state = s;
+    const s2d2_model_config& m = c->m;
+    if (m.dtype != S2D2_DTYPE_BF16 || !c->dc.use_tensor_cores || m.n_experts > 0 || !gemm_tc_available(c)) return S2D2_OK;
+    const int d = m.d_model, hd = m.head_dim, nq = m.n_q_heads * hd, nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, f = m.ffn;
+    if (!(hd == 64 || hd == 128) || d % 128 || f % 128 || nqkv % 128 || nq % 64 || c->page_tokens < 16) return S2D2_OK;
+    if (c->max_rows < pp::MAX_T) return S2D2_OK;
+    int coop = 0, n_sms = 0, optin = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+    cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, c->device);
+    cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
+    if (!coop || n_sms < 1) return S2D2_OK;
+    s->grid = n_sms;
+    s->max_smem = optin;
+    if (stages_for(s, pp::MAX_T, hd) < 3) return S2D2_OK;
+    cudaError_t e = hd == 128 ? prepare_kernel<128>(s, optin) : prepare_kernel<64>(s, optin);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return S2D2_OK;       // the one-kernel-per-operation path stays in charge
+    }
+    // tensor maps
+    const int L = m.n_layers;
+    s->n_weight_maps = L * 4 + 1;
+    s->map_x0 = s->n_weight_maps;
+    s->map_kv = s->map_x0 + 12;
+    std::vector<CUtensorMap> maps(s->map_kv + 1);
+    auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
+        return gemm_encode_map(c, &maps[idx], ptr, rows, cols, box_rows) == 0;
+    };
+    bool good = true;
+    for (int l = 0; l < L && good; ++l) {
+        const LayerWeights& W = c->layers[l];
+        good = enc(l * 4 + 0, W.wqkv, nqkv, d, 128) && enc(l * 4 + 1, W.wo, d, nq, 128) && enc(l * 4 + 2, W.wgu, 2 * f, d, 128) &&
+               enc(l * 4 + 3, W.wdown, d, f, 128);
+        s->weight_bytes += 2.0 * ((double)nqkv * d + (double)d * nq + 2.0 * f * d + (double)d * f);
+    }
+    good = good && enc(L * 4, c->lm_head, m.vocab, d, 128);
+    s->head_bytes = 2.0 * (double)m.vocab * d;
+    for (int t = 0; t < 4 && good; ++t) {
+        const int T = 16 * (t + 1);
+        good = enc(s->map_x0 + t, c->xn, c->max_rows, d, T) && enc(s->map_x0 + 4 + t, c->attn, c->max_rows, nq, T) &&
+               enc(s->map_x0 + 8 + t, c->act, c->max_rows, f, T);
+    }
+    if (!good) {
+        c->err = "cuTensorMapEncodeTiled failed for the persistent pass";
+        return S2D2_ERR_CUDA;
+    }
+    {   // the KV pool map is the attention kernel's
+        PassView dummy{};
+        dummy.n_seqs = 1;
+        att::AttnParams ap;
+        const void* mk = nullptr;
+        if (!attention_plan(c, dummy, 1, 1, 0, &ap, &mk) || !mk) return S2D2_OK;
+        maps[s->map_kv] = *(const CUtensorMap*)mk;
+    }
+    // split-K workspace: the most segments any CTA has in one GEMM
+    const int G = s->grid;
+    auto segs = [&](long long N, long long K) {
+        long long n_tiles = (N + 127) / 128, kbt = K / 64, U = n_tiles * kbt;
+        long long per = (U + G - 1) / G;
+        return (int)((per + kbt - 1) / kbt + 1);
+    };
+    s->max_segs = std::max({segs(nqkv, d), segs(d, nq), segs(2 * f, d), segs(d, f), segs(m.vocab, d)});
+    size_t ws_floats = (size_t)G * s->max_segs * pp::MAX_T * 128;
+    std::vector<pp::LayerGains> gains(L);
+    for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
+    size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
+    if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
+        cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
+        cudaMalloc((void**)&s->ws, ws_floats * 4) != cudaSuccess || cudaMalloc((void**)&s->ssq_a, ssq_bytes) != cudaSuccess ||
+        cudaMalloc((void**)&s->ssq_b, ssq_bytes) != cudaSuccess || cudaMalloc((void**)&s->barrier, 256) != cudaSuccess) {
+        c->err = "cudaMalloc failed for the persistent pass";
+        return S2D2_ERR_CUDA;
+    }
+    if (cudaMemcpy(s->d_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(s->d_gains, gains.data(), gains.size() * sizeof(pp::LayerGains), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(s->ws, 0, ws_floats * 4) != cudaSuccess) {
+        c->err = "device copy failed for the persistent pass";
+        return S2D2_ERR_CUDA;
+    }
+    // rows past the pass's own rows ride along as unused MMA columns: keep them finite
+    size_t es = 2;
+    cudaMemset(c->xn, 0, (size_t)c->max_rows * d * es);
+    cudaMemset(c->attn, 0, (size_t)c->max_rows * nq * es);
+    cudaMemset(c->act, 0, (size_t)c->max_rows * f * es);
+    s->ok = true;
+    return S2D2_OK;
+}
+
+void pass_destroy(s2d2_ctx* c) {
+    PassState* s = state(c);
+    if (!s) return;
+    void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    delete s;
+    c->pass_state = nullptr;
+}
+
+int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long long sum_ctx, float* logits_out, bool* taken) {
+    *taken = false;
+    PassState* s = state(c);
+    const s2d2_model_config& m = c->m;
+    if (!s || !s->ok || pv.n_rows < 1 || pv.n_rows > pp::MAX_T) return S2D2_OK;
+    pp::PassParams p;
+    if (!attention_plan(c, pv, max_ctx, max_rows, s->grid, &p.ap, nullptr)) return S2D2_OK;
+    p.n_layers = m.n_layers;
+    p.d = m.d_model;
+    p.Hq = m.n_q_heads;
+    p.Hkv = m.n_kv_heads;
+    p.hd = m.head_dim;
+    p.f = m.ffn;
+    p.V = m.vocab;
+    p.qk_norm = m.qk_norm;
+    p.eps = m.rms_eps;
+    p.logit_scale = m.logit_scale;
+    p.pv = pv;
+    p.M = pv.n_rows;
+    p.T = (pv.n_rows + 15) / 16 * 16;
+    p.n_logit = logits_out ? pv.n_logit_rows : 0;
+    p.embed = (const bf16*)c->embed;
+    p.gains = s->d_gains;
+    p.final_norm = c->final_norm;
+    p.h = c->h;
+    p.xn = (bf16*)c->xn;
+    p.q = (bf16*)c->q;
+    p.k_rows = (bf16*)c->k_rows;
+    p.v_rows = (bf16*)c->v_rows;
+    p.attn = (bf16*)c->attn;
+    p.act = (bf16*)c->act;
+    p.ws = s->ws;
+    p.max_segs = s->max_segs;
+    p.ssq_a = s->ssq_a;
+    p.ssq_b = s->ssq_b;
+    p.logits = logits_out;
+    p.rope_cos = c->rope_cos;
+    p.rope_sin = c->rope_sin;
+    p.pool.base = (bf16*)c->kv_base;
+    p.pool.page_tokens = c->page_tokens;
+    p.pool.page_shift = c->page_shift;
+    p.pool.n_kv_heads = m.n_kv_heads;
+    p.pool.head_dim = m.head_dim;
+    p.pool.page_stride = (size_t)2 * m.n_kv_heads * c->page_tokens * m.head_dim;
+    p.pool.layer_stride = (size_t)c->n_pages * p.pool.page_stride;
+    p.maps = s->d_maps;
+    const int ti = p.T / 16 - 1;
+    p.map_xn = s->map_x0 + ti;
+    p.map_attn = s->map_x0 + 4 + ti;
+    p.map_act = s->map_x0 + 8 + ti;
+    p.map_kv = s->map_kv;
+    p.barrier = s->barrier;
+    p.status = c->d_status;
+    p.S = stages_for(s, p.T, m.head_dim);
+    size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
+    if (cudaMemsetAsync(s->barrier, 0, 4, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
+    void* args[] = {&p};
+    gemm_prof_begin(c);
+    cudaError_t e = m.head_dim == 128
+                        ? cudaLaunchCooperativeKernel((void*)pp::pass_kernel<128>, dim3(s->grid), dim3(pp::THREADS), args, smem, c->stream)
+                        : cudaLaunchCooperativeKernel((void*)pp::pass_kernel<64>, dim3(s->grid), dim3(pp::THREADS), args, smem, c->stream);
+    // algorithmic bytes of the pass: every matrix once, the cached K/V of every sequence once,
+    // this pass's K/V rows written, logits written
+    double kv_tok = 2.0 * m.n_layers * m.n_kv_heads * m.head_dim * 2.0;
+    double bytes = s->weight_bytes + (p.n_logit > 0 ? s->head_bytes + 4.0 * p.n_logit * m.vocab : 0.0) + kv_tok * (double)sum_ctx +
+                   kv_tok * pv.n_rows;
+    gemm_prof_end(c, bytes);
+    if (e != cudaSuccess) {
+        c->err = std::string("persistent pass launch: ") + cudaGetErrorString(e);
+        return S2D2_ERR_CUDA;
+    }
+    c->cnt.n_kernel_launches++;
+    c->last_pass_rows = pv.n_rows;
+    *taken = true;
+    return S2D2_OK;
+}

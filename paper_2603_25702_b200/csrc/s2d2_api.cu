@@ -16,6 +16,7 @@
 #include "attention.h"
 #include "gemm.h"
 #include "kernels_simt.cuh"
+#include "pass.h"
 #include "vocab_kernels.cuh"
 
 using namespace s2d2;
@@ -305,6 +306,7 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
     int grc = gemm_init(c);
     if (grc != S2D2_OK) return grc;
     if ((grc = attention_init(c)) != S2D2_OK) return grc;
+    if ((grc = pass_init(c)) != S2D2_OK) return grc;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     return S2D2_OK;
 }
@@ -312,6 +314,7 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
 extern "C" int s2d2_destroy(s2d2_ctx* c) {
     if (!c) return S2D2_ERR_INVALID;
     cudaStreamSynchronize(c->stream);
+    pass_destroy(c);
     attention_destroy(c);
     gemm_destroy(c);
     void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
@@ -376,6 +379,7 @@ namespace {
 struct PassBuild {
     int n_rows = 0, n_seqs = 0, n_logit = 0;
     int max_ctx = 0, max_rows = 0;     // over the sequences of the pass
+    long long sum_ctx = 0;             // cached tokens visible to the pass, all sequences
 };
 
 int ensure_pages(s2d2_ctx* c, SeqState& s, int n_tokens) {
@@ -394,6 +398,7 @@ void begin_seq(s2d2_ctx* c, PassBuild& pb, const SeqState& s, int n_ctx) {
     PassMeta& pm = c->meta;
     int q = pb.n_seqs++;
     pb.max_ctx = std::max(pb.max_ctx, n_ctx);
+    pb.sum_ctx += n_ctx;
     pm.hp<int>(pm.off_nctx)[q] = n_ctx;
     pm.hp<int>(pm.off_row0)[q] = pb.n_rows;
     pm.hp<int>(pm.off_nrows)[q] = 0;
@@ -456,6 +461,15 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
     int nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, nq = m.n_q_heads * hd;
     CUDA_TRY(c, cudaMemcpyAsync(c->meta.d, c->meta.h, c->meta.bytes, cudaMemcpyHostToDevice, st));
     c->cnt.h2d_bytes += c->meta.bytes;
+    {   // the persistent kernel runs the whole pass when the shape allows it
+        bool taken = false;
+        int rc = pass_run(c, pv, pb.max_ctx, pb.max_rows, pb.sum_ctx, logits_out, &taken);
+        if (rc) return rc;
+        if (taken) {
+            CUDA_TRY(c, cudaGetLastError());
+            return S2D2_OK;
+        }
+    }
     embed_kernel<TW><<<M, 256, 0, st>>>((const TW*)c->embed, pv.row_token, c->h, d);
     LAUNCHED(c);
     KvPool<TKV> pool = make_pool<TKV>(c);
