@@ -142,30 +142,46 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
         for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
 
     // ---- Q tile: global -> swizzled shared -> A fragments ----
-    for (int i = tid; i < QT * CH; i += THREADS) {
-        int r = i / CH, c = i % CH;
-        int qv = q0 + r;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (qv < nq) {
-            int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
-            val = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+    {   // all loads first, then the stores: one round trip for the tile
+        constexpr int NQ = QT * CH / THREADS;
+        uint4 val[NQ];
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH, qv = q0 + r;
+            val[k] = make_uint4(0, 0, 0, 0);
+            if (qv < nq) {
+                int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
+                val[k] = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+            }
         }
-        *reinterpret_cast<uint4*>(q_s + sw_off(r, c, QT)) = val;
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            *reinterpret_cast<uint4*>(q_s + sw_off(r, c, QT)) = val[k];
+        }
     }
     if (in_pass) {
         // K and V of this pass's rows of the sequence into stage 0 (rows past nrows are zero)
         uint8_t* kd = kv_s;
         uint8_t* vd = kd + tile_bytes;
-        for (int i = tid; i < 64 * CH; i += THREADS) {
-            int r = i / CH, c = i % CH;
-            uint4 kk = make_uint4(0, 0, 0, 0), vv = kk;
+        constexpr int NK = 64 * CH / THREADS;
+        uint4 kk[NK], vv[NK];
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            kk[k] = make_uint4(0, 0, 0, 0);
+            vv[k] = kk[k];
             if (r < nrows) {
                 size_t o = ((size_t)(row0 + r) * p.Hkv + kvh) * HD + c * 8;
-                kk = ldcg16(p.k_rows + o);
-                vv = ldcg16(p.v_rows + o);
+                kk[k] = ldcg16(p.k_rows + o);
+                vv[k] = ldcg16(p.v_rows + o);
             }
-            *reinterpret_cast<uint4*>(kd + sw_off(r, c, 64)) = kk;
-            *reinterpret_cast<uint4*>(vd + sw_off(r, c, 64)) = vv;
+        }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            *reinterpret_cast<uint4*>(kd + sw_off(r, c, 64)) = kk[k];
+            *reinterpret_cast<uint4*>(vd + sw_off(r, c, 64)) = vv[k];
         }
     }
     group_sync(bar_id, THREADS);

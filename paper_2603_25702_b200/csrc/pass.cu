@@ -4,6 +4,8 @@
 
 #include <cuda.h>
 
+#include <stdlib.h>
+
 #include <algorithm>
 #include <vector>
 
@@ -28,6 +30,10 @@ struct PassState {
     int max_segs = 0;
     float *ssq_a = nullptr, *ssq_b = nullptr;
     unsigned* barrier = nullptr;
+    unsigned long long* trace = nullptr;
+    int trace_cap = 0;
+    int last_marks = 0;
+    int* parts[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // split-K part tables per GEMM kind
     double weight_bytes = 0;     // bytes of every matrix a pass streams (without the LM head)
     double head_bytes = 0;
 };
@@ -63,6 +69,7 @@ int pass_init(s2d2_ctx* c) {
     if (!coop || n_sms < 1) return S2D2_OK;
     s->grid = n_sms;
     s->max_smem = optin;
+
     if (stages_for(s, pp::MAX_T, hd) < 3) return S2D2_OK;
     cudaError_t e = hd == 128 ? prepare_kernel<128>(s, optin) : prepare_kernel<64>(s, optin);
     if (e != cudaSuccess) {
@@ -113,9 +120,40 @@ int pass_init(s2d2_ctx* c) {
     };
     s->max_segs = std::max({segs(nqkv, d), segs(d, nq), segs(2 * f, d), segs(d, f), segs(m.vocab, d)});
     size_t ws_floats = (size_t)G * s->max_segs * pp::MAX_T * 128;
+    // per GEMM kind and weight tile: the workspace slots of its split-K partials, in CTA order
+    // (the kernel cuts the tile-major (tile, k-block) units into G equal contiguous ranges)
+    {
+        const long long NK[5][2] = {{nqkv, d}, {d, nq}, {2LL * f, d}, {d, f}, {m.vocab, d}};
+        for (int k = 0; k < 5; ++k) {
+            const long long n_tiles = (NK[k][0] + 127) / 128, kbt = NK[k][1] / 64, U = n_tiles * kbt;
+            if (U * (long long)G >= (1LL << 40)) return S2D2_OK;
+            std::vector<int> tab((size_t)n_tiles * (1 + pp::MAX_PARTS), 0);
+            for (int cta = 0; cta < G; ++cta) {
+                const long long u0 = U * cta / G, u1 = U * (cta + 1) / G;
+                if (u1 <= u0) continue;
+                const long long first = u0 / kbt, last = (u1 - 1) / kbt;
+                for (long long t = first; t <= last; ++t) {
+                    int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
+                    if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
+                    tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs + (int)(t - first);
+                    ++cnt;
+                }
+            }
+            if (cudaMalloc((void**)&s->parts[k], tab.size() * 4) != cudaSuccess ||
+                cudaMemcpy(s->parts[k], tab.data(), tab.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+                c->err = "cudaMalloc failed for the persistent pass";
+                return S2D2_ERR_CUDA;
+            }
+        }
+    }
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
+    s->trace_cap = 2 * (10 * L + 2);
+    if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) {
+        c->err = "cudaMalloc failed for the persistent pass";
+        return S2D2_ERR_CUDA;
+    }
     if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
         cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
         cudaMalloc((void**)&s->ws, ws_floats * 4) != cudaSuccess || cudaMalloc((void**)&s->ssq_a, ssq_bytes) != cudaSuccess ||
@@ -141,7 +179,8 @@ int pass_init(s2d2_ctx* c) {
 void pass_destroy(s2d2_ctx* c) {
     PassState* s = state(c);
     if (!s) return;
-    void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier};
+    void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier, s->trace,
+                    s->parts[0], s->parts[1], s->parts[2], s->parts[3], s->parts[4]};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete s;
@@ -202,6 +241,10 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.barrier = s->barrier;
     p.status = c->d_status;
     p.S = stages_for(s, p.T, m.head_dim);
+    for (int k = 0; k < 5; ++k) p.parts[k] = s->parts[k];
+    p.trace = s->trace;
+    p.trace_cap = s->trace_cap;
+    s->last_marks = 2 * (10 * m.n_layers + 1 + (p.n_logit > 0 ? 1 : 0));
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, 4, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
     void* args[] = {&p};
@@ -222,5 +265,25 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     c->cnt.n_kernel_launches++;
     c->last_pass_rows = pv.n_rows;
     *taken = true;
+    return S2D2_OK;
+}
+
+int pass_copy_trace(s2d2_ctx* c, unsigned long long* out, long long cap, int* n_ctas, int* n_marks) {
+    PassState* s = state(c);
+    if (!s || !s->ok || s->last_marks == 0) {
+        c->err = "no persistent pass has run";
+        return S2D2_ERR_STATE;
+    }
+    if (cap < (long long)s->grid * s->last_marks) {
+        c->err = "trace buffer too small";
+        return S2D2_ERR_INVALID;
+    }
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
+    for (int g = 0; g < s->grid; ++g)
+        if (cudaMemcpy(out + (size_t)g * s->last_marks, s->trace + (size_t)g * s->trace_cap, (size_t)s->last_marks * 8,
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return S2D2_ERR_CUDA;
+    *n_ctas = s->grid;
+    *n_marks = s->last_marks;
     return S2D2_OK;
 }

@@ -10,3 +10,5 @@ void pass_destroy(s2d2_ctx* c);
 // sum_ctx: cached tokens visible to the pass, summed over its sequences (for byte accounting).
 int pass_run(s2d2_ctx* c, const s2d2::PassView& pv, int max_ctx, int max_rows, long long sum_ctx, float* logits_out,
              bool* taken);
+// Timestamps of the last persistent pass (see s2d2_debug_pass_trace).
+int pass_copy_trace(s2d2_ctx* c, unsigned long long* out, long long cap, int* n_ctas, int* n_marks);

@@ -46,6 +46,7 @@ constexpr int ACC_STRIDE = 64;       // tensor-memory columns per accumulator bu
 constexpr int MAX_T = 64;            // most token rows of a pass
 constexpr int W_TILE_BYTES = tc::BLOCK_N * 128;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
+constexpr int MAX_PARTS = 16;        // most split-K partials of one weight tile
 
 struct LayerGains {
     const float *attn_norm, *ffn_norm, *q_norm, *k_norm;
@@ -74,6 +75,9 @@ struct PassParams {
     unsigned* barrier;        // grid barrier counter, zero at launch
     int* status;
     int S;                    // ring stages
+    const int* parts[5];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
+    unsigned long long* trace;   // [grid][trace_cap] globaltimer at entry and exit of every grid barrier
+    int trace_cap;
 };
 
 __host__ __device__ inline size_t stage_bytes(int T) { return (size_t)W_TILE_BYTES + (size_t)T * 128; }
@@ -144,43 +148,88 @@ __device__ __forceinline__ bool wait_counter(const PassParams& p, unsigned targe
     return false;
 }
 
-// Sum of the split-K partials of (tile, row m, column n) in CTA order.
-struct TileParts {
-    int c_lo, c_hi;
-};
-__device__ __forceinline__ TileParts tile_parts(const GemmShape& g, int tile, int G) {
-    long long ua = (long long)tile * g.kbt, ub = ua + g.kbt - 1;
-    TileParts t;
-    int c = (int)(ua * G / g.U);
-    while (unit_begin(g.U, c + 1, G) <= ua) ++c;
-    t.c_lo = c;
-    c = (int)(ub * G / g.U);
-    while (unit_begin(g.U, c + 1, G) <= ub) ++c;
-    t.c_hi = c;
-    return t;
-}
-constexpr int RC = 8;   // rows handled together so that their loads are in flight at once
-// acc[j] = sum of the split-K partials of (tile, row rows[j], column n), parts in CTA order.
-__device__ __forceinline__ void tile_sum_rows(const PassParams& p, const GemmShape& g, const TileParts& tp, int tile, int G,
-                                              const int (&rows)[RC], int n, float (&acc)[RC]) {
-#pragma unroll
-    for (int j = 0; j < RC; ++j) acc[j] = 0.f;
-    for (int c = tp.c_lo; c <= tp.c_hi; ++c) {
-        long long b0 = unit_begin(g.U, c, G), b1 = unit_begin(g.U, c + 1, G);
-        if (b1 <= b0) continue;
-        int local = tile - (int)(b0 / g.kbt);
-        const float* part = p.ws + ((size_t)c * p.max_segs + local) * (size_t)p.T * tc::BLOCK_N + n;
-        float v[RC];
-#pragma unroll
-        for (int j = 0; j < RC; ++j) v[j] = __ldcg(part + (size_t)rows[j] * tc::BLOCK_N);
-#pragma unroll
-        for (int j = 0; j < RC; ++j) acc[j] += v[j];
+// Walks the weight tiles (unit by unit) that one CTA streams during a pass, in order.  The
+// per-unit step is two compares; divisions happen once per GEMM.
+struct UnitCursor {
+    int gi, n_gemms, cta, G;
+    int left, kb, tile, kbt, map_w;
+    __device__ __forceinline__ void open(const PassParams& p) {
+        while (gi < n_gemms) {
+            const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
+            const GemmShape g = gemm_shape(p, l, kind);
+            const long long u = unit_begin(g.U, cta, G), u1 = unit_begin(g.U, cta + 1, G);
+            if (u < u1) {
+                left = (int)(u1 - u);
+                tile = (int)(u / g.kbt);
+                kb = (int)(u - (long long)tile * g.kbt);
+                kbt = g.kbt;
+                map_w = g.map_w;
+                return;
+            }
+            ++gi;
+        }
     }
-}
-// rows m0 .. m0+RC-1, clamped to the last valid row (duplicates are computed and dropped)
-__device__ __forceinline__ void chunk_rows(int m0, int M, int (&rows)[RC]) {
+    __device__ __forceinline__ void init(const PassParams& p, int n_gemms_, int cta_, int G_) {
+        gi = 0;
+        n_gemms = n_gemms_;
+        cta = cta_;
+        G = G_;
+        open(p);
+    }
+    __device__ __forceinline__ bool done() const { return gi >= n_gemms; }
+    // current unit: weight map index, k-block and tile; then advance
+    __device__ __forceinline__ void next(const PassParams& p, int& map_w_, int& kb_, int& tile_) {
+        map_w_ = map_w;
+        kb_ = kb;
+        tile_ = tile;
+        if (--left == 0) {
+            ++gi;
+            open(p);
+        } else if (++kb == kbt) {
+            kb = 0;
+            ++tile;
+        }
+    }
+};
+// Sum over the split-K partials (in CTA order) of 4 consecutive columns of (tile, row): every
+// lane of a warp takes columns 4*lane .. 4*lane+3, all loads of the warp are issued together.
+__device__ __forceinline__ float4 tile_row_sum(const PassParams& p, int kind, int tile, int row, int lane) {
+    const int* tab = p.parts[kind] + (size_t)tile * (1 + MAX_PARTS);
+    const int mine = lane <= MAX_PARTS ? __ldg(tab + lane) : 0;
+    const int cnt = __shfl_sync(0xffffffffu, mine, 0);
+    float4 v[MAX_PARTS];
 #pragma unroll
-    for (int j = 0; j < RC; ++j) rows[j] = min(m0 + j, M - 1);
+    for (int j = 0; j < MAX_PARTS; ++j) {
+        const int slot = __shfl_sync(0xffffffffu, mine, j + 1);
+        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < cnt) v[j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row) * tc::BLOCK_N) + lane);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < MAX_PARTS; ++j) {
+        acc.x += v[j].x;
+        acc.y += v[j].y;
+        acc.z += v[j].z;
+        acc.w += v[j].w;
+    }
+    return acc;
+}
+// 1/rms of a row from the per-tile sums of squares of h, in two steps so that the loads of the
+// first are in flight together with whatever the caller loads next: lanes take the tiles.
+__device__ __forceinline__ float row_ssq_lane(const float* ssq, int d_tiles, int row, int lane) {
+    float s = 0.f;
+    for (int t = lane; t < d_tiles; t += 32) s += __ldcg(ssq + (size_t)t * MAX_T + row);
+    return s;
+}
+__device__ __forceinline__ float inv_rms_from(float lane_part, int d, float eps) {
+    return 1.0f / sqrtf(warp_sum(lane_part) / (float)d + eps);
+}
+__device__ __forceinline__ void store_bf16x4(bf16* dst, float a, float b, float c, float d) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst) = u;
 }
 
 template <int HD>
@@ -202,9 +251,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     volatile int* w_issued = abort_flag + 1;
     volatile int* x_issued = w_issued + 1;
     volatile int* consumed = x_issued + 1;
-    float* red = (float*)(misc + 512);        // [4][MAX_T]
-    float* inv_s = red + 4 * MAX_T;           // [MAX_T]
-    float* stage_f = (float*)attn_s;          // [MAX_T][128] staging of the QKV phase (aliases the attention tiles)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_gemms = p.n_layers * 4 + (p.n_logit > 0 ? 1 : 0);
@@ -239,23 +285,26 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             // ---------------- W producer: free-running over every GEMM of the pass ----------------
             uint64_t policy;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+            UnitCursor ld;
+            ld.init(p, n_gemms, cta, G);
             uint32_t i = 0;
             bool ok = true;
-            for (int gi = 0; gi < n_gemms && ok; ++gi) {
-                const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
-                const GemmShape g = gemm_shape(p, l, kind);
-                const CUtensorMap* mw = p.maps + g.map_w;
-                for_each_segment(g, cta, G, [&](int tile, int kb0, int kb1, int) {
-                    for (int kb = kb0; kb < kb1; ++kb, ++i) {
-                        int s = (int)(i % (uint32_t)S);
-                        if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) return ok = false;
-                        if (*abort_flag) return ok = false;
-                        tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
-                        tc::tma_load_2d_hint(ring + s * sbytes, mw, kb * tc::BLOCK_K, tile * tc::BLOCK_N, &full[s], policy);
-                        *w_issued = (int)i + 1;
-                    }
-                    return true;
-                });
+            while (!ld.done()) {
+                int mw, kb, tile;
+                ld.next(p, mw, kb, tile);
+                const int s = (int)(i % (uint32_t)S);
+                if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                if (*abort_flag) {
+                    ok = false;
+                    break;
+                }
+                tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
+                tc::tma_load_2d_hint(ring + s * sbytes, p.maps + mw, kb * tc::BLOCK_K, tile * tc::BLOCK_N, &full[s], policy);
+                *w_issued = (int)i + 1;
+                ++i;
             }
             if (!ok) {
                 atomicCAS(p.status, 0, 7);
@@ -346,12 +395,20 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             __threadfence();
             att::group_sync(BAR_COMPUTE, CTHREADS);
             if (tid == 0) {
+                const int k = 2 * (int)epoch - 2;
+                unsigned long long t0, t1;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
                 if (!wait_counter(p, epoch * (unsigned)G, abort_flag)) {
                     atomicCAS(p.status, 0, 5);
                     *abort_flag = 1;
                 }
                 __threadfence();
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+                if (p.trace && k + 1 < p.trace_cap) {
+                    p.trace[(size_t)cta * p.trace_cap + k] = t0;
+                    p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
+                }
             }
             att::group_sync(BAR_COMPUTE, CTHREADS);
             asm volatile("fence.proxy.async;" ::: "memory");
@@ -384,62 +441,43 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 *abort_flag = 1;
             }
         };
-        // 1/rms of every row from the per-tile sums of squares
-        auto compute_inv = [&](const float* ssq) {
-            if (tid < M) {
-                float s = 0.f;
-#pragma unroll 8
-                for (int t = 0; t < d_tiles; ++t) s += __ldcg(ssq + (size_t)t * MAX_T + tid);
-                inv_s[tid] = 1.0f / sqrtf(s / (float)d + p.eps);
+        // The element-wise phases work warp by warp on (tile, row) pairs: 128 output columns of one
+        // row, 4 per lane.  A pair's loads (its partials, its residual row, the sums of squares) are
+        // all in flight together, so a phase costs about one round trip to L2.
+        const int gw = cta * 4 + cw, GW = G * 4;
+
+        // h update shared by the embedding and the two residual phases: writes h, the next GEMM's
+        // input bf16(h * gain) and the (tile, row) sum of squares
+        auto h_phase = [&](const float* gain, float* ssq, auto&& value) {
+            for (int pair = gw; pair < d_tiles * M; pair += GW) {
+                const int t = pair / M, m = pair % M;
+                const int col = t * tc::BLOCK_N + 4 * lane;
+                const float4 gn = *reinterpret_cast<const float4*>(gain + col);
+                const float4 x = value(t, m, col);
+                *reinterpret_cast<float4*>(p.h + (size_t)m * d + col) = x;
+                store_bf16x4(p.xn + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
+                const float sq = warp_sum(x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w);
+                if (lane == 0) ssq[(size_t)t * MAX_T + m] = sq;
             }
-            att::group_sync(BAR_COMPUTE, CTHREADS);
         };
-        // h tile update shared by the embedding and the two residual phases: value(rows, x) gives the
-        // new h of RC rows of this thread's column; writes h, the next GEMM's input bf16(h * gain)
-        // and the tile's per-row sums of squares
-        auto h_tile = [&](int t, const float* gain, float* ssq, auto&& value) {
-            const int col = t * tc::BLOCK_N + tid;
-            const float gn = gain[col];
-            for (int m0 = 0; m0 < M; m0 += RC) {
-                int rows[RC];
-                chunk_rows(m0, M, rows);
-                float x[RC];
-                value(rows, col, x);
-#pragma unroll
-                for (int j = 0; j < RC; ++j) {
-                    if (m0 + j < M) {
-                        p.h[(size_t)rows[j] * d + col] = x[j];
-                        p.xn[(size_t)rows[j] * d + col] = __float2bfloat16_rn(x[j] * gn);
-                    }
-                    float sq = warp_sum(x[j] * x[j]);
-                    if (lane == 0 && m0 + j < M) red[cw * MAX_T + m0 + j] = sq;
-                }
-            }
-            att::group_sync(BAR_COMPUTE, CTHREADS);
-            if (tid < M) ssq[(size_t)t * MAX_T + tid] = red[tid] + red[MAX_T + tid] + red[2 * MAX_T + tid] + red[3 * MAX_T + tid];
-            att::group_sync(BAR_COMPUTE, CTHREADS);
-        };
-        auto residual_phase = [&](int l, int kind, const float* gain, float* ssq) {
-            const GemmShape g = gemm_shape(p, l, kind);
-            for (int t = cta; t < d_tiles; t += G) {
-                const TileParts tp = tile_parts(g, t, G);
-                h_tile(t, gain, ssq, [&](const int (&rows)[RC], int col, float (&x)[RC]) {
-                    float hv[RC];
-#pragma unroll
-                    for (int j = 0; j < RC; ++j) hv[j] = __ldcg(p.h + (size_t)rows[j] * d + col);
-                    tile_sum_rows(p, g, tp, t, G, rows, tid, x);
-#pragma unroll
-                    for (int j = 0; j < RC; ++j) x[j] += hv[j];
-                });
-            }
+        auto residual_phase = [&](int kind, const float* gain, float* ssq) {
+            h_phase(gain, ssq, [&](int t, int m, int col) {
+                const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
+                float4 x = tile_row_sum(p, kind, t, m, lane);
+                x.x += hv.x;
+                x.y += hv.y;
+                x.z += hv.z;
+                x.w += hv.w;
+                return x;
+            });
         };
 
         // ---- embedding ----
-        for (int t = cta; t < d_tiles; t += G)
-            h_tile(t, p.gains[0].attn_norm, p.ssq_a, [&](const int (&rows)[RC], int col, float (&x)[RC]) {
-#pragma unroll
-                for (int j = 0; j < RC; ++j) x[j] = __bfloat162float(p.embed[(size_t)p.pv.row_token[rows[j]] * d + col]);
-            });
+        h_phase(p.gains[0].attn_norm, p.ssq_a, [&](int, int m, int col) {
+            const uint2 u = *reinterpret_cast<const uint2*>(p.embed + (size_t)p.pv.row_token[m] * d + col);
+            const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&u.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&u.y);
+            return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+        });
         grid_sync();
 
         for (int l = 0; l < p.n_layers && ok; ++l) {
@@ -449,74 +487,57 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (!ok) break;
             grid_sync();
             if (!ok) break;
-            // ---- 1/rms, q/k norm, RoPE, K/V write ----
-            compute_inv(p.ssq_a);
+            // ---- 1/rms, q/k norm, RoPE, K/V write: one warp per (128-column tile, row) ----
             {
-                const GemmShape g = gemm_shape(p, l, 0);
-                constexpr int HIT = tc::BLOCK_N / HD;      // heads per tile
-                constexpr int E = HD / 32, half = HD / 2;
-                for (int t = cta; t < g.n_tiles; t += G) {
-                    const TileParts tp = tile_parts(g, t, G);
-                    for (int m0 = 0; m0 < M; m0 += RC) {
-                        int rows[RC];
-                        chunk_rows(m0, M, rows);
-                        float x[RC];
-                        tile_sum_rows(p, g, tp, t, G, rows, tid, x);
+                constexpr int half = HD / 2, PART = half / 4;     // PART: lane distance of a RoPE pair
+                const int n_tiles = (p.Hq + 2 * p.Hkv) * HD / tc::BLOCK_N;
+                for (int pair = gw; pair < n_tiles * M; pair += GW) {
+                    const int t = pair / M, m = pair % M;
+                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
+                    float4 s4 = tile_row_sum(p, 0, t, m, lane);
+                    const float inv = inv_rms_from(sq_l, d, p.eps);
+                    float x[4] = {inv * s4.x, inv * s4.y, inv * s4.z, inv * s4.w};
+                    const int c_tile = 4 * lane;                    // column inside the tile
+                    const int head = (t * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
+                    const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
+                    const int pos = p.pv.row_pos[m];
+                    if (p.qk_norm) {
+                        float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
 #pragma unroll
-                        for (int j = 0; j < RC; ++j)
-                            if (m0 + j < M) stage_f[(m0 + j) * tc::BLOCK_N + tid] = inv_s[m0 + j] * x[j];
-                    }
-                    att::group_sync(BAR_COMPUTE, CTHREADS);
-                    for (int pair = cw; pair < M * HIT; pair += 4) {
-                        const int m = pair / HIT, head = t * HIT + pair % HIT;
-                        const float* src = stage_f + m * tc::BLOCK_N + (pair % HIT) * HD;
-                        float x[E];
-#pragma unroll
-                        for (int e = 0; e < E; ++e) x[e] = src[lane + 32 * e];
-                        const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
-                        const int pos = p.pv.row_pos[m];
+                        for (int o = HD / 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);   // over the head's lanes
                         if (is_q || is_k) {
-                            if (p.qk_norm) {
-                                float ss = 0.f;
-#pragma unroll
-                                for (int e = 0; e < E; ++e) ss += x[e] * x[e];
-                                ss = warp_sum(ss);
-                                const float inv = 1.0f / sqrtf(ss / (float)HD + p.eps);
-                                const float* gq = is_q ? lg.q_norm : lg.k_norm;
-#pragma unroll
-                                for (int e = 0; e < E; ++e) x[e] = x[e] * inv * gq[lane + 32 * e];
-                            }
-#pragma unroll
-                            for (int e = 0; e < E / 2; ++e) {
-                                const int i = lane + 32 * e;
-                                const float c = p.rope_cos[(size_t)pos * half + i], s = p.rope_sin[(size_t)pos * half + i];
-                                const float x1 = x[e], x2 = x[e + E / 2];
-                                x[e] = x1 * c - x2 * s;
-                                x[e + E / 2] = x2 * c + x1 * s;
-                            }
-                        }
-                        if (is_q) {
-                            bf16* dst = p.q + ((size_t)m * p.Hq + head) * HD;
-#pragma unroll
-                            for (int e = 0; e < E; ++e) dst[lane + 32 * e] = __float2bfloat16_rn(x[e]);
-                        } else {
-                            const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
-                            bf16* dst = (is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD;
-                            bf16* cdst = nullptr;
-                            if (p.pv.row_flags[m] & ROW_WRITE_KV) {
-                                const int sq = p.pv.row_seq[m];
-                                const int page = p.pv.seq_pages[(size_t)sq * p.pv.max_pages + (pos >> p.pool.page_shift)];
-                                cdst = p.pool.ptr(l, page, is_k ? 0 : 1, kvh, pos & (p.pool.page_tokens - 1));
-                            }
-#pragma unroll
-                            for (int e = 0; e < E; ++e) {
-                                const bf16 v = __float2bfloat16_rn(x[e]);
-                                dst[lane + 32 * e] = v;
-                                if (cdst) cdst[lane + 32 * e] = v;
-                            }
+                            const float hinv = 1.0f / sqrtf(ss / (float)HD + p.eps);
+                            const float4 gq = *reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch);
+                            x[0] *= hinv * gq.x;
+                            x[1] *= hinv * gq.y;
+                            x[2] *= hinv * gq.z;
+                            x[3] *= hinv * gq.w;
                         }
                     }
-                    att::group_sync(BAR_COMPUTE, CTHREADS);
+                    {   // rotate-half RoPE: element i of the first half pairs with i + half
+                        const bool second = ch >= half;
+                        const int i0 = ch - (second ? half : 0);
+                        const float4 cs = *reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * half + i0);
+                        const float4 sn = *reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * half + i0);
+                        const float c4[4] = {cs.x, cs.y, cs.z, cs.w}, s4r[4] = {sn.x, sn.y, sn.z, sn.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float other = __shfl_xor_sync(0xffffffffu, x[e], PART);
+                            const float y = second ? x[e] * c4[e] + other * s4r[e] : x[e] * c4[e] - other * s4r[e];
+                            if (is_q || is_k) x[e] = y;
+                        }
+                    }
+                    if (is_q) {
+                        store_bf16x4(p.q + ((size_t)m * p.Hq + head) * HD + ch, x[0], x[1], x[2], x[3]);
+                    } else {
+                        const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+                        store_bf16x4((is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD + ch, x[0], x[1], x[2], x[3]);
+                        if (p.pv.row_flags[m] & ROW_WRITE_KV) {
+                            const int sq = p.pv.row_seq[m];
+                            const int page = p.pv.seq_pages[(size_t)sq * p.pv.max_pages + (pos >> p.pool.page_shift)];
+                            store_bf16x4(p.pool.ptr(l, page, is_k ? 0 : 1, kvh, pos & (p.pool.page_tokens - 1)) + ch, x[0], x[1], x[2], x[3]);
+                        }
+                    }
                 }
             }
             grid_sync();
@@ -527,9 +548,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 ap.layer = l;
                 const int n_splits = ap.n_cache_splits + 1;
                 const int total = ap.pv.n_seqs * ap.Hkv * ap.n_qtiles * n_splits;
-                // plain stores of the previous phases into the tile region precede TMA writes
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                att::group_sync(BAR_COMPUTE, CTHREADS);
                 for (int idx = cta; idx < total && ok; idx += G) {
                     const int split = idx % n_splits, r = idx / n_splits;
                     if (!att::attn_item<HD>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
@@ -542,7 +560,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 grid_sync();
                 if (!ok) break;
                 // ---- combine the key splits of every (row, query head) ----
-                for (int pair = cta * 4 + cw; pair < M * p.Hq; pair += G * 4) {
+                for (int pair = gw; pair < M * p.Hq; pair += GW) {
                     const int r = pair / p.Hq, hq = pair % p.Hq;
                     const int seq = p.pv.row_seq[r], kvh = hq / ap.group;
                     const int qv = (r - p.pv.seq_row0[seq]) * ap.group + hq % ap.group;
@@ -551,6 +569,9 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     const int n_pages = (n_ctx + ap.page_tokens - 1) >> ap.page_shift;
                     const size_t item0 = ((size_t)(seq * ap.Hkv + kvh) * ap.n_qtiles + qt) * n_splits;
                     // lanes take the splits for the maxima and weights, then the columns for the sums
+                    float acc[HD / 32], lsum = 0.f;
+#pragma unroll
+                    for (int e = 0; e < HD / 32; ++e) acc[e] = 0.f;
                     float mx = -INFINITY;
                     for (int s0 = 0; s0 < n_splits; s0 += 32) {
                         const int s = s0 + lane;
@@ -558,31 +579,30 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const float ms = used ? __ldcg(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2) : -INFINITY;
                         mx = fmaxf(mx, warp_max(ms));
                     }
-                    float acc[HD / 32], lsum = 0.f;
-#pragma unroll
-                    for (int e = 0; e < HD / 32; ++e) acc[e] = 0.f;
                     for (int s0 = 0; s0 < n_splits; s0 += 32) {
                         const int s = s0 + lane;
                         const bool used = s < n_splits && (s == ap.n_cache_splits || s * ap.pages_per_split < n_pages);
-                        float w_l = 0.f, l_l = 0.f;
-                        if (used) {
-                            const float ms = __ldcg(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2);
-                            if (ms != -INFINITY) {
-                                w_l = exp2f(ms - mx);
-                                l_l = __ldcg(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2 + 1);
-                            }
-                        }
+                        float2 ml = make_float2(-INFINITY, 0.f);
+                        if (used) ml = __ldcg(reinterpret_cast<const float2*>(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2));
+                        const float w_l = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
                         const int cnt = min(32, n_splits - s0);
-#pragma unroll 4
-                        for (int k = 0; k < cnt; ++k) {
-                            const float w = __shfl_sync(0xffffffffu, w_l, k);
-                            lsum += w * __shfl_sync(0xffffffffu, l_l, k);
-                            const float* po = ap.part_o + ((item0 + s0 + k) * att::QT + qi) * HD + lane;
+                        for (int k0 = 0; k0 < cnt; k0 += 8) {
+                            float v[8][HD / 32], w[8];
 #pragma unroll
-                            for (int e = 0; e < HD / 32; ++e) {
-                                const float v = w != 0.f ? __ldcg(po + 32 * e) : 0.f;
-                                acc[e] += w * v;
+                            for (int k = 0; k < 8; ++k) {
+                                w[k] = __shfl_sync(0xffffffffu, w_l, (k0 + k) & 31);
+                                const float lk = __shfl_sync(0xffffffffu, ml.y, (k0 + k) & 31);
+                                const bool on = k0 + k < cnt && w[k] != 0.f;
+                                if (!on) w[k] = 0.f;
+                                lsum += w[k] * lk;
+                                const float* po = ap.part_o + ((item0 + s0 + k0 + k) * att::QT + qi) * HD + lane;
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e) v[k][e] = on ? __ldcg(po + 32 * e) : 0.f;
                             }
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                                for (int e = 0; e < HD / 32; ++e) acc[e] += w[k] * v[k][e];
                         }
                     }
 #pragma unroll
@@ -597,7 +617,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (!ok) break;
             grid_sync();
             if (!ok) break;
-            residual_phase(l, 1, lg.ffn_norm, p.ssq_b);
+            residual_phase(1, lg.ffn_norm, p.ssq_b);
             grid_sync();
             if (!ok) break;
             // ---- gate/up GEMM, SwiGLU ----
@@ -605,25 +625,19 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (!ok) break;
             grid_sync();
             if (!ok) break;
-            compute_inv(p.ssq_b);
             {
-                const GemmShape g = gemm_shape(p, l, 2);
                 const int f_tiles = p.f / tc::BLOCK_N;
-                for (int t = cta; t < f_tiles; t += G) {
-                    const TileParts tg = tile_parts(g, t, G), tu = tile_parts(g, t + f_tiles, G);
-                    for (int m0 = 0; m0 < M; m0 += RC) {
-                        int rows[RC];
-                        chunk_rows(m0, M, rows);
-                        float gs[RC], us[RC];
-                        tile_sum_rows(p, g, tg, t, G, rows, tid, gs);
-                        tile_sum_rows(p, g, tu, t + f_tiles, G, rows, tid, us);
+                for (int pair = gw; pair < f_tiles * M; pair += GW) {
+                    const int t = pair / M, m = pair % M;
+                    const float sq_l = row_ssq_lane(p.ssq_b, d_tiles, m, lane);
+                    const float4 g4 = tile_row_sum(p, 2, t, m, lane), u4 = tile_row_sum(p, 2, t + f_tiles, m, lane);
+                    const float inv = inv_rms_from(sq_l, d, p.eps);
+                    const float gv[4] = {inv * g4.x, inv * g4.y, inv * g4.z, inv * g4.w};
+                    const float uv[4] = {inv * u4.x, inv * u4.y, inv * u4.z, inv * u4.w};
+                    float a[4];
 #pragma unroll
-                        for (int j = 0; j < RC; ++j) {
-                            if (m0 + j >= M) continue;
-                            const float gv = inv_s[m0 + j] * gs[j], uv = inv_s[m0 + j] * us[j];
-                            p.act[(size_t)(m0 + j) * p.f + t * tc::BLOCK_N + tid] = __float2bfloat16_rn(gv / (1.f + expf(-gv)) * uv);
-                        }
-                    }
+                    for (int e = 0; e < 4; ++e) a[e] = gv[e] / (1.f + expf(-gv[e])) * uv[e];
+                    store_bf16x4(p.act + (size_t)m * p.f + t * tc::BLOCK_N + 4 * lane, a[0], a[1], a[2], a[3]);
                 }
             }
             grid_sync();
@@ -633,7 +647,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (!ok) break;
             grid_sync();
             if (!ok) break;
-            residual_phase(l, 3, l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm, p.ssq_a);
+            residual_phase(3, l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm, p.ssq_a);
             grid_sync();
         }
         if (ok && p.n_logit > 0) {
@@ -641,21 +655,23 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             drain(p.n_layers, 4);
             if (ok) grid_sync();
             if (ok) {
-                compute_inv(p.ssq_a);
-                const GemmShape g = gemm_shape(p, p.n_layers, 4);
-                for (int t = cta; t < g.n_tiles; t += G) {
-                    const TileParts tp = tile_parts(g, t, G);
-                    const int col = t * tc::BLOCK_N + tid;
-                    for (int r0 = 0; r0 < p.n_logit; r0 += RC) {
-                        int rows[RC];
+                const int n_tiles = (p.V + tc::BLOCK_N - 1) / tc::BLOCK_N;
+                const bool vec = (p.V & 3) == 0;
+                for (int pair = gw; pair < n_tiles * p.n_logit; pair += GW) {
+                    const int t = pair / p.n_logit, lr = pair % p.n_logit;
+                    const int m = p.pv.logit_rows[lr];
+                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
+                    const float4 s4 = tile_row_sum(p, 4, t, m, lane);
+                    const float sc = p.logit_scale * inv_rms_from(sq_l, d, p.eps);
+                    const int col = t * tc::BLOCK_N + 4 * lane;
+                    float* dst = p.logits + (size_t)lr * p.V + col;
+                    if (vec && col + 3 < p.V) {
+                        *reinterpret_cast<float4*>(dst) = make_float4(sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w);
+                    } else {
+                        const float o[4] = {sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w};
 #pragma unroll
-                        for (int j = 0; j < RC; ++j) rows[j] = p.pv.logit_rows[min(r0 + j, p.n_logit - 1)];
-                        float x[RC];
-                        tile_sum_rows(p, g, tp, t, G, rows, tid, x);
-#pragma unroll
-                        for (int j = 0; j < RC; ++j)
-                            if (r0 + j < p.n_logit && col < p.V)
-                                p.logits[(size_t)(r0 + j) * p.V + col] = p.logit_scale * inv_s[rows[j]] * x[j];
+                        for (int e = 0; e < 4; ++e)
+                            if (col + e < p.V) dst[e] = o[e];
                     }
                 }
             }

@@ -1192,3 +1192,8 @@ extern "C" int s2d2_debug_copy_expert_ids(s2d2_ctx* c, int32_t* out, int64_t cap
     *n_rows = M;
     return S2D2_OK;
 }
+
+extern "C" int s2d2_debug_pass_trace(s2d2_ctx* c, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks) {
+    if (!c || !out || !n_ctas || !n_marks) return S2D2_ERR_INVALID;
+    return pass_copy_trace(c, (unsigned long long*)out, cap, n_ctas, n_marks);
+}
