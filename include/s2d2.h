@@ -250,12 +250,13 @@ int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int3
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);
 
-/* Phase timeline of the last pass that ran as the persistent kernel: for every CTA, the GPU
- * global timer (ns) at entry to and exit from each of its grid barriers, out[cta * n_marks + 2*b]
- * and [.. + 2*b + 1] for barrier b.  Barrier 0 follows the embedding; per layer the barriers
- * follow, in order, the QKV GEMM, q/k-norm+RoPE+K/V write, attention, its combine, the O GEMM,
- * the residual add, the gate/up GEMM, SwiGLU, the down GEMM and the residual add; a last one
- * follows the LM head when the pass had logit rows.  S2D2_ERR_STATE if no such pass has run. */
+/* Phase timeline of the last pass that ran as the persistent kernel: for every CTA, a row of
+ * n_marks + 1 values: the GPU global timer (ns) at entry to and exit from each of its grid
+ * barriers, out[cta * (n_marks + 1) + 2*b] and [.. + 2*b + 1] for barrier b, then the id of the
+ * SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
+ * QKV GEMM + q/k-norm + RoPE + K/V write, attention, its combine, O GEMM + residual add,
+ * gate/up GEMM + SwiGLU, down GEMM + residual add.  Marks are recorded only while
+ * s2d2_set_profiling is on.  S2D2_ERR_STATE if no such pass has run. */
 int s2d2_debug_pass_trace(s2d2_ctx* ctx, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks);
 
 /* y[M, N] = x[M, K] w[N, K]^T on device buffers, without any allocation.

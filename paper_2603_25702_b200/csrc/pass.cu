@@ -29,7 +29,9 @@ struct PassState {
     float* ws = nullptr;
     int max_segs = 0;
     float *ssq_a = nullptr, *ssq_b = nullptr;
-    unsigned* barrier = nullptr;
+    unsigned* barrier = nullptr;     // [64 | tile counters of the 5 GEMM kinds], zeroed before every launch
+    size_t sync_bytes = 0;
+    size_t cnt_off[5] = {0, 0, 0, 0, 0};
     unsigned long long* trace = nullptr;
     int trace_cap = 0;
     int last_marks = 0;
@@ -120,6 +122,19 @@ int pass_init(s2d2_ctx* c) {
     };
     s->max_segs = std::max({segs(nqkv, d), segs(d, nq), segs(2 * f, d), segs(d, f), segs(m.vocab, d)});
     size_t ws_floats = (size_t)G * s->max_segs * pp::MAX_T * 128;
+    {
+        const long long Ns[5] = {nqkv, d, 2LL * f, d, m.vocab};
+        size_t o = 64;
+        for (int k = 0; k < 5; ++k) {
+            s->cnt_off[k] = o;
+            o += (size_t)((Ns[k] + 127) / 128);
+        }
+        s->sync_bytes = o * 4;
+        if (cudaMalloc((void**)&s->barrier, s->sync_bytes) != cudaSuccess) {
+            c->err = "cudaMalloc failed for the persistent pass";
+            return S2D2_ERR_CUDA;
+        }
+    }
     // per GEMM kind and weight tile: the workspace slots of its split-K partials, in CTA order
     // (the kernel cuts the tile-major (tile, k-block) units into G equal contiguous ranges)
     {
@@ -149,7 +164,7 @@ int pass_init(s2d2_ctx* c) {
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
-    s->trace_cap = 2 * (10 * L + 2);
+    s->trace_cap = 2 * (6 * L + 1) + 1;      // two marks per grid barrier + the SM id
     if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) {
         c->err = "cudaMalloc failed for the persistent pass";
         return S2D2_ERR_CUDA;
@@ -157,7 +172,7 @@ int pass_init(s2d2_ctx* c) {
     if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
         cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
         cudaMalloc((void**)&s->ws, ws_floats * 4) != cudaSuccess || cudaMalloc((void**)&s->ssq_a, ssq_bytes) != cudaSuccess ||
-        cudaMalloc((void**)&s->ssq_b, ssq_bytes) != cudaSuccess || cudaMalloc((void**)&s->barrier, 256) != cudaSuccess) {
+        cudaMalloc((void**)&s->ssq_b, ssq_bytes) != cudaSuccess) {
         c->err = "cudaMalloc failed for the persistent pass";
         return S2D2_ERR_CUDA;
     }
@@ -242,11 +257,12 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.status = c->d_status;
     p.S = stages_for(s, p.T, m.head_dim);
     for (int k = 0; k < 5; ++k) p.parts[k] = s->parts[k];
-    p.trace = s->trace;
+    p.trace = c->profiling ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    s->last_marks = 2 * (10 * m.n_layers + 1 + (p.n_logit > 0 ? 1 : 0));
+    if (c->profiling) s->last_marks = 2 * (6 * m.n_layers + 1);
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
-    if (cudaMemsetAsync(s->barrier, 0, 4, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
+    if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
+    for (int k = 0; k < 5; ++k) p.tile_cnt[k] = s->barrier + s->cnt_off[k];
     void* args[] = {&p};
     gemm_prof_begin(c);
     cudaError_t e = m.head_dim == 128
@@ -274,13 +290,16 @@ int pass_copy_trace(s2d2_ctx* c, unsigned long long* out, long long cap, int* n_
         c->err = "no persistent pass has run";
         return S2D2_ERR_STATE;
     }
-    if (cap < (long long)s->grid * s->last_marks) {
+    if (cap < (long long)s->grid * (s->last_marks + 1)) {
         c->err = "trace buffer too small";
         return S2D2_ERR_INVALID;
     }
     if (cudaStreamSynchronize(c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
+    const size_t row = (size_t)s->last_marks + 1;
     for (int g = 0; g < s->grid; ++g)
-        if (cudaMemcpy(out + (size_t)g * s->last_marks, s->trace + (size_t)g * s->trace_cap, (size_t)s->last_marks * 8,
+        if (cudaMemcpy(out + g * row, s->trace + (size_t)g * s->trace_cap, (size_t)s->last_marks * 8, cudaMemcpyDeviceToHost) !=
+                cudaSuccess ||
+            cudaMemcpy(out + g * row + s->last_marks, s->trace + (size_t)g * s->trace_cap + s->trace_cap - 1, 8,
                        cudaMemcpyDeviceToHost) != cudaSuccess)
             return S2D2_ERR_CUDA;
     *n_ctas = s->grid;

@@ -73,6 +73,7 @@ struct PassParams {
     int map_xn, map_attn, map_act, map_kv;
     att::AttnParams ap;       // attention geometry of this pass (layer filled in per layer)
     unsigned* barrier;        // grid barrier counter, zero at launch
+    unsigned* tile_cnt[5];    // per GEMM kind and weight tile: partials published so far (zero at launch)
     int* status;
     int S;                    // ring stages
     const int* parts[5];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
@@ -110,8 +111,8 @@ __device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int 
 }
 // Grid barriers passed before the inputs of a GEMM are published.
 __device__ __forceinline__ unsigned gemm_epoch(const PassParams& p, int l, int kind) {
-    const unsigned off[5] = {1u, 5u, 7u, 9u, 1u};
-    return off[kind] + 10u * (unsigned)(kind == 4 ? p.n_layers : l);
+    const unsigned off[5] = {1u, 4u, 5u, 6u, 1u};
+    return off[kind] + 6u * (unsigned)(kind == 4 ? p.n_layers : l);
 }
 __device__ __forceinline__ long long unit_begin(long long U, int c, int G) { return U * c / G; }
 
@@ -192,25 +193,49 @@ struct UnitCursor {
     }
 };
 // Sum over the split-K partials (in CTA order) of 4 consecutive columns of (tile, row): every
-// lane of a warp takes columns 4*lane .. 4*lane+3, all loads of the warp are issued together.
-__device__ __forceinline__ float4 tile_row_sum(const PassParams& p, int kind, int tile, int row, int lane) {
-    const int* tab = p.parts[kind] + (size_t)tile * (1 + MAX_PARTS);
-    const int mine = lane <= MAX_PARTS ? __ldg(tab + lane) : 0;
-    const int cnt = __shfl_sync(0xffffffffu, mine, 0);
-    float4 v[MAX_PARTS];
-#pragma unroll
-    for (int j = 0; j < MAX_PARTS; ++j) {
-        const int slot = __shfl_sync(0xffffffffu, mine, j + 1);
-        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < cnt) v[j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row) * tc::BLOCK_N) + lane);
-    }
+// lane of a warp takes columns 4*lane .. 4*lane+3; the loads of up to PCH parts are in flight
+// together.  tile_row_tab fetches the tile's slot list (one entry per lane) ahead of time.
+constexpr int PCH = 8;
+__device__ __forceinline__ int tile_row_tab(const PassParams& p, int kind, int tile, int lane) {
+    return lane <= MAX_PARTS ? __ldg(p.parts[kind] + (size_t)tile * (1 + MAX_PARTS) + lane) : 0;
+}
+// Before reading, the warp waits (bounded) until all `cnt * round` partials of the tile have been
+// published by the CTAs that drained them (round = layer + 1: the counters only grow).
+__device__ __forceinline__ float4 tile_row_sum(const PassParams& p, int tab_lane, int row, int lane, const unsigned* published,
+                                               unsigned round, volatile int* abort_flag) {
+    const int cnt = __shfl_sync(0xffffffffu, tab_lane, 0);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    {
+        const unsigned target = (unsigned)cnt * round;
+        bool ready = false;
+        for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+            if (ld_acquire(published) >= target) {
+                ready = true;
+                break;
+            }
+            if ((it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
+        }
+        if (!ready) {
+            atomicCAS(p.status, 0, 8);
+            *abort_flag = 1;
+            return acc;
+        }
+    }
+    for (int j0 = 0; j0 < cnt; j0 += PCH) {
+        float4 v[PCH];
 #pragma unroll
-    for (int j = 0; j < MAX_PARTS; ++j) {
-        acc.x += v[j].x;
-        acc.y += v[j].y;
-        acc.z += v[j].z;
-        acc.w += v[j].w;
+        for (int j = 0; j < PCH; ++j) {
+            const int slot = __shfl_sync(0xffffffffu, tab_lane, (j0 + j + 1) & 31);
+            v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j0 + j < cnt) v[j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row) * tc::BLOCK_N) + lane);
+        }
+#pragma unroll
+        for (int j = 0; j < PCH; ++j) {
+            acc.x += v[j].x;
+            acc.y += v[j].y;
+            acc.z += v[j].z;
+            acc.w += v[j].w;
+        }
     }
     return acc;
 }
@@ -389,35 +414,36 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         const int M = p.M, d = p.d;
         const int d_tiles = d / tc::BLOCK_N;
 
-        auto grid_sync = [&]() {
+        // Grid barrier.  tma_out: this phase wrote data that other CTAs read through TMA (GEMM
+        // inputs, K/V pages), which needs the generic-to-async proxy fence on the writer side.
+        // One thread publishes for the CTA: its release covers the writes the CTA barrier ordered
+        // before it.
+        auto grid_sync = [&](bool tma_out) {
             ++epoch;
-            asm volatile("fence.proxy.async;" ::: "memory");
-            __threadfence();
+            if (tma_out) asm volatile("fence.proxy.async;" ::: "memory");
             att::group_sync(BAR_COMPUTE, CTHREADS);
             if (tid == 0) {
                 const int k = 2 * (int)epoch - 2;
-                unsigned long long t0, t1;
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+                unsigned long long t0 = 0, t1 = 0;
+                if (p.trace) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
                 if (!wait_counter(p, epoch * (unsigned)G, abort_flag)) {
                     atomicCAS(p.status, 0, 5);
                     *abort_flag = 1;
                 }
-                __threadfence();
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                if (p.trace && k + 1 < p.trace_cap) {
+                if (p.trace && k + 1 < p.trace_cap - 1) {
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
                     p.trace[(size_t)cta * p.trace_cap + k] = t0;
                     p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
                 }
             }
             att::group_sync(BAR_COMPUTE, CTHREADS);
-            asm volatile("fence.proxy.async;" ::: "memory");
             if (*abort_flag) ok = false;
         };
         // accumulators of this CTA's segments of one GEMM -> split-K partials
         auto drain = [&](int l, int kind) {
             const GemmShape g = gemm_shape(p, l, kind);
-            for_each_segment(g, cta, G, [&](int, int, int, int local) {
+            for_each_segment(g, cta, G, [&](int tile, int, int, int local) {
                 const uint32_t b = seg & 1u;
                 if (!tc::mbar_wait(&acc_full[b], (seg >> 1) & 1, abort_flag)) return ok = false;
                 tc::tc_fence_after();
@@ -433,6 +459,9 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[b]);
+                // publish: every thread's part of the partial is stored, then one release for the CTA
+                att::group_sync(BAR_COMPUTE, CTHREADS);
+                if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.tile_cnt[kind] + tile) : "memory");
                 ++seg;
                 return true;
             });
@@ -460,10 +489,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 if (lane == 0) ssq[(size_t)t * MAX_T + m] = sq;
             }
         };
-        auto residual_phase = [&](int kind, const float* gain, float* ssq) {
+        auto residual_phase = [&](int kind, unsigned round, const float* gain, float* ssq) {
             h_phase(gain, ssq, [&](int t, int m, int col) {
+                const int tab = tile_row_tab(p, kind, t, lane);
                 const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
-                float4 x = tile_row_sum(p, kind, t, m, lane);
+                float4 x = tile_row_sum(p, tab, m, lane, p.tile_cnt[kind] + t, round, abort_flag);
                 x.x += hv.x;
                 x.y += hv.y;
                 x.z += hv.z;
@@ -472,20 +502,23 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             });
         };
 
+        if (tid == 0 && p.trace) {
+            unsigned smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            p.trace[(size_t)cta * p.trace_cap + p.trace_cap - 1] = smid;
+        }
         // ---- embedding ----
         h_phase(p.gains[0].attn_norm, p.ssq_a, [&](int, int m, int col) {
             const uint2 u = *reinterpret_cast<const uint2*>(p.embed + (size_t)p.pv.row_token[m] * d + col);
             const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&u.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&u.y);
             return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
         });
-        grid_sync();
+        grid_sync(true);
 
         for (int l = 0; l < p.n_layers && ok; ++l) {
             const LayerGains lg = p.gains[l];
             // ---- QKV GEMM ----
             drain(l, 0);
-            if (!ok) break;
-            grid_sync();
             if (!ok) break;
             // ---- 1/rms, q/k norm, RoPE, K/V write: one warp per (128-column tile, row) ----
             {
@@ -493,21 +526,29 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 const int n_tiles = (p.Hq + 2 * p.Hkv) * HD / tc::BLOCK_N;
                 for (int pair = gw; pair < n_tiles * M; pair += GW) {
                     const int t = pair / M, m = pair % M;
-                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
-                    float4 s4 = tile_row_sum(p, 0, t, m, lane);
-                    const float inv = inv_rms_from(sq_l, d, p.eps);
-                    float x[4] = {inv * s4.x, inv * s4.y, inv * s4.z, inv * s4.w};
                     const int c_tile = 4 * lane;                    // column inside the tile
                     const int head = (t * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
                     const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
-                    const int pos = p.pv.row_pos[m];
+                    // everything this pair reads is requested before anything is used
+                    const int tab = tile_row_tab(p, 0, t, lane);
+                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
+                    const int pos = __ldg(p.pv.row_pos + m), flags = __ldg(p.pv.row_flags + m), sq = __ldg(p.pv.row_seq + m);
+                    const bool second = ch >= half;
+                    const int i0 = ch - (second ? half : 0);
+                    const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * half + i0));
+                    const float4 sn = __ldg(reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * half + i0));
+                    const int page = (flags & ROW_WRITE_KV) ? __ldg(p.pv.seq_pages + (size_t)sq * p.pv.max_pages + (pos >> p.pool.page_shift)) : 0;
+                    float4 gq = make_float4(1.f, 1.f, 1.f, 1.f);
+                    if (p.qk_norm && (is_q || is_k)) gq = __ldg(reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch));
+                    float4 s4 = tile_row_sum(p, tab, m, lane, p.tile_cnt[0] + t, (unsigned)l + 1u, abort_flag);
+                    const float inv = inv_rms_from(sq_l, d, p.eps);
+                    float x[4] = {inv * s4.x, inv * s4.y, inv * s4.z, inv * s4.w};
                     if (p.qk_norm) {
                         float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
 #pragma unroll
                         for (int o = HD / 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);   // over the head's lanes
                         if (is_q || is_k) {
                             const float hinv = 1.0f / sqrtf(ss / (float)HD + p.eps);
-                            const float4 gq = *reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch);
                             x[0] *= hinv * gq.x;
                             x[1] *= hinv * gq.y;
                             x[2] *= hinv * gq.z;
@@ -515,10 +556,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         }
                     }
                     {   // rotate-half RoPE: element i of the first half pairs with i + half
-                        const bool second = ch >= half;
-                        const int i0 = ch - (second ? half : 0);
-                        const float4 cs = *reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * half + i0);
-                        const float4 sn = *reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * half + i0);
                         const float c4[4] = {cs.x, cs.y, cs.z, cs.w}, s4r[4] = {sn.x, sn.y, sn.z, sn.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
@@ -532,15 +569,13 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     } else {
                         const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
                         store_bf16x4((is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD + ch, x[0], x[1], x[2], x[3]);
-                        if (p.pv.row_flags[m] & ROW_WRITE_KV) {
-                            const int sq = p.pv.row_seq[m];
-                            const int page = p.pv.seq_pages[(size_t)sq * p.pv.max_pages + (pos >> p.pool.page_shift)];
+                        if (flags & ROW_WRITE_KV) {
                             store_bf16x4(p.pool.ptr(l, page, is_k ? 0 : 1, kvh, pos & (p.pool.page_tokens - 1)) + ch, x[0], x[1], x[2], x[3]);
                         }
                     }
                 }
             }
-            grid_sync();
+            grid_sync(true);
             if (!ok) break;
             // ---- attention items ----
             {
@@ -557,111 +592,132 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                 }
                 if (!ok) break;
-                grid_sync();
+                grid_sync(false);
                 if (!ok) break;
                 // ---- combine the key splits of every (row, query head) ----
                 for (int pair = gw; pair < M * p.Hq; pair += GW) {
                     const int r = pair / p.Hq, hq = pair % p.Hq;
-                    const int seq = p.pv.row_seq[r], kvh = hq / ap.group;
-                    const int qv = (r - p.pv.seq_row0[seq]) * ap.group + hq % ap.group;
+                    const int seq = __ldg(p.pv.row_seq + r), kvh = hq / ap.group;
+                    const int qv = (r - __ldg(p.pv.seq_row0 + seq)) * ap.group + hq % ap.group;
                     const int qt = qv / att::QT, qi = qv % att::QT;
-                    const int n_ctx = p.pv.seq_nctx[seq];
+                    const int n_ctx = __ldg(p.pv.seq_nctx + seq);
                     const int n_pages = (n_ctx + ap.page_tokens - 1) >> ap.page_shift;
                     const size_t item0 = ((size_t)(seq * ap.Hkv + kvh) * ap.n_qtiles + qt) * n_splits;
-                    // lanes take the splits for the maxima and weights, then the columns for the sums
-                    float acc[HD / 32], lsum = 0.f;
-#pragma unroll
-                    for (int e = 0; e < HD / 32; ++e) acc[e] = 0.f;
-                    float mx = -INFINITY;
-                    for (int s0 = 0; s0 < n_splits; s0 += 32) {
-                        const int s = s0 + lane;
-                        const bool used = s < n_splits && (s == ap.n_cache_splits || s * ap.pages_per_split < n_pages);
-                        const float ms = used ? __ldcg(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2) : -INFINITY;
-                        mx = fmaxf(mx, warp_max(ms));
-                    }
+                    // Lanes take the splits for maxima and weights, and 4 output columns each (the
+                    // first HD/4 lanes) for the sums.  Whether a split was written follows from the
+                    // page count alone, so the loads of the partial outputs do not wait for the weights.
+                    constexpr int CCH = 12;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float lsum = 0.f;
                     for (int s0 = 0; s0 < n_splits; s0 += 32) {
                         const int s = s0 + lane;
                         const bool used = s < n_splits && (s == ap.n_cache_splits || s * ap.pages_per_split < n_pages);
                         float2 ml = make_float2(-INFINITY, 0.f);
                         if (used) ml = __ldcg(reinterpret_cast<const float2*>(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2));
+                        // the maximum over all splits is needed before any weight: second sweep when n_splits > 32
+                        float mx = warp_max(ml.x);
+                        for (int z0 = 0; z0 < n_splits; z0 += 32) {
+                            if (z0 == s0) continue;
+                            const int z = z0 + lane;
+                            const bool uz = z < n_splits && (z == ap.n_cache_splits || z * ap.pages_per_split < n_pages);
+                            mx = fmaxf(mx, warp_max(uz ? __ldcg(ap.part_ml + (item0 + z) * att::QT * 2 + qi * 2) : -INFINITY));
+                        }
                         const float w_l = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
+                        lsum += warp_sum(w_l * ml.y);
                         const int cnt = min(32, n_splits - s0);
-                        for (int k0 = 0; k0 < cnt; k0 += 8) {
-                            float v[8][HD / 32], w[8];
+                        for (int k0 = 0; k0 < cnt; k0 += CCH) {
+                            float4 v[CCH];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                w[k] = __shfl_sync(0xffffffffu, w_l, (k0 + k) & 31);
-                                const float lk = __shfl_sync(0xffffffffu, ml.y, (k0 + k) & 31);
-                                const bool on = k0 + k < cnt && w[k] != 0.f;
-                                if (!on) w[k] = 0.f;
-                                lsum += w[k] * lk;
-                                const float* po = ap.part_o + ((item0 + s0 + k0 + k) * att::QT + qi) * HD + lane;
-#pragma unroll
-                                for (int e = 0; e < HD / 32; ++e) v[k][e] = on ? __ldcg(po + 32 * e) : 0.f;
+                            for (int k = 0; k < CCH; ++k) {
+                                const int z = s0 + k0 + k;
+                                const bool uz = k0 + k < cnt && (z == ap.n_cache_splits || z * ap.pages_per_split < n_pages);
+                                v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (uz && lane < HD / 4) v[k] = __ldcg(reinterpret_cast<const float4*>(ap.part_o + ((item0 + z) * att::QT + qi) * HD) + lane);
                             }
 #pragma unroll
-                            for (int k = 0; k < 8; ++k)
-#pragma unroll
-                                for (int e = 0; e < HD / 32; ++e) acc[e] += w[k] * v[k][e];
+                            for (int k = 0; k < CCH; ++k) {
+                                const float w = __shfl_sync(0xffffffffu, w_l, (k0 + k) & 31);
+                                if (k0 + k < cnt && w != 0.f) {
+                                    acc.x += w * v[k].x;
+                                    acc.y += w * v[k].y;
+                                    acc.z += w * v[k].z;
+                                    acc.w += w * v[k].w;
+                                }
+                            }
                         }
                     }
-#pragma unroll
-                    for (int e = 0; e < HD / 32; ++e)
-                        p.attn[((size_t)r * p.Hq + hq) * HD + lane + 32 * e] = __float2bfloat16_rn(acc[e] / lsum);
+                    if (lane < HD / 4) {
+                        store_bf16x4(p.attn + ((size_t)r * p.Hq + hq) * HD + 4 * lane, acc.x / lsum, acc.y / lsum, acc.z / lsum, acc.w / lsum);
+                    }
                 }
             }
-            grid_sync();
+            grid_sync(true);
             if (!ok) break;
             // ---- O GEMM, residual ----
             drain(l, 1);
             if (!ok) break;
-            grid_sync();
-            if (!ok) break;
-            residual_phase(1, lg.ffn_norm, p.ssq_b);
-            grid_sync();
+            residual_phase(1, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b);
+            grid_sync(true);
             if (!ok) break;
             // ---- gate/up GEMM, SwiGLU ----
             drain(l, 2);
             if (!ok) break;
-            grid_sync();
-            if (!ok) break;
             {
-                const int f_tiles = p.f / tc::BLOCK_N;
-                for (int pair = gw; pair < f_tiles * M; pair += GW) {
-                    const int t = pair / M, m = pair % M;
-                    const float sq_l = row_ssq_lane(p.ssq_b, d_tiles, m, lane);
-                    const float4 g4 = tile_row_sum(p, 2, t, m, lane), u4 = tile_row_sum(p, 2, t + f_tiles, m, lane);
-                    const float inv = inv_rms_from(sq_l, d, p.eps);
-                    const float gv[4] = {inv * g4.x, inv * g4.y, inv * g4.z, inv * g4.w};
-                    const float uv[4] = {inv * u4.x, inv * u4.y, inv * u4.z, inv * u4.w};
-                    float a[4];
+                const int f_tiles = p.f / tc::BLOCK_N, n_pairs = f_tiles * M;
+                // two (tile, row) pairs per step so that both pairs' loads overlap
+                for (int pair = gw; pair < n_pairs; pair += 2 * GW) {
+                    int tt[2], mm[2], tg[2], tu[2];
+                    float sq_l[2];
+                    bool on[2];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) a[e] = gv[e] / (1.f + expf(-gv[e])) * uv[e];
-                    store_bf16x4(p.act + (size_t)m * p.f + t * tc::BLOCK_N + 4 * lane, a[0], a[1], a[2], a[3]);
+                    for (int q = 0; q < 2; ++q) {
+                        const int pr = pair + q * GW;
+                        on[q] = pr < n_pairs;
+                        tt[q] = on[q] ? pr / M : 0;
+                        mm[q] = on[q] ? pr % M : 0;
+                        tg[q] = tile_row_tab(p, 2, tt[q], lane);
+                        tu[q] = tile_row_tab(p, 2, tt[q] + f_tiles, lane);
+                        sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane);
+                    }
+                    float4 g4[2], u4[2];
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        g4[q] = tile_row_sum(p, tg[q], mm[q], lane, p.tile_cnt[2] + tt[q], (unsigned)l + 1u, abort_flag);
+                        u4[q] = tile_row_sum(p, tu[q], mm[q], lane, p.tile_cnt[2] + tt[q] + f_tiles, (unsigned)l + 1u, abort_flag);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const float inv = inv_rms_from(sq_l[q], d, p.eps);
+                        if (!on[q]) continue;
+                        const float gv[4] = {inv * g4[q].x, inv * g4[q].y, inv * g4[q].z, inv * g4[q].w};
+                        const float uv[4] = {inv * u4[q].x, inv * u4[q].y, inv * u4[q].z, inv * u4[q].w};
+                        float a[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) a[e] = gv[e] / (1.f + expf(-gv[e])) * uv[e];
+                        store_bf16x4(p.act + (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane, a[0], a[1], a[2], a[3]);
+                    }
                 }
             }
-            grid_sync();
+            grid_sync(true);
             if (!ok) break;
             // ---- down GEMM, residual; prepares the next layer's (or the head's) input ----
             drain(l, 3);
             if (!ok) break;
-            grid_sync();
-            if (!ok) break;
-            residual_phase(3, l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm, p.ssq_a);
-            grid_sync();
+            residual_phase(3, (unsigned)l + 1u, l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm, p.ssq_a);
+            grid_sync(true);
         }
         if (ok && p.n_logit > 0) {
             // ---- LM head on the rows that need logits ----
             drain(p.n_layers, 4);
-            if (ok) grid_sync();
             if (ok) {
                 const int n_tiles = (p.V + tc::BLOCK_N - 1) / tc::BLOCK_N;
                 const bool vec = (p.V & 3) == 0;
                 for (int pair = gw; pair < n_tiles * p.n_logit; pair += GW) {
                     const int t = pair / p.n_logit, lr = pair % p.n_logit;
                     const int m = p.pv.logit_rows[lr];
+                    const int tab = tile_row_tab(p, 4, t, lane);
                     const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
-                    const float4 s4 = tile_row_sum(p, 4, t, m, lane);
+                    const float4 s4 = tile_row_sum(p, tab, m, lane, p.tile_cnt[4] + t, 1u, abort_flag);
                     const float sc = p.logit_scale * inv_rms_from(sq_l, d, p.eps);
                     const int col = t * tc::BLOCK_N + 4 * lane;
                     float* dst = p.logits + (size_t)lr * p.V + col;
