@@ -107,6 +107,9 @@ struct s2d2_ctx {
     int *d_xhat = nullptr;
     float *d_conf = nullptr, *d_margin = nullptr, *d_entropy = nullptr;
     double* d_lse = nullptr;
+    void *chunk_d = nullptr, *chunk_v = nullptr;   // per (logit row, vocabulary chunk) statistics of the two passes
+    void* rej_info = nullptr;                      // per sequence: the rejected position to resample
+    double *res_rsum = nullptr, *res_vsum = nullptr;   // per (sequence, chunk) residual and pi_v mass
     char *acc_h = nullptr, *acc_d = nullptr;      // staging for the acceptance kernel's inputs and outputs
     size_t acc_bytes = 0;
     char* stats_h = nullptr;                       // pinned mirror of the draft statistics

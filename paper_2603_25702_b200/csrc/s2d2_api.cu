@@ -292,6 +292,12 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
         if ((rc = dmalloc(c, &c->d_margin, R))) return rc;
         if ((rc = dmalloc(c, &c->d_entropy, R))) return rc;
         if ((rc = dmalloc(c, &c->d_lse, R))) return rc;
+        size_t nch = vocab_chunks(m->vocab), Sq = dc->max_batch;
+        if ((rc = dmalloc(c, (ChunkStats**)&c->chunk_d, R * nch))) return rc;
+        if ((rc = dmalloc(c, (ChunkStats**)&c->chunk_v, R * nch))) return rc;
+        if ((rc = dmalloc(c, (RejectInfo**)&c->rej_info, Sq))) return rc;
+        if ((rc = dmalloc(c, &c->res_rsum, Sq * nch))) return rc;
+        if ((rc = dmalloc(c, &c->res_vsum, Sq * nch))) return rc;
         CUDA_TRY(c, cudaMallocHost((void**)&c->stats_h, R * 16));
         size_t S = dc->max_batch;
         c->acc_bytes = S * 4 * 12 + S * S2D2_MAX_BLOCK * 4 * 3 + 256;
@@ -320,7 +326,8 @@ extern "C" int s2d2_destroy(s2d2_ctx* c) {
     void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
                     c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
-                    c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status};
+                    c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status, c->chunk_d, c->chunk_v, c->rej_info,
+                    c->res_rsum, c->res_vsum};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->meta.h) cudaFreeHost(c->meta.h);
@@ -667,8 +674,14 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     CUDA_TRY(c, cudaEventRecord(c->ev[0], c->stream));
     if ((rc = run_pass(c, pb, c->logits_draft))) return rc;
     DraftStatsOut so{c->d_xhat, c->d_conf, c->d_margin, c->d_entropy, c->d_lse};
-    draft_stats_kernel<<<pb.n_logit, VOCAB_THREADS, 0, c->stream>>>(c->logits_draft, c->m.vocab, so);
-    LAUNCHED(c);
+    {
+        const int nch = vocab_chunks(c->m.vocab);
+        vocab_chunk_stats_kernel<<<dim3(nch, pb.n_logit), VCHUNK_THREADS, 0, c->stream>>>(c->logits_draft, c->m.vocab,
+                                                                                         (ChunkStats*)c->chunk_d);
+        LAUNCHED(c);
+        draft_finish_kernel<<<(pb.n_logit + 3) / 4, 128, 0, c->stream>>>((const ChunkStats*)c->chunk_d, nch, pb.n_logit, so);
+        LAUNCHED(c);
+    }
     size_t R = pb.n_logit;
     int* hx = (int*)c->stats_h;
     float* hc = (float*)(c->stats_h + R * 4);
@@ -831,8 +844,9 @@ struct AccStage {     // layout of acc_h / acc_d for S sequences
     }
 };
 
+// n_draft_rows / n_verify_rows: logit rows of the two buffers that the sequences refer to.
 int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, const float* d_verify, const int* d_xhat,
-                  const double* d_lse, const float* d_conf) {
+                  const double* d_lse, const float* d_conf, int n_draft_rows, int n_verify_rows) {
     CUDA_TRY(c, cudaMemcpyAsync(c->acc_d, c->acc_h, a.in_bytes, cudaMemcpyHostToDevice, c->stream));
     c->cnt.h2d_bytes += a.in_bytes;
     c->cnt.d2h_bytes += a.total - a.in_bytes;
@@ -864,8 +878,26 @@ int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, c
     out.u = (float*)(c->acc_d + a.o_u);
     out.a = (float*)(c->acc_d + a.o_a);
     out.v = (float*)(c->acc_d + a.o_v);
-    accept_block_kernel<<<n, VOCAB_THREADS, 0, c->stream>>>(in, out);
+    const int nch = vocab_chunks(c->m.vocab);
+    in.verify_chunks = (const ChunkStats*)c->chunk_v;
+    in.draft_chunks = (const ChunkStats*)c->chunk_d;
+    if (n_verify_rows > 0) {
+        vocab_chunk_stats_kernel<<<dim3(nch, n_verify_rows), VCHUNK_THREADS, 0, c->stream>>>(d_verify, c->m.vocab, (ChunkStats*)c->chunk_v);
+        LAUNCHED(c);
+    }
+    if (!d_lse && n_draft_rows > 0) {
+        vocab_chunk_stats_kernel<<<dim3(nch, n_draft_rows), VCHUNK_THREADS, 0, c->stream>>>(d_draft, c->m.vocab, (ChunkStats*)c->chunk_d);
+        LAUNCHED(c);
+    }
+    RejectInfo* rej = (RejectInfo*)c->rej_info;
+    accept_scan_kernel<<<n, 128, 0, c->stream>>>(in, out, rej);
     LAUNCHED(c);
+    if (c->dc.resample && n_verify_rows > 0) {
+        residual_chunk_kernel<<<dim3(nch, n), VCHUNK_THREADS, 0, c->stream>>>(in, rej, c->res_rsum, c->res_vsum);
+        LAUNCHED(c);
+        residual_pick_kernel<<<n, VCHUNK_THREADS, 0, c->stream>>>(in, rej, c->res_rsum, c->res_vsum, nch, out.resampled);
+        LAUNCHED(c);
+    }
     CUDA_TRY(c, cudaMemcpyAsync(c->acc_h + a.in_bytes, c->acc_d + a.in_bytes, a.total - a.in_bytes,
                                 cudaMemcpyDeviceToHost, c->stream));
     return S2D2_OK;
@@ -896,7 +928,8 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
         ((int*)(c->acc_h + a.o_mode))[i] = flags[i] ? 1 : 0;
     }
     CUDA_TRY(c, cudaEventRecord(c->ev[4], c->stream));
-    int rc = launch_accept(c, a, n, c->logits_draft, c->logits_verify, c->d_xhat, c->d_lse, c->d_conf);
+    int rc = launch_accept(c, a, n, c->logits_draft, c->logits_verify, c->d_xhat, c->d_lse, c->d_conf, c->n_draft_logit_rows,
+                           c->n_verify_logit_rows);
     if (rc) return rc;
     if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[5], c->stream));
@@ -997,7 +1030,7 @@ extern "C" int s2d2_accept_logits(s2d2_ctx* c, const float* d_draft, const float
         ((int*)(c->acc_h + a.o_mode))[i] = 1;
     }
     CUDA_TRY(c, cudaMemcpyAsync(c->d_xhat, xhat, (size_t)n * l_max * 4, cudaMemcpyHostToDevice, c->stream));
-    int rc = launch_accept(c, a, n, d_draft, d_verify, c->d_xhat, nullptr, nullptr);
+    int rc = launch_accept(c, a, n, d_draft, d_verify, c->d_xhat, nullptr, nullptr, n * l_max, n * l_max);
     if (rc) return rc;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     for (int i = 0; i < n; ++i) {

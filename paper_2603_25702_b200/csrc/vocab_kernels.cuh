@@ -12,7 +12,6 @@
 
 namespace s2d2 {
 
-constexpr int VOCAB_THREADS = 1024;
 
 struct Top2 {
     float v1;   // best value
@@ -88,30 +87,128 @@ struct DraftStatsOut {
     double* lse;      // log-sum-exp of the row, fp64
 };
 
-// SampleFromLogits, greedy: one block per logit row.
-__global__ void draft_stats_kernel(const float* __restrict__ logits, int V, DraftStatsOut o) {
+// ---------------------------------------------------------------------------------------------
+// Stage 1, shared by the draft statistics and the acceptance step: the vocabulary of every logit
+// row is cut into chunks of VCHUNK entries, one CTA per (chunk, row), so that a handful of rows
+// still fills the GPU.  Per chunk: its top-2, and sum exp(x - max_chunk), sum x exp(x - max_chunk)
+// in fp64.  Stage 2 kernels merge the chunks of a row in chunk order.
+// ---------------------------------------------------------------------------------------------
+constexpr int VCHUNK = 4096;
+constexpr int VCHUNK_THREADS = 256;
+constexpr int VPER = VCHUNK / VCHUNK_THREADS;   // 16 entries per thread
+
+struct ChunkStats {
+    float mx;      // largest logit of the chunk
+    int arg;       // its index (lowest id among equals)
+    float mx2;     // second largest (== mx when attained twice)
+    int pad;
+    double s;      // sum exp(x - mx)
+    double sx;     // sum x * exp(x - mx)
+};
+__host__ __device__ inline int vocab_chunks(int V) { return (V + VCHUNK - 1) / VCHUNK; }
+
+// Loads the VPER entries of thread t of a chunk: entries (k * 256 + t) * 4 .. + 3 for k = 0..3
+// (ids ascending inside a thread); entries past V read as -inf.
+__device__ __forceinline__ void load_chunk_strided(const float* row, int V, int base, int t, float (&x)[VPER]) {
+    const bool vec = (V & 3) == 0;
+#pragma unroll
+    for (int k = 0; k < VPER / 4; ++k) {
+        const int i0 = base + (k * VCHUNK_THREADS + t) * 4;
+        if (vec && i0 + 3 < V) {
+            const float4 v = *reinterpret_cast<const float4*>(row + i0);
+            x[4 * k] = v.x;
+            x[4 * k + 1] = v.y;
+            x[4 * k + 2] = v.z;
+            x[4 * k + 3] = v.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[4 * k + e] = i0 + e < V ? row[i0 + e] : -INFINITY;
+        }
+    }
+}
+
+static __global__ void __launch_bounds__(VCHUNK_THREADS) vocab_chunk_stats_kernel(const float* __restrict__ logits, int V,
+                                                                                  ChunkStats* __restrict__ out) {
     __shared__ Top2 sh_t[32];
     __shared__ double sh_d[32];
-    int r = blockIdx.x;
-    const float* x = logits + (size_t)r * V;
+    const int chunk = blockIdx.x, r = blockIdx.y, n_chunks = gridDim.x;
+    const float* row = logits + (size_t)r * V;
+    const int base = chunk * VCHUNK;
+    float x[VPER];
+    load_chunk_strided(row, V, base, threadIdx.x, x);
     Top2 t{-INFINITY, 0x7fffffff, -INFINITY};
-    for (int i = threadIdx.x; i < V; i += blockDim.x) t = top2_push(t, x[i], i);
+#pragma unroll
+    for (int k = 0; k < VPER; ++k) t = top2_push(t, x[k], base + ((k >> 2) * VCHUNK_THREADS + threadIdx.x) * 4 + (k & 3));
     t = block_top2(t, sh_t);
-    double mx = (double)t.v1, s = 0.0, sx = 0.0;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
-        double xi = (double)x[i];
-        double e = exp(xi - mx);
-        s += e;
-        sx += e * xi;
+    const double mx = (double)t.v1;
+    double s = 0.0, sx = 0.0;
+#pragma unroll
+    for (int k = 0; k < VPER; ++k) {
+        if (x[k] != -INFINITY) {
+            const double xi = (double)x[k], e = exp(xi - mx);
+            s += e;
+            sx += e * xi;
+        }
     }
     s = block_sum_d(s, sh_d);
     sx = block_sum_d(sx, sh_d);
     if (threadIdx.x == 0) {
-        double lse = mx + log(s);
-        o.xhat[r] = t.i1;
-        o.conf[r] = (float)(1.0 / s);
-        o.margin[r] = (float)((1.0 - exp((double)t.v2 - mx)) / s);
-        o.entropy[r] = (float)(lse - sx / s);
+        ChunkStats o;
+        o.mx = t.v1;
+        o.arg = t.i1;
+        o.mx2 = t.v2;
+        o.pad = 0;
+        o.s = s;
+        o.sx = sx;
+        out[(size_t)r * n_chunks + chunk] = o;
+    }
+}
+
+// Merge of a row's chunks by one warp: top-2 in chunk order, then the sums rescaled to the row
+// maximum.  Every lane returns the same values.
+struct RowStats {
+    Top2 t;
+    double s, sx;
+};
+__device__ __forceinline__ RowStats warp_row_stats(const ChunkStats* cs, int n_chunks, int lane) {
+    Top2 t{-INFINITY, 0x7fffffff, -INFINITY};
+    for (int c = lane; c < n_chunks; c += 32) {
+        Top2 o{cs[c].mx, cs[c].arg, cs[c].mx2};
+        t = top2_merge(t, o);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Top2 other;
+        other.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        other.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        other.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t = top2_merge(t, other);
+    }
+    const double mx = (double)t.v1;
+    double s = 0.0, sx = 0.0;
+    for (int c = lane; c < n_chunks; c += 32) {
+        const double w = exp((double)cs[c].mx - mx);
+        s += cs[c].s * w;
+        sx += cs[c].sx * w;
+    }
+    RowStats r;
+    r.t = t;
+    r.s = warp_sum(s);
+    r.sx = warp_sum(sx);
+    return r;
+}
+
+// SampleFromLogits, greedy, stage 2: one warp per logit row.
+static __global__ void draft_finish_kernel(const ChunkStats* __restrict__ cs, int n_chunks, int n_rows, DraftStatsOut o) {
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= n_rows) return;
+    const RowStats st = warp_row_stats(cs + (size_t)r * n_chunks, n_chunks, lane);
+    if (lane == 0) {
+        const double mx = (double)st.t.v1, lse = mx + log(st.s);
+        o.xhat[r] = st.t.i1;
+        o.conf[r] = (float)(1.0 / st.s);
+        o.margin[r] = (float)((1.0 - exp((double)st.t.v2 - mx)) / st.s);
+        o.entropy[r] = (float)(lse - st.sx / st.s);
         o.lse[r] = lse;
     }
 }
@@ -127,9 +224,11 @@ struct AcceptIn {
     const unsigned* seq_stream;   // Philox sequence stream
     const int* seq_step;          // Philox step word
     const int* xhat;              // per draft-logit row
-    const double* draft_lse;      // per draft-logit row (may be null: recomputed)
+    const double* draft_lse;      // per draft-logit row (may be null: taken from draft_chunks)
     const int* seq_mode;          // 1: acceptance scan; 0: confidence branch (may be null: all 1)
     const float* conf;            // per draft-logit row, for the confidence branch
+    const ChunkStats* verify_chunks;   // stage-1 output over the verifier-logit rows
+    const ChunkStats* draft_chunks;    // stage-1 output over the draft-logit rows (when draft_lse is null)
     float tau_conf;
     unsigned seed;
     float gamma;
@@ -146,26 +245,25 @@ struct AcceptOut {
     float* a;
     float* v;
 };
+// What the residual kernels need to know about a sequence's rejected position.
+struct RejectInfo {
+    int draft_row, verify_row;   // logit rows; draft_row < 0: nothing to resample
+    unsigned pos;
+    int pad;
+    double lse_d, lse_v;
+};
 
-__device__ __forceinline__ double row_lse_block(const float* x, int V, double* sh_d, Top2* sh_t) {
-    Top2 t{-INFINITY, 0x7fffffff, -INFINITY};
-    for (int i = threadIdx.x; i < V; i += blockDim.x) t = top2_push(t, x[i], i);
-    t = block_top2(t, sh_t);
-    double mx = (double)t.v1, s = 0.0;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) s += exp((double)x[i] - mx);
-    s = block_sum_d(s, sh_d);
-    return mx + log(s);
-}
-
-// Reference form of the acceptance step: one block per sequence, rows scanned
-// left to right, stopping at the first rejection.
-__global__ void accept_block_kernel(AcceptIn in, AcceptOut out) {
-    __shared__ Top2 sh_t[32];
-    __shared__ double sh_d[32];
-    __shared__ double sh_pref[VOCAB_THREADS];
-    __shared__ int sh_pick;
-    int s = blockIdx.x;
-    int L = in.seq_len[s];
+// Acceptance scan, one CTA of 128 threads per sequence (Algorithm "SampleBlock for S2D2", the
+// left-to-right loop; the else-branch for sequences that were not verified).  Warps merge the
+// verifier chunks of the span's rows, thread i evaluates position i (v_i, d_i, a_i, u_i), thread 0
+// scans left to right up to the first rejection.
+static __global__ void __launch_bounds__(128) accept_scan_kernel(AcceptIn in, AcceptOut out, RejectInfo* rej) {
+    __shared__ double sh_lse_v[32], sh_lse_d[32];
+    __shared__ double sh_a[32], sh_u[32], sh_v[32];
+    const int s = blockIdx.x, L = in.seq_len[s];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_chunks = vocab_chunks(in.V);
+    if (threadIdx.x == 0) rej[s].draft_row = -1;
     if (in.seq_mode && in.seq_mode[s] == 0) {
         // Not verified: S = {i in M_t : d_i > tau} U {argmax d_i} (ties -> leftmost); L = |M_t| here.
         if (threadIdx.x == 0) {
@@ -184,87 +282,192 @@ __global__ void accept_block_kernel(AcceptIn in, AcceptOut out) {
         }
         return;
     }
-    int n_acc = 0, first_rej = -1, resampled = -1, near = 0;
-    for (int i = 0; i < L; ++i) {
-        int dr = in.seq_draft_row0[s] + i;
-        const float* xd = in.draft_logits + (size_t)dr * in.V;
-        const float* xv = in.verify_logits + (size_t)(in.seq_verify_row0[s] + i) * in.V;
-        double lse_v = row_lse_block(xv, in.V, sh_d, sh_t);
-        double lse_d = in.draft_lse ? in.draft_lse[dr] : row_lse_block(xd, in.V, sh_d, sh_t);
-        int tok = in.xhat[dr];
-        double v = exp((double)xv[tok] - lse_v), d = exp((double)xd[tok] - lse_d);
+    const int dr0 = in.seq_draft_row0[s], vr0 = in.seq_verify_row0[s];
+    for (int i = warp; i < L; i += 4) {
+        const RowStats sv = warp_row_stats(in.verify_chunks + (size_t)(vr0 + i) * n_chunks, n_chunks, lane);
+        if (lane == 0) sh_lse_v[i] = (double)sv.t.v1 + log(sv.s);
+        if (in.draft_lse) {
+            if (lane == 0) sh_lse_d[i] = in.draft_lse[dr0 + i];
+        } else {
+            const RowStats sd = warp_row_stats(in.draft_chunks + (size_t)(dr0 + i) * n_chunks, n_chunks, lane);
+            if (lane == 0) sh_lse_d[i] = (double)sd.t.v1 + log(sd.s);
+        }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < L) {
+        const int i = threadIdx.x, tok = in.xhat[dr0 + i];
+        const double xv = (double)in.verify_logits[(size_t)(vr0 + i) * in.V + tok];
+        const double xd = (double)in.draft_logits[(size_t)(dr0 + i) * in.V + tok];
+        const double v = exp(xv - sh_lse_v[i]), d = exp(xd - sh_lse_d[i]);
         double ratio = v / d;
         if (in.gamma != 1.f) ratio = pow(ratio, (double)in.gamma);
-        double a = fmin(1.0, ratio);
-        unsigned pos = (unsigned)(in.seq_pos0[s] + i);
-        double u = philox_uniform(in.seed, pos, in.seq_stream[s], (unsigned)in.seq_step[s], STREAM_ACCEPT);
-        if (threadIdx.x == 0) {
+        sh_v[i] = v;
+        sh_a[i] = fmin(1.0, ratio);
+        sh_u[i] = philox_uniform(in.seed, (unsigned)(in.seq_pos0[s] + i), in.seq_stream[s], (unsigned)in.seq_step[s], STREAM_ACCEPT);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int n_acc = 0, first_rej = -1, near = 0;
+        for (int i = 0; i < L; ++i) {
+            const double u = sh_u[i], a = sh_a[i];
             out.u[(size_t)s * in.l_cap + i] = (float)u;
             out.a[(size_t)s * in.l_cap + i] = (float)a;
-            out.v[(size_t)s * in.l_cap + i] = (float)v;
-        }
-        if (fabs(u - a) < 1e-4) ++near;
-        if (u < a) {
-            ++n_acc;
-            continue;
-        }
-        first_rej = i;
-        if (in.resample) {
-            // residual (pi_v - pi_d)_+ : each thread owns a contiguous slice so that the
-            // block prefix over threads is the vocabulary-order CDF
-            int per = (in.V + blockDim.x - 1) / blockDim.x;
-            int lo = min(in.V, (int)threadIdx.x * per), hi = min(in.V, lo + per);
-            double mine = 0.0;
-            for (int w = lo; w < hi; ++w) mine += fmax(0.0, exp((double)xv[w] - lse_v) - exp((double)xd[w] - lse_d));
-            double Z = block_sum_d(mine, sh_d);
-            bool use_residual = Z > 0.0;
-            if (!use_residual) {   // unreachable after a true rejection in exact arithmetic
-                mine = 0.0;
-                for (int w = lo; w < hi; ++w) mine += exp((double)xv[w] - lse_v);
+            out.v[(size_t)s * in.l_cap + i] = (float)sh_v[i];
+            if (fabs(u - a) < 1e-4) ++near;
+            if (u < a) {
+                ++n_acc;
+                continue;
             }
-            sh_pref[threadIdx.x] = mine;
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                double run = 0.0;
-                for (int t = 0; t < (int)blockDim.x; ++t) {
-                    double x = sh_pref[t];
-                    sh_pref[t] = run;          // exclusive prefix
-                    run += x;
-                }
-                sh_d[0] = run;
-                sh_pick = in.V - 1;
-            }
-            __syncthreads();
-            double total = sh_d[0];
-            double u2 = philox_uniform(in.seed, pos, in.seq_stream[s], (unsigned)in.seq_step[s], STREAM_RESAMPLE);
-            double target = u2 * total;
-            double before = sh_pref[threadIdx.x];
-            __syncthreads();
-            if (before <= target && before + mine > target) {
-                double c = before;
-                int pick = hi - 1;
-                for (int w = lo; w < hi; ++w) {
-                    double wgt = use_residual ? fmax(0.0, exp((double)xv[w] - lse_v) - exp((double)xd[w] - lse_d))
-                                              : exp((double)xv[w] - lse_v);
-                    c += wgt;
-                    if (c > target) {
-                        pick = w;
-                        break;
-                    }
-                }
-                atomicMin(&sh_pick, pick);
-            }
-            __syncthreads();
-            resampled = sh_pick;
+            first_rej = i;
+            break;
         }
-        break;
-    }
-    if (threadIdx.x == 0) {
         out.n_accepted[s] = n_acc;
         out.first_reject[s] = first_rej;
-        out.resampled[s] = resampled;
+        out.resampled[s] = -1;
         out.n_near[s] = near;
+        if (first_rej >= 0 && in.resample) {
+            RejectInfo r;
+            r.draft_row = dr0 + first_rej;
+            r.verify_row = vr0 + first_rej;
+            r.pos = (unsigned)(in.seq_pos0[s] + first_rej);
+            r.pad = 0;
+            r.lse_d = sh_lse_d[first_rej];
+            r.lse_v = sh_lse_v[first_rej];
+            rej[s] = r;
+        }
     }
+}
+
+// Residual (pi_v - pi_d)_+ of the rejected position, stage 1: per (chunk, sequence) the chunk's
+// residual mass and its pi_v mass in fp64.  Thread t owns the 16 consecutive entries
+// [base + 16 t, base + 16 t + 16) so that prefixes over threads follow the vocabulary order.
+__device__ __forceinline__ void load_chunk_contiguous(const float* row, int V, int base, int t, float (&x)[VPER]) {
+    const bool vec = (V & 3) == 0;
+#pragma unroll
+    for (int k = 0; k < VPER / 4; ++k) {
+        const int i0 = base + t * VPER + 4 * k;
+        if (vec && i0 + 3 < V) {
+            const float4 v = *reinterpret_cast<const float4*>(row + i0);
+            x[4 * k] = v.x;
+            x[4 * k + 1] = v.y;
+            x[4 * k + 2] = v.z;
+            x[4 * k + 3] = v.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[4 * k + e] = i0 + e < V ? row[i0 + e] : -INFINITY;
+        }
+    }
+}
+static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_chunk_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
+                                                                               double* __restrict__ rsum, double* __restrict__ vsum) {
+    __shared__ double sh_d[32];
+    const int chunk = blockIdx.x, s = blockIdx.y, n_chunks = gridDim.x;
+    const RejectInfo r = rej[s];
+    if (r.draft_row < 0) return;
+    float xv[VPER], xd[VPER];
+    load_chunk_contiguous(in.verify_logits + (size_t)r.verify_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xv);
+    load_chunk_contiguous(in.draft_logits + (size_t)r.draft_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xd);
+    double rs = 0.0, vs = 0.0;
+#pragma unroll
+    for (int k = 0; k < VPER; ++k) {
+        if (xv[k] == -INFINITY && xd[k] == -INFINITY) continue;      // past the vocabulary
+        const double pv = exp((double)xv[k] - r.lse_v), pd = exp((double)xd[k] - r.lse_d);
+        rs += fmax(0.0, pv - pd);
+        vs += pv;
+    }
+    rs = block_sum_d(rs, sh_d);
+    vs = block_sum_d(vs, sh_d);
+    if (threadIdx.x == 0) {
+        rsum[(size_t)s * n_chunks + chunk] = rs;
+        vsum[(size_t)s * n_chunks + chunk] = vs;
+    }
+}
+
+// Stage 2: inverse CDF in vocabulary order with one uniform.  Thread 0 walks the chunk masses to
+// the chunk that holds u * Z, the CTA then walks that chunk (prefix over threads, then the
+// owning thread over its 16 entries).  If the residual mass is zero (cannot follow a true
+// rejection in exact arithmetic) the draw is from pi_v.
+static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_pick_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
+                                                                              const double* __restrict__ rsum,
+                                                                              const double* __restrict__ vsum, int n_chunks,
+                                                                              int* __restrict__ resampled) {
+    __shared__ double sh_warp[VCHUNK_THREADS / 32];
+    __shared__ double sh_target;
+    __shared__ int sh_chunk, sh_use_res, sh_pick;
+    const int s = blockIdx.x;
+    const RejectInfo r = rej[s];
+    if (r.draft_row < 0) return;
+    if (threadIdx.x == 0) {
+        double Z = 0.0;
+        for (int c = 0; c < n_chunks; ++c) Z += rsum[(size_t)s * n_chunks + c];
+        const bool use_res = Z > 0.0;
+        const double* mass = (use_res ? rsum : vsum) + (size_t)s * n_chunks;
+        double total = 0.0;
+        for (int c = 0; c < n_chunks; ++c) total += mass[c];
+        const double u2 = philox_uniform(in.seed, r.pos, in.seq_stream[s], (unsigned)in.seq_step[s], STREAM_RESAMPLE);
+        const double target = u2 * total;
+        double before = 0.0;
+        int pick_chunk = -1;
+        for (int c = 0; c < n_chunks; ++c) {
+            if (before + mass[c] > target) {
+                pick_chunk = c;
+                break;
+            }
+            before += mass[c];
+        }
+        sh_chunk = pick_chunk;
+        sh_use_res = use_res;
+        sh_target = target - before;
+        sh_pick = in.V - 1;
+    }
+    __syncthreads();
+    const int chunk = sh_chunk;
+    if (chunk >= 0) {
+        const bool use_res = sh_use_res != 0;
+        const double target = sh_target;
+        float xv[VPER], xd[VPER];
+        load_chunk_contiguous(in.verify_logits + (size_t)r.verify_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xv);
+        load_chunk_contiguous(in.draft_logits + (size_t)r.draft_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xd);
+        double w[VPER], mine = 0.0;
+#pragma unroll
+        for (int k = 0; k < VPER; ++k) {
+            w[k] = 0.0;
+            if (!(xv[k] == -INFINITY && xd[k] == -INFINITY)) {
+                const double pv = exp((double)xv[k] - r.lse_v), pd = exp((double)xd[k] - r.lse_d);
+                w[k] = use_res ? fmax(0.0, pv - pd) : pv;
+            }
+            mine += w[k];
+        }
+        // exclusive prefix over threads in thread order
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sh_warp[warp] = incl;
+        __syncthreads();
+        double before = incl - mine;
+        for (int k = 0; k < warp; ++k) before += sh_warp[k];
+        if (before <= target && before + mine > target) {
+            double c = before;
+            int pick = VPER - 1;
+#pragma unroll
+            for (int k = VPER - 1; k >= 0; --k) {
+                // prefix(k) in the same left-to-right order for every k; keep the smallest k that passes
+                double upto = before;
+#pragma unroll
+                for (int j = 0; j < VPER; ++j)
+                    if (j <= k) upto += w[j];
+                if (upto > target) pick = k;
+            }
+            (void)c;
+            atomicMin(&sh_pick, min(in.V - 1, chunk * VCHUNK + (int)threadIdx.x * VPER + pick));
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) resampled[s] = sh_pick;
 }
 
 }  // namespace s2d2
