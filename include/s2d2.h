@@ -74,7 +74,8 @@ typedef struct {
     float tau_conf;             /* threshold of the confidence branch            */
     float ratio_gamma;          /* accept iff u < min(1, (v/d)^gamma)            */
     uint32_t seed;              /* Philox key                                    */
-    int32_t use_tensor_cores;   /* 0: portable SIMT kernels only (debug)         */
+    int32_t use_tensor_cores;   /* 1: default. 0: portable SIMT kernels only (debug).
+                                   2: tensor-core kernels, one per operation (no persistent pass kernel) */
 } s2d2_decode_config;
 
 typedef struct {
@@ -212,10 +213,13 @@ int s2d2_release_seq(s2d2_ctx* ctx, int32_t seq_id);
 int s2d2_get_counters(s2d2_ctx* ctx, s2d2_counters* out);
 int s2d2_reset_counters(s2d2_ctx* ctx);
 
-/* Kernel-level timing for roofline reports: while on, every GEMM launch of the
- * forward pass is bracketed by a CUDA event pair on the context's stream.
- * s2d2_get_gemm_profile synchronises and returns the launches, their summed
- * device time and their summed algorithmic bytes (weight matrix read once +
+/* Kernel-level timing for roofline reports.  on >= 1: the dominant launches of the forward
+ * pass (the persistent pass kernel; on the one-kernel-per-operation path every GEMM) are
+ * bracketed by a CUDA event pair on the context's stream.  on >= 2: the persistent kernel also
+ * records its phase marks (s2d2_debug_pass_trace), which costs it a few percent.
+ * s2d2_get_gemm_profile synchronises and returns the bracketed launches, their summed device
+ * time and their summed algorithmic bytes (every weight matrix read once, the cached K/V of the
+ * pass's sequences read once, K/V rows and logits written; for a single GEMM: weights +
  * activations read + output written) since profiling was switched on. */
 int s2d2_set_profiling(s2d2_ctx* ctx, int32_t on);
 int s2d2_get_gemm_profile(s2d2_ctx* ctx, int64_t* n_launches, double* total_ms, double* total_bytes);
@@ -256,7 +260,7 @@ int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t
  * SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
  * QKV GEMM + q/k-norm + RoPE + K/V write, attention, its combine, O GEMM + residual add,
  * gate/up GEMM + SwiGLU, down GEMM + residual add.  Marks are recorded only while
- * s2d2_set_profiling is on.  S2D2_ERR_STATE if no such pass has run. */
+ * s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */
 int s2d2_debug_pass_trace(s2d2_ctx* ctx, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks);
 
 /* y[M, N] = x[M, K] w[N, K]^T on device buffers, without any allocation.

@@ -285,7 +285,8 @@ class Engine:
     def reset_counters(self):
         self._check(self.lib.s2d2_reset_counters(self._h))
 
-    def set_profiling(self, on: bool):
+    def set_profiling(self, on):
+        """0: off; 1: event pairs around the dominant kernels; 2: also the persistent kernel's phase marks."""
         self._check(self.lib.s2d2_set_profiling(self._h, int(on)))
 
     def get_gemm_profile(self):

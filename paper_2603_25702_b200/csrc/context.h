@@ -126,6 +126,7 @@ struct s2d2_ctx {
     bool verify_timing_pending = false;
     // per-GEMM profiling (off by default)
     bool profiling = false;
+    bool tracing = false;                   // in-kernel phase marks of the persistent pass
     std::vector<cudaEvent_t> prof_events;   // pairs
     size_t prof_used = 0;
     double prof_bytes = 0, prof_ms_done = 0;

@@ -60,7 +60,7 @@ int pass_init(s2d2_ctx* c) {
     PassState* s = new PassState();
     c->pass_state = s;
     const s2d2_model_config& m = c->m;
-    if (m.dtype != S2D2_DTYPE_BF16 || !c->dc.use_tensor_cores || m.n_experts > 0 || !gemm_tc_available(c)) return S2D2_OK;
+    if (m.dtype != S2D2_DTYPE_BF16 || c->dc.use_tensor_cores != 1 || m.n_experts > 0 || !gemm_tc_available(c)) return S2D2_OK;
     const int d = m.d_model, hd = m.head_dim, nq = m.n_q_heads * hd, nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, f = m.ffn;
     if (!(hd == 64 || hd == 128) || d % 128 || f % 128 || nqkv % 128 || nq % 64 || c->page_tokens < 16) return S2D2_OK;
     if (c->max_rows < pp::MAX_T) return S2D2_OK;
@@ -257,9 +257,9 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.status = c->d_status;
     p.S = stages_for(s, p.T, m.head_dim);
     for (int k = 0; k < 5; ++k) p.parts[k] = s->parts[k];
-    p.trace = c->profiling ? s->trace : nullptr;
+    p.trace = c->tracing ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    if (c->profiling) s->last_marks = 2 * (6 * m.n_layers + 1);
+    if (c->tracing) s->last_marks = 2 * (6 * m.n_layers + 1);
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
     for (int k = 0; k < 5; ++k) p.tile_cnt[k] = s->barrier + s->cnt_off[k];

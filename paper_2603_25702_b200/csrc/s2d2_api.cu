@@ -1126,6 +1126,7 @@ extern "C" int s2d2_set_profiling(s2d2_ctx* c, int32_t on) {
         c->prof_launches = 0;
     }
     c->profiling = on != 0;
+    c->tracing = on >= 2;
     return S2D2_OK;
 }
 extern "C" int s2d2_get_gemm_profile(s2d2_ctx* c, int64_t* n, double* ms, double* bytes) {
