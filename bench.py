@@ -139,8 +139,8 @@ def model_pass_bytes(m):
 # DRAM traffic of one pass_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu
 # capture summarised in profiles/pass_kernel_c2.md, as a ratio to the launch's algorithmic bytes; the
 # capture is of the 1.7B-class shape (a few GB on the device) and is scaled by algorithmic bytes, which
-# the traffic follows (weights dominate both).  None until a capture of the current kernel exists.
-PASS_TRAFFIC_RATIO = None
+# the traffic follows (weights dominate both).  Set to None when the kernel changes until it is re-captured.
+PASS_TRAFFIC_RATIO = 1.006
 
 
 def pass_traffic_bytes(m, algorithmic_bytes_per_launch):
