@@ -255,9 +255,10 @@ int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int3
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);
 
 /* Phase timeline of the last pass that ran as the persistent kernel: for every CTA, a row of
- * n_marks + 1 values: the GPU global timer (ns) at entry to and exit from each of its grid
- * barriers, out[cta * (n_marks + 1) + 2*b] and [.. + 2*b + 1] for barrier b, then the id of the
- * SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
+ * n_marks + 1 values: for each of its grid barriers b the GPU global timer (ns) at entry
+ * (out[cta * (n_marks + 1) + 3*b]), at exit (.. + 3*b + 1) and at the moment the CTA had drained
+ * its last accumulator of the phase that ends at the barrier (.. + 3*b + 2; 0 for phases without
+ * a GEMM), then the id of the SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
  * QKV GEMM + q/k-norm + RoPE + K/V write, attention, its combine, O GEMM + residual add,
  * gate/up GEMM + SwiGLU, down GEMM + residual add.  Marks are recorded only while
  * s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */

@@ -336,13 +336,14 @@ class Engine:
         return y
 
     def debug_pass_trace(self) -> np.ndarray:
-        """(marks [n_ctas, n_barriers, 2], sm_ids [n_ctas]): global-timer ns at entry/exit of every grid
-        barrier of the last persistent pass, and the SM each CTA ran on."""
-        buf = np.zeros(256 * (2 * (10 * self.model.n_layers + 2) + 1), dtype=np.uint64)
+        """(marks [n_ctas, n_barriers, 3], sm_ids [n_ctas]): global-timer ns at entry to / exit from every grid
+        barrier of the last persistent pass and at the end of the phase's accumulator drain (0 if none), and
+        the SM each CTA ran on."""
+        buf = np.zeros(256 * (3 * (6 * self.model.n_layers + 1) + 1), dtype=np.uint64)
         nc, nm = C.c_int32(), C.c_int32()
         self._check(self.lib.s2d2_debug_pass_trace(self._h, buf.ctypes.data, buf.size, C.byref(nc), C.byref(nm)))
         rows = buf[: nc.value * (nm.value + 1)].reshape(nc.value, nm.value + 1)
-        return rows[:, :nm.value].reshape(nc.value, nm.value // 2, 2), rows[:, nm.value].astype(np.int64)
+        return rows[:, :nm.value].reshape(nc.value, nm.value // 3, 3), rows[:, nm.value].astype(np.int64)
 
     def debug_copy_expert_ids(self, max_rows: int) -> np.ndarray:
         k, nl = self.model.top_k, self.model.n_layers

@@ -32,6 +32,7 @@ struct PassState {
     unsigned* barrier = nullptr;     // [64 | tile counters of the 5 GEMM kinds], zeroed before every launch
     size_t sync_bytes = 0;
     size_t cnt_off[5] = {0, 0, 0, 0, 0};
+    size_t xcnt_off[3] = {0, 0, 0};
     unsigned long long* trace = nullptr;
     int trace_cap = 0;
     int last_marks = 0;
@@ -129,6 +130,11 @@ int pass_init(s2d2_ctx* c) {
             s->cnt_off[k] = o;
             o += (size_t)((Ns[k] + 127) / 128);
         }
+        const long long Xs[3] = {d, nq, f};       // columns of xn, attn, act
+        for (int k = 0; k < 3; ++k) {
+            s->xcnt_off[k] = o;
+            o += (size_t)((Xs[k] + 127) / 128);
+        }
         s->sync_bytes = o * 4;
         if (cudaMalloc((void**)&s->barrier, s->sync_bytes) != cudaSuccess) {
             c->err = "cudaMalloc failed for the persistent pass";
@@ -164,7 +170,7 @@ int pass_init(s2d2_ctx* c) {
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
-    s->trace_cap = 2 * (6 * L + 1) + 1;      // two marks per grid barrier + the SM id
+    s->trace_cap = 3 * (6 * L + 1) + 1;      // three marks per grid barrier + the SM id
     if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) {
         c->err = "cudaMalloc failed for the persistent pass";
         return S2D2_ERR_CUDA;
@@ -259,10 +265,11 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     for (int k = 0; k < 5; ++k) p.parts[k] = s->parts[k];
     p.trace = c->tracing ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    if (c->tracing) s->last_marks = 2 * (6 * m.n_layers + 1);
+    if (c->tracing) s->last_marks = 3 * (6 * m.n_layers + 1);
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
     for (int k = 0; k < 5; ++k) p.tile_cnt[k] = s->barrier + s->cnt_off[k];
+    for (int k = 0; k < 3; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];
     void* args[] = {&p};
     gemm_prof_begin(c);
     cudaError_t e = m.head_dim == 128

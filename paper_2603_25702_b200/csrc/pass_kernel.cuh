@@ -12,7 +12,7 @@
 //             other operation, so while the CTA sits in a grid barrier, an element-wise phase or
 //             attention, the next GEMM's weights are already arriving.
 //   warp 1    X producer: TMA-loads the matching 64-column slices of the token rows into the same
-//             stages once the grid barrier that publishes them has been passed.
+//             stages as soon as the phase that writes them has counted their columns complete.
 //   warp 2    issues tcgen05.mma (weight tile = M operand, token rows = N operand, fp32
 //             accumulators double-buffered in tensor memory).
 //   warps 4-7 everything else: drain accumulators to split-K partials, then between grid barriers
@@ -74,10 +74,12 @@ struct PassParams {
     att::AttnParams ap;       // attention geometry of this pass (layer filled in per layer)
     unsigned* barrier;        // grid barrier counter, zero at launch
     unsigned* tile_cnt[5];    // per GEMM kind and weight tile: partials published so far (zero at launch)
+    unsigned* x_cnt[3];       // per 128-column tile of xn / attn / act: (tile, row) pairs written so far (zero at launch)
     int* status;
     int S;                    // ring stages
     const int* parts[5];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
-    unsigned long long* trace;   // [grid][trace_cap] globaltimer at entry and exit of every grid barrier
+    unsigned long long* trace;   // [grid][trace_cap] per grid barrier: globaltimer at entry, at exit, and when the
+                                 // CTA's last accumulator of the phase had been drained (0 if the phase has no GEMM)
     int trace_cap;
 };
 
@@ -109,11 +111,6 @@ __device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int 
     g.U = (long long)g.n_tiles * g.kbt;
     return g;
 }
-// Grid barriers passed before the inputs of a GEMM are published.
-__device__ __forceinline__ unsigned gemm_epoch(const PassParams& p, int l, int kind) {
-    const unsigned off[5] = {1u, 4u, 5u, 6u, 1u};
-    return off[kind] + 6u * (unsigned)(kind == 4 ? p.n_layers : l);
-}
 __device__ __forceinline__ long long unit_begin(long long U, int c, int G) { return U * c / G; }
 
 // Calls f(tile, kb0, kb1, local_segment) for the segments of this CTA's unit range.
@@ -132,6 +129,11 @@ __device__ __forceinline__ void for_each_segment(const GemmShape& g, int cta, in
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc::smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ unsigned ld_relaxed(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -193,61 +195,87 @@ struct UnitCursor {
     }
 };
 // Sum over the split-K partials (in CTA order) of 4 consecutive columns of (tile, row): every
-// lane of a warp takes columns 4*lane .. 4*lane+3; the loads of up to PCH parts are in flight
-// together.  tile_row_tab fetches the tile's slot list (one entry per lane) ahead of time.
-constexpr int PCH = 8;
+// lane of a warp takes columns 4*lane .. 4*lane+3.  tile_row_tab fetches the tile's slot list
+// (count, then slots; one entry per lane) ahead of time.
 __device__ __forceinline__ int tile_row_tab(const PassParams& p, int kind, int tile, int lane) {
     return lane <= MAX_PARTS ? __ldg(p.parts[kind] + (size_t)tile * (1 + MAX_PARTS) + lane) : 0;
 }
-// Before reading, the warp waits (bounded) until all `cnt * round` partials of the tile have been
-// published by the CTAs that drained them (round = layer + 1: the counters only grow).
-__device__ __forceinline__ float4 tile_row_sum(const PassParams& p, int tab_lane, int row, int lane, const unsigned* published,
-                                               unsigned round, volatile int* abort_flag) {
-    const int cnt = __shfl_sync(0xffffffffu, tab_lane, 0);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+// NS such sums at once (tab_lane[s] = 0 marks an unused one).  Before reading, the warp waits
+// (bounded) until all `cnt * round` partials of each tile have been published by the CTAs that
+// drained them (round = layer + 1: the counters only grow).  Then the loads of up to PC parts of
+// every sum are issued together, and each sum is accumulated in part order.
+template <int NS, int PC>
+__device__ __forceinline__ bool tile_row_sums(const PassParams& p, const int (&tab_lane)[NS], const int (&row)[NS],
+                                              const unsigned* const (&published)[NS], unsigned round, int lane,
+                                              volatile int* abort_flag, float4 (&out)[NS]) {
+    int cnt[NS], max_cnt = 0;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        cnt[s] = __shfl_sync(0xffffffffu, tab_lane[s], 0);
+        max_cnt = max(max_cnt, cnt[s]);
+        out[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     {
-        const unsigned target = (unsigned)cnt * round;
         bool ready = false;
-        for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-            if (ld_acquire(published) >= target) {
-                ready = true;
-                break;
-            }
-            if ((it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
+        // relaxed polls of all counters at once (acquire loads would complete one after the other),
+        // then one fence orders the data loads after what the counters published
+        for (uint32_t it = 0; it < SPIN_LIMIT && !ready; ++it) {
+            unsigned seen[NS];
+#pragma unroll
+            for (int s = 0; s < NS; ++s) seen[s] = cnt[s] > 0 ? ld_relaxed(published[s]) : 0u;
+            ready = true;
+#pragma unroll
+            for (int s = 0; s < NS; ++s)
+                if (cnt[s] > 0 && seen[s] < (unsigned)cnt[s] * round) ready = false;
+            if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
         }
+        asm volatile("fence.acq_rel.gpu;" ::: "memory");
         if (!ready) {
             atomicCAS(p.status, 0, 8);
             *abort_flag = 1;
-            return acc;
+            return false;
         }
     }
-    for (int j0 = 0; j0 < cnt; j0 += PCH) {
-        float4 v[PCH];
+    for (int j0 = 0; j0 < max_cnt; j0 += PC) {
+        float4 v[NS][PC];
 #pragma unroll
-        for (int j = 0; j < PCH; ++j) {
-            const int slot = __shfl_sync(0xffffffffu, tab_lane, (j0 + j + 1) & 31);
-            v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (j0 + j < cnt) v[j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row) * tc::BLOCK_N) + lane);
-        }
+        for (int s = 0; s < NS; ++s)
 #pragma unroll
-        for (int j = 0; j < PCH; ++j) {
-            acc.x += v[j].x;
-            acc.y += v[j].y;
-            acc.z += v[j].z;
-            acc.w += v[j].w;
-        }
+            for (int j = 0; j < PC; ++j) {
+                const int slot = __shfl_sync(0xffffffffu, tab_lane[s], (j0 + j + 1) & 31);
+                v[s][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (j0 + j < cnt[s])
+                    v[s][j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row[s]) * tc::BLOCK_N) + lane);
+            }
+#pragma unroll
+        for (int s = 0; s < NS; ++s)
+#pragma unroll
+            for (int j = 0; j < PC; ++j) {
+                out[s].x += v[s][j].x;
+                out[s].y += v[s][j].y;
+                out[s].z += v[s][j].z;
+                out[s].w += v[s][j].w;
+            }
     }
-    return acc;
+    return true;
 }
-// 1/rms of a row from the per-tile sums of squares of h, in two steps so that the loads of the
-// first are in flight together with whatever the caller loads next: lanes take the tiles.
-__device__ __forceinline__ float row_ssq_lane(const float* ssq, int d_tiles, int row, int lane) {
-    float s = 0.f;
-    for (int t = lane; t < d_tiles; t += 32) s += __ldcg(ssq + (size_t)t * MAX_T + row);
-    return s;
+// 1/rms of a row from the per-tile sums of squares of h, in two steps: the loads (lanes take
+// the tiles; nothing consumes them here, so they stay in flight with whatever the caller loads
+// next), and later the sum.  Up to 128 tiles (d <= 16384).
+struct SsqLane {
+    float v[4];
+};
+__device__ __forceinline__ SsqLane row_ssq_lane(const float* ssq, int d_tiles, int row, int lane) {
+    SsqLane r;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int t = lane + 32 * k;
+        r.v[k] = t < d_tiles ? __ldcg(ssq + (size_t)t * MAX_T + row) : 0.f;
+    }
+    return r;
 }
-__device__ __forceinline__ float inv_rms_from(float lane_part, int d, float eps) {
-    return 1.0f / sqrtf(warp_sum(lane_part) / (float)d + eps);
+__device__ __forceinline__ float inv_rms_from(const SsqLane& r, int d, float eps) {
+    return 1.0f / sqrtf(warp_sum((r.v[0] + r.v[1]) + (r.v[2] + r.v[3])) / (float)d + eps);
 }
 __device__ __forceinline__ void store_bf16x4(bf16* dst, float a, float b, float c, float d) {
     __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
@@ -337,37 +365,59 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- X producer: token-row slices, after their grid barrier ----------------
-            uint32_t i = 0;
-            bool ok = true;
-            for (int gi = 0; gi < n_gemms && ok; ++gi) {
-                const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
-                const GemmShape g = gemm_shape(p, l, kind);
-                const CUtensorMap* mx = p.maps + g.map_x;
-                if (unit_begin(g.U, cta + 1, G) > unit_begin(g.U, cta, G)) {
-                    if (!wait_counter(p, gemm_epoch(p, l, kind) * (unsigned)G, abort_flag)) {
-                        ok = false;
-                        break;
+        // ---------------- X producer: token-row slices, as soon as their columns are written ----------------
+        // The phases that write a GEMM's input count the finished (128-column tile, row) pairs per
+        // tile; the lanes of this warp poll the tiles a segment needs in parallel, lane 0 issues the
+        // copies.  The inputs are therefore fetched without waiting for the grid barrier, which only
+        // guards buffer reuse.
+        uint32_t i = 0;
+        bool ok = true;
+        for (int gi = 0; gi < n_gemms && ok; ++gi) {
+            const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
+            const GemmShape g = gemm_shape(p, l, kind);
+            const CUtensorMap* mx = p.maps + g.map_x;
+            // which counter set, and how many pairs make a tile complete for this GEMM
+            const unsigned* cnt;
+            unsigned target;
+            switch (kind) {
+                case 0: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 1u); break;
+                case 1: cnt = p.x_cnt[1]; target = (unsigned)p.M * (unsigned)(tc::BLOCK_N / HD) * (l + 1u); break;
+                case 2: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 2u); break;
+                case 3: cnt = p.x_cnt[2]; target = (unsigned)p.M * (l + 1u); break;
+                default: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * p.n_layers + 1u); break;
+            }
+            for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
+                // tiles of 128 columns = 2 k-blocks
+                for (int t0 = kb0 >> 1; t0 <= (kb1 - 1) >> 1; t0 += 32) {
+                    const int t = t0 + lane;
+                    bool ready = t > ((kb1 - 1) >> 1);
+                    for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
+                        ready = ld_acquire(cnt + t) >= target;
+                        if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
                     }
-                    asm volatile("fence.proxy.async;" ::: "memory");
+                    if (!__all_sync(0xffffffffu, ready)) return ok = false;
                 }
-                for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
-                    for (int kb = kb0; kb < kb1; ++kb, ++i) {
-                        int s = (int)(i % (uint32_t)S);
-                        if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) return ok = false;
-                        if (*abort_flag) return ok = false;
-                        tc::mbar_expect_tx(&full[s], (uint32_t)T * 128u);
-                        tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, 0, &full[s]);
-                        *x_issued = (int)i + 1;
+                asm volatile("fence.proxy.async;" ::: "memory");
+                for (int kb = kb0; kb < kb1; ++kb, ++i) {
+                    int s = (int)(i % (uint32_t)S);
+                    bool fine = true;
+                    if (lane == 0) {
+                        if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) fine = false;
+                        if (*abort_flag) fine = false;
+                        if (fine) {
+                            tc::mbar_expect_tx(&full[s], (uint32_t)T * 128u);
+                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, 0, &full[s]);
+                            *x_issued = (int)i + 1;
+                        }
                     }
-                    return true;
-                });
-            }
-            if (!ok) {
-                atomicCAS(p.status, 0, 3);
-                *abort_flag = 1;
-            }
+                    if (!__all_sync(0xffffffffu, fine)) return ok = false;
+                }
+                return true;
+            });
+        }
+        if (!ok && lane == 0) {
+            atomicCAS(p.status, 0, 3);
+            *abort_flag = 1;
         }
     } else if (warp == 2) {
         if (lane == 0) {
@@ -418,12 +468,13 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // inputs, K/V pages), which needs the generic-to-async proxy fence on the writer side.
         // One thread publishes for the CTA: its release covers the writes the CTA barrier ordered
         // before it.
+        unsigned long long t_drained = 0;
         auto grid_sync = [&](bool tma_out) {
             ++epoch;
             if (tma_out) asm volatile("fence.proxy.async;" ::: "memory");
             att::group_sync(BAR_COMPUTE, CTHREADS);
             if (tid == 0) {
-                const int k = 2 * (int)epoch - 2;
+                const int k = 3 * (int)epoch - 3;
                 unsigned long long t0 = 0, t1 = 0;
                 if (p.trace) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
@@ -431,10 +482,12 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     atomicCAS(p.status, 0, 5);
                     *abort_flag = 1;
                 }
-                if (p.trace && k + 1 < p.trace_cap - 1) {
+                if (p.trace && k + 2 < p.trace_cap - 1) {
                     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
                     p.trace[(size_t)cta * p.trace_cap + k] = t0;
                     p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
+                    p.trace[(size_t)cta * p.trace_cap + k + 2] = t_drained;
+                    t_drained = 0;
                 }
             }
             att::group_sync(BAR_COMPUTE, CTHREADS);
@@ -469,6 +522,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 atomicCAS(p.status, 0, 6);
                 *abort_flag = 1;
             }
+            if (p.trace && tid == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_drained));
         };
         // The element-wise phases work warp by warp on (tile, row) pairs: 128 output columns of one
         // row, 4 per lane.  A pair's loads (its partials, its residual row, the sums of squares) are
@@ -477,6 +531,12 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
 
         // h update shared by the embedding and the two residual phases: writes h, the next GEMM's
         // input bf16(h * gain) and the (tile, row) sum of squares
+        // A (tile, row) pair of a GEMM input is written: make it visible to TMA readers and count it.
+        auto publish_x = [&](unsigned* counter) {
+            asm volatile("fence.proxy.async;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
+        };
         auto h_phase = [&](const float* gain, float* ssq, auto&& value) {
             for (int pair = gw; pair < d_tiles * M; pair += GW) {
                 const int t = pair / M, m = pair % M;
@@ -487,13 +547,18 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 store_bf16x4(p.xn + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
                 const float sq = warp_sum(x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w);
                 if (lane == 0) ssq[(size_t)t * MAX_T + m] = sq;
+                publish_x(p.x_cnt[0] + t);
             }
         };
         auto residual_phase = [&](int kind, unsigned round, const float* gain, float* ssq) {
             h_phase(gain, ssq, [&](int t, int m, int col) {
                 const int tab = tile_row_tab(p, kind, t, lane);
                 const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
-                float4 x = tile_row_sum(p, tab, m, lane, p.tile_cnt[kind] + t, round, abort_flag);
+                const int tabs[1] = {tab}, rows[1] = {m};
+                const unsigned* const pubs[1] = {p.tile_cnt[kind] + t};
+                float4 sums[1];
+                tile_row_sums<1, 8>(p, tabs, rows, pubs, round, lane, abort_flag, sums);
+                float4 x = sums[0];
                 x.x += hv.x;
                 x.y += hv.y;
                 x.z += hv.z;
@@ -524,53 +589,77 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             {
                 constexpr int half = HD / 2, PART = half / 4;     // PART: lane distance of a RoPE pair
                 const int n_tiles = (p.Hq + 2 * p.Hkv) * HD / tc::BLOCK_N;
-                for (int pair = gw; pair < n_tiles * M; pair += GW) {
-                    const int t = pair / M, m = pair % M;
-                    const int c_tile = 4 * lane;                    // column inside the tile
-                    const int head = (t * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
-                    const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
-                    // everything this pair reads is requested before anything is used
-                    const int tab = tile_row_tab(p, 0, t, lane);
-                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
-                    const int pos = __ldg(p.pv.row_pos + m), flags = __ldg(p.pv.row_flags + m), sq = __ldg(p.pv.row_seq + m);
-                    const bool second = ch >= half;
-                    const int i0 = ch - (second ? half : 0);
-                    const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * half + i0));
-                    const float4 sn = __ldg(reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * half + i0));
-                    const int page = (flags & ROW_WRITE_KV) ? __ldg(p.pv.seq_pages + (size_t)sq * p.pv.max_pages + (pos >> p.pool.page_shift)) : 0;
-                    float4 gq = make_float4(1.f, 1.f, 1.f, 1.f);
-                    if (p.qk_norm && (is_q || is_k)) gq = __ldg(reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch));
-                    float4 s4 = tile_row_sum(p, tab, m, lane, p.tile_cnt[0] + t, (unsigned)l + 1u, abort_flag);
-                    const float inv = inv_rms_from(sq_l, d, p.eps);
-                    float x[4] = {inv * s4.x, inv * s4.y, inv * s4.z, inv * s4.w};
-                    if (p.qk_norm) {
-                        float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
+                const int c_tile = 4 * lane;                        // column inside the tile
+                const int n_pairs = n_tiles * M;
+                // two pairs per step; everything a step reads is requested before anything is used
+                for (int pair0 = gw; pair0 < n_pairs; pair0 += 2 * GW) {
+                    int tt[2], mm[2], tabs[2], pos[2], flags[2], page[2];
+                    SsqLane sq_l[2];
+                    float4 cs[2], sn[2], gq[2];
+                    bool on[2];
+                    const unsigned* pubs[2];
 #pragma unroll
-                        for (int o = HD / 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);   // over the head's lanes
-                        if (is_q || is_k) {
-                            const float hinv = 1.0f / sqrtf(ss / (float)HD + p.eps);
-                            x[0] *= hinv * gq.x;
-                            x[1] *= hinv * gq.y;
-                            x[2] *= hinv * gq.z;
-                            x[3] *= hinv * gq.w;
-                        }
+                    for (int q = 0; q < 2; ++q) {
+                        const int pr = pair0 + q * GW;
+                        on[q] = pr < n_pairs;
+                        tt[q] = on[q] ? pr / M : 0;
+                        mm[q] = on[q] ? pr % M : 0;
+                        const int head = (tt[q] * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
+                        const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
+                        tabs[q] = on[q] ? tile_row_tab(p, 0, tt[q], lane) : 0;
+                        pubs[q] = p.tile_cnt[0] + tt[q];
+                        sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, mm[q], lane);
+                        pos[q] = __ldg(p.pv.row_pos + mm[q]);
+                        flags[q] = __ldg(p.pv.row_flags + mm[q]);
+                        const int sq = __ldg(p.pv.row_seq + mm[q]);
+                        const int i0 = ch - (ch >= half ? half : 0);
+                        cs[q] = __ldg(reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos[q] * half + i0));
+                        sn[q] = __ldg(reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos[q] * half + i0));
+                        page[q] = (flags[q] & ROW_WRITE_KV) ? __ldg(p.pv.seq_pages + (size_t)sq * p.pv.max_pages + (pos[q] >> p.pool.page_shift)) : 0;
+                        gq[q] = make_float4(1.f, 1.f, 1.f, 1.f);
+                        if (p.qk_norm && (is_q || is_k)) gq[q] = __ldg(reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch));
                     }
-                    {   // rotate-half RoPE: element i of the first half pairs with i + half
-                        const float c4[4] = {cs.x, cs.y, cs.z, cs.w}, s4r[4] = {sn.x, sn.y, sn.z, sn.w};
+                    float4 sums[2];
+                    const unsigned* const pubs_c[2] = {pubs[0], pubs[1]};
+                    tile_row_sums<2, 8>(p, tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float other = __shfl_xor_sync(0xffffffffu, x[e], PART);
-                            const float y = second ? x[e] * c4[e] + other * s4r[e] : x[e] * c4[e] - other * s4r[e];
-                            if (is_q || is_k) x[e] = y;
+                    for (int q = 0; q < 2; ++q) {
+                        const float inv = inv_rms_from(sq_l[q], d, p.eps);
+                        if (!on[q]) continue;                          // warp-uniform
+                        const int t = tt[q], m = mm[q];
+                        const int head = (t * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
+                        const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
+                        const bool second = ch >= half;
+                        float x[4] = {inv * sums[q].x, inv * sums[q].y, inv * sums[q].z, inv * sums[q].w};
+                        if (p.qk_norm) {
+                            float ss = x[0] * x[0] + x[1] * x[1] + x[2] * x[2] + x[3] * x[3];
+#pragma unroll
+                            for (int o = HD / 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);   // over the head's lanes
+                            if (is_q || is_k) {
+                                const float hinv = 1.0f / sqrtf(ss / (float)HD + p.eps);
+                                x[0] *= hinv * gq[q].x;
+                                x[1] *= hinv * gq[q].y;
+                                x[2] *= hinv * gq[q].z;
+                                x[3] *= hinv * gq[q].w;
+                            }
                         }
-                    }
-                    if (is_q) {
-                        store_bf16x4(p.q + ((size_t)m * p.Hq + head) * HD + ch, x[0], x[1], x[2], x[3]);
-                    } else {
-                        const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
-                        store_bf16x4((is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD + ch, x[0], x[1], x[2], x[3]);
-                        if (flags & ROW_WRITE_KV) {
-                            store_bf16x4(p.pool.ptr(l, page, is_k ? 0 : 1, kvh, pos & (p.pool.page_tokens - 1)) + ch, x[0], x[1], x[2], x[3]);
+                        {   // rotate-half RoPE: element i of the first half pairs with i + half
+                            const float c4[4] = {cs[q].x, cs[q].y, cs[q].z, cs[q].w}, s4r[4] = {sn[q].x, sn[q].y, sn[q].z, sn[q].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float other = __shfl_xor_sync(0xffffffffu, x[e], PART);
+                                const float y = second ? x[e] * c4[e] + other * s4r[e] : x[e] * c4[e] - other * s4r[e];
+                                if (is_q || is_k) x[e] = y;
+                            }
+                        }
+                        if (is_q) {
+                            store_bf16x4(p.q + ((size_t)m * p.Hq + head) * HD + ch, x[0], x[1], x[2], x[3]);
+                        } else {
+                            const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+                            store_bf16x4((is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD + ch, x[0], x[1], x[2], x[3]);
+                            if (flags[q] & ROW_WRITE_KV)
+                                store_bf16x4(p.pool.ptr(l, page[q], is_k ? 0 : 1, kvh, pos[q] & (p.pool.page_tokens - 1)) + ch, x[0], x[1], x[2],
+                                             x[3]);
                         }
                     }
                 }
@@ -649,6 +738,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     if (lane < HD / 4) {
                         store_bf16x4(p.attn + ((size_t)r * p.Hq + hq) * HD + 4 * lane, acc.x / lsum, acc.y / lsum, acc.z / lsum, acc.w / lsum);
                     }
+                    publish_x(p.x_cnt[1] + hq * HD / tc::BLOCK_N);
                 }
             }
             grid_sync(true);
@@ -664,37 +754,49 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (!ok) break;
             {
                 const int f_tiles = p.f / tc::BLOCK_N, n_pairs = f_tiles * M;
-                // two (tile, row) pairs per step so that both pairs' loads overlap
-                for (int pair = gw; pair < n_pairs; pair += 2 * GW) {
-                    int tt[2], mm[2], tg[2], tu[2];
-                    float sq_l[2];
-                    bool on[2];
+                // three (tile, row) pairs per step so that all their loads overlap
+                constexpr int NP = 3;
+                for (int pair = gw; pair < n_pairs; pair += NP * GW) {
+                    int tt[NP], mm[NP], tabs[2 * NP], rows[2 * NP];
+                    const unsigned* pubs[2 * NP];
+                    SsqLane sq_l[NP];
+                    bool on[NP];
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
+                    for (int q = 0; q < NP; ++q) {
                         const int pr = pair + q * GW;
                         on[q] = pr < n_pairs;
                         tt[q] = on[q] ? pr / M : 0;
                         mm[q] = on[q] ? pr % M : 0;
-                        tg[q] = tile_row_tab(p, 2, tt[q], lane);
-                        tu[q] = tile_row_tab(p, 2, tt[q] + f_tiles, lane);
+                        tabs[2 * q] = on[q] ? tile_row_tab(p, 2, tt[q], lane) : 0;
+                        tabs[2 * q + 1] = on[q] ? tile_row_tab(p, 2, tt[q] + f_tiles, lane) : 0;
+                        rows[2 * q] = rows[2 * q + 1] = mm[q];
+                        pubs[2 * q] = p.tile_cnt[2] + tt[q];
+                        pubs[2 * q + 1] = p.tile_cnt[2] + tt[q] + f_tiles;
                         sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane);
                     }
-                    float4 g4[2], u4[2];
+                    float4 sums[2 * NP];
+                    const unsigned* const pubs_c[2 * NP] = {pubs[0], pubs[1], pubs[2], pubs[3], pubs[4], pubs[5]};
+                    tile_row_sums<2 * NP, 4>(p, tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        g4[q] = tile_row_sum(p, tg[q], mm[q], lane, p.tile_cnt[2] + tt[q], (unsigned)l + 1u, abort_flag);
-                        u4[q] = tile_row_sum(p, tu[q], mm[q], lane, p.tile_cnt[2] + tt[q] + f_tiles, (unsigned)l + 1u, abort_flag);
-                    }
-#pragma unroll
-                    for (int q = 0; q < 2; ++q) {
+                    for (int q = 0; q < NP; ++q) {
                         const float inv = inv_rms_from(sq_l[q], d, p.eps);
                         if (!on[q]) continue;
-                        const float gv[4] = {inv * g4[q].x, inv * g4[q].y, inv * g4[q].z, inv * g4[q].w};
-                        const float uv[4] = {inv * u4[q].x, inv * u4[q].y, inv * u4[q].z, inv * u4[q].w};
+                        const float4 g4 = sums[2 * q], u4 = sums[2 * q + 1];
+                        const float gv[4] = {inv * g4.x, inv * g4.y, inv * g4.z, inv * g4.w};
+                        const float uv[4] = {inv * u4.x, inv * u4.y, inv * u4.z, inv * u4.w};
                         float a[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) a[e] = gv[e] / (1.f + expf(-gv[e])) * uv[e];
+                        for (int e = 0; e < 4; ++e) a[e] = __fdividef(gv[e], 1.f + __expf(-gv[e])) * uv[e];   // bf16 output: 2^-9 rounding dominates
                         store_bf16x4(p.act + (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane, a[0], a[1], a[2], a[3]);
+                    }
+                    // one fence for the step's stores, then one count per finished pair
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("fence.acq_rel.gpu;" ::: "memory");
+#pragma unroll
+                        for (int q = 0; q < NP; ++q)
+                            if (on[q]) asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p.x_cnt[2] + tt[q]) : "memory");
                     }
                 }
             }
@@ -716,8 +818,12 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     const int t = pair / p.n_logit, lr = pair % p.n_logit;
                     const int m = p.pv.logit_rows[lr];
                     const int tab = tile_row_tab(p, 4, t, lane);
-                    const float sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
-                    const float4 s4 = tile_row_sum(p, tab, m, lane, p.tile_cnt[4] + t, 1u, abort_flag);
+                    const SsqLane sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
+                    const int tabs[1] = {tab}, rows[1] = {m};
+                    const unsigned* const pubs[1] = {p.tile_cnt[4] + t};
+                    float4 sums[1];
+                    tile_row_sums<1, 8>(p, tabs, rows, pubs, 1u, lane, abort_flag, sums);
+                    const float4 s4 = sums[0];
                     const float sc = p.logit_scale * inv_rms_from(sq_l, d, p.eps);
                     const int col = t * tc::BLOCK_N + 4 * lane;
                     float* dst = p.logits + (size_t)lr * p.V + col;
