@@ -30,6 +30,18 @@ def widen(w: np.ndarray) -> np.ndarray:
     return w.astype(np.float64)
 
 
+def as_stored_kv(x: np.ndarray, cfg) -> np.ndarray:
+    """K and V as the cache holds them.  The cache of a bf16 model stores bfloat16 (the
+    workloads name a "paged bf16 KV cache"), so for such a model K and V are bfloat16 values
+    wherever they are used: rounded once, to nearest even, where they are produced (after
+    RoPE for K).  fp32 models keep them unrounded in the oracle.  Returned widened to fp64."""
+    if cfg.dtype != "bf16":
+        return x
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
 def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
     """x / sqrt(mean(x^2) + eps) * gain over the last axis."""
     ms = np.mean(x * x, axis=-1, keepdims=True)
@@ -126,7 +138,8 @@ def forward(W: Dict[str, np.ndarray], cfg, tokens, positions, inblock_mask,
             q = rmsnorm(q, widen(W[p + "q_norm"]), cfg.rms_eps)
             k = rmsnorm(k, widen(W[p + "k_norm"]), cfg.rms_eps)
         q = rope(q, positions, cfg.rope_base)
-        k = rope(k, positions, cfg.rope_base)
+        k = as_stored_kv(rope(k, positions, cfg.rope_base), cfg)
+        v = as_stored_kv(v, cfg)
         kv_rows.append((k, v))
         if kv_prefix is not None and kv_prefix[l][0].shape[0] > 0:
             K_all = np.concatenate([kv_prefix[l][0], k], axis=0)

@@ -104,6 +104,7 @@ bool attention_plan(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, 
     if (!a || !a->tc_ok) return false;
     att::AttnParams p;
     p.q = (const bf16*)c->q;
+    p.q_lo = nullptr;
     p.k_rows = (const bf16*)c->k_rows;
     p.v_rows = (const bf16*)c->v_rows;
     p.out = (bf16*)c->attn;

@@ -27,6 +27,7 @@ constexpr int STAGES = 2;
 
 struct AttnParams {
     const bf16* q;              // [M, Hq, HD]
+    const bf16* q_lo;           // low halves of q (q = hi + lo, both bf16) for the two-term variant, else unused
     const bf16* k_rows;         // [M, Hkv, HD] K of this pass's rows
     const bf16* v_rows;
     bf16* out;                  // [M, Hq*HD]
@@ -94,7 +95,10 @@ __device__ __forceinline__ uint4 ldcg16(const void* p) { return __ldcg(reinterpr
 // far (it carries the barrier phase from one item to the next).  Activations are read with
 // L2-only loads: inside a persistent kernel they are rewritten by other CTAs between items.
 // Returns false when a bounded wait ran out (the status word is raised).
-template <int HD>
+// HL: two-term arithmetic.  q arrives as hi + lo (both bf16) and the probabilities are split the
+// same way, so that S = (q_hi + q_lo) K^T and O += (p_hi + p_lo) V carry 16 significant bits of q
+// and p; K and V are bf16 as the cache stores them.  Costs twice the (tiny) tensor work.
+template <int HD, bool HL = false>
 __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
                                           uint8_t* base, uint64_t* full, uint32_t& ring_pos, int tid, int bar_id) {
     constexpr int CH = HD / 8;          // 16-byte chunks per row
@@ -142,16 +146,19 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
         for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
 
     // ---- Q tile: global -> swizzled shared -> A fragments ----
+    constexpr int NQ = QT * CH / THREADS;
+    uint4 q_lo_val[HL ? NQ : 1];
     {   // all loads first, then the stores: one round trip for the tile
-        constexpr int NQ = QT * CH / THREADS;
         uint4 val[NQ];
 #pragma unroll
         for (int k = 0; k < NQ; ++k) {
             const int i = tid + k * THREADS, r = i / CH, c = i % CH, qv = q0 + r;
             val[k] = make_uint4(0, 0, 0, 0);
+            if (HL) q_lo_val[k] = val[k];
             if (qv < nq) {
                 int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
                 val[k] = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+                if (HL) q_lo_val[k] = ldcg16(p.q_lo + ((size_t)row * p.Hq + hq) * HD + c * 8);
             }
         }
 #pragma unroll
@@ -185,7 +192,7 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
         }
     }
     group_sync(bar_id, THREADS);
-    uint32_t qf[KS][4];
+    uint32_t qf[KS][4], qf_lo[HL ? KS : 1][4];
     {
         const uint32_t qb = tc::smem_u32(q_s);
         int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -193,6 +200,20 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
         for (int ks = 0; ks < KS; ++ks) {
             int c = ks * 2 + (lane >> 4);
             ldsm_x4(qb + sw_off(r, c, QT), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+        }
+        if (HL) {   // the low halves pass through the same tile
+            group_sync(bar_id, THREADS);
+#pragma unroll
+            for (int k = 0; k < NQ; ++k) {
+                const int i = tid + k * THREADS, rr = i / CH, c = i % CH;
+                *reinterpret_cast<uint4*>(q_s + sw_off(rr, c, QT)) = q_lo_val[k];
+            }
+            group_sync(bar_id, THREADS);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                int c = ks * 2 + (lane >> 4);
+                ldsm_x4(qb + sw_off(r, c, QT), qf_lo[ks][0], qf_lo[ks][1], qf_lo[ks][2], qf_lo[ks][3]);
+            }
         }
     }
     // masks of this thread's two query vectors (rows g and g + 8 of the warp's 16)
@@ -236,6 +257,10 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
                     ldsm_x4(kb + sw_off(r, c, rows_t), b0, b1, b2, b3);
                     mma_bf16(sc[np * 2], qf[ks], b0, b1);
                     mma_bf16(sc[np * 2 + 1], qf[ks], b2, b3);
+                    if (HL) {
+                        mma_bf16(sc[np * 2], qf_lo[ks], b0, b1);
+                        mma_bf16(sc[np * 2 + 1], qf_lo[ks], b2, b3);
+                    }
                 }
             }
         }
@@ -266,7 +291,7 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
         m_a = mn_a;
         m_b = mn_b;
         float sum_a = 0.f, sum_b = 0.f;
-        uint32_t pf[4][4];
+        uint32_t pf[4][4], pf_lo[HL ? 4 : 1][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
             float p0 = exp2f(sc[nt][0] - ref_a), p1 = exp2f(sc[nt][1] - ref_a);
@@ -274,8 +299,14 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
             sum_a += p0 + p1;
             sum_b += p2 + p3;
             // C fragments of two adjacent key n-tiles are the A fragment of one 16-key k-step
-            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+            const uint32_t h01 = pack_bf16(p0, p1), h23 = pack_bf16(p2, p3);
+            pf[nt >> 1][(nt & 1) * 2 + 0] = h01;
+            pf[nt >> 1][(nt & 1) * 2 + 1] = h23;
+            if (HL) {
+                const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&h01), b = *reinterpret_cast<const __nv_bfloat162*>(&h23);
+                pf_lo[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0 - __low2float(a), p1 - __high2float(a));
+                pf_lo[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2 - __low2float(b), p3 - __high2float(b));
+            }
         }
         l_a = l_a * corr_a + sum_a;
         l_b = l_b * corr_b + sum_b;
@@ -298,6 +329,10 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
                     ldsm_x4_t(vb + sw_off(r, c, rows_t), b0, b1, b2, b3);
                     mma_bf16(o[np * 2], pf[kk], b0, b1);
                     mma_bf16(o[np * 2 + 1], pf[kk], b2, b3);
+                    if (HL) {
+                        mma_bf16(o[np * 2], pf_lo[kk], b0, b1);
+                        mma_bf16(o[np * 2 + 1], pf_lo[kk], b2, b3);
+                    }
                 }
             }
         }

@@ -27,6 +27,7 @@ struct PassState {
     CUtensorMap* d_maps = nullptr;
     pp::LayerGains* d_gains = nullptr;
     float* ws = nullptr;
+    bf16 *xn_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr, *q_lo = nullptr;
     int max_segs = 0;
     float *ssq_a = nullptr, *ssq_b = nullptr;
     unsigned* barrier = nullptr;     // [64 | tile counters of the 5 GEMM kinds], zeroed before every launch
@@ -83,7 +84,7 @@ int pass_init(s2d2_ctx* c) {
     const int L = m.n_layers;
     s->n_weight_maps = L * 4 + 1;
     s->map_x0 = s->n_weight_maps;
-    s->map_kv = s->map_x0 + 12;
+    s->map_kv = s->map_x0 + 24;      // 12 maps of the high halves, 12 of the low halves
     std::vector<CUtensorMap> maps(s->map_kv + 1);
     auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
         return gemm_encode_map(c, &maps[idx], ptr, rows, cols, box_rows) == 0;
@@ -97,8 +98,23 @@ int pass_init(s2d2_ctx* c) {
     }
     good = good && enc(L * 4, c->lm_head, m.vocab, d, 128);
     s->head_bytes = 2.0 * (double)m.vocab * d;
+    {
+        size_t rows = c->max_rows;
+        if (cudaMalloc((void**)&s->xn_lo, rows * d * 2) != cudaSuccess || cudaMalloc((void**)&s->attn_lo, rows * nq * 2) != cudaSuccess ||
+            cudaMalloc((void**)&s->act_lo, rows * f * 2) != cudaSuccess || cudaMalloc((void**)&s->q_lo, rows * nq * 2) != cudaSuccess) {
+            c->err = "cudaMalloc failed for the persistent pass";
+            return S2D2_ERR_CUDA;
+        }
+        cudaMemset(s->xn_lo, 0, rows * d * 2);
+        cudaMemset(s->attn_lo, 0, rows * nq * 2);
+        cudaMemset(s->act_lo, 0, rows * f * 2);
+        cudaMemset(s->q_lo, 0, rows * nq * 2);
+    }
     for (int t = 0; t < 4 && good; ++t) {
         const int T = 16 * (t + 1);
+        good = enc(s->map_x0 + 12 + t, s->xn_lo, c->max_rows, d, T) && enc(s->map_x0 + 16 + t, s->attn_lo, c->max_rows, nq, T) &&
+               enc(s->map_x0 + 20 + t, s->act_lo, c->max_rows, f, T);
+        if (!good) break;
         good = enc(s->map_x0 + t, c->xn, c->max_rows, d, T) && enc(s->map_x0 + 4 + t, c->attn, c->max_rows, nq, T) &&
                enc(s->map_x0 + 8 + t, c->act, c->max_rows, f, T);
     }
@@ -201,7 +217,7 @@ void pass_destroy(s2d2_ctx* c) {
     PassState* s = state(c);
     if (!s) return;
     void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier, s->trace,
-                    s->parts[0], s->parts[1], s->parts[2], s->parts[3], s->parts[4]};
+                    s->parts[0], s->parts[1], s->parts[2], s->parts[3], s->parts[4], s->xn_lo, s->attn_lo, s->act_lo, s->q_lo};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     delete s;
@@ -239,6 +255,12 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.v_rows = (bf16*)c->v_rows;
     p.attn = (bf16*)c->attn;
     p.act = (bf16*)c->act;
+    p.xn_lo = s->xn_lo;
+    p.attn_lo = s->attn_lo;
+    p.act_lo = s->act_lo;
+    p.map_lo_off = 12;
+    p.q_lo = s->q_lo;
+    p.ap.q_lo = s->q_lo;
     p.ws = s->ws;
     p.max_segs = s->max_segs;
     p.ssq_a = s->ssq_a;

@@ -42,7 +42,7 @@ namespace pp {
 constexpr int THREADS = 256;
 constexpr int CTHREADS = 128;        // compute warps 4..7
 constexpr int BAR_COMPUTE = 1;       // named barrier of the compute warps
-constexpr int ACC_STRIDE = 64;       // tensor-memory columns per accumulator buffer
+constexpr int ACC_STRIDE = 128;      // tensor-memory columns per accumulator buffer (2 T: high and low halves)
 constexpr int MAX_T = 64;            // most token rows of a pass
 constexpr int W_TILE_BYTES = tc::BLOCK_N * 128;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
@@ -63,6 +63,9 @@ struct PassParams {
     const float* final_norm;
     float* h;                 // [M, d] residual stream
     bf16 *xn, *q, *k_rows, *v_rows, *attn, *act;
+    bf16 *xn_lo, *attn_lo, *act_lo;   // low halves of the GEMM inputs: x = hi + lo, both bf16
+    bf16* q_lo;                       // low halves of q, same split, for the attention items
+    int map_lo_off;                   // tensor map of a buffer's low half = that of its high half + this
     float* ws;                // split-K partials [grid][max_segs][T][128]
     int max_segs;
     float *ssq_a, *ssq_b;     // per-tile sums of squares of h rows [d/128][MAX_T]
@@ -83,7 +86,7 @@ struct PassParams {
     int trace_cap;
 };
 
-__host__ __device__ inline size_t stage_bytes(int T) { return (size_t)W_TILE_BYTES + (size_t)T * 128; }
+__host__ __device__ inline size_t stage_bytes(int T) { return (size_t)W_TILE_BYTES + (size_t)2 * T * 128; }
 __host__ __device__ inline size_t misc_bytes() { return 2048; }
 __host__ __device__ inline size_t smem_bytes(int T, int S, int hd) {
     return 1024 + (size_t)S * stage_bytes(T) + att::attn_tiles_bytes(hd) + misc_bytes();
@@ -277,6 +280,16 @@ __device__ __forceinline__ SsqLane row_ssq_lane(const float* ssq, int d_tiles, i
 __device__ __forceinline__ float inv_rms_from(const SsqLane& r, int d, float eps) {
     return 1.0f / sqrtf(warp_sum((r.v[0] + r.v[1]) + (r.v[2] + r.v[3])) / (float)d + eps);
 }
+__device__ __forceinline__ void store_bf16x4(bf16* dst, float a, float b, float c, float d);
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): the GEMMs take both halves as token rows, so
+// their inputs carry 16 significant bits instead of 8 (the tensor pipe is nearly idle in this
+// kernel; the second half costs 2 KB of shared memory per stage).
+__device__ __forceinline__ void store_hi_lo_x4(bf16* hi, bf16* lo, float a, float b, float c, float d) {
+    const float ha = __bfloat162float(__float2bfloat16_rn(a)), hb = __bfloat162float(__float2bfloat16_rn(b));
+    const float hc = __bfloat162float(__float2bfloat16_rn(c)), hd = __bfloat162float(__float2bfloat16_rn(d));
+    store_bf16x4(hi, ha, hb, hc, hd);
+    store_bf16x4(lo, a - ha, b - hb, c - hc, d - hd);
+}
 __device__ __forceinline__ void store_bf16x4(bf16* dst, float a, float b, float c, float d) {
     __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
     uint2 u;
@@ -405,8 +418,9 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) fine = false;
                         if (*abort_flag) fine = false;
                         if (fine) {
-                            tc::mbar_expect_tx(&full[s], (uint32_t)T * 128u);
+                            tc::mbar_expect_tx(&full[s], (uint32_t)T * 256u);
                             tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, 0, &full[s]);
+                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES + T * 128, mx + p.map_lo_off, kb * tc::BLOCK_K, 0, &full[s]);
                             *x_issued = (int)i + 1;
                         }
                     }
@@ -422,7 +436,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     } else if (warp == 2) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            const uint32_t idesc = tc::instr_desc_bf16(T);
+            const uint32_t idesc = tc::instr_desc_bf16(2 * T);     // token rows twice: high halves, then low halves
             uint32_t i = 0, seg = 0;
             bool ok = true;
             for (int gi = 0; gi < n_gemms && ok; ++gi) {
@@ -503,11 +517,12 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 float* mine = p.ws + ((size_t)cta * p.max_segs + local) * (size_t)T * tc::BLOCK_N + tid;
                 const uint32_t taddr = tmem_base + ((uint32_t)(cw * 32) << 16) + b * ACC_STRIDE;
                 for (int c0 = 0; c0 < T; c0 += 16) {
-                    float v[16];
-                    tc::tmem_ld16(taddr + c0, v);
+                    float v[16], w[16];
+                    tc::tmem_ld16(taddr + c0, v);          // W x_hi
+                    tc::tmem_ld16(taddr + T + c0, w);      // W x_lo
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (c0 + j < M) mine[(size_t)(c0 + j) * tc::BLOCK_N] = v[j];
+                        if (c0 + j < M) mine[(size_t)(c0 + j) * tc::BLOCK_N] = v[j] + w[j];
                 }
                 tc::tc_fence_before();
                 __syncwarp();
@@ -544,7 +559,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 const float4 gn = *reinterpret_cast<const float4*>(gain + col);
                 const float4 x = value(t, m, col);
                 *reinterpret_cast<float4*>(p.h + (size_t)m * d + col) = x;
-                store_bf16x4(p.xn + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
+                store_hi_lo_x4(p.xn + (size_t)m * d + col, p.xn_lo + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
                 const float sq = warp_sum(x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w);
                 if (lane == 0) ssq[(size_t)t * MAX_T + m] = sq;
                 publish_x(p.x_cnt[0] + t);
@@ -653,7 +668,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                             }
                         }
                         if (is_q) {
-                            store_bf16x4(p.q + ((size_t)m * p.Hq + head) * HD + ch, x[0], x[1], x[2], x[3]);
+                            const size_t o = ((size_t)m * p.Hq + head) * HD + ch;
+                            store_hi_lo_x4(p.q + o, p.q_lo + o, x[0], x[1], x[2], x[3]);
                         } else {
                             const int kvh = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
                             store_bf16x4((is_k ? p.k_rows : p.v_rows) + ((size_t)m * p.Hkv + kvh) * HD + ch, x[0], x[1], x[2], x[3]);
@@ -674,7 +690,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 const int total = ap.pv.n_seqs * ap.Hkv * ap.n_qtiles * n_splits;
                 for (int idx = cta; idx < total && ok; idx += G) {
                     const int split = idx % n_splits, r = idx / n_splits;
-                    if (!att::attn_item<HD>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
+                    if (!att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
                                             kv_ring, tid, BAR_COMPUTE)) {
                         ok = false;
                         *abort_flag = 1;
@@ -736,7 +752,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         }
                     }
                     if (lane < HD / 4) {
-                        store_bf16x4(p.attn + ((size_t)r * p.Hq + hq) * HD + 4 * lane, acc.x / lsum, acc.y / lsum, acc.z / lsum, acc.w / lsum);
+                        const size_t o = ((size_t)r * p.Hq + hq) * HD + 4 * lane;
+                        store_hi_lo_x4(p.attn + o, p.attn_lo + o, acc.x / lsum, acc.y / lsum, acc.z / lsum, acc.w / lsum);
                     }
                     publish_x(p.x_cnt[1] + hq * HD / tc::BLOCK_N);
                 }
@@ -786,8 +803,9 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const float uv[4] = {inv * u4.x, inv * u4.y, inv * u4.z, inv * u4.w};
                         float a[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) a[e] = __fdividef(gv[e], 1.f + __expf(-gv[e])) * uv[e];   // bf16 output: 2^-9 rounding dominates
-                        store_bf16x4(p.act + (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane, a[0], a[1], a[2], a[3]);
+                        for (int e = 0; e < 4; ++e) a[e] = __fdividef(gv[e], 1.f + __expf(-gv[e])) * uv[e];   // fast exp and divide: 2^-21, far below what the later stages add
+                        const size_t o = (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane;
+                        store_hi_lo_x4(p.act + o, p.act_lo + o, a[0], a[1], a[2], a[3]);
                     }
                     // one fence for the step's stores, then one count per finished pair
                     asm volatile("fence.proxy.async;" ::: "memory");

@@ -1,0 +1,38 @@
+"""Parity at the full model shapes of the workloads, in the launch configuration bench.py times
+(persistent pass kernel, 64-token pages): a few decode steps after a short prompt, so that the
+fp64 oracle forward of the same rows stays within a minute or two per workload.
+
+Stage A (proposals, accepted length, first rejection, resampled ids on the engine's own logits) and
+stage B (the oracle's forward of the same rows against the engine's logits, 2e-2 absolute) are the
+same checks as in test_gpu_parity.py; here the matrices have the workloads' real sizes (d_model
+2048 / 4096, 28 / 36 layers, vocabulary 151936), which is what spans many tiles, split-K parts and
+vocabulary chunks and lets rounding accumulate over the real depth."""
+import pytest
+
+from s2d2_inputs import generate_prompts, generate_weights, get_config
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.mark.parametrize("name,n_steps", [("c2", 3), ("c4", 1)])
+def test_full_shape_steps_match_oracle(name, n_steps):
+    from paper_2603_25702_b200 import Engine
+    from tests.parity_util import check_kv, register_prompt_lens, run_steps
+    wl = get_config(name, prompt_len=(6, 6), gen_tokens=2 * get_config(name).block_size)
+    W = generate_weights(wl.model, seed=wl.weight_seed)
+    e = Engine(wl.model, block_size=wl.block_size, max_batch=1, max_seq_len=256, kv_page_tokens=wl.kv_page_tokens,
+               seed=wl.philox_seed, stream=torch.cuda.current_stream().cuda_stream)
+    e.load_weights(W)
+    prompts = generate_prompts(wl)
+    ids = e.prefill(prompts)
+    register_prompt_lens(ids, prompts)
+    e.seq_set_rng_stream(ids[0], 0)
+    rep = run_steps(e, W, wl, ids, {ids[0]: 0}, n_steps=n_steps, logit_atol=2e-2)
+    print(name, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.stage_b_passes >= n_steps and rep.verified_steps == n_steps
+    assert e.get_counters().n_kernel_launches < 40 * n_steps      # the persistent kernel ran, not one kernel per operation
+    if name == "c2":
+        check_kv(e, W, wl.model, ids[0], atol=4e-2)
+    e.close()

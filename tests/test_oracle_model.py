@@ -45,6 +45,8 @@ def _torch_causal_forward(W, cfg, tokens):
             q = F.rms_norm(q, (hd,), _t(W[p + "q_norm"]), cfg.rms_eps)
             k = F.rms_norm(k, (hd,), _t(W[p + "k_norm"]), cfg.rms_eps)
         q, k = _torch_rope_complex(q, pos, cfg.rope_base), _torch_rope_complex(k, pos, cfg.rope_base)
+        if cfg.dtype == "bf16":      # K and V are held as the cache stores them: torch's own bfloat16 rounding
+            k, v = k.float().bfloat16().double(), v.float().bfloat16().double()
         o = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None], v.transpose(0, 1)[None],
                                            is_causal=True, enable_gqa=True)[0]
         h = h + F.linear(o.transpose(0, 1).reshape(R, Hq * hd), _t(W[p + "wo"]))
@@ -142,3 +144,26 @@ def test_moe_model_forward_runs_and_is_finite(tiny_moe):
     logits, kv = M.forward(W, cfg, [1, 2, cfg.mask_id], [0, 1, 2], M.causal_mask(3))
     assert logits.shape == (3, cfg.vocab) and np.isfinite(logits).all()
     assert kv[0][0].shape == (3, cfg.n_kv_heads, cfg.head_dim)
+
+
+def test_kv_is_held_as_the_cache_stores_it():
+    """bf16 models: every K/V value the oracle hands out is a bfloat16 number (low 16 bits of
+    its fp32 pattern are zero) and equals torch's rounding of the unrounded value; fp32 models
+    keep fp64 K/V."""
+    class Cfg:
+        dtype = "bf16"
+    x = np.random.default_rng(5).standard_normal(4096) * np.logspace(-6, 3, 4096)
+    got = M.as_stored_kv(x, Cfg)
+    assert (got.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all()
+    want = torch.from_numpy(x).float().bfloat16().double().numpy()
+    assert (got == want).all()
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8])      # exactly between two bfloat16 neighbours: to even
+    assert M.as_stored_kv(ties, Cfg).tolist() == [1.0, 1.0 + 2.0 ** -6]
+    Cfg.dtype = "fp32"
+    assert M.as_stored_kv(x, Cfg) is x
+    wl = get_config("t_bf16")
+    W = generate_weights(wl.model, seed=2)
+    _, kv = M.forward(W, wl.model, [1, 2, 3], np.arange(3), M.causal_mask(3), need_logits=[])
+    for k, v in kv:
+        for a in (k, v):
+            assert (a.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all() and (a.astype(np.float32) == a).all()
