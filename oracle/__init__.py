@@ -11,7 +11,8 @@ Pins (what each part is checked against, see tests/test_oracle_*.py):
   philox.py   published known-answer vectors of Philox4x32-10.
   model.py    a separately written composition of torch fp64 library ops for a
               plain causal pass; RoPE shift invariance; cached == recomputed;
-              MoE top-k == dense evaluation with zeroed gates.
+              MoE top-k == dense evaluation with zeroed gates; K/V of bf16 models held
+              as bfloat16 (the cache's storage format) == torch's bfloat16 conversion.
   accept.py   scipy logsumexp; closed forms of speculative sampling (exact
               enumeration on tiny vocabularies); brute-force inverse CDF.
   s2d2.py     verifier rows of the 2L pass == L literal single-row passes;

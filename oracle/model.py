@@ -12,7 +12,8 @@ which rows of the same pass a row may attend to (this is where the verifier
 mask and the partially causal drafting mask of Section "Self-Verification Mode"
 enter), and the cached prefix K/V, which every row sees in full.
 Weights arrive as the stored values (bfloat16 bit patterns or fp32) and are
-widened exactly to fp64; all arithmetic is fp64.
+widened exactly to fp64; all arithmetic is fp64.  One storage format besides the weights'
+enters: K and V of a bf16 model are bfloat16 values, as its KV cache stores them (as_stored_kv).
 """
 from __future__ import annotations
 
