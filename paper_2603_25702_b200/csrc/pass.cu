@@ -213,6 +213,11 @@ int pass_init(s2d2_ctx* c) {
     return S2D2_OK;
 }
 
+int pass_max_rows(s2d2_ctx* c) {
+    PassState* s = state(c);
+    return s && s->ok ? pp::MAX_T : 0;
+}
+
 void pass_destroy(s2d2_ctx* c) {
     PassState* s = state(c);
     if (!s) return;

@@ -12,3 +12,5 @@ int pass_run(s2d2_ctx* c, const s2d2::PassView& pv, int max_ctx, int max_rows, l
              bool* taken);
 // Timestamps of the last persistent pass (see s2d2_debug_pass_trace).
 int pass_copy_trace(s2d2_ctx* c, unsigned long long* out, long long cap, int* n_ctas, int* n_marks);
+// Most rows the persistent kernel takes in one pass on this context (0: it is not available).
+int pass_max_rows(s2d2_ctx* c);

@@ -587,27 +587,32 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
     }
     CUDA_TRY(c, cudaEventRecord(c->ev[6], c->stream));
     const int CH = S2D2_MAX_ROWS_PER_SEQ;
+    // Rows per pass: where the persistent pass kernel is available a chunk is cut to what that kernel
+    // takes (it is both faster and carries two-term operands); otherwise one chunk of every sequence.
+    const int budget = pass_max_rows(c) > 0 ? pass_max_rows(c) : CH * (int)ids.size();
+    std::vector<int> took(ids.size());
     for (;;) {
         PassBuild pb;
-        for (int id : ids) {
-            SeqState& s = c->seqs[id];
+        int room = budget;
+        for (size_t k = 0; k < ids.size(); ++k) {
+            SeqState& s = c->seqs[ids[k]];
+            took[k] = 0;
             int left = s.n_final - s.n_c;
-            if (left <= 0) continue;
-            int rows = std::min(left, CH);
+            if (left <= 0 || room <= 0) continue;
+            int rows = std::min(std::min(left, CH), room);
             if ((rc = ensure_pages(c, s, s.n_c + rows))) return rc;
             begin_seq(c, pb, s, s.n_c);
             for (int r = 0; r < rows; ++r)
                 add_row(c, pb, s.tok[s.n_c + r], s.n_c + r, (r == 63) ? ~0ull : ((1ull << (r + 1)) - 1), ROW_WRITE_KV, false);
+            took[k] = rows;
+            room -= rows;
         }
         if (pb.n_rows == 0) break;
         if ((rc = run_pass(c, pb, nullptr))) return rc;
         c->cnt.n_prefill_passes++;
         // the metadata buffer is reused by the next chunk: wait for this pass to have consumed it
         CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-        for (int id : ids) {
-            SeqState& s = c->seqs[id];
-            s.n_c = std::min(s.n_final, s.n_c + CH);
-        }
+        for (size_t k = 0; k < ids.size(); ++k) c->seqs[ids[k]].n_c += took[k];
     }
     if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[7], c->stream));

@@ -15,24 +15,26 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
-@pytest.mark.parametrize("name,n_steps", [("c2", 3), ("c4", 1)])
-def test_full_shape_steps_match_oracle(name, n_steps):
+@pytest.mark.parametrize("name,n_steps,batch", [("c2", 3, 1), ("c4", 1, 1), ("c3", 1, 3)])
+def test_full_shape_steps_match_oracle(name, n_steps, batch):
     from paper_2603_25702_b200 import Engine
     from tests.parity_util import check_kv, register_prompt_lens, run_steps
-    wl = get_config(name, prompt_len=(6, 6), gen_tokens=2 * get_config(name).block_size)
+    wl = get_config(name, prompt_len=(5, 9), gen_tokens=2 * get_config(name).block_size, batch=batch)
     W = generate_weights(wl.model, seed=wl.weight_seed)
-    e = Engine(wl.model, block_size=wl.block_size, max_batch=1, max_seq_len=256, kv_page_tokens=wl.kv_page_tokens,
+    e = Engine(wl.model, block_size=wl.block_size, max_batch=batch, max_seq_len=256, kv_page_tokens=wl.kv_page_tokens,
                seed=wl.philox_seed, stream=torch.cuda.current_stream().cuda_stream)
     e.load_weights(W)
     prompts = generate_prompts(wl)
     ids = e.prefill(prompts)
     register_prompt_lens(ids, prompts)
-    e.seq_set_rng_stream(ids[0], 0)
-    rep = run_steps(e, W, wl, ids, {ids[0]: 0}, n_steps=n_steps, logit_atol=2e-2)
+    for k, sid in enumerate(ids):
+        e.seq_set_rng_stream(sid, k)
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=n_steps, logit_atol=2e-2)
     print(name, rep)
     assert not rep.mismatches, rep.mismatches[:5]
-    assert rep.stage_b_passes >= n_steps and rep.verified_steps == n_steps
+    assert rep.stage_b_passes >= n_steps and rep.verified_steps == n_steps * batch
     assert e.get_counters().n_kernel_launches < 40 * n_steps      # the persistent kernel ran, not one kernel per operation
     if name == "c2":
         check_kv(e, W, wl.model, ids[0], atol=4e-2)
     e.close()
+
