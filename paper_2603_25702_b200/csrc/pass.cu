@@ -5,6 +5,7 @@
 #include <cuda.h>
 
 #include <stdlib.h>
+#include <string.h>
 
 #include <algorithm>
 #include <vector>
@@ -19,26 +20,33 @@ using namespace s2d2;
 namespace {
 struct PassState {
     bool ok = false;
+    bool moe = false;
     int grid = 0;
     int max_smem = 0;
-    int n_weight_maps = 0;
-    int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act
+    int maps_per_layer = 4;
+    int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act; then their low halves
+    int map_act_e = 0;           // per T: experts' SwiGLU output, high halves then low halves
     int map_kv = 0;
     CUtensorMap* d_maps = nullptr;
     pp::LayerGains* d_gains = nullptr;
     float* ws = nullptr;
-    bf16 *xn_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr, *q_lo = nullptr;
-    int max_segs = 0;
+    bf16 *xn_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr, *q_lo = nullptr, *act_e = nullptr, *act_e_lo = nullptr;
+    long long ws_off[pp::N_KINDS] = {};
+    int max_segs[pp::N_KINDS] = {};
     float *ssq_a = nullptr, *ssq_b = nullptr;
-    unsigned* barrier = nullptr;     // [64 | tile counters of the 5 GEMM kinds], zeroed before every launch
+    unsigned* barrier = nullptr;     // [64 | tile counters of the static GEMM kinds | x counters], zeroed before every launch
     size_t sync_bytes = 0;
-    size_t cnt_off[5] = {0, 0, 0, 0, 0};
+    long long cnt_off[pp::N_KINDS] = {};     // -1: the kind publishes through a grid barrier
     size_t xcnt_off[3] = {0, 0, 0};
     unsigned long long* trace = nullptr;
     int trace_cap = 0;
     int last_marks = 0;
-    int* parts[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // split-K part tables per GEMM kind
-    double weight_bytes = 0;     // bytes of every matrix a pass streams (without the LM head)
+    int barriers_per_layer = 6;
+    int* parts[pp::N_KINDS] = {};    // split-K part tables of the static GEMM kinds
+    int* n_touched = nullptr;        // [n_layers] device, touched experts of the last pass
+    int* n_touched_h = nullptr;      // pinned mirror
+    double weight_bytes = 0;         // bytes of every matrix a pass always streams (without the LM head)
+    double expert_bytes = 0;         // bytes of one routed expert's three matrices
     double head_bytes = 0;
 };
 PassState* state(s2d2_ctx* c) { return (PassState*)c->pass_state; }
@@ -56,15 +64,23 @@ int stages_for(const PassState* s, int T, int hd) {
     long avail = (long)s->max_smem - 1024 - (long)att::attn_tiles_bytes(hd) - (long)pp::misc_bytes();
     return (int)std::min<long>(12, avail / (long)pp::stage_bytes(T));
 }
+int fail_alloc(s2d2_ctx* c) {
+    c->err = "cudaMalloc failed for the persistent pass";
+    return S2D2_ERR_CUDA;
+}
 }  // namespace
 
 int pass_init(s2d2_ctx* c) {
     PassState* s = new PassState();
     c->pass_state = s;
     const s2d2_model_config& m = c->m;
-    if (m.dtype != S2D2_DTYPE_BF16 || c->dc.use_tensor_cores != 1 || m.n_experts > 0 || !gemm_tc_available(c)) return S2D2_OK;
-    const int d = m.d_model, hd = m.head_dim, nq = m.n_q_heads * hd, nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd, f = m.ffn;
-    if (!(hd == 64 || hd == 128) || d % 128 || f % 128 || nqkv % 128 || nq % 64 || c->page_tokens < 16) return S2D2_OK;
+    if (m.dtype != S2D2_DTYPE_BF16 || c->dc.use_tensor_cores != 1 || !gemm_tc_available(c)) return S2D2_OK;
+    const bool moe = m.n_experts > 0;
+    const int d = m.d_model, hd = m.head_dim, nq = m.n_q_heads * hd, nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd;
+    const int fe = m.expert_ffn, fs = moe ? m.expert_ffn * m.n_shared : 0, E = m.n_experts;
+    const int f = moe ? fs : m.ffn;                 // width of the dense / shared-expert SwiGLU
+    if (!(hd == 64 || hd == 128) || d % 128 || f % 128 || f < 128 || nqkv % 128 || nq % 64 || c->page_tokens < 16) return S2D2_OK;
+    if (moe && (E % 128 || E > pp::MAX_EXPERTS || fe % 128 || m.top_k > 32 || m.top_k < 1 || m.n_shared < 1)) return S2D2_OK;
     if (c->max_rows < pp::MAX_T) return S2D2_OK;
     int coop = 0, n_sms = 0, optin = 0;
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
@@ -73,18 +89,21 @@ int pass_init(s2d2_ctx* c) {
     if (!coop || n_sms < 1) return S2D2_OK;
     s->grid = n_sms;
     s->max_smem = optin;
-
+    s->moe = moe;
+    const int G = s->grid;
     if (stages_for(s, pp::MAX_T, hd) < 3) return S2D2_OK;
     cudaError_t e = hd == 128 ? prepare_kernel<128>(s, optin) : prepare_kernel<64>(s, optin);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return S2D2_OK;       // the one-kernel-per-operation path stays in charge
     }
-    // tensor maps
+    // ---- tensor maps: weights [layer][maps_per_layer], LM head, activations per T, KV pool ----
     const int L = m.n_layers;
-    s->n_weight_maps = L * 4 + 1;
-    s->map_x0 = s->n_weight_maps;
-    s->map_kv = s->map_x0 + 24;      // 12 maps of the high halves, 12 of the low halves
+    s->maps_per_layer = moe ? 8 : 4;
+    s->barriers_per_layer = moe ? 9 : 6;
+    s->map_x0 = L * s->maps_per_layer + 1;
+    s->map_act_e = s->map_x0 + 24;
+    s->map_kv = s->map_act_e + 8;
     std::vector<CUtensorMap> maps(s->map_kv + 1);
     auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
         return gemm_encode_map(c, &maps[idx], ptr, rows, cols, box_rows) == 0;
@@ -92,31 +111,51 @@ int pass_init(s2d2_ctx* c) {
     bool good = true;
     for (int l = 0; l < L && good; ++l) {
         const LayerWeights& W = c->layers[l];
-        good = enc(l * 4 + 0, W.wqkv, nqkv, d, 128) && enc(l * 4 + 1, W.wo, d, nq, 128) && enc(l * 4 + 2, W.wgu, 2 * f, d, 128) &&
-               enc(l * 4 + 3, W.wdown, d, f, 128);
-        s->weight_bytes += 2.0 * ((double)nqkv * d + (double)d * nq + 2.0 * f * d + (double)d * f);
+        const int b = l * s->maps_per_layer;
+        good = enc(b + 0, W.wqkv, nqkv, d, 128) && enc(b + 1, W.wo, d, nq, 128);
+        s->weight_bytes += 2.0 * ((double)nqkv * d + (double)d * nq);
+        if (!moe) {
+            good = good && enc(b + 2, W.wgu, 2 * f, d, 128) && enc(b + 3, W.wdown, d, f, 128);
+            s->weight_bytes += 2.0 * (3.0 * f * d);
+        } else {
+            good = good && enc(b + 2, W.router, E, d, 128) && enc(b + 3, W.s_gu, 2 * fs, d, 128) &&
+                   enc(b + 4, W.e_gate, (unsigned long long)E * fe, d, 128) && enc(b + 5, W.e_up, (unsigned long long)E * fe, d, 128) &&
+                   enc(b + 6, W.s_down, d, fs, 128) && enc(b + 7, W.e_down, (unsigned long long)E * d, fe, 128);
+            s->weight_bytes += 2.0 * ((double)E * d + 3.0 * fs * d);
+        }
     }
-    good = good && enc(L * 4, c->lm_head, m.vocab, d, 128);
+    s->expert_bytes = 2.0 * 3.0 * fe * d;
+    good = good && enc(L * s->maps_per_layer, c->lm_head, m.vocab, d, 128);
     s->head_bytes = 2.0 * (double)m.vocab * d;
     {
         size_t rows = c->max_rows;
         if (cudaMalloc((void**)&s->xn_lo, rows * d * 2) != cudaSuccess || cudaMalloc((void**)&s->attn_lo, rows * nq * 2) != cudaSuccess ||
-            cudaMalloc((void**)&s->act_lo, rows * f * 2) != cudaSuccess || cudaMalloc((void**)&s->q_lo, rows * nq * 2) != cudaSuccess) {
-            c->err = "cudaMalloc failed for the persistent pass";
-            return S2D2_ERR_CUDA;
-        }
+            cudaMalloc((void**)&s->act_lo, rows * f * 2) != cudaSuccess || cudaMalloc((void**)&s->q_lo, rows * nq * 2) != cudaSuccess)
+            return fail_alloc(c);
         cudaMemset(s->xn_lo, 0, rows * d * 2);
         cudaMemset(s->attn_lo, 0, rows * nq * 2);
         cudaMemset(s->act_lo, 0, rows * f * 2);
         cudaMemset(s->q_lo, 0, rows * nq * 2);
+        if (moe) {
+            // SwiGLU outputs of the touched experts: [expert slot][T rows][fe]
+            size_t bytes = (size_t)E * pp::MAX_T * fe * 2;
+            if (cudaMalloc((void**)&s->act_e, bytes) != cudaSuccess || cudaMalloc((void**)&s->act_e_lo, bytes) != cudaSuccess ||
+                cudaMalloc((void**)&s->n_touched, L * 4) != cudaSuccess || cudaMallocHost((void**)&s->n_touched_h, L * 4) != cudaSuccess)
+                return fail_alloc(c);
+            cudaMemset(s->act_e, 0, bytes);
+            cudaMemset(s->act_e_lo, 0, bytes);
+            cudaMemset(s->n_touched, 0, L * 4);
+            memset(s->n_touched_h, 0, L * 4);
+        }
     }
     for (int t = 0; t < 4 && good; ++t) {
         const int T = 16 * (t + 1);
-        good = enc(s->map_x0 + 12 + t, s->xn_lo, c->max_rows, d, T) && enc(s->map_x0 + 16 + t, s->attn_lo, c->max_rows, nq, T) &&
-               enc(s->map_x0 + 20 + t, s->act_lo, c->max_rows, f, T);
-        if (!good) break;
         good = enc(s->map_x0 + t, c->xn, c->max_rows, d, T) && enc(s->map_x0 + 4 + t, c->attn, c->max_rows, nq, T) &&
-               enc(s->map_x0 + 8 + t, c->act, c->max_rows, f, T);
+               enc(s->map_x0 + 8 + t, c->act, c->max_rows, f, T) && enc(s->map_x0 + 12 + t, s->xn_lo, c->max_rows, d, T) &&
+               enc(s->map_x0 + 16 + t, s->attn_lo, c->max_rows, nq, T) && enc(s->map_x0 + 20 + t, s->act_lo, c->max_rows, f, T);
+        if (moe && good)
+            good = enc(s->map_act_e + t, s->act_e, (unsigned long long)E * pp::MAX_T, fe, T) &&
+                   enc(s->map_act_e + 4 + t, s->act_e_lo, (unsigned long long)E * pp::MAX_T, fe, T);
     }
     if (!good) {
         c->err = "cuTensorMapEncodeTiled failed for the persistent pass";
@@ -130,77 +169,81 @@ int pass_init(s2d2_ctx* c) {
         if (!attention_plan(c, dummy, 1, 1, 0, &ap, &mk) || !mk) return S2D2_OK;
         maps[s->map_kv] = *(const CUtensorMap*)mk;
     }
-    // split-K workspace: the most segments any CTA has in one GEMM
-    const int G = s->grid;
-    auto segs = [&](long long N, long long K) {
-        long long n_tiles = (N + 127) / 128, kbt = K / 64, U = n_tiles * kbt;
-        long long per = (U + G - 1) / G;
-        return (int)((per + kbt - 1) / kbt + 1);
-    };
-    s->max_segs = std::max({segs(nqkv, d), segs(d, nq), segs(2 * f, d), segs(d, f), segs(m.vocab, d)});
-    size_t ws_floats = (size_t)G * s->max_segs * pp::MAX_T * 128;
-    {
-        const long long Ns[5] = {nqkv, d, 2LL * f, d, m.vocab};
-        size_t o = 64;
-        for (int k = 0; k < 5; ++k) {
-            s->cnt_off[k] = o;
-            o += (size_t)((Ns[k] + 127) / 128);
+    // ---- per GEMM kind: shape, split-K workspace region, publish counters, part tables ----
+    // N < 0 marks a kind this model does not run; for the two routed-expert GEMMs N is the largest (all experts touched).
+    long long NK[pp::N_KINDS][2];
+    for (auto& nk : NK) nk[0] = -1, nk[1] = 64;
+    NK[pp::K_QKV][0] = nqkv, NK[pp::K_QKV][1] = d;
+    NK[pp::K_O][0] = d, NK[pp::K_O][1] = nq;
+    NK[pp::K_LM][0] = m.vocab, NK[pp::K_LM][1] = d;
+    if (!moe) {
+        NK[pp::K_GU][0] = 2LL * f, NK[pp::K_GU][1] = d;
+        NK[pp::K_DOWN][0] = d, NK[pp::K_DOWN][1] = f;
+    } else {
+        NK[pp::K_ROUTER][0] = E, NK[pp::K_ROUTER][1] = d;
+        NK[pp::K_SGU][0] = 2LL * fs, NK[pp::K_SGU][1] = d;
+        NK[pp::K_EGU][0] = 2LL * fe * E, NK[pp::K_EGU][1] = d;
+        NK[pp::K_SDOWN][0] = d, NK[pp::K_SDOWN][1] = fs;
+        NK[pp::K_EDOWN][0] = (long long)d * E, NK[pp::K_EDOWN][1] = fe;
+    }
+    long long ws_floats = 0;
+    size_t sync_words = 64;
+    for (int k = 0; k < pp::N_KINDS; ++k) {
+        s->cnt_off[k] = -1;
+        if (NK[k][0] < 0) continue;
+        const bool dynamic = k == pp::K_EGU || k == pp::K_EDOWN;
+        const long long n_tiles = (NK[k][0] + 127) / 128, kbt = NK[k][1] / 64, U = n_tiles * kbt;
+        if (U * (long long)G >= (1LL << 40)) return S2D2_OK;
+        // the kernel shares a GEMM's units among Geff CTAs (pp::effective_ctas); for the routed-expert GEMMs the
+        // largest per-CTA share is that of the largest U, since Geff only grows with U
+        const int Geff = pp::effective_ctas(U, (int)kbt, G);
+        const long long per = (U + Geff - 1) / Geff;
+        s->max_segs[k] = (int)((per + kbt - 1) / kbt + 1);
+        s->ws_off[k] = ws_floats;
+        ws_floats += (long long)G * s->max_segs[k] * pp::MAX_T * 128;
+        if (dynamic) continue;
+        s->cnt_off[k] = (long long)sync_words;
+        sync_words += (size_t)n_tiles;
+        // per weight tile: the workspace slots of its split-K partials, in CTA order (the kernel cuts the
+        // tile-major (tile, k-block) units into G equal contiguous ranges)
+        std::vector<int> tab((size_t)n_tiles * (1 + pp::MAX_PARTS), 0);
+        for (int cta = 0; cta < Geff; ++cta) {
+            const long long u0 = U * cta / Geff, u1 = U * (cta + 1) / Geff;
+            if (u1 <= u0) continue;
+            const long long first = u0 / kbt, last = (u1 - 1) / kbt;
+            for (long long t = first; t <= last; ++t) {
+                int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
+                if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
+                tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs[k] + (int)(t - first);
+                ++cnt;
+            }
         }
+        if (cudaMalloc((void**)&s->parts[k], tab.size() * 4) != cudaSuccess ||
+            cudaMemcpy(s->parts[k], tab.data(), tab.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+            return fail_alloc(c);
+    }
+    {
         const long long Xs[3] = {d, nq, f};       // columns of xn, attn, act
         for (int k = 0; k < 3; ++k) {
-            s->xcnt_off[k] = o;
-            o += (size_t)((Xs[k] + 127) / 128);
+            s->xcnt_off[k] = sync_words;
+            sync_words += (size_t)((Xs[k] + 127) / 128);
         }
-        s->sync_bytes = o * 4;
-        if (cudaMalloc((void**)&s->barrier, s->sync_bytes) != cudaSuccess) {
-            c->err = "cudaMalloc failed for the persistent pass";
-            return S2D2_ERR_CUDA;
-        }
-    }
-    // per GEMM kind and weight tile: the workspace slots of its split-K partials, in CTA order
-    // (the kernel cuts the tile-major (tile, k-block) units into G equal contiguous ranges)
-    {
-        const long long NK[5][2] = {{nqkv, d}, {d, nq}, {2LL * f, d}, {d, f}, {m.vocab, d}};
-        for (int k = 0; k < 5; ++k) {
-            const long long n_tiles = (NK[k][0] + 127) / 128, kbt = NK[k][1] / 64, U = n_tiles * kbt;
-            if (U * (long long)G >= (1LL << 40)) return S2D2_OK;
-            std::vector<int> tab((size_t)n_tiles * (1 + pp::MAX_PARTS), 0);
-            for (int cta = 0; cta < G; ++cta) {
-                const long long u0 = U * cta / G, u1 = U * (cta + 1) / G;
-                if (u1 <= u0) continue;
-                const long long first = u0 / kbt, last = (u1 - 1) / kbt;
-                for (long long t = first; t <= last; ++t) {
-                    int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
-                    if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
-                    tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs + (int)(t - first);
-                    ++cnt;
-                }
-            }
-            if (cudaMalloc((void**)&s->parts[k], tab.size() * 4) != cudaSuccess ||
-                cudaMemcpy(s->parts[k], tab.data(), tab.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
-                c->err = "cudaMalloc failed for the persistent pass";
-                return S2D2_ERR_CUDA;
-            }
-        }
+        s->sync_bytes = sync_words * 4;
+        if (cudaMalloc((void**)&s->barrier, s->sync_bytes) != cudaSuccess) return fail_alloc(c);
     }
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
-    s->trace_cap = 3 * (6 * L + 1) + 1;      // three marks per grid barrier + the SM id
-    if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) {
-        c->err = "cudaMalloc failed for the persistent pass";
-        return S2D2_ERR_CUDA;
-    }
+    s->trace_cap = 3 * (s->barriers_per_layer * L + 1) + 1;      // three marks per grid barrier + the SM id
+    if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) return fail_alloc(c);
     if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
         cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
-        cudaMalloc((void**)&s->ws, ws_floats * 4) != cudaSuccess || cudaMalloc((void**)&s->ssq_a, ssq_bytes) != cudaSuccess ||
-        cudaMalloc((void**)&s->ssq_b, ssq_bytes) != cudaSuccess) {
-        c->err = "cudaMalloc failed for the persistent pass";
-        return S2D2_ERR_CUDA;
-    }
+        cudaMalloc((void**)&s->ws, (size_t)ws_floats * 4) != cudaSuccess || cudaMalloc((void**)&s->ssq_a, ssq_bytes) != cudaSuccess ||
+        cudaMalloc((void**)&s->ssq_b, ssq_bytes) != cudaSuccess)
+        return fail_alloc(c);
     if (cudaMemcpy(s->d_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(s->d_gains, gains.data(), gains.size() * sizeof(pp::LayerGains), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemset(s->ws, 0, ws_floats * 4) != cudaSuccess) {
+        cudaMemset(s->ws, 0, (size_t)ws_floats * 4) != cudaSuccess) {
         c->err = "device copy failed for the persistent pass";
         return S2D2_ERR_CUDA;
     }
@@ -221,10 +264,13 @@ int pass_max_rows(s2d2_ctx* c) {
 void pass_destroy(s2d2_ctx* c) {
     PassState* s = state(c);
     if (!s) return;
-    void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier, s->trace,
-                    s->parts[0], s->parts[1], s->parts[2], s->parts[3], s->parts[4], s->xn_lo, s->attn_lo, s->act_lo, s->q_lo};
+    void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier, s->trace, s->xn_lo, s->attn_lo, s->act_lo, s->q_lo,
+                    s->act_e, s->act_e_lo, s->n_touched};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (int* p : s->parts)
+        if (p) cudaFree(p);
+    if (s->n_touched_h) cudaFreeHost(s->n_touched_h);
     delete s;
     c->pass_state = nullptr;
 }
@@ -241,7 +287,13 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.Hq = m.n_q_heads;
     p.Hkv = m.n_kv_heads;
     p.hd = m.head_dim;
-    p.f = m.ffn;
+    p.moe = s->moe;
+    p.n_experts = m.n_experts;
+    p.top_k = m.top_k;
+    p.fe = m.expert_ffn;
+    p.fs = s->moe ? m.expert_ffn * m.n_shared : 0;
+    p.f = s->moe ? p.fs : m.ffn;
+    p.maps_per_layer = s->maps_per_layer;
     p.V = m.vocab;
     p.qk_norm = m.qk_norm;
     p.eps = m.rms_eps;
@@ -267,7 +319,19 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.q_lo = s->q_lo;
     p.ap.q_lo = s->q_lo;
     p.ws = s->ws;
-    p.max_segs = s->max_segs;
+    for (int k = 0; k < pp::N_KINDS; ++k) {
+        p.ws_off[k] = s->ws_off[k];
+        p.max_segs[k] = s->max_segs[k];
+        p.parts[k] = s->parts[k];
+        p.tile_cnt[k] = s->cnt_off[k] >= 0 ? s->barrier + s->cnt_off[k] : nullptr;
+    }
+    p.act_e = s->act_e;
+    p.act_e_lo = s->act_e_lo;
+    p.moe_ids = c->moe_ids;
+    p.moe_gates = c->moe_gates;
+    p.moe_ids_trace = c->moe_ids_trace;
+    p.trace_stride = c->max_rows * std::max(1, m.top_k);
+    p.n_touched_out = s->n_touched;
     p.ssq_a = s->ssq_a;
     p.ssq_b = s->ssq_b;
     p.logits = logits_out;
@@ -285,28 +349,35 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.map_xn = s->map_x0 + ti;
     p.map_attn = s->map_x0 + 4 + ti;
     p.map_act = s->map_x0 + 8 + ti;
+    p.map_act_e = s->map_act_e + ti;
     p.map_kv = s->map_kv;
     p.barrier = s->barrier;
     p.status = c->d_status;
     p.S = stages_for(s, p.T, m.head_dim);
-    for (int k = 0; k < 5; ++k) p.parts[k] = s->parts[k];
     p.trace = c->tracing ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    if (c->tracing) s->last_marks = 3 * (6 * m.n_layers + 1);
+    if (c->tracing) s->last_marks = 3 * (s->barriers_per_layer * m.n_layers + 1);
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
-    for (int k = 0; k < 5; ++k) p.tile_cnt[k] = s->barrier + s->cnt_off[k];
     for (int k = 0; k < 3; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];
     void* args[] = {&p};
     gemm_prof_begin(c);
     cudaError_t e = m.head_dim == 128
                         ? cudaLaunchCooperativeKernel((void*)pp::pass_kernel<128>, dim3(s->grid), dim3(pp::THREADS), args, smem, c->stream)
                         : cudaLaunchCooperativeKernel((void*)pp::pass_kernel<64>, dim3(s->grid), dim3(pp::THREADS), args, smem, c->stream);
-    // algorithmic bytes of the pass: every matrix once, the cached K/V of every sequence once,
-    // this pass's K/V rows written, logits written
+    // algorithmic bytes of the pass: every matrix once (for routed experts: those the previous pass of this
+    // context touched, the closest count the host has without a read-back), the cached K/V of every sequence
+    // once, this pass's K/V rows written, logits written
     double kv_tok = 2.0 * m.n_layers * m.n_kv_heads * m.head_dim * 2.0;
     double bytes = s->weight_bytes + (p.n_logit > 0 ? s->head_bytes + 4.0 * p.n_logit * m.vocab : 0.0) + kv_tok * (double)sum_ctx +
                    kv_tok * pv.n_rows;
+    if (s->moe) {
+        long long touched = 0;
+        for (int l = 0; l < m.n_layers; ++l) touched += s->n_touched_h[l];
+        bytes += s->expert_bytes * (double)touched;
+        c->cnt.moe_expert_tiles_touched += touched;
+        cudaMemcpyAsync(s->n_touched_h, s->n_touched, m.n_layers * 4, cudaMemcpyDeviceToHost, c->stream);
+    }
     gemm_prof_end(c, bytes);
     if (e != cudaSuccess) {
         c->err = std::string("persistent pass launch: ") + cudaGetErrorString(e);

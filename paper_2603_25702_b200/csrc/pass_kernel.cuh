@@ -47,6 +47,10 @@ constexpr int MAX_T = 64;            // most token rows of a pass
 constexpr int W_TILE_BYTES = tc::BLOCK_N * 128;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
 constexpr int MAX_PARTS = 16;        // most split-K partials of one weight tile
+// GEMM kinds of a pass.  Dense layers run QKV, O, GU, DOWN; mixture-of-experts layers run QKV, O,
+// ROUTER, SGU (shared expert gate/up), EGU (gate/up of the touched routed experts), SDOWN, EDOWN.
+enum : int { K_QKV = 0, K_O = 1, K_GU = 2, K_DOWN = 3, K_LM = 4, K_ROUTER = 5, K_SGU = 6, K_EGU = 7, K_SDOWN = 8, K_EDOWN = 9, N_KINDS = 10 };
+constexpr int MAX_EXPERTS = 256;
 
 struct LayerGains {
     const float *attn_norm, *ffn_norm, *q_norm, *k_norm;
@@ -54,6 +58,8 @@ struct LayerGains {
 
 struct PassParams {
     int n_layers, d, Hq, Hkv, hd, f, V;
+    int moe, n_experts, top_k, fe, fs;   // mixture of experts: routed experts of width fe, shared width fs (f = fs)
+    int maps_per_layer;                  // weight tensor maps per layer (4 dense, 8 mixture of experts)
     int qk_norm;
     float eps, logit_scale;
     PassView pv;
@@ -66,8 +72,16 @@ struct PassParams {
     bf16 *xn_lo, *attn_lo, *act_lo;   // low halves of the GEMM inputs: x = hi + lo, both bf16
     bf16* q_lo;                       // low halves of q, same split, for the attention items
     int map_lo_off;                   // tensor map of a buffer's low half = that of its high half + this
-    float* ws;                // split-K partials [grid][max_segs][T][128]
-    int max_segs;
+    float* ws;                // split-K partials, one region per GEMM kind: [grid][max_segs][T][128]
+    long long ws_off[N_KINDS];   // region offsets in floats
+    int max_segs[N_KINDS];
+    bf16 *act_e, *act_e_lo;   // SwiGLU outputs of the touched experts [expert slot][T][fe], hi and lo halves
+    int map_act_e;
+    int* moe_ids;             // [M, top_k] chosen experts of the current layer
+    float* moe_gates;         // [M, top_k] renormalised gates
+    int* moe_ids_trace;       // [n_layers][trace_stride] copy of the ids of every layer (test tap)
+    int trace_stride;
+    int* n_touched_out;       // [n_layers] touched experts per layer (for byte accounting)
     float *ssq_a, *ssq_b;     // per-tile sums of squares of h rows [d/128][MAX_T]
     float* logits;            // [n_logit, V]
     const float *rope_cos, *rope_sin;
@@ -76,50 +90,109 @@ struct PassParams {
     int map_xn, map_attn, map_act, map_kv;
     att::AttnParams ap;       // attention geometry of this pass (layer filled in per layer)
     unsigned* barrier;        // grid barrier counter, zero at launch
-    unsigned* tile_cnt[5];    // per GEMM kind and weight tile: partials published so far (zero at launch)
+    unsigned* tile_cnt[N_KINDS];    // per GEMM kind and weight tile: partials published so far (zero at launch)
     unsigned* x_cnt[3];       // per 128-column tile of xn / attn / act: (tile, row) pairs written so far (zero at launch)
     int* status;
     int S;                    // ring stages
-    const int* parts[5];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
+    const int* parts[N_KINDS];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
     unsigned long long* trace;   // [grid][trace_cap] per grid barrier: globaltimer at entry, at exit, and when the
                                  // CTA's last accumulator of the phase had been drained (0 if the phase has no GEMM)
     int trace_cap;
 };
 
 __host__ __device__ inline size_t stage_bytes(int T) { return (size_t)W_TILE_BYTES + (size_t)2 * T * 128; }
-__host__ __device__ inline size_t misc_bytes() { return 2048; }
+__host__ __device__ inline size_t misc_bytes() { return 4096; }
 __host__ __device__ inline size_t smem_bytes(int T, int S, int hd) {
     return 1024 + (size_t)S * stage_bytes(T) + att::attn_tiles_bytes(hd) + misc_bytes();
 }
 
 struct GemmShape {
     int n_tiles, kbt, map_w, map_x;
+    int tpe;           // weight tiles per expert for the two routed-expert GEMMs, else 0
+    int Geff;          // CTAs that share the GEMM's units: all of them, or fewer for a small GEMM so that
+                       // no CTA gets less than an eighth of a tile's k-blocks and a tile has few parts
     long long U;
 };
-// kind 0: QKV, 1: O, 2: gate/up, 3: down (layer l), 4: LM head.
-__device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int kind) {
-    int N, K, mx;
-    switch (kind) {
-        case 0: N = (p.Hq + 2 * p.Hkv) * p.hd; K = p.d; mx = p.map_xn; break;
-        case 1: N = p.d; K = p.Hq * p.hd; mx = p.map_attn; break;
-        case 2: N = 2 * p.f; K = p.d; mx = p.map_xn; break;
-        case 3: N = p.d; K = p.f; mx = p.map_act; break;
-        default: N = p.V; K = p.d; mx = p.map_xn; break;
-    }
+__host__ __device__ inline int effective_ctas(long long U, int kbt, int G) {
+    const long long min_units = kbt / 8 > 1 ? kbt / 8 : 1;
+    const long long n = U / min_units;
+    return (int)(n < 1 ? 1 : (n < G ? n : G));
+}
+// Shape of one GEMM of layer l; n_touched: touched routed experts of that layer (K_EGU, K_EDOWN).
+__device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int kind, int n_touched) {
+    int N, K, mx, mw;
     GemmShape g;
+    g.tpe = 0;
+    switch (kind) {
+        case K_QKV: N = (p.Hq + 2 * p.Hkv) * p.hd; K = p.d; mx = p.map_xn; mw = 0; break;
+        case K_O: N = p.d; K = p.Hq * p.hd; mx = p.map_attn; mw = 1; break;
+        case K_GU: N = 2 * p.f; K = p.d; mx = p.map_xn; mw = 2; break;
+        case K_DOWN: N = p.d; K = p.f; mx = p.map_act; mw = 3; break;
+        case K_ROUTER: N = p.n_experts; K = p.d; mx = p.map_xn; mw = 2; break;
+        case K_SGU: N = 2 * p.fs; K = p.d; mx = p.map_xn; mw = 3; break;
+        case K_EGU: g.tpe = 2 * p.fe / tc::BLOCK_N; N = n_touched * 2 * p.fe; K = p.d; mx = p.map_xn; mw = 4; break;   // gate map 4, up map 5
+        case K_SDOWN: N = p.d; K = p.fs; mx = p.map_act; mw = 6; break;
+        case K_EDOWN: g.tpe = p.d / tc::BLOCK_N; N = n_touched * p.d; K = p.fe; mx = p.map_act_e; mw = 7; break;
+        default: N = p.V; K = p.d; mx = p.map_xn; mw = 0; break;
+    }
     g.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
     g.kbt = K / tc::BLOCK_K;
-    g.map_w = kind == 4 ? p.n_layers * 4 : l * 4 + kind;
+    g.map_w = kind == K_LM ? p.n_layers * p.maps_per_layer : l * p.maps_per_layer + mw;
     g.map_x = mx;
     g.U = (long long)g.n_tiles * g.kbt;
+    g.Geff = effective_ctas(g.U, g.kbt, (int)gridDim.x);
     return g;
 }
-__device__ __forceinline__ long long unit_begin(long long U, int c, int G) { return U * c / G; }
+// The gi-th GEMM of the pass: its layer and kind.
+__device__ __forceinline__ void gemm_at(const PassParams& p, int gi, int& l, int& kind) {
+    const int gpl = p.moe ? 7 : 4;
+    if (gi >= p.n_layers * gpl) {
+        l = p.n_layers;
+        kind = K_LM;
+        return;
+    }
+    l = gi / gpl;
+    const int j = gi - l * gpl;
+    kind = !p.moe ? j : (j < 2 ? j : K_ROUTER + (j - 2));
+}
+// What the routed-expert GEMMs of the current layer need to know; lives in shared memory, written by
+// the compute warps after the layer's routing, read by every role (layer_ready says for which layer).
+struct Routing {
+    volatile int layer_ready;      // 1 + the layer whose list is valid
+    volatile int n_touched;
+    int mask[MAX_EXPERTS / 32];
+    short list[MAX_EXPERTS];       // touched expert ids, ascending
+    short slot_of[MAX_EXPERTS];    // expert id -> position in list
+};
+__device__ __forceinline__ bool wait_routing(const PassParams& p, const Routing* r, int l, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (r->layer_ready > l) return true;
+        if ((it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) return false;
+        __nanosleep(50);
+    }
+    return false;
+}
+// Tensor map and row coordinate of weight tile `tile` of a GEMM.
+__device__ __forceinline__ void weight_tile_coord(const PassParams& p, const GemmShape& g, int kind, int tile, const Routing* r,
+                                                  int& map_w, int& y) {
+    map_w = g.map_w;
+    if (kind == K_EGU) {
+        const int e = r->list[tile / g.tpe], t = tile % g.tpe, half = g.tpe / 2;
+        map_w += t >= half;                                   // gate rows, then up rows
+        y = e * p.fe + (t % half) * tc::BLOCK_N;
+    } else if (kind == K_EDOWN) {
+        y = r->list[tile / g.tpe] * p.d + (tile % g.tpe) * tc::BLOCK_N;
+    } else {
+        y = tile * tc::BLOCK_N;
+    }
+}
+// First unit of CTA c: the units are cut into Geff equal contiguous ranges, CTAs past Geff get none.
+__device__ __forceinline__ long long unit_begin(const GemmShape& g, int c) { return c >= g.Geff ? g.U : g.U * c / g.Geff; }
 
 // Calls f(tile, kb0, kb1, local_segment) for the segments of this CTA's unit range.
 template <class F>
 __device__ __forceinline__ void for_each_segment(const GemmShape& g, int cta, int G, F f) {
-    long long u = unit_begin(g.U, cta, G), u1 = unit_begin(g.U, cta + 1, G);
+    long long u = unit_begin(g, cta), u1 = unit_begin(g, cta + 1);
     const int first_tile = (int)(u / g.kbt);
     while (u < u1) {
         int tile = (int)(u / g.kbt);
@@ -155,46 +228,62 @@ __device__ __forceinline__ bool wait_counter(const PassParams& p, unsigned targe
 }
 
 // Walks the weight tiles (unit by unit) that one CTA streams during a pass, in order.  The
-// per-unit step is two compares; divisions happen once per GEMM.
+// per-unit step is two compares; divisions happen once per GEMM.  Before a layer's routed-expert
+// GEMMs the cursor waits for that layer's routing.
 struct UnitCursor {
     int gi, n_gemms, cta, G;
-    int left, kb, tile, kbt, map_w;
-    __device__ __forceinline__ void open(const PassParams& p) {
-        while (gi < n_gemms) {
-            const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
-            const GemmShape g = gemm_shape(p, l, kind);
-            const long long u = unit_begin(g.U, cta, G), u1 = unit_begin(g.U, cta + 1, G);
-            if (u < u1) {
-                left = (int)(u1 - u);
-                tile = (int)(u / g.kbt);
-                kb = (int)(u - (long long)tile * g.kbt);
-                kbt = g.kbt;
-                map_w = g.map_w;
-                return;
-            }
-            ++gi;
-        }
-    }
-    __device__ __forceinline__ void init(const PassParams& p, int n_gemms_, int cta_, int G_) {
+    int left, kb, tile, kind;
+    GemmShape g;
+    const Routing* routing;
+    volatile int* abort_flag;
+    bool failed, opened;
+    __device__ __forceinline__ void init(const PassParams&, int n_gemms_, int cta_, int G_, const Routing* r, volatile int* abort) {
         gi = 0;
         n_gemms = n_gemms_;
         cta = cta_;
         G = G_;
-        open(p);
+        routing = r;
+        abort_flag = abort;
+        failed = false;
+        opened = false;
     }
-    __device__ __forceinline__ bool done() const { return gi >= n_gemms; }
-    // current unit: weight map index, k-block and tile; then advance
-    __device__ __forceinline__ void next(const PassParams& p, int& map_w_, int& kb_, int& tile_) {
-        map_w_ = map_w;
+    // Next unit: weight map index, k-block and row coordinate; false when the pass is through (or a
+    // wait gave up: `failed`).  A GEMM is opened only when its first unit is asked for, so the wait for a
+    // layer's routing never holds back a unit of an earlier GEMM.
+    __device__ __forceinline__ bool next(const PassParams& p, int& map_w_, int& kb_, int& y_) {
+        while (!opened) {
+            if (gi >= n_gemms) return false;
+            int l;
+            gemm_at(p, gi, l, kind);
+            int n_touched = 0;
+            if (kind == K_EGU || kind == K_EDOWN) {
+                if (!wait_routing(p, routing, l, abort_flag)) {
+                    failed = true;
+                    return false;
+                }
+                n_touched = routing->n_touched;
+            }
+            g = gemm_shape(p, l, kind, n_touched);
+            const long long u = unit_begin(g, cta), u1 = unit_begin(g, cta + 1);
+            if (u < u1) {
+                left = (int)(u1 - u);
+                tile = (int)(u / g.kbt);
+                kb = (int)(u - (long long)tile * g.kbt);
+                opened = true;
+            } else {
+                ++gi;
+            }
+        }
+        weight_tile_coord(p, g, kind, tile, routing, map_w_, y_);
         kb_ = kb;
-        tile_ = tile;
         if (--left == 0) {
             ++gi;
-            open(p);
-        } else if (++kb == kbt) {
+            opened = false;
+        } else if (++kb == g.kbt) {
             kb = 0;
             ++tile;
         }
+        return true;
     }
 };
 // Sum over the split-K partials (in CTA order) of 4 consecutive columns of (tile, row): every
@@ -203,18 +292,50 @@ struct UnitCursor {
 __device__ __forceinline__ int tile_row_tab(const PassParams& p, int kind, int tile, int lane) {
     return lane <= MAX_PARTS ? __ldg(p.parts[kind] + (size_t)tile * (1 + MAX_PARTS) + lane) : 0;
 }
+// The same list for a GEMM whose tile count is only known at run time (routed experts): the
+// contiguous unit ranges of the CTAs that touch the tile, by the arithmetic of for_each_segment
+// (CTAs whose range is empty are skipped).  Returns -1 in lane 0 when the tile has more parts than
+// the list holds.
+__device__ __forceinline__ int dyn_tab(const GemmShape& g, int tile, int G, int max_segs, int lane) {
+    const long long ua = (long long)tile * g.kbt, ub = ua + g.kbt - 1;
+    int c_lo = (int)(ua * g.Geff / g.U);
+    while (unit_begin(g, c_lo + 1) <= ua) ++c_lo;
+    int c_hi = (int)(ub * g.Geff / g.U);
+    while (unit_begin(g, c_hi + 1) <= ub) ++c_hi;
+    const int c = c_lo + lane;                       // lane i looks at the i-th CTA from c_lo
+    long long b0 = 0;
+    bool valid = c <= c_hi;
+    if (valid) {
+        b0 = unit_begin(g, c);
+        valid = unit_begin(g, c + 1) > b0;
+    }
+    const unsigned have = __ballot_sync(0xffffffffu, valid);
+    const int cnt = __popc(have);
+    const int mine = c * max_segs + (tile - (int)(b0 / g.kbt));
+    // entry j (lane j >= 1) is the slot of the (j-1)-th valid CTA
+    const int src = lane >= 1 && lane <= cnt ? (int)__fns(have, 0, lane) : 0;
+    const int got = __shfl_sync(0xffffffffu, mine, src & 31);
+    if (lane == 0) return (cnt > MAX_PARTS || c_hi - c_lo > 31) ? -1 : cnt;
+    return lane <= cnt ? got : 0;
+}
 // NS such sums at once (tab_lane[s] = 0 marks an unused one).  Before reading, the warp waits
 // (bounded) until all `cnt * round` partials of each tile have been published by the CTAs that
 // drained them (round = layer + 1: the counters only grow).  Then the loads of up to PC parts of
 // every sum are issued together, and each sum is accumulated in part order.
+// published[s] == nullptr: no wait (a grid barrier already ordered the partials).
 template <int NS, int PC>
-__device__ __forceinline__ bool tile_row_sums(const PassParams& p, const int (&tab_lane)[NS], const int (&row)[NS],
+__device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* ws, const int (&tab_lane)[NS], const int (&row)[NS],
                                               const unsigned* const (&published)[NS], unsigned round, int lane,
                                               volatile int* abort_flag, float4 (&out)[NS]) {
     int cnt[NS], max_cnt = 0;
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
         cnt[s] = __shfl_sync(0xffffffffu, tab_lane[s], 0);
+        if (cnt[s] < 0) {      // a tile split into more parts than the lists hold
+            atomicCAS(p.status, 0, 9);
+            *abort_flag = 1;
+            cnt[s] = 0;
+        }
         max_cnt = max(max_cnt, cnt[s]);
         out[s] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
@@ -225,7 +346,7 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const int (&t
         for (uint32_t it = 0; it < SPIN_LIMIT && !ready; ++it) {
             unsigned seen[NS];
 #pragma unroll
-            for (int s = 0; s < NS; ++s) seen[s] = cnt[s] > 0 ? ld_relaxed(published[s]) : 0u;
+            for (int s = 0; s < NS; ++s) seen[s] = cnt[s] > 0 && published[s] ? ld_relaxed(published[s]) : 0xffffffffu;
             ready = true;
 #pragma unroll
             for (int s = 0; s < NS; ++s)
@@ -248,7 +369,7 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const int (&t
                 const int slot = __shfl_sync(0xffffffffu, tab_lane[s], (j0 + j + 1) & 31);
                 v[s][j] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (j0 + j < cnt[s])
-                    v[s][j] = __ldcg(reinterpret_cast<const float4*>(p.ws + ((size_t)slot * p.T + row[s]) * tc::BLOCK_N) + lane);
+                    v[s][j] = __ldcg(reinterpret_cast<const float4*>(ws + ((size_t)slot * p.T + row[s]) * tc::BLOCK_N) + lane);
             }
 #pragma unroll
         for (int s = 0; s < NS; ++s)
@@ -317,9 +438,10 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     volatile int* w_issued = abort_flag + 1;
     volatile int* x_issued = w_issued + 1;
     volatile int* consumed = x_issued + 1;
+    Routing* routing = (Routing*)(misc + 1024);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_gemms = p.n_layers * 4 + (p.n_logit > 0 ? 1 : 0);
+    const int n_gemms = p.n_layers * (p.moe ? 7 : 4) + (p.n_logit > 0 ? 1 : 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -335,6 +457,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         *w_issued = 0;
         *x_issued = 0;
         *consumed = 0;
+        routing->layer_ready = 0;
+        routing->n_touched = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 2) {
@@ -352,12 +476,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             uint64_t policy;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
             UnitCursor ld;
-            ld.init(p, n_gemms, cta, G);
+            ld.init(p, n_gemms, cta, G, routing, abort_flag);
             uint32_t i = 0;
             bool ok = true;
-            while (!ld.done()) {
-                int mw, kb, tile;
-                ld.next(p, mw, kb, tile);
+            int mw, kb, y;
+            while (ld.next(p, mw, kb, y)) {
                 const int s = (int)(i % (uint32_t)S);
                 if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
                     ok = false;
@@ -368,11 +491,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     break;
                 }
                 tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
-                tc::tma_load_2d_hint(ring + s * sbytes, p.maps + mw, kb * tc::BLOCK_K, tile * tc::BLOCK_N, &full[s], policy);
+                tc::tma_load_2d_hint(ring + s * sbytes, p.maps + mw, kb * tc::BLOCK_K, y, &full[s], policy);
                 *w_issued = (int)i + 1;
                 ++i;
             }
-            if (!ok) {
+            if (!ok || ld.failed) {
                 atomicCAS(p.status, 0, 7);
                 *abort_flag = 1;
             }
@@ -386,22 +509,39 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         uint32_t i = 0;
         bool ok = true;
         for (int gi = 0; gi < n_gemms && ok; ++gi) {
-            const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
-            const GemmShape g = gemm_shape(p, l, kind);
+            int l, kind;
+            gemm_at(p, gi, l, kind);
+            int n_touched = 0;
+            if (kind == K_EGU || kind == K_EDOWN) {
+                if (!wait_routing(p, routing, l, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                n_touched = routing->n_touched;
+            }
+            const GemmShape g = gemm_shape(p, l, kind, n_touched);
             const CUtensorMap* mx = p.maps + g.map_x;
             // which counter set, and how many pairs make a tile complete for this GEMM
-            const unsigned* cnt;
-            unsigned target;
+            const unsigned* cnt = nullptr;
+            unsigned target = 0;
             switch (kind) {
-                case 0: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 1u); break;
-                case 1: cnt = p.x_cnt[1]; target = (unsigned)p.M * (unsigned)(tc::BLOCK_N / HD) * (l + 1u); break;
-                case 2: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 2u); break;
-                case 3: cnt = p.x_cnt[2]; target = (unsigned)p.M * (l + 1u); break;
+                case K_QKV: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 1u); break;
+                case K_O: cnt = p.x_cnt[1]; target = (unsigned)p.M * (unsigned)(tc::BLOCK_N / HD) * (l + 1u); break;
+                case K_GU: case K_ROUTER: case K_SGU: case K_EGU: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 2u); break;
+                case K_DOWN: case K_SDOWN: cnt = p.x_cnt[2]; target = (unsigned)p.M * (l + 1u); break;
+                case K_EDOWN: break;     // its input is published by the grid barrier that follows the experts' SwiGLU
                 default: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * p.n_layers + 1u); break;
             }
-            for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
+            if (kind == K_EDOWN && unit_begin(g, cta + 1) > unit_begin(g, cta)) {
+                if (!wait_counter(p, (2u + 9u * l + 6u) * (unsigned)G, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+            }
+            for_each_segment(g, cta, G, [&](int tile, int kb0, int kb1, int) {
+                const int x_row = kind == K_EDOWN ? (tile / g.tpe) * T : 0;     // the expert slot's rows of act_e
                 // tiles of 128 columns = 2 k-blocks
-                for (int t0 = kb0 >> 1; t0 <= (kb1 - 1) >> 1; t0 += 32) {
+                for (int t0 = kb0 >> 1; cnt && t0 <= (kb1 - 1) >> 1; t0 += 32) {
                     const int t = t0 + lane;
                     bool ready = t > ((kb1 - 1) >> 1);
                     for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
@@ -419,8 +559,9 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         if (*abort_flag) fine = false;
                         if (fine) {
                             tc::mbar_expect_tx(&full[s], (uint32_t)T * 256u);
-                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, 0, &full[s]);
-                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES + T * 128, mx + p.map_lo_off, kb * tc::BLOCK_K, 0, &full[s]);
+                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, x_row, &full[s]);
+                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES + T * 128, mx + (kind == K_EDOWN ? 4 : p.map_lo_off), kb * tc::BLOCK_K,
+                                            x_row, &full[s]);
                             *x_issued = (int)i + 1;
                         }
                     }
@@ -440,8 +581,17 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             uint32_t i = 0, seg = 0;
             bool ok = true;
             for (int gi = 0; gi < n_gemms && ok; ++gi) {
-                const int l = gi >> 2, kind = gi < p.n_layers * 4 ? (gi & 3) : 4;
-                const GemmShape g = gemm_shape(p, l, kind);
+                int l, kind;
+                gemm_at(p, gi, l, kind);
+                int n_touched = 0;
+                if (kind == K_EGU || kind == K_EDOWN) {
+                    if (!wait_routing(p, routing, l, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    n_touched = routing->n_touched;
+                }
+                const GemmShape g = gemm_shape(p, l, kind, n_touched);
                 for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
                     const uint32_t b = seg & 1u;
                     if (seg >= 2 && !tc::mbar_wait(&acc_empty[b], ((seg >> 1) - 1) & 1, abort_flag)) return ok = false;
@@ -509,12 +659,12 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         };
         // accumulators of this CTA's segments of one GEMM -> split-K partials
         auto drain = [&](int l, int kind) {
-            const GemmShape g = gemm_shape(p, l, kind);
+            const GemmShape g = gemm_shape(p, l, kind, routing->n_touched);
             for_each_segment(g, cta, G, [&](int tile, int, int, int local) {
                 const uint32_t b = seg & 1u;
                 if (!tc::mbar_wait(&acc_full[b], (seg >> 1) & 1, abort_flag)) return ok = false;
                 tc::tc_fence_after();
-                float* mine = p.ws + ((size_t)cta * p.max_segs + local) * (size_t)T * tc::BLOCK_N + tid;
+                float* mine = p.ws + p.ws_off[kind] + ((size_t)cta * p.max_segs[kind] + local) * (size_t)T * tc::BLOCK_N + tid;
                 const uint32_t taddr = tmem_base + ((uint32_t)(cw * 32) << 16) + b * ACC_STRIDE;
                 for (int c0 = 0; c0 < T; c0 += 16) {
                     float v[16], w[16];
@@ -529,7 +679,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 if (lane == 0) mbar_arrive(&acc_empty[b]);
                 // publish: every thread's part of the partial is stored, then one release for the CTA
                 att::group_sync(BAR_COMPUTE, CTHREADS);
-                if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.tile_cnt[kind] + tile) : "memory");
+                if (tid == 0 && p.tile_cnt[kind]) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.tile_cnt[kind] + tile) : "memory");
                 ++seg;
                 return true;
             });
@@ -572,7 +722,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 const int tabs[1] = {tab}, rows[1] = {m};
                 const unsigned* const pubs[1] = {p.tile_cnt[kind] + t};
                 float4 sums[1];
-                tile_row_sums<1, 8>(p, tabs, rows, pubs, round, lane, abort_flag, sums);
+                tile_row_sums<1, 8>(p, p.ws + p.ws_off[kind], tabs, rows, pubs, round, lane, abort_flag, sums);
                 float4 x = sums[0];
                 x.x += hv.x;
                 x.y += hv.y;
@@ -598,7 +748,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         for (int l = 0; l < p.n_layers && ok; ++l) {
             const LayerGains lg = p.gains[l];
             // ---- QKV GEMM ----
-            drain(l, 0);
+            drain(l, K_QKV);
             if (!ok) break;
             // ---- 1/rms, q/k norm, RoPE, K/V write: one warp per (128-column tile, row) ----
             {
@@ -636,7 +786,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                     float4 sums[2];
                     const unsigned* const pubs_c[2] = {pubs[0], pubs[1]};
-                    tile_row_sums<2, 8>(p, tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
+                    tile_row_sums<2, 8>(p, p.ws + p.ws_off[K_QKV], tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
                     for (int q = 0; q < 2; ++q) {
                         const float inv = inv_rms_from(sq_l[q], d, p.eps);
@@ -761,15 +911,13 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             grid_sync(true);
             if (!ok) break;
             // ---- O GEMM, residual ----
-            drain(l, 1);
+            drain(l, K_O);
             if (!ok) break;
-            residual_phase(1, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b);
+            residual_phase(K_O, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b);
             grid_sync(true);
             if (!ok) break;
-            // ---- gate/up GEMM, SwiGLU ----
-            drain(l, 2);
-            if (!ok) break;
-            {
+            // SwiGLU of a dense or shared-expert gate/up GEMM -> act (hi/lo), counted per tile
+            auto swiglu_phase = [&](int gu_kind) {
                 const int f_tiles = p.f / tc::BLOCK_N, n_pairs = f_tiles * M;
                 // three (tile, row) pairs per step so that all their loads overlap
                 constexpr int NP = 3;
@@ -784,16 +932,16 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         on[q] = pr < n_pairs;
                         tt[q] = on[q] ? pr / M : 0;
                         mm[q] = on[q] ? pr % M : 0;
-                        tabs[2 * q] = on[q] ? tile_row_tab(p, 2, tt[q], lane) : 0;
-                        tabs[2 * q + 1] = on[q] ? tile_row_tab(p, 2, tt[q] + f_tiles, lane) : 0;
+                        tabs[2 * q] = on[q] ? tile_row_tab(p, gu_kind, tt[q], lane) : 0;
+                        tabs[2 * q + 1] = on[q] ? tile_row_tab(p, gu_kind, tt[q] + f_tiles, lane) : 0;
                         rows[2 * q] = rows[2 * q + 1] = mm[q];
-                        pubs[2 * q] = p.tile_cnt[2] + tt[q];
-                        pubs[2 * q + 1] = p.tile_cnt[2] + tt[q] + f_tiles;
+                        pubs[2 * q] = p.tile_cnt[gu_kind] + tt[q];
+                        pubs[2 * q + 1] = p.tile_cnt[gu_kind] + tt[q] + f_tiles;
                         sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane);
                     }
                     float4 sums[2 * NP];
                     const unsigned* const pubs_c[2 * NP] = {pubs[0], pubs[1], pubs[2], pubs[3], pubs[4], pubs[5]};
-                    tile_row_sums<2 * NP, 4>(p, tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
+                    tile_row_sums<2 * NP, 4>(p, p.ws + p.ws_off[gu_kind], tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
                     for (int q = 0; q < NP; ++q) {
                         const float inv = inv_rms_from(sq_l[q], d, p.eps);
@@ -817,18 +965,219 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                             if (on[q]) asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p.x_cnt[2] + tt[q]) : "memory");
                     }
                 }
+            };
+            const float* next_gain = l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm;
+            if (!p.moe) {
+                // ---- gate/up GEMM, SwiGLU ----
+                drain(l, K_GU);
+                if (!ok) break;
+                swiglu_phase(K_GU);
+                grid_sync(true);
+                if (!ok) break;
+                // ---- down GEMM, residual; prepares the next layer's (or the head's) input ----
+                drain(l, K_DOWN);
+                if (!ok) break;
+                residual_phase(K_DOWN, (unsigned)l + 1u, next_gain, p.ssq_a);
+                grid_sync(true);
+                continue;
+            }
+            // ================= mixture of experts =================
+            // ---- router GEMM; per row: softmax over the experts, top-k (ties -> lowest id), gates renormalised ----
+            drain(l, K_ROUTER);
+            if (!ok) break;
+            {
+                const int e_tiles = p.n_experts / tc::BLOCK_N;     // 1 or 2
+                for (int m = gw; m < M; m += GW) {
+                    int tabs[2], rows[2] = {m, m};
+                    const unsigned* pubs[2];
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        tabs[t] = t < e_tiles ? tile_row_tab(p, K_ROUTER, t, lane) : 0;
+                        pubs[t] = p.tile_cnt[K_ROUTER] + t;
+                    }
+                    const SsqLane sq_l = row_ssq_lane(p.ssq_b, d_tiles, m, lane);
+                    float4 sums[2];
+                    const unsigned* const pubs_c[2] = {pubs[0], pubs[1]};
+                    tile_row_sums<2, 8>(p, p.ws + p.ws_off[K_ROUTER], tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
+                    const float inv = inv_rms_from(sq_l, d, p.eps);
+                    // lane holds logits of experts 4*lane .. +3 (tile 0) and 128 + 4*lane .. +3 (tile 1)
+                    float x[8] = {inv * sums[0].x, inv * sums[0].y, inv * sums[0].z, inv * sums[0].w,
+                                  inv * sums[1].x, inv * sums[1].y, inv * sums[1].z, inv * sums[1].w};
+                    const int n_mine = 4 * e_tiles;
+                    float mx = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i < n_mine) mx = fmaxf(mx, x[i]);
+                    mx = warp_max(mx);
+                    float sum = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i < n_mine) sum += expf(x[i] - mx);
+                    sum = warp_sum(sum);
+                    float last_v = INFINITY, kept = 0.f, my_gate = 0.f;
+                    int last_i = -1, my_id = 0;
+                    for (int k = 0; k < p.top_k; ++k) {
+                        // candidates strictly after (last_v, last_i) in the order (value desc, id asc)
+                        float bv = -INFINITY;
+                        int bi = 0x7fffffff;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (i >= n_mine) continue;
+                            const int e = (i >> 2) * tc::BLOCK_N + 4 * lane + (i & 3);
+                            const float v = x[i];
+                            const bool after = (v < last_v) || (v == last_v && e > last_i);
+                            if (after && (v > bv || (v == bv && e < bi))) {
+                                bv = v;
+                                bi = e;
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                            if (ov > bv || (ov == bv && oi < bi)) {
+                                bv = ov;
+                                bi = oi;
+                            }
+                        }
+                        last_v = bv;
+                        last_i = bi;
+                        const float pk = expf(bv - mx) / sum;
+                        kept += pk;
+                        if (lane == k) {
+                            my_gate = pk;
+                            my_id = bi;
+                        }
+                    }
+                    if (lane < p.top_k) {
+                        p.moe_ids[(size_t)m * p.top_k + lane] = my_id;
+                        p.moe_gates[(size_t)m * p.top_k + lane] = my_gate / kept;
+                        p.moe_ids_trace[(size_t)l * p.trace_stride + (size_t)m * p.top_k + lane] = my_id;
+                    }
+                }
+            }
+            grid_sync(false);
+            if (!ok) break;
+            // ---- the touched experts of this layer, ascending; every CTA builds the same list ----
+            {
+                if (tid < MAX_EXPERTS / 32) routing->mask[tid] = 0;
+                att::group_sync(BAR_COMPUTE, CTHREADS);
+                for (int i = tid; i < M * p.top_k; i += CTHREADS) {
+                    const int e = __ldcg(p.moe_ids + i);
+                    atomicOr(&routing->mask[e >> 5], 1 << (e & 31));
+                }
+                att::group_sync(BAR_COMPUTE, CTHREADS);
+                int before = 0;
+                for (int w = 0; w < MAX_EXPERTS / 32; ++w) {
+                    const unsigned mword = (unsigned)routing->mask[w];
+                    for (int e = tid; e < 32; e += CTHREADS)   // tid < 32: one word per round
+                        if (mword >> e & 1u) {
+                            const int pos = before + __popc(mword & ((1u << e) - 1u));
+                            routing->list[pos] = (short)(w * 32 + e);
+                            routing->slot_of[w * 32 + e] = (short)pos;
+                        }
+                    before += __popc(mword);
+                }
+                att::group_sync(BAR_COMPUTE, CTHREADS);
+                if (tid == 0) {
+                    routing->n_touched = before;
+                    __threadfence_block();
+                    routing->layer_ready = l + 1;
+                    if (cta == 0) p.n_touched_out[l] = before;
+                }
+                att::group_sync(BAR_COMPUTE, CTHREADS);
+            }
+            const int n_touched = routing->n_touched;
+            // ---- shared expert gate/up, SwiGLU (its weights do not depend on the routing) ----
+            drain(l, K_SGU);
+            if (!ok) break;
+            swiglu_phase(K_SGU);
+            // ---- routed experts gate/up over all rows; SwiGLU only for the (row, expert) pairs that were routed ----
+            drain(l, K_EGU);
+            if (!ok) break;
+            grid_sync(true);
+            if (!ok) break;
+            {
+                const GemmShape g = gemm_shape(p, l, K_EGU, n_touched);
+                const int fe_tiles = p.fe / tc::BLOCK_N;
+                const int n_items = M * p.top_k * fe_tiles;
+                const float* wsb = p.ws + p.ws_off[K_EGU];
+                for (int item = gw; item < n_items; item += GW) {
+                    const int j = item % fe_tiles, rs = item / fe_tiles, m = rs / p.top_k;
+                    const int slot = routing->slot_of[__ldcg(p.moe_ids + rs)];
+                    const SsqLane sq_l = row_ssq_lane(p.ssq_b, d_tiles, m, lane);
+                    const int tg = slot * g.tpe + j, tu = tg + fe_tiles;
+                    const int tabs[2] = {dyn_tab(g, tg, G, p.max_segs[K_EGU], lane), dyn_tab(g, tu, G, p.max_segs[K_EGU], lane)};
+                    const int rows[2] = {m, m};
+                    const unsigned* const pubs[2] = {nullptr, nullptr};
+                    float4 sums[2];
+                    tile_row_sums<2, 8>(p, wsb, tabs, rows, pubs, 0u, lane, abort_flag, sums);
+                    const float inv = inv_rms_from(sq_l, d, p.eps);
+                    const float gv[4] = {inv * sums[0].x, inv * sums[0].y, inv * sums[0].z, inv * sums[0].w};
+                    const float uv[4] = {inv * sums[1].x, inv * sums[1].y, inv * sums[1].z, inv * sums[1].w};
+                    float a[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) a[e] = __fdividef(gv[e], 1.f + __expf(-gv[e])) * uv[e];
+                    const size_t o = ((size_t)slot * T + m) * p.fe + j * tc::BLOCK_N + 4 * lane;
+                    store_hi_lo_x4(p.act_e + o, p.act_e_lo + o, a[0], a[1], a[2], a[3]);
+                }
             }
             grid_sync(true);
             if (!ok) break;
-            // ---- down GEMM, residual; prepares the next layer's (or the head's) input ----
-            drain(l, 3);
+            // ---- shared and routed down GEMMs; h += shared + sum_k gate_k * expert_k; next layer's input ----
+            drain(l, K_SDOWN);
             if (!ok) break;
-            residual_phase(3, (unsigned)l + 1u, l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm, p.ssq_a);
+            drain(l, K_EDOWN);
+            if (!ok) break;
+            grid_sync(false);
+            if (!ok) break;
+            {
+                const GemmShape g = gemm_shape(p, l, K_EDOWN, n_touched);
+                const float* wsb = p.ws + p.ws_off[K_EDOWN];
+                h_phase(next_gain, p.ssq_a, [&](int t, int m, int col) {
+                    const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
+                    float4 x;
+                    {   // shared expert
+                        const int tabs[1] = {tile_row_tab(p, K_SDOWN, t, lane)}, rows[1] = {m};
+                        const unsigned* const pubs[1] = {nullptr};
+                        float4 sums[1];
+                        tile_row_sums<1, 8>(p, p.ws + p.ws_off[K_SDOWN], tabs, rows, pubs, 0u, lane, abort_flag, sums);
+                        x = sums[0];
+                    }
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int k0 = 0; k0 < p.top_k; k0 += 4) {     // routed experts in slot order, four at a time
+                        int tabs[4], rows[4] = {m, m, m, m};
+                        float gk[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const bool on = k0 + q < p.top_k;
+                            const int e = on ? __ldcg(p.moe_ids + (size_t)m * p.top_k + k0 + q) : 0;
+                            gk[q] = on ? __ldcg(p.moe_gates + (size_t)m * p.top_k + k0 + q) : 0.f;
+                            tabs[q] = on ? dyn_tab(g, routing->slot_of[e] * g.tpe + t, G, p.max_segs[K_EDOWN], lane) : 0;
+                        }
+                        const unsigned* const pubs[4] = {nullptr, nullptr, nullptr, nullptr};
+                        float4 sums[4];
+                        tile_row_sums<4, 4>(p, wsb, tabs, rows, pubs, 0u, lane, abort_flag, sums);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            acc.x += gk[q] * sums[q].x;
+                            acc.y += gk[q] * sums[q].y;
+                            acc.z += gk[q] * sums[q].z;
+                            acc.w += gk[q] * sums[q].w;
+                        }
+                    }
+                    x.x = hv.x + (acc.x + x.x);
+                    x.y = hv.y + (acc.y + x.y);
+                    x.z = hv.z + (acc.z + x.z);
+                    x.w = hv.w + (acc.w + x.w);
+                    return x;
+                });
+            }
             grid_sync(true);
         }
         if (ok && p.n_logit > 0) {
             // ---- LM head on the rows that need logits ----
-            drain(p.n_layers, 4);
+            drain(p.n_layers, K_LM);
             if (ok) {
                 const int n_tiles = (p.V + tc::BLOCK_N - 1) / tc::BLOCK_N;
                 const bool vec = (p.V & 3) == 0;
@@ -840,7 +1189,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     const int tabs[1] = {tab}, rows[1] = {m};
                     const unsigned* const pubs[1] = {p.tile_cnt[4] + t};
                     float4 sums[1];
-                    tile_row_sums<1, 8>(p, tabs, rows, pubs, 1u, lane, abort_flag, sums);
+                    tile_row_sums<1, 8>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs, 1u, lane, abort_flag, sums);
                     const float4 s4 = sums[0];
                     const float sc = p.logit_scale * inv_rms_from(sq_l, d, p.eps);
                     const int col = t * tc::BLOCK_N + 4 * lane;

@@ -365,9 +365,11 @@ static int enqueue_status_read(s2d2_ctx* c) {
 }
 static int check_status(s2d2_ctx* c) {
     if (*c->h_status == 0) return S2D2_OK;
+    const int code = *c->h_status;
     *c->h_status = 0;
     cudaMemsetAsync(c->d_status, 0, 4, c->stream);
-    FAIL(c, S2D2_ERR_TIMEOUT, "a kernel gave up on a bounded wait (results of this call are invalid)");
+    FAIL(c, S2D2_ERR_TIMEOUT, "a kernel gave up on a bounded wait (results of this call are invalid; device status word " +
+                                   std::to_string(code) + ")");
 }
 
 static int check_weights(s2d2_ctx* c) {

@@ -73,6 +73,8 @@ _t_bf16 = ModelConfig("t-dense-bf16", 2, 256, 4, 2, 64, 512, 1000)
 _t_bf16_128 = ModelConfig("t-dense-bf16-hd128", 2, 512, 4, 2, 128, 768, 2000)
 _t_moe = ModelConfig("t-moe-bf16", 2, 256, 4, 2, 64, 0, 1000,
                      n_experts=16, top_k=4, expert_ffn=128, n_shared=1)
+_t_moe128 = ModelConfig("t-moe128-bf16", 2, 256, 4, 2, 64, 0, 1000,
+                        n_experts=128, top_k=8, expert_ffn=128, n_shared=1)
 _t_f32 = ModelConfig("t-dense-fp32", 2, 64, 2, 1, 32, 96, 50, dtype="fp32",
                      rope_base=1.0e4, qk_norm=True, logit_scale=3.0)
 
@@ -86,6 +88,7 @@ CONFIGS = {
     "t_bf16": WorkloadConfig("t_bf16", _t_bf16, 3, (5, 70), 4, 16, kv_page_tokens=16),
     "t_bf16_128": WorkloadConfig("t_bf16_128", _t_bf16_128, 2, (60, 130), 8, 24),
     "t_moe": WorkloadConfig("t_moe", _t_moe, 2, (9, 40), 8, 16, kv_page_tokens=16),
+    "t_moe128": WorkloadConfig("t_moe128", _t_moe128, 2, (9, 40), 8, 16, kv_page_tokens=16),
     "t_f32": WorkloadConfig("t_f32", _t_f32, 2, (3, 20), 4, 12, kv_page_tokens=8),
 }
 

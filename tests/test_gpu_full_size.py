@@ -38,3 +38,25 @@ def test_full_shape_steps_match_oracle(name, n_steps, batch):
         check_kv(e, W, wl.model, ids[0], atol=4e-2)
     e.close()
 
+
+
+def test_full_shape_moe_step_matches_oracle():
+    """The MoE workload's shape (20 layers, 256 experts of width 512, top-8, vocabulary 157184) with a
+    block of 8 so that the oracle's per-row expert loop stays affordable."""
+    from paper_2603_25702_b200 import Engine
+    from tests.parity_util import moe_prefill_shadows, register_prompt_lens, run_steps
+    wl = get_config("c5", prompt_len=(6, 6), block_size=8, gen_tokens=8)
+    W = generate_weights(wl.model, seed=wl.weight_seed)
+    e = Engine(wl.model, block_size=wl.block_size, max_batch=1, max_seq_len=128, kv_page_tokens=wl.kv_page_tokens,
+               seed=wl.philox_seed, stream=torch.cuda.current_stream().cuda_stream)
+    e.load_weights(W)
+    prompts = generate_prompts(wl)
+    ids = e.prefill(prompts)
+    register_prompt_lens(ids, prompts)
+    e.seq_set_rng_stream(ids[0], 0)
+    shadows = moe_prefill_shadows(e, W, wl.model, ids, prompts)
+    rep = run_steps(e, W, wl, ids, {ids[0]: 0}, n_steps=1, logit_atol=2e-2, shadows=shadows)
+    print("c5", rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.stage_b_passes >= 1
+    e.close()

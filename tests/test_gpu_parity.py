@@ -109,9 +109,12 @@ def test_batch_composition_does_not_change_results():
         e1.close()
 
 
-def test_moe_stepwise_parity():
+@pytest.mark.parametrize("name", ["t_moe", "t_moe128"])
+def test_moe_stepwise_parity(name):
+    """t_moe (16 experts) runs the per-operation kernels, t_moe128 (128 experts, top-8) the persistent pass."""
     from tests.parity_util import moe_prefill_shadows, run_steps
-    wl = get_config("t_moe")
+    # the shadows mirror the engine's expert choice of one prefill pass: both prompts must fit 64 rows together
+    wl = get_config(name, prompt_len=(9, 30))
     W = generate_weights(wl.model, seed=4, gain_jitter=0.1)
     e, ids, prompts = _start(wl, W)
     shadows = moe_prefill_shadows(e, W, wl.model, ids, prompts)
