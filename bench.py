@@ -49,24 +49,39 @@ class ClockSampler:
 
     def __init__(self, gpu_index: int):
         self.rows, self.proc, self.gpu = [], None, gpu_index
+        self.t0 = self.t1 = None
 
     def start(self):
+        """Started before the warm-up steps: nvidia-smi takes a few hundred ms to deliver its first sample."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.perf_counter(), [x.strip() for x in line.split(",")]))
+
+    def mark_begin(self):
+        self.t0 = time.perf_counter()
+
+    def mark_end(self):
+        self.t1 = time.perf_counter()
 
     def stop(self):
         if self.proc:
             self.proc.terminate()
+        # samples inside the timed region; if it was shorter than the sampling period, the samples under load
+        # around it (warm-up steps run the same work)
+        inside = [r for t, r in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t)]
+        window = "timed region"
+        if len(inside) < 2:
+            inside = [r for t, r in self.rows if self.t0 is None or t >= self.t0 - 1.0]
+            window = "timed region and the second before it (warm-up)"
         sm, mx, reasons = [], 0.0, set()
-        for r in self.rows:
+        for r in inside:
             try:
                 sm.append(float(r[1]))
                 mx = max(mx, float(r[2]))
@@ -76,7 +91,7 @@ class ClockSampler:
             except Exception:
                 pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "window": window}
 
 
 def oracle_decode_steps(wl, W, n_steps: int, prompt_len: int = 8):
@@ -180,7 +195,7 @@ def main():
     from paper_2603_25702_b200.build import build
     build()
     m, B = wl.model, wl.block_size
-    total_steps = args.warmup + args.steps + args.profile_steps + 2
+    total_steps = args.warmup + args.steps + args.profile_steps + 2 + 400     # 400: room for the time-based part of the warm-up
     max_seq = wl.prompt_len[1] + total_steps * B + 2 * B
     t_setup = time.perf_counter()
     W = generate_weights(m, seed=wl.weight_seed)
@@ -201,16 +216,22 @@ def main():
         eng.verify_block(ids, fl)
         return eng.accept_and_commit(ids, fl)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_w = time.perf_counter()
     for _ in range(args.warmup):
         step()
+    n_extra = 0
+    while time.perf_counter() - t_w < 0.6 and n_extra < 390:      # same load until the clock sampler delivers
+        step()
+        n_extra += 1
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     eng.reset_counters()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    sampler.mark_begin()
     t0 = time.perf_counter()
     ev0.record()
     committed = 0
@@ -221,6 +242,7 @@ def main():
     ev1.record()
     torch.cuda.synchronize()
     wall = time.perf_counter() - t0
+    sampler.mark_end()
     dev_ms = ev0.elapsed_time(ev1)
     cnt = eng.get_counters()
     clocks = sampler.stop()
