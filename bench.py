@@ -193,13 +193,14 @@ def main():
 
     from paper_2603_25702_b200 import Engine
     from paper_2603_25702_b200.build import build
+    from paper_2603_25702_b200.replicas import aggregate_over_ranks, rank_prompt_seed
     build()
     m, B = wl.model, wl.block_size
     total_steps = args.warmup + args.steps + args.profile_steps + 2 + 400     # 400: room for the time-based part of the warm-up
     max_seq = wl.prompt_len[1] + total_steps * B + 2 * B
     t_setup = time.perf_counter()
     W = generate_weights(m, seed=wl.weight_seed)
-    prompts = generate_prompts(wl, seed=wl.prompt_seed + rank)
+    prompts = generate_prompts(wl, seed=rank_prompt_seed(wl.prompt_seed, rank))
     eng = Engine(m, block_size=B, max_batch=wl.batch, max_seq_len=max_seq, kv_page_tokens=wl.kv_page_tokens,
                  seed=wl.philox_seed, tau_conf=wl.tau_conf, stream=torch.cuda.current_stream().cuda_stream)
     eng.load_weights(W)
@@ -248,11 +249,7 @@ def main():
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
-        t = torch.tensor([dev_ms, wall], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        n = torch.tensor([committed], device="cuda", dtype=torch.float64)
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        dev_ms, wall, committed = float(t[0]), float(t[1]), int(n[0])
+    dev_ms, wall, committed = aggregate_over_ranks(dev_ms, wall, committed)
 
     # roofline of the dominant kernel: its launches are bracketed by CUDA event pairs on the library's
     # own stream (the persistent pass kernel, one launch per draft or verifier pass; on shapes it does

@@ -264,6 +264,12 @@ int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t
  * s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */
 int s2d2_debug_pass_trace(s2d2_ctx* ctx, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks);
 
+/* Failure-path tap: runs the kernels' bounded-wait pattern on a word that nothing sets.  With
+ * target > 0 the wait runs out after limit_polls polls (<= 2^20, about 0.1 us each), the kernel raises
+ * the status word and returns normally, and the call returns S2D2_ERR_TIMEOUT; the context stays
+ * usable.  With target == 0 the wait is satisfied at once and the call returns S2D2_OK. */
+int s2d2_debug_wait_timeout(s2d2_ctx* ctx, uint32_t target, uint32_t limit_polls);
+
 /* y[M, N] = x[M, K] w[N, K]^T on device buffers, without any allocation.
  * (The paper has no counterpart: this is a service entry for hosts that must not
  * allocate.)  Some callers cannot call cudaMalloc: a serving process whose framework

@@ -78,7 +78,7 @@ EXPORTS = [
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
     "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
-    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace",
+    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace", "s2d2_debug_wait_timeout",
     "s2d2_gemm_bf16_noalloc", "s2d2_noalloc_last_error",
 ]
 
@@ -131,6 +131,7 @@ def load_library() -> C.CDLL:
     lib.s2d2_debug_seq_state.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.s2d2_debug_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.s2d2_debug_copy_expert_ids.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int64, C.POINTER(C.c_int32)]
+    lib.s2d2_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32]
     lib.s2d2_debug_pass_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     _LIB = lib
     return lib
@@ -334,6 +335,10 @@ class Engine:
         y = np.empty((M, N), dtype=np.float32)
         self._check(self.lib.s2d2_debug_gemm(self._h, x.ctypes.data, w.ctypes.data, M, N, K, y.ctypes.data))
         return y
+
+    def debug_wait_timeout(self, target: int, limit_polls: int = 1000):
+        """Runs the bounded-wait pattern on a word nothing sets; raises S2D2Error(-5) when target > 0."""
+        self._check(self.lib.s2d2_debug_wait_timeout(self._h, target, limit_polls))
 
     def debug_pass_trace(self) -> np.ndarray:
         """(marks [n_ctas, n_barriers, 3], sm_ids [n_ctas]): global-timer ns at entry to / exit from every grid

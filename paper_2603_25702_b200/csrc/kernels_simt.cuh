@@ -292,6 +292,18 @@ static __global__ void moe_combine_kernel(const float* __restrict__ pair_out, co
     h[idx] += acc;
 }
 
+// The bounded-wait pattern of the tensor-core kernels in isolation (test tap): poll a word that is
+// expected to reach `target`; after `limit` polls raise the status word and return normally.
+static __global__ void bounded_wait_probe_kernel(const unsigned* __restrict__ word, unsigned target, unsigned limit, int* status) {
+    for (unsigned it = 0; it < limit; ++it) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+        if (v >= target) return;
+        __nanosleep(100);
+    }
+    atomicCAS(status, 0, 10);
+}
+
 // Copy K/V of cache positions [0, n) of one layer to fp32 (test tap).
 template <typename TKV>
 __global__ void kv_export_kernel(KvPool<TKV> pool, const int* __restrict__ pages, int layer, int n, float* __restrict__ k,

@@ -1238,3 +1238,20 @@ extern "C" int s2d2_debug_pass_trace(s2d2_ctx* c, uint64_t* out, int64_t cap, in
     if (!c || !out || !n_ctas || !n_marks) return S2D2_ERR_INVALID;
     return pass_copy_trace(c, (unsigned long long*)out, cap, n_ctas, n_marks);
 }
+
+extern "C" int s2d2_debug_wait_timeout(s2d2_ctx* c, uint32_t target, uint32_t limit_polls) {
+    if (!c || limit_polls == 0 || limit_polls > (1u << 20)) return S2D2_ERR_INVALID;
+    // the word polled is the status word's neighbour in a zeroed 8-byte allocation: nothing ever sets it
+    unsigned* word = nullptr;
+    CUDA_TRY(c, cudaMalloc((void**)&word, 8));
+    CUDA_TRY(c, cudaMemsetAsync(word, 0, 8, c->stream));
+    bounded_wait_probe_kernel<<<1, 1, 0, c->stream>>>(word, target, limit_polls, c->d_status);
+    LAUNCHED(c);
+    int rc = enqueue_status_read(c);
+    if (!rc) {
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        rc = check_status(c);
+    }
+    cudaFree(word);
+    return rc;
+}

@@ -191,3 +191,19 @@ def test_error_paths_return_codes_not_faults():
     with pytest.raises(S2D2Error):
         e.draft_block([sid])
     e.close()
+
+
+def test_bounded_wait_times_out_with_a_status_not_a_hang():
+    """A wait that nothing satisfies ends after its poll limit with S2D2_ERR_TIMEOUT; the context then
+    decodes as usual (the status word is cleared, nothing is left in flight)."""
+    from paper_2603_25702_b200 import S2D2Error
+    wl = get_config("t_bf16")
+    W = generate_weights(wl.model, seed=1)
+    e, ids, _ = _start(wl, W)
+    e.debug_wait_timeout(0)                       # satisfied at once
+    with pytest.raises(S2D2Error) as ei:
+        e.debug_wait_timeout(1, limit_polls=2000)
+    assert ei.value.code == -5 and "status word 10" in str(ei.value)
+    e.generate(ids, wl.block_size)                # still usable
+    assert all(len(e.get_tokens(s)) > 0 for s in ids)
+    e.close()
