@@ -185,19 +185,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int n = n0 + n_local;
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
         const int m_hi = min(T, p.M - m0);
+        // In both epilogues the loads of 16 rows (previous y for an accumulating GEMM, split-K partials)
+        // are issued together before anything is stored: one round trip per 16 rows instead of one per row.
         if (p.splits == 1) {
             for (int c = 0; c < T; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);      // executed by the whole warp even past m_hi (aligned instruction)
                 if (n < p.N) {
+                    float old[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        int m = c + j;
-                        if (m < m_hi) {
-                            float* y = p.Y + (size_t)(m0 + m) * p.ldy + n;
-                            *y = p.accumulate ? (*y + p.scale * v[j]) : p.scale * v[j];
-                        }
-                    }
+                    for (int j = 0; j < 16; ++j)
+                        old[j] = (p.accumulate && c + j < m_hi) ? __ldcg(p.Y + (size_t)(m0 + c + j) * p.ldy + n) : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c + j < m_hi) p.Y[(size_t)(m0 + c + j) * p.ldy + n] = old[j] + p.scale * v[j];
                 }
             }
         } else {
@@ -219,13 +220,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             __syncthreads();
             if (*last_flag) {
                 __threadfence();
-                const float* base = p.ws + (size_t)tile * p.splits * (size_t)T * BLOCK_N;
+                const float* base = p.ws + (size_t)tile * p.splits * (size_t)T * BLOCK_N + n_local;
                 if (n < p.N) {
-                    for (int m = 0; m < m_hi; ++m) {
-                        float acc = 0.f;
-                        for (int s = 0; s < p.splits; ++s) acc += __ldcg(base + ((size_t)s * T + m) * BLOCK_N + n_local);
-                        float* y = p.Y + (size_t)(m0 + m) * p.ldy + n;
-                        *y = p.accumulate ? (*y + p.scale * acc) : p.scale * acc;
+                    for (int c = 0; c < m_hi; c += 16) {
+                        float acc[16], old[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            acc[j] = 0.f;
+                            old[j] = (p.accumulate && c + j < m_hi) ? __ldcg(p.Y + (size_t)(m0 + c + j) * p.ldy + n) : 0.f;
+                        }
+                        for (int s0 = 0; s0 < p.splits; s0 += 2) {       // partials summed in split order, two splits per round trip
+                            float t0[16], t1[16];
+                            const bool two = s0 + 1 < p.splits;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const bool in = c + j < m_hi;
+                                t0[j] = in ? __ldcg(base + ((size_t)s0 * T + c + j) * BLOCK_N) : 0.f;
+                                t1[j] = in && two ? __ldcg(base + ((size_t)(s0 + 1) * T + c + j) * BLOCK_N) : 0.f;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                acc[j] += t0[j];
+                                if (two) acc[j] += t1[j];
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c + j < m_hi) p.Y[(size_t)(m0 + c + j) * p.ldy + n] = old[j] + p.scale * acc[j];
                     }
                 }
                 if (threadIdx.x == 0) p.tickets[tile] = 0;   // ready for the next launch

@@ -591,7 +591,8 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
     const int CH = S2D2_MAX_ROWS_PER_SEQ;
     // Rows per pass: where the persistent pass kernel is available a chunk is cut to what that kernel
     // takes (it is both faster and carries two-term operands); otherwise one chunk of every sequence.
-    const int budget = pass_max_rows(c) > 0 ? pass_max_rows(c) : CH * (int)ids.size();
+    // (a few sequences only: a large batch prefills faster as wide per-operation passes, which are tensor-bound)
+    const int budget = pass_max_rows(c) > 0 && ids.size() <= 4 ? pass_max_rows(c) : CH * (int)ids.size();
     std::vector<int> took(ids.size());
     for (;;) {
         PassBuild pb;
