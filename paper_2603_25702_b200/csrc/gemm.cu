@@ -97,7 +97,10 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
         if ((size_t)tiles * s * p.T * tc::BLOCK_N > g->ws_floats && s > 1) break;
         if ((size_t)tiles > g->n_tickets && s > 1) break;
         int waves = (tiles * s + slots - 1) / slots;
-        double cost = waves * ((double)(p.kb_total + s - 1) / s + 6.0) + (s > 1 ? 2.0 : 0.0);
+        // per CTA: its k-blocks, a fixed set-up cost, and an epilogue that grows with the token tile (a split adds
+        // the partial tile's round trip through the workspace); all in units of one k-block of a 16-row tile
+        const double kb_cost = 1.0 + p.T / 64.0, epi = p.T / 16.0;
+        double cost = waves * ((double)(p.kb_total + s - 1) / s * kb_cost + 6.0 + epi * (s > 1 ? 3.0 : 1.0)) + (s > 1 ? 2.0 : 0.0);
         if (cost < best_cost - 1e-9) {
             best_cost = cost;
             best = s;
