@@ -173,6 +173,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-steps", type=int, default=6)
+    ap.add_argument("--shaped-steps", type=int, default=20,
+                    help="extra timed steps with the accept test overridden by u < 0.77 (the paper's per-token acceptance), reported under 'shaped'; 0: skip")
     ap.add_argument("--warmup-seconds", type=float, default=0.6,
                     help="keep stepping after the --warmup steps until the clock sampler has had this long to deliver (0: exactly --warmup steps, for profiler runs)")
     args = ap.parse_args()
@@ -198,7 +200,7 @@ def main():
     from paper_2603_25702_b200.replicas import aggregate_over_ranks, rank_prompt_seed
     build()
     m, B = wl.model, wl.block_size
-    total_steps = args.warmup + args.steps + args.profile_steps + 2 + 400     # 400: room for the time-based part of the warm-up
+    total_steps = args.warmup + args.steps + args.profile_steps + args.shaped_steps + 5 + 400     # 400: room for the time-based part of the warm-up
     max_seq = wl.prompt_len[1] + total_steps * B + 2 * B
     t_setup = time.perf_counter()
     W = generate_weights(m, seed=wl.weight_seed)
@@ -262,9 +264,35 @@ def main():
     prof = eng.get_gemm_profile()
     eng.set_profiling(0)
     peak, peak_kind = measured_peaks()
+    n_ctx = eng.debug_seq_state(ids[0])["n_cached"]
+
+    # Shaped run: random weights accept few drafted tokens, the paper's trained models about 0.77 of
+    # the verified ones (its table of confidence/ratio quadrants).  Same steps with the accept test
+    # replaced by u < 0.77: a throughput figure at the paper's accepted-length profile, never a parity case.
+    shaped = None
+    if args.shaped_steps > 0:
+        eng.set_accept_override(0.77)
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        eng.reset_counters()
+        sv0, sv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sv0.record()
+        s_committed = 0
+        for _ in range(args.shaped_steps):
+            s_committed += sum(r.n_committed for r in step())
+        sv1.record()
+        torch.cuda.synchronize()
+        s_ms = sv0.elapsed_time(sv1)
+        sc = eng.get_counters()
+        eng.set_accept_override(0.0)
+        shaped = {"accept_test": "u < 0.77", "steps": args.shaped_steps, "value": s_committed / (s_ms * 1e-3), "unit": "tokens/s",
+                  "ms_per_step": s_ms / args.shaped_steps,
+                  "mean_accepted_per_verify": sc.n_accepted_tokens / max(1, sc.n_verify_passes * wl.batch),
+                  "tokens_per_step": s_committed / args.shaped_steps,
+                  "accepted_len_hist": [int(x) for x in list(sc.accepted_len_hist)[:B + 1]]}
     achieved = prof["bytes"] / (prof["ms"] * 1e-3) / 1e9 if prof["ms"] > 0 else 0.0
     persistent = prof["launches"] <= 2 * args.profile_steps + 1
-    n_ctx = eng.debug_seq_state(ids[0])["n_cached"]
 
     pass_bytes = model_pass_bytes(m)
     verify_ms = cnt.ms_verify / max(1, cnt.n_verify_passes)
@@ -300,7 +328,9 @@ def main():
                         "hbm_frac_of_8TBs": verify_step_bytes / ((verify_ms + accept_ms) * 1e-3) / 1e9 / 8000.0},
         "acceptance": {"mean_accepted_per_verify": cnt.n_accepted_tokens / max(1, cnt.n_verify_passes * wl.batch),
                        "tokens_per_step": committed / args.steps / world, "resampled": int(cnt.n_resampled),
-                       "near_boundary": int(cnt.n_near_boundary)},
+                       "near_boundary": int(cnt.n_near_boundary),
+                       "accepted_len_hist": [int(x) for x in list(cnt.accepted_len_hist)[:B + 1]]},
+        "shaped": shaped,
         "setup_s": setup_s, "prefill_ms": c0.ms_prefill,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

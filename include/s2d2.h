@@ -213,6 +213,15 @@ int s2d2_release_seq(s2d2_ctx* ctx, int32_t seq_id);
 int s2d2_get_counters(s2d2_ctx* ctx, s2d2_counters* out);
 int s2d2_reset_counters(s2d2_ctx* ctx);
 
+/* Throughput studies on models whose acceptance profile is not the one of interest (random
+ * weights accept far fewer tokens than the trained models of the paper's Table "Per-token
+ * draft-confidence versus verifier-ratio analysis", whose quadrants average to 0.77 per verified
+ * token).  prob in (0, 1]: the accept test of every scanned position becomes u_i < prob, whatever
+ * the two distributions say; a rejected position is still resampled from the residual.  The
+ * output no longer follows the verifier's law, so such a run measures speed only.  prob = 0
+ * restores the rule of Algorithm "SampleBlock for S2D2".  S2D2_ERR_INVALID outside [0, 1]. */
+int s2d2_set_accept_override(s2d2_ctx* ctx, float prob);
+
 /* Kernel-level timing for roofline reports.  on >= 1: the dominant launches of the forward
  * pass (the persistent pass kernel; on the one-kernel-per-operation path every GEMM) are
  * bracketed by a CUDA event pair on the context's stream.  on >= 2: the persistent kernel also

@@ -77,7 +77,7 @@ EXPORTS = [
     "s2d2_create", "s2d2_destroy", "s2d2_last_error", "s2d2_load_weights", "s2d2_prefill",
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
-    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
+    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_set_accept_override", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
     "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace", "s2d2_debug_wait_timeout",
     "s2d2_gemm_bf16_noalloc", "s2d2_noalloc_last_error",
 ]
@@ -122,6 +122,7 @@ def load_library() -> C.CDLL:
     lib.s2d2_get_counters.argtypes = [C.c_void_p, C.POINTER(Counters)]
     lib.s2d2_reset_counters.argtypes = [C.c_void_p]
     lib.s2d2_set_profiling.argtypes = [C.c_void_p, C.c_int32]
+    lib.s2d2_set_accept_override.argtypes = [C.c_void_p, C.c_float]
     lib.s2d2_get_gemm_profile.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.s2d2_accept_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
                                        C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_uint32),
@@ -285,6 +286,10 @@ class Engine:
 
     def reset_counters(self):
         self._check(self.lib.s2d2_reset_counters(self._h))
+
+    def set_accept_override(self, prob: float):
+        """prob in (0, 1]: accept test u < prob for every scanned position (speed studies only); 0: the paper's rule."""
+        self._check(self.lib.s2d2_set_accept_override(self._h, float(prob)))
 
     def set_profiling(self, on):
         """0: off; 1: event pairs around the dominant kernels; 2: also the persistent kernel's phase marks."""

@@ -126,6 +126,7 @@ struct s2d2_ctx {
     bool verify_timing_pending = false;
     // per-GEMM profiling (off by default)
     bool profiling = false;
+    float accept_override = 0.f;            // > 0: every accept test is u < accept_override (throughput studies)
     bool tracing = false;                   // in-kernel phase marks of the persistent pass
     std::vector<cudaEvent_t> prof_events;   // pairs
     size_t prof_used = 0;

@@ -339,26 +339,33 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* 
         max_cnt = max(max_cnt, cnt[s]);
         out[s] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // Relaxed polls of all counters at once (acquire loads would complete one after the other).
+    // The partials are then read by L2 loads whose addresses depend on the polled values: such a
+    // load is issued after the counts it depends on have arrived, and the writers made their
+    // partials visible in L2 before they counted, so no fence is needed between the two.
+    unsigned dep = 0;
     {
         bool ready = false;
-        // relaxed polls of all counters at once (acquire loads would complete one after the other),
-        // then one fence orders the data loads after what the counters published
+        unsigned low = 0xffffffffu;
         for (uint32_t it = 0; it < SPIN_LIMIT && !ready; ++it) {
             unsigned seen[NS];
 #pragma unroll
             for (int s = 0; s < NS; ++s) seen[s] = cnt[s] > 0 && published[s] ? ld_relaxed(published[s]) : 0xffffffffu;
             ready = true;
+            low = 0xffffffffu;
 #pragma unroll
-            for (int s = 0; s < NS; ++s)
+            for (int s = 0; s < NS; ++s) {
                 if (cnt[s] > 0 && seen[s] < (unsigned)cnt[s] * round) ready = false;
+                low = min(low, seen[s] + 0x7fffffffu);        // wraps for the "no counter" value; never 0 for a real count
+            }
             if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
         }
-        asm volatile("fence.acq_rel.gpu;" ::: "memory");
         if (!ready) {
             atomicCAS(p.status, 0, 8);
             *abort_flag = 1;
             return false;
         }
+        dep = low == 0u ? 1u : 0u;     // always 0, but only known once every poll has returned
     }
     for (int j0 = 0; j0 < max_cnt; j0 += PC) {
         float4 v[NS][PC];
@@ -369,7 +376,7 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* 
                 const int slot = __shfl_sync(0xffffffffu, tab_lane[s], (j0 + j + 1) & 31);
                 v[s][j] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (j0 + j < cnt[s])
-                    v[s][j] = __ldcg(reinterpret_cast<const float4*>(ws + ((size_t)slot * p.T + row[s]) * tc::BLOCK_N) + lane);
+                    v[s][j] = __ldcg(reinterpret_cast<const float4*>(ws + ((size_t)slot * p.T + row[s]) * tc::BLOCK_N) + lane + dep);
             }
 #pragma unroll
         for (int s = 0; s < NS; ++s)

@@ -875,6 +875,7 @@ int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, c
     in.tau_conf = c->dc.tau_conf;
     in.seed = c->dc.seed;
     in.gamma = c->dc.ratio_gamma;
+    in.accept_override = c->accept_override;
     in.resample = c->dc.resample;
     in.l_cap = S2D2_MAX_BLOCK;
     AcceptOut out;
@@ -1122,6 +1123,12 @@ extern "C" int s2d2_get_counters(s2d2_ctx* c, s2d2_counters* out) {
 extern "C" int s2d2_reset_counters(s2d2_ctx* c) {
     if (!c) return S2D2_ERR_INVALID;
     memset(&c->cnt, 0, sizeof(c->cnt));
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_set_accept_override(s2d2_ctx* c, float prob) {
+    if (!c || !(prob >= 0.f && prob <= 1.f)) return S2D2_ERR_INVALID;
+    c->accept_override = prob;
     return S2D2_OK;
 }
 

@@ -232,6 +232,7 @@ struct AcceptIn {
     float tau_conf;
     unsigned seed;
     float gamma;
+    float accept_override;        // > 0: a_i is this constant instead of min(1, (v_i/d_i)^gamma)
     int resample;
     int l_cap;                    // stride of the per-position outputs
 };
@@ -302,7 +303,7 @@ static __global__ void __launch_bounds__(128) accept_scan_kernel(AcceptIn in, Ac
         double ratio = v / d;
         if (in.gamma != 1.f) ratio = pow(ratio, (double)in.gamma);
         sh_v[i] = v;
-        sh_a[i] = fmin(1.0, ratio);
+        sh_a[i] = in.accept_override > 0.f ? (double)in.accept_override : fmin(1.0, ratio);
         sh_u[i] = philox_uniform(in.seed, (unsigned)(in.seq_pos0[s] + i), in.seq_stream[s], (unsigned)in.seq_step[s], STREAM_ACCEPT);
     }
     __syncthreads();

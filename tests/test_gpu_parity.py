@@ -207,3 +207,42 @@ def test_bounded_wait_times_out_with_a_status_not_a_hang():
     e.generate(ids, wl.block_size)                # still usable
     assert all(len(e.get_tokens(s)) > 0 for s in ids)
     e.close()
+
+
+def test_accept_override_replaces_only_the_accept_probability():
+    """The speed-study switch: with u < 1 every drafted token of the span is accepted, with a
+    probability below the smallest uniform none is and position 0 is resampled from the residual,
+    and switching it off restores the rule (same results as an engine that never had it on)."""
+    from paper_2603_25702_b200 import S2D2Error
+    wl = get_config("t_bf16")
+    W = generate_weights(wl.model, seed=1)
+
+    def one_step(e, ids):
+        st = e.draft_block(ids)
+        fl = [1] * len(ids)
+        e.verify_block(ids, fl)
+        return st, e.accept_and_commit(ids, fl)
+
+    e, ids, _ = _start(wl, W)
+    with pytest.raises(S2D2Error):
+        e.set_accept_override(1.5)
+    e.set_accept_override(1.0)
+    st, res = one_step(e, ids)
+    for s, r in zip(st, res):
+        assert r.n_accepted == s.span_len and r.first_reject == -1 and r.resampled_id == -1
+        assert all(a == 1.0 for a in r.a[:s.span_len])
+    e.set_accept_override(1e-9)                    # uniforms are at least 2^-25
+    st, res = one_step(e, ids)
+    for s, r in zip(st, res):
+        assert r.n_accepted == 0 and r.first_reject == 0 and r.resampled_id >= 0 and r.resampled_id != s.xhat[0]
+    e.close()
+
+    a, ids_a, _ = _start(wl, W)
+    b, ids_b, _ = _start(wl, W)
+    b.set_accept_override(0.5)
+    b.set_accept_override(0.0)
+    for _ in range(3):
+        ra, rb = one_step(a, ids_a)[1], one_step(b, ids_b)[1]
+        assert [(r.n_accepted, r.first_reject, r.resampled_id) for r in ra] == [(r.n_accepted, r.first_reject, r.resampled_id) for r in rb]
+    a.close()
+    b.close()
