@@ -76,11 +76,13 @@ int attention_init(s2d2_ctx* c) {
     a->cap_items = std::max<size_t>(2048, base_items * 2);
     if (cudaMalloc((void**)&a->part_o, a->cap_items * att::QT * m.head_dim * 4) != cudaSuccess) return S2D2_ERR_CUDA;
     if (cudaMalloc((void**)&a->part_ml, a->cap_items * att::QT * 2 * 4) != cudaSuccess) return S2D2_ERR_CUDA;
-    cudaError_t e = m.head_dim == 128
-                        ? cudaFuncSetAttribute(att::attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)att::attn_smem_bytes(128))
-                        : cudaFuncSetAttribute(att::attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)att::attn_smem_bytes(64));
+    const int smem = (int)att::attn_smem_bytes(m.head_dim);
+    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = m.head_dim == 128 ? cudaFuncSetAttribute(att::attn_tc_kernel<128, true>, attr, smem)
+                                      : cudaFuncSetAttribute(att::attn_tc_kernel<64, true>, attr, smem);
+    if (e == cudaSuccess)
+        e = m.head_dim == 128 ? cudaFuncSetAttribute(att::attn_tc_kernel<128, false>, attr, smem)
+                              : cudaFuncSetAttribute(att::attn_tc_kernel<64, false>, attr, smem);
     if (e != cudaSuccess) return S2D2_ERR_CUDA;
     a->tc_ok = true;
     return S2D2_OK;
@@ -104,10 +106,11 @@ bool attention_plan(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, 
     if (!a || !a->tc_ok) return false;
     att::AttnParams p;
     p.q = (const bf16*)c->q;
-    p.q_lo = nullptr;
+    p.q_lo = (const bf16*)c->q_lo;
     p.k_rows = (const bf16*)c->k_rows;
     p.v_rows = (const bf16*)c->v_rows;
     p.out = (bf16*)c->attn;
+    p.out_lo = (bf16*)c->attn_lo;
     p.part_o = a->part_o;
     p.part_ml = a->part_ml;
     p.pv = pv;
@@ -149,11 +152,15 @@ int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_r
     }
     p.layer = layer;
     dim3 grid(p.n_cache_splits + 1, p.n_qtiles, pv.n_seqs * m.n_kv_heads);
+    const size_t smem = att::attn_smem_bytes(m.head_dim);
+    // two-term queries and probabilities whenever the low halves of q exist (always on this path)
     if (m.head_dim == 128) {
-        att::attn_tc_kernel<128><<<grid, att::THREADS, att::attn_smem_bytes(128), c->stream>>>(a->map_kv, p);
+        if (p.q_lo) att::attn_tc_kernel<128, true><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
+        else att::attn_tc_kernel<128, false><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
         att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);
     } else {
-        att::attn_tc_kernel<64><<<grid, att::THREADS, att::attn_smem_bytes(64), c->stream>>>(a->map_kv, p);
+        if (p.q_lo) att::attn_tc_kernel<64, true><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
+        else att::attn_tc_kernel<64, false><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
         att::attn_combine_kernel<64><<<dim3(pv.n_rows, m.n_q_heads), 64, 0, c->stream>>>(p);
     }
     c->cnt.n_kernel_launches += 2;

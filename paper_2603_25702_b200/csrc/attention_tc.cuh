@@ -28,6 +28,7 @@ constexpr int STAGES = 2;
 struct AttnParams {
     const bf16* q;              // [M, Hq, HD]
     const bf16* q_lo;           // low halves of q (q = hi + lo, both bf16) for the two-term variant, else unused
+    bf16* out_lo;               // low halves of the combined output (attn_combine_kernel; may be null)
     const bf16* k_rows;         // [M, Hkv, HD] K of this pass's rows
     const bf16* v_rows;
     bf16* out;                  // [M, Hq*HD]
@@ -370,7 +371,7 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
     return true;
 }
 
-template <int HD>
+template <int HD, bool HL>
 __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -381,7 +382,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
     }
     __syncthreads();
     uint32_t ring_pos = 0;
-    bool ok = attn_item<HD>(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, full, ring_pos, threadIdx.x, 0);
+    bool ok = attn_item<HD, HL>(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, full, ring_pos, threadIdx.x, 0);
     if (!ok && threadIdx.x == 0) {
         // copies already issued target this CTA's shared memory: give them one more bounded wait
         // before the CTA leaves
@@ -389,7 +390,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant_
     }
 }
 
-// Merges the partials of all splits of one query vector (fixed split order) and writes bf16.
+// Merges the partials of all splits of one query vector (fixed split order) and writes bf16 (two terms when out_lo is given).
 template <int HD>
 __global__ void attn_combine_kernel(AttnParams p) {
     int r = blockIdx.x, hq = blockIdx.y;
@@ -417,7 +418,10 @@ __global__ void attn_combine_kernel(AttnParams p) {
             l += w * p.part_ml[(item0 + s) * QT * 2 + qi * 2 + 1];
             acc += w * p.part_o[((item0 + s) * QT + qi) * HD + c];
         }
-        p.out[((size_t)r * p.Hq + hq) * HD + c] = __float2bfloat16_rn(acc / l);
+        const float o = acc / l;
+        const bf16 hi = __float2bfloat16_rn(o);
+        p.out[((size_t)r * p.Hq + hq) * HD + c] = hi;
+        if (p.out_lo) p.out_lo[((size_t)r * p.Hq + hq) * HD + c] = __float2bfloat16_rn(o - __bfloat162float(hi));
     }
 }
 

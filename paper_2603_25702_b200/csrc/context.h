@@ -92,6 +92,8 @@ struct s2d2_ctx {
     int max_rows = 0, max_logit_rows = 0;
     float *h = nullptr, *qkv = nullptr, *gu = nullptr, *tmp = nullptr;
     void *xn = nullptr, *q = nullptr, *k_rows = nullptr, *v_rows = nullptr, *attn = nullptr, *act = nullptr;
+    // low halves of the two-term activations (bf16 models): x = hi + lo
+    void *xn_lo = nullptr, *q_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr;
     float *logits_draft = nullptr, *logits_verify = nullptr;
     float *rope_cos = nullptr, *rope_sin = nullptr;
     // MoE scratch

@@ -67,7 +67,7 @@ void gemm_simt(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N
 }
 
 int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
-            int accumulate) {
+            int accumulate, const void* X_lo) {
     GemmState* g = state(c);
     tc::GemmParams p;
     p.Y = Y;
@@ -79,14 +79,17 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
     p.accumulate = accumulate;
     p.kb_total = K / tc::BLOCK_K;
     p.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
-    p.m_tiles = (M + 255) / 256;
+    p.hilo = X_lo != nullptr;
+    const int t_max = p.hilo ? 128 : 256;       // the MMA takes up to 256 token rows, the low halves count
+    p.m_tiles = (M + t_max - 1) / t_max;
     int per = (M + p.m_tiles - 1) / p.m_tiles;
-    p.T = std::min(256, (per + 15) / 16 * 16);
+    p.T = std::min(t_max, (per + 15) / 16 * 16);
     p.m_tiles = (M + p.T - 1) / p.T;
+    const int TN = p.hilo ? 2 * p.T : p.T;
     // two CTAs per SM while the token tile is small, one otherwise
-    bool two = p.T <= 64;
+    bool two = TN <= 64;
     size_t budget = two ? 100 * 1024 : 200 * 1024;
-    p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(p.T));
+    p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(TN));
     p.stages = std::max(2, std::min(p.stages, p.kb_total));
     // K splits: fill the resident CTA slots; cost model in K-blocks per CTA plus a fixed set-up cost
     int slots = g->n_sms * (two ? 2 : 1);
@@ -99,7 +102,7 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
         int waves = (tiles * s + slots - 1) / slots;
         // per CTA: its k-blocks, a fixed set-up cost, and an epilogue that grows with the token tile (a split adds
         // the partial tile's round trip through the workspace); all in units of one k-block of a 16-row tile
-        const double kb_cost = 1.0 + p.T / 64.0, epi = p.T / 16.0;
+        const double kb_cost = 1.0 + TN / 64.0, epi = p.T / 16.0;
         double cost = waves * ((double)(p.kb_total + s - 1) / s * kb_cost + 6.0 + epi * (s > 1 ? 3.0 : 1.0)) + (s > 1 ? 2.0 : 0.0);
         if (cost < best_cost - 1e-9) {
             best_cost = cost;
@@ -113,10 +116,11 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
     p.evict_first = (M <= 64);
     const CUtensorMap* mw = get_map(c, W, N, K, tc::BLOCK_N);
     const CUtensorMap* mx = get_map(c, X, M, K, p.T);
-    if (!mw || !mx) return S2D2_ERR_CUDA;
-    size_t smem = tc::smem_bytes(p.T, p.stages);
+    const CUtensorMap* mx_lo = p.hilo ? get_map(c, X_lo, M, K, p.T) : mx;
+    if (!mw || !mx || !mx_lo) return S2D2_ERR_CUDA;
+    size_t smem = tc::smem_bytes(TN, p.stages);
     int grid = tiles * p.splits;
-    tc::gemm_tc_kernel<<<grid, tc::THREADS, smem, c->stream>>>(*mw, *mx, p);
+    tc::gemm_tc_kernel<<<grid, tc::THREADS, smem, c->stream>>>(*mw, *mx, *mx_lo, p);
     c->cnt.n_kernel_launches++;
     return S2D2_OK;
 }
@@ -216,20 +220,22 @@ int gemm_prof_collect(s2d2_ctx* c) {
     return S2D2_OK;
 }
 
-int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate) {
+int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate,
+         const void* X_lo) {
     size_t es = c->m.dtype == S2D2_DTYPE_F32 ? 4 : 2;
     gemm_prof_begin(c);
     struct End {
         s2d2_ctx* c;
         double b;
         ~End() { gemm_prof_end(c, b); }
-    } end{c, (double)N * K * es + (double)M * K * es + (double)M * N * 4 * (accumulate ? 2 : 1)};
+    } end{c, (double)N * K * es + (double)M * K * es * (X_lo ? 2 : 1) + (double)M * N * 4 * (accumulate ? 2 : 1)};
     if (c->m.dtype == S2D2_DTYPE_F32) {
         gemm_simt<float, float>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
         return S2D2_OK;
     }
-    if (state(c)->tc_ok && K % tc::BLOCK_K == 0) return gemm_tc(c, X, W, Y, M, N, K, ldy, scale, accumulate);
+    if (state(c)->tc_ok && K % tc::BLOCK_K == 0) return gemm_tc(c, X, W, Y, M, N, K, ldy, scale, accumulate, X_lo);
     gemm_simt<bf16, bf16>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
+    if (X_lo) gemm_simt<bf16, bf16>(c, X_lo, W, Y, M, N, K, ldy, scale, 1);
     return S2D2_OK;
 }
 
@@ -352,6 +358,7 @@ extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d
     p.tickets = nd.tickets;
     p.status = nd.status;
     p.evict_first = 0;
+    p.hilo = 0;
     CUtensorMap mw, mx;
     if (noalloc_map(&mw, d_w, N, K, tc::BLOCK_N) || noalloc_map(&mx, d_x, M, K, p.T))
         return noalloc_fail(S2D2_ERR_CUDA, "cuTensorMapEncodeTiled failed");
@@ -360,7 +367,7 @@ extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d
         return noalloc_fail(S2D2_ERR_CUDA, "cudaMemsetAsync", e);
     if ((e = cudaMemsetAsync(nd.status, 0, sizeof(int), st)) != cudaSuccess)
         return noalloc_fail(S2D2_ERR_CUDA, "cudaMemsetAsync", e);
-    tc::gemm_tc_kernel<<<p.n_tiles * p.splits, tc::THREADS, tc::smem_bytes(p.T, p.stages), st>>>(mw, mx, p);
+    tc::gemm_tc_kernel<<<p.n_tiles * p.splits, tc::THREADS, tc::smem_bytes(p.T, p.stages), st>>>(mw, mx, mx, p);
     if ((e = cudaGetLastError()) != cudaSuccess) return noalloc_fail(S2D2_ERR_CUDA, "kernel launch", e);
     int status = 0;
     if ((e = cudaMemcpyAsync(&status, nd.status, sizeof(int), cudaMemcpyDeviceToHost, st)) != cudaSuccess)

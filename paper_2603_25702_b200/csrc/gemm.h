@@ -1,10 +1,12 @@
 // Y[M, N] (+)= scale * X[M, K] * W[N, K]^T for the model's storage type.
 // X is fp32 (fp32 model) or bf16 (bf16 model); W is the stored matrix; Y is fp32.
+// X_lo (bf16 models, may be null): the low halves of a two-term input, X = X + X_lo.
 #pragma once
 struct s2d2_ctx;
 int gemm_init(s2d2_ctx* c);
 void gemm_destroy(s2d2_ctx* c);
-int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate);
+int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate,
+         const void* X_lo = nullptr);
 // Profiling helpers: bracket a launch with an event pair while profiling is on.
 void gemm_prof_begin(s2d2_ctx* c);
 void gemm_prof_end(s2d2_ctx* c, double algorithmic_bytes);

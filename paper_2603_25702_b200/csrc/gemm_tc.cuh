@@ -8,7 +8,9 @@
 // GEMM: a tile of 128 weight rows is the MMA "M" operand (A, K-major, staged by
 // TMA with the 128-byte swizzle), the token rows are the MMA "N" operand
 // (B, K-major, T = 16..256 rows), and the fp32 accumulator D[128 x T] lives in
-// tensor memory.  One CTA owns one (weight tile, token tile, K split):
+// tensor memory.  With two-term inputs (x = hi + lo, both bf16: 16 significant bits, which a
+// network of 30 and more layers needs to keep its logits within 2e-2) the low halves are T more
+// token rows of the same MMA and the epilogue adds the two accumulator halves.  One CTA owns one (weight tile, token tile, K split):
 //   warp 0 / lane 0   TMA producer: W and X K-blocks of 64 into a ring of stages
 //   warp 1 / lane 0   tcgen05.mma issuer, 4 MMAs (K = 16 each) per stage;
 //                     tcgen05.commit frees the stage and finally signals the epilogue
@@ -48,6 +50,7 @@ struct GemmParams {
     unsigned* tickets;   // one counter per (n_tile, m_tile), zero between launches
     int* status;         // device status word (0 = ok)
     int evict_first;     // stream W with an evict-first L2 policy
+    int hilo;            // X arrives as two bf16 terms (X = X_hi + X_lo): both are token rows of one MMA (N = 2T, T <= 128)
 };
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
@@ -67,16 +70,18 @@ __host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int T) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T >> 3) << 17) | ((uint32_t)(BLOCK_N >> 4) << 24);
 }
 
-__host__ __device__ __forceinline__ size_t stage_bytes(int T) { return (size_t)BLOCK_N * 128 + (size_t)T * 128; }
-__host__ __device__ __forceinline__ size_t smem_bytes(int T, int stages) { return stages * stage_bytes(T) + 1024 + 256; }
+// TN: token rows of one stage (T, or 2T with two-term inputs)
+__host__ __device__ __forceinline__ size_t stage_bytes(int TN) { return (size_t)BLOCK_N * 128 + (size_t)TN * 128; }
+__host__ __device__ __forceinline__ size_t smem_bytes(int TN, int stages) { return stages * stage_bytes(TN) + 1024 + 256; }
 
 static __global__ void __launch_bounds__(THREADS)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+               const __grid_constant__ CUtensorMap map_x_lo, GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     // tiles need 1024-byte alignment for the 128-byte swizzle
     uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int S = p.stages, T = p.T;
-    const size_t sbytes = stage_bytes(T);
+    const int S = p.stages, T = p.T, TN = p.hilo ? 2 * p.T : p.T;
+    const size_t sbytes = stage_bytes(TN);
     uint64_t* full = (uint64_t*)(tiles + S * sbytes);
     uint64_t* empty = full + S;
     uint64_t* acc_ready = empty + S;
@@ -98,7 +103,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int kb1 = (int)((long long)p.kb_total * (split + 1) / p.splits);
     const int n0 = n_tile * BLOCK_N, m0 = m_tile * T;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < T) tmem_cols <<= 1;
+    while ((int)tmem_cols < TN) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -113,6 +118,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        if (p.hilo) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x_lo) : "memory");
     }
     if (warp == 0) {
         tmem_alloc(tmem_slot, tmem_cols);
@@ -140,11 +146,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (p.evict_first) tma_load_2d_hint(a, &map_w, kb * BLOCK_K, n0, &full[s], policy);
             else tma_load_2d(a, &map_w, kb * BLOCK_K, n0, &full[s]);
             tma_load_2d(b, &map_x, kb * BLOCK_K, m0, &full[s]);
+            if (p.hilo) tma_load_2d(b + (size_t)T * 128, &map_x_lo, kb * BLOCK_K, m0, &full[s]);
             *issued = i + 1;
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer ----------------
-        const uint32_t idesc = instr_desc_bf16(T);
+        const uint32_t idesc = instr_desc_bf16(TN);
         int i = 0;
         for (int kb = kb0; kb < kb1; ++kb, ++i) {
             int s = i % S;
@@ -191,6 +198,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int c = 0; c < T; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);      // executed by the whole warp even past m_hi (aligned instruction)
+                if (p.hilo) {
+                    float w[16];
+                    tmem_ld16(taddr + T + c, w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                }
                 if (n < p.N) {
                     float old[16];
 #pragma unroll
@@ -207,6 +220,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int c = 0; c < T; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);
+                if (p.hilo) {
+                    float w[16];
+                    tmem_ld16(taddr + T + c, w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     if (c + j < m_hi) mine[(size_t)(c + j) * BLOCK_N + n_local] = v[j];

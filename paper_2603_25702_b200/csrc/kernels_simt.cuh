@@ -32,10 +32,18 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
     return sh[0];
 }
 
-// out[i, :] = rmsnorm(h[rows ? rows[i] : i, :]) * gain, written as TO.
+// Stores v as hi = T(v) and, when a second buffer is given, lo = T(v - hi): the GEMMs and the
+// attention of bf16 models take such two-term inputs (16 significant bits instead of 8).
+template <typename T>
+__device__ __forceinline__ void store_two_term(T* hi, T* lo, size_t i, float v) {
+    const T h = from_f32<T>(v);
+    hi[i] = h;
+    if (lo) lo[i] = from_f32<T>(v - to_f32(h));
+}
+// out[i, :] = rmsnorm(h[rows ? rows[i] : i, :]) * gain, written as TO (out_lo: low halves, may be null).
 template <typename TO>
 __global__ void rmsnorm_kernel(const float* __restrict__ h, const int* __restrict__ rows, const float* __restrict__ gain,
-                               TO* __restrict__ out, int d, float eps) {
+                               TO* __restrict__ out, TO* __restrict__ out_lo, int d, float eps) {
     __shared__ float sh[32];
     int i = blockIdx.x;
     const float* x = h + (size_t)(rows ? rows[i] : i) * d;
@@ -46,7 +54,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ h, const int* __restric
     // rsqrtf is approximate (2 ulp); refine once so the fp32 model stays within 1e-4 relative
     float m = ss / (float)d + eps;
     inv = inv * (1.5f - 0.5f * m * inv * inv);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) out[(size_t)i * d + c] = from_f32<TO>(x[c] * inv * gain[c]);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) store_two_term(out, out_lo, (size_t)i * d + c, x[c] * inv * gain[c]);
 }
 
 // Y[m, n] (+)= scale * sum_k X[m, k] * W[n, k].  One warp per output column and
@@ -85,7 +93,7 @@ __global__ void gemm_simt_kernel(const TX* __restrict__ X, const TW* __restrict_
 template <typename TA, typename TKV>
 __global__ void qk_rope_kv_kernel(const float* __restrict__ qkv, PassView pv, const float* __restrict__ q_gain,
                                   const float* __restrict__ k_gain, const float* __restrict__ rope_cos,
-                                  const float* __restrict__ rope_sin, TA* __restrict__ q_out, TKV* __restrict__ k_rows,
+                                  const float* __restrict__ rope_sin, TA* __restrict__ q_out, TA* __restrict__ q_lo, TKV* __restrict__ k_rows,
                                   TKV* __restrict__ v_rows, KvPool<TKV> pool, int layer, int Hq, int Hkv, int hd,
                                   float eps, int qk_norm) {
     __shared__ float sh[32];
@@ -112,9 +120,9 @@ __global__ void qk_rope_kv_kernel(const float* __restrict__ qkv, PassView pv, co
         x2 = y2;
     }
     if (is_q) {
-        TA* dst = q_out + ((size_t)r * Hq + head) * hd;
-        dst[i] = from_f32<TA>(x1);
-        dst[i + half] = from_f32<TA>(x2);
+        const size_t o = ((size_t)r * Hq + head) * hd;
+        store_two_term(q_out, q_lo, o + i, x1);
+        store_two_term(q_out, q_lo, o + i + half, x2);
         return;
     }
     int kvh = is_k ? head - Hq : head - Hq - Hkv;
@@ -190,12 +198,12 @@ __global__ void attention_simt_kernel(const TA* __restrict__ q, const TKV* __res
 
 // act[m, i] = silu(gu[m, i]) * gu[m, f + i]
 template <typename TA>
-__global__ void swiglu_kernel(const float* __restrict__ gu, TA* __restrict__ act, int M, int f) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, TA* __restrict__ act, TA* __restrict__ act_lo, int M, int f) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)M * f) return;
     size_t m = idx / f, i = idx % f;
     float g = gu[m * 2 * f + i], u = gu[m * 2 * f + f + i];
-    act[idx] = from_f32<TA>(g / (1.f + expf(-g)) * u);
+    store_two_term(act, act_lo, idx, g / (1.f + expf(-g)) * u);
 }
 
 // ---- mixture of experts, plain form -------------------------------------------------------------

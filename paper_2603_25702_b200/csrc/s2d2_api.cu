@@ -229,6 +229,12 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
     if ((rc = dmalloc(c, (char**)&c->v_rows, M * m->n_kv_heads * m->head_dim * es))) return rc;
     if ((rc = dmalloc(c, (char**)&c->attn, M * nq * es))) return rc;
     if ((rc = dmalloc(c, (char**)&c->act, M * f * es))) return rc;
+    if (m->dtype == S2D2_DTYPE_BF16 && dc->use_tensor_cores) {
+        if ((rc = dmalloc(c, (char**)&c->xn_lo, M * d * es))) return rc;
+        if ((rc = dmalloc(c, (char**)&c->q_lo, M * nq * es))) return rc;
+        if ((rc = dmalloc(c, (char**)&c->attn_lo, M * nq * es))) return rc;
+        if ((rc = dmalloc(c, (char**)&c->act_lo, M * f * es))) return rc;
+    }
     if ((rc = dmalloc(c, &c->logits_draft, (size_t)c->max_logit_rows * m->vocab))) return rc;
     if ((rc = dmalloc(c, &c->logits_verify, (size_t)c->max_logit_rows * m->vocab))) return rc;
     if (m->n_experts > 0) {
@@ -323,7 +329,7 @@ extern "C" int s2d2_destroy(s2d2_ctx* c) {
     pass_destroy(c);
     attention_destroy(c);
     gemm_destroy(c);
-    void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act,
+    void* ptrs[] = {c->w_arena, c->kv_base, c->h, c->qkv, c->gu, c->xn, c->q, c->k_rows, c->v_rows, c->attn, c->act, c->xn_lo, c->q_lo, c->attn_lo, c->act_lo,
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
                     c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
                     c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status, c->chunk_d, c->chunk_v, c->rej_info,
@@ -484,21 +490,21 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
     KvPool<TKV> pool = make_pool<TKV>(c);
     for (int l = 0; l < m.n_layers; ++l) {
         const LayerWeights& L = c->layers[l];
-        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.attn_norm, (TA*)c->xn, d, m.rms_eps);
+        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.attn_norm, (TA*)c->xn, (TA*)c->xn_lo, d, m.rms_eps);
         LAUNCHED(c);
-        int rc = gemm(c, c->xn, L.wqkv, c->qkv, M, nqkv, d, nqkv, 1.f, 0);
+        int rc = gemm(c, c->xn, L.wqkv, c->qkv, M, nqkv, d, nqkv, 1.f, 0, c->xn_lo);
         if (rc) return rc;
         qk_rope_kv_kernel<TA, TKV><<<dim3(M, m.n_q_heads + 2 * m.n_kv_heads), hd / 2, 0, st>>>(
-            c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
+            c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TA*)c->q_lo, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
             l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
         LAUNCHED(c);
         if ((rc = attention(c, pv, l, pb.max_ctx, pb.max_rows))) return rc;
-        if ((rc = gemm(c, c->attn, L.wo, c->h, M, d, nq, d, 1.f, 1))) return rc;
-        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.ffn_norm, (TA*)c->xn, d, m.rms_eps);
+        if ((rc = gemm(c, c->attn, L.wo, c->h, M, d, nq, d, 1.f, 1, c->attn_lo))) return rc;
+        rmsnorm_kernel<TA><<<M, 256, 0, st>>>(c->h, nullptr, L.ffn_norm, (TA*)c->xn, (TA*)c->xn_lo, d, m.rms_eps);
         LAUNCHED(c);
         if (m.n_experts > 0) {
             int E = m.n_experts, k = m.top_k, fe = m.expert_ffn, P = M * k;
-            if ((rc = gemm(c, c->xn, L.router, c->router_logits, M, E, d, E, 1.f, 0))) return rc;
+            if ((rc = gemm(c, c->xn, L.router, c->router_logits, M, E, d, E, 1.f, 0, c->xn_lo))) return rc;
             moe_topk_kernel<<<M, 32, 0, st>>>(c->router_logits, M, E, k, c->moe_ids, c->moe_gates);
             LAUNCHED(c);
             CUDA_TRY(c, cudaMemcpyAsync(c->moe_ids_trace + (size_t)l * c->max_rows * k, c->moe_ids, (size_t)P * 4,
@@ -506,7 +512,7 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
             moe_gateup_kernel<TW, TA><<<dim3((2 * fe + 3) / 4, P), 128, 0, st>>>(
                 (const TA*)c->xn, (const TW*)L.e_gate, (const TW*)L.e_up, c->moe_ids, c->moe_gu, k, fe, d);
             LAUNCHED(c);
-            swiglu_kernel<TA><<<(unsigned)(((size_t)P * fe + 255) / 256), 256, 0, st>>>(c->moe_gu, (TA*)c->moe_act, P, fe);
+            swiglu_kernel<TA><<<(unsigned)(((size_t)P * fe + 255) / 256), 256, 0, st>>>(c->moe_gu, (TA*)c->moe_act, (TA*)nullptr, P, fe);
             LAUNCHED(c);
             moe_down_kernel<TW, TA><<<dim3((d + 3) / 4, P), 128, 0, st>>>((const TA*)c->moe_act, (const TW*)L.e_down,
                                                                          c->moe_ids, c->moe_out, fe, d);
@@ -517,24 +523,24 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
             c->cnt.moe_expert_tiles_touched += 0;   // filled by the grouped kernel when it is in use
             if (m.n_shared > 0) {
                 int fs = fe * m.n_shared;
-                if ((rc = gemm(c, c->xn, L.s_gu, c->gu, M, 2 * fs, d, 2 * fs, 1.f, 0))) return rc;
-                swiglu_kernel<TA><<<(unsigned)(((size_t)M * fs + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, M, fs);
+                if ((rc = gemm(c, c->xn, L.s_gu, c->gu, M, 2 * fs, d, 2 * fs, 1.f, 0, c->xn_lo))) return rc;
+                swiglu_kernel<TA><<<(unsigned)(((size_t)M * fs + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, (TA*)c->act_lo, M, fs);
                 LAUNCHED(c);
-                if ((rc = gemm(c, c->act, L.s_down, c->h, M, d, fs, d, 1.f, 1))) return rc;
+                if ((rc = gemm(c, c->act, L.s_down, c->h, M, d, fs, d, 1.f, 1, c->act_lo))) return rc;
             }
         } else {
             int f = m.ffn;
-            if ((rc = gemm(c, c->xn, L.wgu, c->gu, M, 2 * f, d, 2 * f, 1.f, 0))) return rc;
-            swiglu_kernel<TA><<<(unsigned)(((size_t)M * f + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, M, f);
+            if ((rc = gemm(c, c->xn, L.wgu, c->gu, M, 2 * f, d, 2 * f, 1.f, 0, c->xn_lo))) return rc;
+            swiglu_kernel<TA><<<(unsigned)(((size_t)M * f + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, (TA*)c->act_lo, M, f);
             LAUNCHED(c);
-            if ((rc = gemm(c, c->act, L.wdown, c->h, M, d, f, d, 1.f, 1))) return rc;
+            if ((rc = gemm(c, c->act, L.wdown, c->h, M, d, f, d, 1.f, 1, c->act_lo))) return rc;
         }
     }
     c->last_pass_rows = M;
     if (pb.n_logit > 0 && logits_out) {
-        rmsnorm_kernel<TA><<<pb.n_logit, 256, 0, st>>>(c->h, pv.logit_rows, c->final_norm, (TA*)c->xn, d, m.rms_eps);
+        rmsnorm_kernel<TA><<<pb.n_logit, 256, 0, st>>>(c->h, pv.logit_rows, c->final_norm, (TA*)c->xn, (TA*)c->xn_lo, d, m.rms_eps);
         LAUNCHED(c);
-        int rc = gemm(c, c->xn, c->lm_head, logits_out, pb.n_logit, m.vocab, d, m.vocab, m.logit_scale, 0);
+        int rc = gemm(c, c->xn, c->lm_head, logits_out, pb.n_logit, m.vocab, d, m.vocab, m.logit_scale, 0, c->xn_lo);
         if (rc) return rc;
     }
     CUDA_TRY(c, cudaGetLastError());

@@ -61,9 +61,11 @@ class OracleShadow:
 
 def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: int = 1, seed: Optional[int] = None,
               gamma: float = 1.0, tau_conf: float = 0.9, logit_atol: float = 2e-2, logit_rtol: float = 0.0,
-              route=None, shadows=None) -> ParityReport:
+              route=None, shadows=None, stage_b_seqs=None) -> ParityReport:
     """Run up to ``n_steps`` decode steps on all sequences (stops when every one has
-    generated wl.gen_tokens) and check both parity stages."""
+    generated wl.gen_tokens) and check both parity stages.  ``stage_b_seqs``: restrict the
+    oracle's forward (stage B) to these sequence ids (large batches at full model size); stage A
+    always covers every sequence."""
     cfg, B = wl.model, wl.block_size
     MASK = cfg.mask_id
     seed = wl.philox_seed if seed is None else seed
@@ -160,7 +162,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
             # ---- stage B: the oracle's own forward ------------------------------------------------
             n_c0 = bf["n_cached"]
             n_draft_rows = (s0 + j - n_c0) + (B - j)
-            if do_b:
+            if do_b and (stage_b_seqs is None or sid in stage_b_seqs):
                 sh = shadows[sid]
                 if not cfg.is_moe:
                     sh.extend(full, n_c0)

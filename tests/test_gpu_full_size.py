@@ -39,6 +39,32 @@ def test_full_shape_steps_match_oracle(name, n_steps, batch):
     e.close()
 
 
+@pytest.mark.parametrize("name,n_steps,batch,checked", [("c2", 2, 20, (0, 9, 19)), ("c4", 1, 9, (4,))])
+def test_full_shape_large_batch_matches_oracle(name, n_steps, batch, checked):
+    """More rows per pass than the persistent kernel takes (batch x block > 64): prefill, draft and
+    verifier passes run as one kernel per operation, the regime of the batch-32 workload.  Every
+    sequence goes through stage A; the oracle's forward (stage B, 2e-2) follows a few of them."""
+    from paper_2603_25702_b200 import Engine
+    from tests.parity_util import register_prompt_lens, run_steps
+    wl = get_config(name, prompt_len=(5, 9), gen_tokens=2 * get_config(name).block_size, batch=batch)
+    W = generate_weights(wl.model, seed=wl.weight_seed)
+    e = Engine(wl.model, block_size=wl.block_size, max_batch=batch, max_seq_len=256, kv_page_tokens=wl.kv_page_tokens,
+               seed=wl.philox_seed, stream=torch.cuda.current_stream().cuda_stream)
+    e.load_weights(W)
+    prompts = generate_prompts(wl)
+    ids = e.prefill(prompts)
+    register_prompt_lens(ids, prompts)
+    for k, sid in enumerate(ids):
+        e.seq_set_rng_stream(sid, k)
+    e.reset_counters()
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=n_steps, logit_atol=2e-2,
+                    stage_b_seqs={ids[k] for k in checked})
+    print(name, batch, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps == n_steps * batch and rep.stage_b_passes >= n_steps * len(checked)
+    assert e.get_counters().n_kernel_launches > 100 * n_steps     # one kernel per operation
+    e.close()
+
 
 def test_full_shape_moe_step_matches_oracle():
     """The MoE workload's shape (20 layers, 256 experts of width 512, top-8, vocabulary 157184) with a
