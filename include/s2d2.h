@@ -269,7 +269,9 @@ int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t
  * its last accumulator of the phase that ends at the barrier (.. + 3*b + 2; 0 for phases without
  * a GEMM), then the id of the SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
  * QKV GEMM + q/k-norm + RoPE + K/V write, attention, its combine, O GEMM + residual add,
- * gate/up GEMM + SwiGLU, down GEMM + residual add.  Marks are recorded only while
+ * gate/up GEMM + SwiGLU, down GEMM + residual add (nine per layer for mixture-of-experts models).  One
+ * more triple closes the row for the LM-head phase, which ends without a barrier: entry and exit both
+ * hold the time the CTA finished its logits.  Marks are recorded only while
  * s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */
 int s2d2_debug_pass_trace(s2d2_ctx* ctx, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks);
 

@@ -348,8 +348,8 @@ class Engine:
     def debug_pass_trace(self) -> np.ndarray:
         """(marks [n_ctas, n_barriers, 3], sm_ids [n_ctas]): global-timer ns at entry to / exit from every grid
         barrier of the last persistent pass and at the end of the phase's accumulator drain (0 if none), and
-        the SM each CTA ran on."""
-        buf = np.zeros(256 * (3 * (6 * self.model.n_layers + 1) + 1), dtype=np.uint64)
+        the SM each CTA ran on.  The last triple is the LM-head phase (entry = exit = the CTA's logits are written)."""
+        buf = np.zeros(256 * (3 * (9 * self.model.n_layers + 2) + 1), dtype=np.uint64)
         nc, nm = C.c_int32(), C.c_int32()
         self._check(self.lib.s2d2_debug_pass_trace(self._h, buf.ctypes.data, buf.size, C.byref(nc), C.byref(nm)))
         rows = buf[: nc.value * (nm.value + 1)].reshape(nc.value, nm.value + 1)

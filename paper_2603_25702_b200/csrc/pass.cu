@@ -234,7 +234,7 @@ int pass_init(s2d2_ctx* c) {
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
-    s->trace_cap = 3 * (s->barriers_per_layer * L + 1) + 1;      // three marks per grid barrier + the SM id
+    s->trace_cap = 3 * (s->barriers_per_layer * L + 2) + 1;      // three marks per grid barrier and for the LM-head phase + the SM id
     if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) return fail_alloc(c);
     if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
         cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
@@ -356,7 +356,7 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.S = stages_for(s, p.T, m.head_dim);
     p.trace = c->tracing ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    if (c->tracing) s->last_marks = 3 * (s->barriers_per_layer * m.n_layers + 1);
+    if (c->tracing) s->last_marks = 3 * (s->barriers_per_layer * m.n_layers + 2);
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
     for (int k = 0; k < 3; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];

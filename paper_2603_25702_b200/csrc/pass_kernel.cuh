@@ -1188,28 +1188,56 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             if (ok) {
                 const int n_tiles = (p.V + tc::BLOCK_N - 1) / tc::BLOCK_N;
                 const bool vec = (p.V & 3) == 0;
-                for (int pair = gw; pair < n_tiles * p.n_logit; pair += GW) {
-                    const int t = pair / p.n_logit, lr = pair % p.n_logit;
-                    const int m = p.pv.logit_rows[lr];
+                // one item = a 128-column tile and up to four logit rows: the tile's part list and
+                // counter are fetched once and the partials of all four rows are in flight together
+                constexpr int NR = 4;
+                const int groups = (p.n_logit + NR - 1) / NR;
+                for (int item = gw; item < n_tiles * groups; item += GW) {
+                    const int t = item / groups, lr0 = (item % groups) * NR;
                     const int tab = tile_row_tab(p, 4, t, lane);
-                    const SsqLane sq_l = row_ssq_lane(p.ssq_a, d_tiles, m, lane);
-                    const int tabs[1] = {tab}, rows[1] = {m};
-                    const unsigned* const pubs[1] = {p.tile_cnt[4] + t};
-                    float4 sums[1];
-                    tile_row_sums<1, 8>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs, 1u, lane, abort_flag, sums);
-                    const float4 s4 = sums[0];
-                    const float sc = p.logit_scale * inv_rms_from(sq_l, d, p.eps);
-                    const int col = t * tc::BLOCK_N + 4 * lane;
-                    float* dst = p.logits + (size_t)lr * p.V + col;
-                    if (vec && col + 3 < p.V) {
-                        *reinterpret_cast<float4*>(dst) = make_float4(sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w);
-                    } else {
-                        const float o[4] = {sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w};
+                    int tabs[NR], rows[NR];
+                    const unsigned* pubs[NR];
+                    SsqLane sq_l[NR];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (col + e < p.V) dst[e] = o[e];
+                    for (int q = 0; q < NR; ++q) {
+                        const bool on = lr0 + q < p.n_logit;
+                        rows[q] = on ? __ldg(p.pv.logit_rows + lr0 + q) : 0;
+                        tabs[q] = on ? tab : 0;
+                        pubs[q] = p.tile_cnt[4] + t;
+                        sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, rows[q], lane);
+                    }
+                    const unsigned* const pubs_c[NR] = {pubs[0], pubs[1], pubs[2], pubs[3]};
+                    float4 sums[NR];
+                    tile_row_sums<NR, 2>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs_c, 1u, lane, abort_flag, sums);
+                    const int col = t * tc::BLOCK_N + 4 * lane;
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) {
+                        const float sc = p.logit_scale * inv_rms_from(sq_l[q], d, p.eps);
+                        if (lr0 + q >= p.n_logit) continue;        // warp-uniform
+                        const float4 s4 = sums[q];
+                        float* dst = p.logits + (size_t)(lr0 + q) * p.V + col;
+                        if (vec && col + 3 < p.V) {
+                            *reinterpret_cast<float4*>(dst) = make_float4(sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w);
+                        } else {
+                            const float o[4] = {sc * s4.x, sc * s4.y, sc * s4.z, sc * s4.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (col + e < p.V) dst[e] = o[e];
+                        }
                     }
                 }
+            }
+        }
+        // the LM-head phase ends without a barrier: its marks are the time this CTA finished its
+        // logits (entry and exit) and the time it had drained its LM-head accumulators
+        if (p.trace && tid == 0) {
+            const int k = 3 * (int)epoch;
+            if (k + 2 < p.trace_cap - 1) {
+                unsigned long long t1;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+                p.trace[(size_t)cta * p.trace_cap + k] = t1;
+                p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
+                p.trace[(size_t)cta * p.trace_cap + k + 2] = t_drained;
             }
         }
     }
