@@ -111,6 +111,8 @@ bool attention_plan(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, 
     p.v_rows = (const bf16*)c->v_rows;
     p.out = (bf16*)c->attn;
     p.out_lo = (bf16*)c->attn_lo;
+    p.sched_off = nullptr;
+    p.sched_items = nullptr;
     p.part_o = a->part_o;
     p.part_ml = a->part_ml;
     p.pv = pv;

@@ -29,6 +29,8 @@ struct AttnParams {
     const bf16* q;              // [M, Hq, HD]
     const bf16* q_lo;           // low halves of q (q = hi + lo, both bf16) for the two-term variant, else unused
     bf16* out_lo;               // low halves of the combined output (attn_combine_kernel; may be null)
+    const int* sched_off;       // persistent kernel, several sequences: items of CTA c are sched_items[sched_off[c] .. sched_off[c+1])
+    const int* sched_items;     // item index = ((seq * Hkv + kv head) * n_qtiles + q tile) * (n_cache_splits + 1) + split; null: idx = cta, cta + G, ..
     const bf16* k_rows;         // [M, Hkv, HD] K of this pass's rows
     const bf16* v_rows;
     bf16* out;                  // [M, Hq*HD]

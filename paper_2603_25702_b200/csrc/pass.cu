@@ -8,6 +8,8 @@
 #include <string.h>
 
 #include <algorithm>
+#include <queue>
+#include <utility>
 #include <vector>
 
 #include "attention.h"
@@ -45,11 +47,90 @@ struct PassState {
     int* parts[pp::N_KINDS] = {};    // split-K part tables of the static GEMM kinds
     int* n_touched = nullptr;        // [n_layers] device, touched experts of the last pass
     int* n_touched_h = nullptr;      // pinned mirror
+    // attention schedule of passes with several sequences: [grid + 1 offsets | items], two slots used in turn
+    int* sched_h[2] = {nullptr, nullptr};   // pinned
+    int* sched_d[2] = {nullptr, nullptr};
+    cudaEvent_t sched_copied[2] = {nullptr, nullptr};
+    size_t sched_cap = 0;            // items per slot
+    int sched_next = 0;
     double weight_bytes = 0;         // bytes of every matrix a pass always streams (without the LM head)
     double expert_bytes = 0;         // bytes of one routed expert's three matrices
     double head_bytes = 0;
 };
 PassState* state(s2d2_ctx* c) { return (PassState*)c->pass_state; }
+
+// Attention items of a pass with several sequences, dealt out to the CTAs by cost (longest first,
+// each to the least loaded CTA): context lengths differ between sequences, and dealing items out
+// by index leaves some CTAs with twice the median work.  Item cost in units of about a
+// microsecond: a fixed part (query tile, first page latency, partial store) + one per 64-key page.
+// Returns the device pointer of [grid + 1 offsets | items], or null (the caller falls back to
+// the index order) when a copy could not be set up.
+const int* attention_schedule(s2d2_ctx* c, PassState* s, const att::AttnParams& ap) {
+    const PassMeta& pm = c->meta;
+    const int* nctx = pm.hp<int>(pm.off_nctx);
+    const int* nrows = pm.hp<int>(pm.off_nrows);
+    const int n_splits = ap.n_cache_splits + 1, G = s->grid;
+    std::vector<std::pair<float, int>> items;      // (cost, item index)
+    for (int seq = 0; seq < ap.pv.n_seqs; ++seq) {
+        const int n_pages = (nctx[seq] + ap.page_tokens - 1) >> ap.page_shift;
+        const int nq = nrows[seq] * ap.group;
+        for (int kvh = 0; kvh < ap.Hkv; ++kvh)
+            for (int qt = 0; qt < ap.n_qtiles && qt * att::QT < nq; ++qt)
+                for (int split = 0; split < n_splits; ++split) {
+                    const int idx = ((seq * ap.Hkv + kvh) * ap.n_qtiles + qt) * n_splits + split;
+                    if (split == ap.n_cache_splits) {
+                        items.emplace_back(5.f, idx);
+                    } else {
+                        const int pg0 = split * ap.pages_per_split;
+                        if (pg0 >= n_pages) continue;
+                        items.emplace_back(3.f + 3.f * (float)(std::min(n_pages, pg0 + ap.pages_per_split) - pg0), idx);
+                    }
+                }
+    }
+    const size_t need = (size_t)G + 1 + items.size();
+    const int k = s->sched_next;
+    if (need > s->sched_cap || !s->sched_h[k]) {
+        if (s->sched_copied[k]) cudaEventSynchronize(s->sched_copied[k]);
+        if (cudaStreamSynchronize(c->stream) != cudaSuccess) return nullptr;
+        for (int j = 0; j < 2; ++j) {
+            if (s->sched_h[j]) cudaFreeHost(s->sched_h[j]);
+            if (s->sched_d[j]) cudaFree(s->sched_d[j]);
+            s->sched_h[j] = s->sched_d[j] = nullptr;
+        }
+        s->sched_cap = std::max<size_t>(2 * need, 4096);
+        for (int j = 0; j < 2; ++j) {
+            if (cudaMallocHost((void**)&s->sched_h[j], s->sched_cap * 4) != cudaSuccess ||
+                cudaMalloc((void**)&s->sched_d[j], s->sched_cap * 4) != cudaSuccess)
+                return nullptr;
+            if (!s->sched_copied[j] && cudaEventCreateWithFlags(&s->sched_copied[j], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+    } else if (cudaEventSynchronize(s->sched_copied[k]) != cudaSuccess) {      // the slot's previous copy has left the host buffer
+        return nullptr;
+    }
+    std::stable_sort(items.begin(), items.end(), [](const std::pair<float, int>& a, const std::pair<float, int>& b) { return a.first > b.first; });
+    typedef std::pair<float, int> Load;           // (load, cta): the least loaded CTA, lowest id first
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int g = 0; g < G; ++g) heap.push(Load(0.f, g));
+    std::vector<std::vector<int>> mine(G);
+    for (const auto& it : items) {
+        Load l = heap.top();
+        heap.pop();
+        mine[l.second].push_back(it.second);
+        heap.push(Load(l.first + it.first, l.second));
+    }
+    int* h = s->sched_h[k];
+    int o = 0;
+    for (int g = 0; g < G; ++g) {
+        h[g] = o;
+        for (int idx : mine[g]) h[G + 1 + o++] = idx;
+    }
+    h[G] = o;
+    if (cudaMemcpyAsync(s->sched_d[k], h, need * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return nullptr;
+    cudaEventRecord(s->sched_copied[k], c->stream);
+    c->cnt.h2d_bytes += need * 4;
+    s->sched_next = k ^ 1;
+    return s->sched_d[k];
+}
 
 template <int HD>
 cudaError_t prepare_kernel(PassState* s, int smem) {
@@ -271,6 +352,11 @@ void pass_destroy(s2d2_ctx* c) {
     for (int* p : s->parts)
         if (p) cudaFree(p);
     if (s->n_touched_h) cudaFreeHost(s->n_touched_h);
+    for (int k = 0; k < 2; ++k) {
+        if (s->sched_h[k]) cudaFreeHost(s->sched_h[k]);
+        if (s->sched_d[k]) cudaFree(s->sched_d[k]);
+        if (s->sched_copied[k]) cudaEventDestroy(s->sched_copied[k]);
+    }
     delete s;
     c->pass_state = nullptr;
 }
@@ -281,7 +367,15 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     const s2d2_model_config& m = c->m;
     if (!s || !s->ok || pv.n_rows < 1 || pv.n_rows > pp::MAX_T) return S2D2_OK;
     pp::PassParams p;
-    if (!attention_plan(c, pv, max_ctx, max_rows, s->grid, &p.ap, nullptr)) return S2D2_OK;
+    // several sequences: finer key splits (about two items per CTA), dealt out by cost
+    if (!attention_plan(c, pv, max_ctx, max_rows, pv.n_seqs > 1 ? 2 * s->grid : s->grid, &p.ap, nullptr)) return S2D2_OK;
+    if (pv.n_seqs > 1) {
+        const int* sched = attention_schedule(c, s, p.ap);
+        if (sched) {
+            p.ap.sched_off = sched;
+            p.ap.sched_items = sched + s->grid + 1;
+        }
+    }
     p.n_layers = m.n_layers;
     p.d = m.d_model;
     p.Hq = m.n_q_heads;

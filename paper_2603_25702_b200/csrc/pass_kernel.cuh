@@ -409,6 +409,25 @@ __device__ __forceinline__ float inv_rms_from(const SsqLane& r, int d, float eps
     return 1.0f / sqrtf(warp_sum((r.v[0] + r.v[1]) + (r.v[2] + r.v[3])) / (float)d + eps);
 }
 __device__ __forceinline__ void store_bf16x4(bf16* dst, float a, float b, float c, float d);
+// x = q * d + r for 0 <= x < 2^22 and a run-time d: one multiplication by the precomputed 1/d
+// instead of an integer division (about 40 dependent instructions, which a warp that has its
+// scheduler to itself pays in full).
+struct FastDiv {
+    int d;
+    float inv;
+    __device__ __forceinline__ explicit FastDiv(int d_) : d(d_), inv(1.0f / (float)d_) {}
+    __device__ __forceinline__ void divmod(int x, int& q, int& r) const {
+        q = (int)(((float)x + 0.5f) * inv);
+        r = x - q * d;
+        if (r < 0) {
+            --q;
+            r += d;
+        } else if (r >= d) {
+            ++q;
+            r -= d;
+        }
+    }
+};
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi): the GEMMs take both halves as token rows, so
 // their inputs carry 16 significant bits instead of 8 (the tensor pipe is nearly idle in this
 // kernel; the second half costs 2 KB of shared memory per stage).
@@ -700,6 +719,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // row, 4 per lane.  A pair's loads (its partials, its residual row, the sums of squares) are
         // all in flight together, so a phase costs about one round trip to L2.
         const int gw = cta * 4 + cw, GW = G * 4;
+        const FastDiv by_M(M), by_Hq(p.Hq);
 
         // h update shared by the embedding and the two residual phases: writes h, the next GEMM's
         // input bf16(h * gain) and the (tile, row) sum of squares
@@ -711,7 +731,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         };
         auto h_phase = [&](const float* gain, float* ssq, auto&& value) {
             for (int pair = gw; pair < d_tiles * M; pair += GW) {
-                const int t = pair / M, m = pair % M;
+                int t, m;
+                by_M.divmod(pair, t, m);
                 const int col = t * tc::BLOCK_N + 4 * lane;
                 const float4 gn = *reinterpret_cast<const float4*>(gain + col);
                 const float4 x = value(t, m, col);
@@ -774,8 +795,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     for (int q = 0; q < 2; ++q) {
                         const int pr = pair0 + q * GW;
                         on[q] = pr < n_pairs;
-                        tt[q] = on[q] ? pr / M : 0;
-                        mm[q] = on[q] ? pr % M : 0;
+                        by_M.divmod(on[q] ? pr : 0, tt[q], mm[q]);
                         const int head = (tt[q] * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
                         const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
                         tabs[q] = on[q] ? tile_row_tab(p, 0, tt[q], lane) : 0;
@@ -845,7 +865,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 ap.layer = l;
                 const int n_splits = ap.n_cache_splits + 1;
                 const int total = ap.pv.n_seqs * ap.Hkv * ap.n_qtiles * n_splits;
-                for (int idx = cta; idx < total && ok; idx += G) {
+                // Items of this CTA: a host-made list when the pass has several sequences (their context
+                // lengths differ, so items are dealt out by cost), else every G-th item.
+                const int i_end = ap.sched_off ? __ldg(ap.sched_off + cta + 1) : total;
+                for (int i = ap.sched_off ? __ldg(ap.sched_off + cta) : cta; i < i_end && ok; i += ap.sched_off ? 1 : G) {
+                    const int idx = ap.sched_off ? __ldg(ap.sched_items + i) : i;
                     const int split = idx % n_splits, r = idx / n_splits;
                     if (!att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
                                             kv_ring, tid, BAR_COMPUTE)) {
@@ -858,7 +882,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 if (!ok) break;
                 // ---- combine the key splits of every (row, query head) ----
                 for (int pair = gw; pair < M * p.Hq; pair += GW) {
-                    const int r = pair / p.Hq, hq = pair % p.Hq;
+                    int r, hq;
+                    by_Hq.divmod(pair, r, hq);
                     const int seq = __ldg(p.pv.row_seq + r), kvh = hq / ap.group;
                     const int qv = (r - __ldg(p.pv.seq_row0 + seq)) * ap.group + hq % ap.group;
                     const int qt = qv / att::QT, qi = qv % att::QT;
@@ -937,8 +962,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     for (int q = 0; q < NP; ++q) {
                         const int pr = pair + q * GW;
                         on[q] = pr < n_pairs;
-                        tt[q] = on[q] ? pr / M : 0;
-                        mm[q] = on[q] ? pr % M : 0;
+                        by_M.divmod(on[q] ? pr : 0, tt[q], mm[q]);
                         tabs[2 * q] = on[q] ? tile_row_tab(p, gu_kind, tt[q], lane) : 0;
                         tabs[2 * q + 1] = on[q] ? tile_row_tab(p, gu_kind, tt[q] + f_tiles, lane) : 0;
                         rows[2 * q] = rows[2 * q + 1] = mm[q];
@@ -1192,8 +1216,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 // counter are fetched once and the partials of all four rows are in flight together
                 constexpr int NR = 4;
                 const int groups = (p.n_logit + NR - 1) / NR;
+                const FastDiv by_groups(groups);
                 for (int item = gw; item < n_tiles * groups; item += GW) {
-                    const int t = item / groups, lr0 = (item % groups) * NR;
+                    int t, lr0;
+                    by_groups.divmod(item, t, lr0);
+                    lr0 *= NR;
                     const int tab = tile_row_tab(p, 4, t, lane);
                     int tabs[NR], rows[NR];
                     const unsigned* pubs[NR];
