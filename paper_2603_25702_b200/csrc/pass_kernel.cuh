@@ -723,9 +723,10 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
 
         // h update shared by the embedding and the two residual phases: writes h, the next GEMM's
         // input bf16(h * gain) and the (tile, row) sum of squares
-        // A (tile, row) pair of a GEMM input is written: make it visible to TMA readers and count it.
+        // A (tile, row) pair of a GEMM input is written: count it.  The release orders the warp's stores
+        // before the count; the reader (the X producer) acquires the count and then crosses to the async
+        // proxy with its own fence before its TMA loads, which is the one proxy fence the chain needs.
         auto publish_x = [&](unsigned* counter) {
-            asm volatile("fence.proxy.async;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
         };
@@ -811,12 +812,14 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         gq[q] = make_float4(1.f, 1.f, 1.f, 1.f);
                         if (p.qk_norm && (is_q || is_k)) gq[q] = __ldg(reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch));
                     }
+                    // 1/rms before the wait for the partials: it only needs what the last barrier ordered
+                    const float inv_q[2] = {inv_rms_from(sq_l[0], d, p.eps), inv_rms_from(sq_l[1], d, p.eps)};
                     float4 sums[2];
                     const unsigned* const pubs_c[2] = {pubs[0], pubs[1]};
                     tile_row_sums<2, 8>(p, p.ws + p.ws_off[K_QKV], tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
                     for (int q = 0; q < 2; ++q) {
-                        const float inv = inv_rms_from(sq_l[q], d, p.eps);
+                        const float inv = inv_q[q];
                         if (!on[q]) continue;                          // warp-uniform
                         const int t = tt[q], m = mm[q];
                         const int head = (t * tc::BLOCK_N + c_tile) / HD, ch = c_tile % HD;
@@ -901,6 +904,19 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const bool used = s < n_splits && (s == ap.n_cache_splits || s * ap.pages_per_split < n_pages);
                         float2 ml = make_float2(-INFINITY, 0.f);
                         if (used) ml = __ldcg(reinterpret_cast<const float2*>(ap.part_ml + (item0 + s) * att::QT * 2 + qi * 2));
+                        // the first partial outputs are requested together with the maxima, before any weight is known
+                        const int cnt = min(32, n_splits - s0);
+                        float4 v[CCH];
+                        auto load_chunk = [&](int k0) {
+#pragma unroll
+                            for (int k = 0; k < CCH; ++k) {
+                                const int z = s0 + k0 + k;
+                                const bool uz = k0 + k < cnt && (z == ap.n_cache_splits || z * ap.pages_per_split < n_pages);
+                                v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (uz && lane < HD / 4) v[k] = __ldcg(reinterpret_cast<const float4*>(ap.part_o + ((item0 + z) * att::QT + qi) * HD) + lane);
+                            }
+                        };
+                        load_chunk(0);
                         // the maximum over all splits is needed before any weight: second sweep when n_splits > 32
                         float mx = warp_max(ml.x);
                         for (int z0 = 0; z0 < n_splits; z0 += 32) {
@@ -911,16 +927,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         }
                         const float w_l = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
                         lsum += warp_sum(w_l * ml.y);
-                        const int cnt = min(32, n_splits - s0);
                         for (int k0 = 0; k0 < cnt; k0 += CCH) {
-                            float4 v[CCH];
-#pragma unroll
-                            for (int k = 0; k < CCH; ++k) {
-                                const int z = s0 + k0 + k;
-                                const bool uz = k0 + k < cnt && (z == ap.n_cache_splits || z * ap.pages_per_split < n_pages);
-                                v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (uz && lane < HD / 4) v[k] = __ldcg(reinterpret_cast<const float4*>(ap.part_o + ((item0 + z) * att::QT + qi) * HD) + lane);
-                            }
+                            if (k0 > 0) load_chunk(k0);
 #pragma unroll
                             for (int k = 0; k < CCH; ++k) {
                                 const float w = __shfl_sync(0xffffffffu, w_l, (k0 + k) & 31);
@@ -970,12 +978,15 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         pubs[2 * q + 1] = p.tile_cnt[gu_kind] + tt[q] + f_tiles;
                         sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane);
                     }
+                    float inv_q[NP];      // before the wait for the partials: it only needs what the last barrier ordered
+#pragma unroll
+                    for (int q = 0; q < NP; ++q) inv_q[q] = inv_rms_from(sq_l[q], d, p.eps);
                     float4 sums[2 * NP];
                     const unsigned* const pubs_c[2 * NP] = {pubs[0], pubs[1], pubs[2], pubs[3], pubs[4], pubs[5]};
                     tile_row_sums<2 * NP, 4>(p, p.ws + p.ws_off[gu_kind], tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
 #pragma unroll
                     for (int q = 0; q < NP; ++q) {
-                        const float inv = inv_rms_from(sq_l[q], d, p.eps);
+                        const float inv = inv_q[q];
                         if (!on[q]) continue;
                         const float4 g4 = sums[2 * q], u4 = sums[2 * q + 1];
                         const float gv[4] = {inv * g4.x, inv * g4.y, inv * g4.z, inv * g4.w};
@@ -986,8 +997,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const size_t o = (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane;
                         store_hi_lo_x4(p.act + o, p.act_lo + o, a[0], a[1], a[2], a[3]);
                     }
-                    // one fence for the step's stores, then one count per finished pair
-                    asm volatile("fence.proxy.async;" ::: "memory");
+                    // one release for the step's stores, then one count per finished pair (the proxy fence is the reader's)
                     __syncwarp();
                     if (lane == 0) {
                         asm volatile("fence.acq_rel.gpu;" ::: "memory");
@@ -1233,13 +1243,16 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         pubs[q] = p.tile_cnt[4] + t;
                         sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, rows[q], lane);
                     }
+                    float sc_q[NR];
+#pragma unroll
+                    for (int q = 0; q < NR; ++q) sc_q[q] = p.logit_scale * inv_rms_from(sq_l[q], d, p.eps);
                     const unsigned* const pubs_c[NR] = {pubs[0], pubs[1], pubs[2], pubs[3]};
                     float4 sums[NR];
                     tile_row_sums<NR, 2>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs_c, 1u, lane, abort_flag, sums);
                     const int col = t * tc::BLOCK_N + 4 * lane;
 #pragma unroll
                     for (int q = 0; q < NR; ++q) {
-                        const float sc = p.logit_scale * inv_rms_from(sq_l[q], d, p.eps);
+                        const float sc = sc_q[q];
                         if (lr0 + q >= p.n_logit) continue;        // warp-uniform
                         const float4 s4 = sums[q];
                         float* dst = p.logits + (size_t)(lr0 + q) * p.V + col;
