@@ -78,7 +78,6 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
     p.scale = scale;
     p.accumulate = accumulate;
     p.kb_total = K / tc::BLOCK_K;
-    p.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
     p.hilo = X_lo != nullptr;
     const int t_max = p.hilo ? 128 : 256;       // the MMA takes up to 256 token rows, the low halves count
     p.m_tiles = (M + t_max - 1) / t_max;
@@ -86,30 +85,50 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
     p.T = std::min(t_max, (per + 15) / 16 * 16);
     p.m_tiles = (M + p.T - 1) / p.T;
     const int TN = p.hilo ? 2 * p.T : p.T;
-    // two CTAs per SM while the token tile is small, one otherwise
-    bool two = TN <= 64;
-    size_t budget = two ? 100 * 1024 : 200 * 1024;
-    p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(TN));
-    p.stages = std::max(2, std::min(p.stages, p.kb_total));
-    // K splits: fill the resident CTA slots; cost model in K-blocks per CTA plus a fixed set-up cost
-    int slots = g->n_sms * (two ? 2 : 1);
-    int tiles = p.n_tiles * p.m_tiles;
-    int best = 1;
+    // Weight sub-tiles per CTA (1 or 2) and K splits, by a time model fitted to measurements on the 8B-class
+    // shapes (microseconds, KB).  A k-block (weight sub-tiles + token block) takes the slowest of: what one SM
+    // takes into shared memory (80 KB/us, shared by the CTAs resident on it), the same for all busy SMs together
+    // (10.5 MB/us), the weights' part from HBM (50 KB/us per SM, 6.5 MB/us in all).  A wave of CTAs adds about
+    // 10 us of set-up and epilogue (5 us where two CTAs per SM overlap them); a K split adds the partial tile's
+    // round trip through the workspace (0.22 us per token row and sub-tile).
+    int best = 1, best_wt = 1;
     double best_cost = 1e30;
-    for (int s = 1; s <= 16 && s <= p.kb_total / 2 + (p.kb_total < 2 ? 1 : 0); ++s) {
-        if ((size_t)tiles * s * p.T * tc::BLOCK_N > g->ws_floats && s > 1) break;
-        if ((size_t)tiles > g->n_tickets && s > 1) break;
-        int waves = (tiles * s + slots - 1) / slots;
-        // per CTA: its k-blocks, a fixed set-up cost, and an epilogue that grows with the token tile (a split adds
-        // the partial tile's round trip through the workspace); all in units of one k-block of a 16-row tile
-        const double kb_cost = 1.0 + TN / 64.0, epi = p.T / 16.0;
-        double cost = waves * ((double)(p.kb_total + s - 1) / s * kb_cost + 6.0 + epi * (s > 1 ? 3.0 : 1.0)) + (s > 1 ? 2.0 : 0.0);
-        if (cost < best_cost - 1e-9) {
-            best_cost = cost;
-            best = s;
+    for (int wt = 1; wt <= 2; ++wt) {
+        if (wt == 2 && (2 * TN > 512 || N < 2 * tc::BLOCK_N)) break;       // two accumulators of TN columns in tensor memory
+        const bool two = TN <= 64 && wt == 1;                               // two CTAs per SM while the stage is small
+        const size_t budget = two ? 100 * 1024 : 200 * 1024;
+        if ((budget - 1280) / tc::stage_bytes(TN, wt) < 2) break;
+        const int slots = g->n_sms * (two ? 2 : 1);
+        const int tiles = (N + wt * tc::BLOCK_N - 1) / (wt * tc::BLOCK_N) * p.m_tiles;
+        const double w_kb = wt * 16.0, kb_bytes = w_kb + TN * 0.125;       // KB per k-block
+        for (int s = 1; s <= 16 && s <= p.kb_total / 2 + (p.kb_total < 2 ? 1 : 0); ++s) {
+            if ((size_t)tiles * s * p.T * tc::BLOCK_N * wt > g->ws_floats && s > 1) break;
+            if ((size_t)tiles > g->n_tickets && s > 1) break;
+            const int ctas = tiles * s;
+            const int waves = (ctas + slots - 1) / slots;
+            const int streaming = std::min(ctas, slots);                    // CTAs streaming at once
+            const int share = (two && ctas > g->n_sms) ? 2 : 1;           // of them on one SM
+            const double kb_us = std::max(std::max(kb_bytes * share / 80.0, kb_bytes * streaming / 10500.0),
+                                          std::max(w_kb * share / 50.0, w_kb * streaming / 6500.0));
+            const double cost = waves * ((double)((p.kb_total + s - 1) / s) * kb_us + (two ? 5.0 : 10.0)) +
+                                (s > 1 ? 2.0 + 0.22 * p.T * wt : 0.0);
+            if (cost < best_cost - 1e-9) {
+                best_cost = cost;
+                best = s;
+                best_wt = wt;
+            }
         }
     }
     p.splits = best;
+    p.wtiles = best_wt;
+    p.n_tiles = (N + best_wt * tc::BLOCK_N - 1) / (best_wt * tc::BLOCK_N);
+    const int tiles = p.n_tiles * p.m_tiles;
+    {
+        const bool two = TN <= 64 && best_wt == 1;
+        const size_t budget = two ? 100 * 1024 : 200 * 1024;
+        p.stages = (int)std::min<size_t>(8, (budget - 1280) / tc::stage_bytes(TN, best_wt));
+        p.stages = std::max(2, std::min(p.stages, p.kb_total));
+    }
     p.ws = g->ws;
     p.tickets = g->tickets;
     p.status = c->d_status;
@@ -118,7 +137,7 @@ int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, i
     const CUtensorMap* mx = get_map(c, X, M, K, p.T);
     const CUtensorMap* mx_lo = p.hilo ? get_map(c, X_lo, M, K, p.T) : mx;
     if (!mw || !mx || !mx_lo) return S2D2_ERR_CUDA;
-    size_t smem = tc::smem_bytes(TN, p.stages);
+    size_t smem = tc::smem_bytes(TN, p.stages, p.wtiles);
     int grid = tiles * p.splits;
     tc::gemm_tc_kernel<<<grid, tc::THREADS, smem, c->stream>>>(*mw, *mx, *mx_lo, p);
     c->cnt.n_kernel_launches++;
@@ -359,6 +378,7 @@ extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d
     p.status = nd.status;
     p.evict_first = 0;
     p.hilo = 0;
+    p.wtiles = 1;
     CUtensorMap mw, mx;
     if (noalloc_map(&mw, d_w, N, K, tc::BLOCK_N) || noalloc_map(&mx, d_x, M, K, p.T))
         return noalloc_fail(S2D2_ERR_CUDA, "cuTensorMapEncodeTiled failed");

@@ -19,6 +19,9 @@
 //                     the last CTA to arrive for a tile (ticket counter) sums the
 //                     partials in split order, so the result does not depend on timing.
 // Two CTAs fit on one SM, so one CTA's set-up and epilogue overlap the other's stream.
+// With more than about 128 token rows the kernel is bound by what enters shared memory, and most of
+// that is the token block, re-read for every weight tile: a CTA then takes two weight sub-tiles
+// (256 rows, one accumulator each) per token block.
 // Every wait on an mbarrier is bounded; on time-out the kernel raises a status word
 // that the host turns into S2D2_ERR_TIMEOUT, drains its copies and frees its TMEM.
 #pragma once
@@ -50,6 +53,7 @@ struct GemmParams {
     unsigned* tickets;   // one counter per (n_tile, m_tile), zero between launches
     int* status;         // device status word (0 = ok)
     int evict_first;     // stream W with an evict-first L2 policy
+    int wtiles;          // 128-row weight sub-tiles per CTA (1 or 2): two halve the re-reads of the token block
     int hilo;            // X arrives as two bf16 terms (X = X_hi + X_lo): both are token rows of one MMA (N = 2T, T <= 128)
 };
 
@@ -70,9 +74,9 @@ __host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int T) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(T >> 3) << 17) | ((uint32_t)(BLOCK_N >> 4) << 24);
 }
 
-// TN: token rows of one stage (T, or 2T with two-term inputs)
-__host__ __device__ __forceinline__ size_t stage_bytes(int TN) { return (size_t)BLOCK_N * 128 + (size_t)TN * 128; }
-__host__ __device__ __forceinline__ size_t smem_bytes(int TN, int stages) { return stages * stage_bytes(TN) + 1024 + 256; }
+// TN: token rows of one stage (T, or 2T with two-term inputs); wtiles: weight sub-tiles of one stage
+__host__ __device__ __forceinline__ size_t stage_bytes(int TN, int wtiles = 1) { return (size_t)wtiles * BLOCK_N * 128 + (size_t)TN * 128; }
+__host__ __device__ __forceinline__ size_t smem_bytes(int TN, int stages, int wtiles = 1) { return stages * stage_bytes(TN, wtiles) + 1024 + 256; }
 
 static __global__ void __launch_bounds__(THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
@@ -81,7 +85,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     // tiles need 1024-byte alignment for the 128-byte swizzle
     uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int S = p.stages, T = p.T, TN = p.hilo ? 2 * p.T : p.T;
-    const size_t sbytes = stage_bytes(TN);
+    const int WT = p.wtiles, NW = WT * BLOCK_N;      // weight rows of this CTA's tile
+    const size_t sbytes = stage_bytes(TN, WT);
     uint64_t* full = (uint64_t*)(tiles + S * sbytes);
     uint64_t* empty = full + S;
     uint64_t* acc_ready = empty + S;
@@ -101,9 +106,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int n_tile = item / p.splits;
     const int kb0 = (int)((long long)p.kb_total * split / p.splits);
     const int kb1 = (int)((long long)p.kb_total * (split + 1) / p.splits);
-    const int n0 = n_tile * BLOCK_N, m0 = m_tile * T;
+    const int n0 = n_tile * NW, m0 = m_tile * T;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < TN) tmem_cols <<= 1;
+    while ((int)tmem_cols < WT * TN) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -141,10 +146,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             if (*abort_flag) break;
             uint8_t* a = tiles + s * sbytes;
-            uint8_t* b = a + BLOCK_N * 128;
+            uint8_t* b = a + (size_t)WT * BLOCK_N * 128;
             mbar_expect_tx(&full[s], (uint32_t)sbytes);
-            if (p.evict_first) tma_load_2d_hint(a, &map_w, kb * BLOCK_K, n0, &full[s], policy);
-            else tma_load_2d(a, &map_w, kb * BLOCK_K, n0, &full[s]);
+            for (int h = 0; h < WT; ++h) {      // a sub-tile past the matrix is zero-filled
+                if (p.evict_first) tma_load_2d_hint(a + h * BLOCK_N * 128, &map_w, kb * BLOCK_K, n0 + h * BLOCK_N, &full[s], policy);
+                else tma_load_2d(a + h * BLOCK_N * 128, &map_w, kb * BLOCK_K, n0 + h * BLOCK_N, &full[s]);
+            }
             tma_load_2d(b, &map_x, kb * BLOCK_K, m0, &full[s]);
             if (p.hilo) tma_load_2d(b + (size_t)T * 128, &map_x_lo, kb * BLOCK_K, m0, &full[s]);
             *issued = i + 1;
@@ -161,12 +168,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             tc_fence_after();
             uint32_t a_addr = smem_u32(tiles + s * sbytes);
-            uint32_t b_addr = a_addr + BLOCK_N * 128;
-            uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+            uint32_t b_addr = a_addr + WT * BLOCK_N * 128;
+            uint64_t b_desc = smem_desc_sw128(b_addr);
+            for (int h = 0; h < WT; ++h) {      // one accumulator of TN columns per weight sub-tile
+                uint64_t a_desc = smem_desc_sw128(a_addr + h * BLOCK_N * 128);
 #pragma unroll
-            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                // stepping 16 elements (32 bytes) along K inside the swizzled row: +2 in the address field
-                umma_bf16(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                    // stepping 16 elements (32 bytes) along K inside the swizzled row: +2 in the address field
+                    umma_bf16(tmem_base + h * TN, a_desc + 2 * k, b_desc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                }
             }
             umma_commit(&empty[s]);   // arrives when the MMAs that read this stage are done
             *consumed = i + 1;
@@ -188,13 +198,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int i = *consumed; i < *issued; ++i) mbar_wait(&full[i % S], (i / S) & 1);
         }
     } else {
-        const int n_local = warp * 32 + lane;
-        const int n = n0 + n_local;
-        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const uint32_t taddr0 = tmem_base + ((uint32_t)(warp * 32) << 16);
         const int m_hi = min(T, p.M - m0);
         // In both epilogues the loads of 16 rows (previous y for an accumulating GEMM, split-K partials)
         // are issued together before anything is stored: one round trip per 16 rows instead of one per row.
         if (p.splits == 1) {
+            for (int h = 0; h < WT; ++h) {
+            const int n = n0 + h * BLOCK_N + warp * 32 + lane;
+            const uint32_t taddr = taddr0 + h * TN;
             for (int c = 0; c < T; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);      // executed by the whole warp even past m_hi (aligned instruction)
@@ -214,9 +225,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         if (c + j < m_hi) p.Y[(size_t)(m0 + c + j) * p.ldy + n] = old[j] + p.scale * v[j];
                 }
             }
+            }
         } else {
             const int tile = n_tile * p.m_tiles + m_tile;
-            float* mine = p.ws + ((size_t)tile * p.splits + split) * (size_t)T * BLOCK_N;
+            float* mine = p.ws + ((size_t)tile * p.splits + split) * (size_t)T * NW;
+            for (int h = 0; h < WT; ++h) {
+            const int n_local = h * BLOCK_N + warp * 32 + lane;
+            const uint32_t taddr = taddr0 + h * TN;
             for (int c = 0; c < T; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);
@@ -228,7 +243,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    if (c + j < m_hi) mine[(size_t)(c + j) * BLOCK_N + n_local] = v[j];
+                    if (c + j < m_hi) mine[(size_t)(c + j) * NW + n_local] = v[j];
+            }
             }
             __threadfence();
             __syncthreads();
@@ -239,7 +255,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             __syncthreads();
             if (*last_flag) {
                 __threadfence();
-                const float* base = p.ws + (size_t)tile * p.splits * (size_t)T * BLOCK_N + n_local;
+                for (int h = 0; h < WT; ++h) {
+                const int n_local = h * BLOCK_N + warp * 32 + lane, n = n0 + n_local;
+                const float* base = p.ws + (size_t)tile * p.splits * (size_t)T * NW + n_local;
                 if (n < p.N) {
                     for (int c = 0; c < m_hi; c += 16) {
                         float acc[16], old[16];
@@ -254,8 +272,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const bool in = c + j < m_hi;
-                                t0[j] = in ? __ldcg(base + ((size_t)s0 * T + c + j) * BLOCK_N) : 0.f;
-                                t1[j] = in && two ? __ldcg(base + ((size_t)(s0 + 1) * T + c + j) * BLOCK_N) : 0.f;
+                                t0[j] = in ? __ldcg(base + ((size_t)s0 * T + c + j) * NW) : 0.f;
+                                t1[j] = in && two ? __ldcg(base + ((size_t)(s0 + 1) * T + c + j) * NW) : 0.f;
                             }
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
@@ -267,6 +285,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         for (int j = 0; j < 16; ++j)
                             if (c + j < m_hi) p.Y[(size_t)(m0 + c + j) * p.ldy + n] = old[j] + p.scale * acc[j];
                     }
+                }
                 }
                 if (threadIdx.x == 0) p.tickets[tile] = 0;   // ready for the next launch
             }

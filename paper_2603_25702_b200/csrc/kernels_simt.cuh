@@ -40,6 +40,24 @@ __device__ __forceinline__ void store_two_term(T* hi, T* lo, size_t i, float v) 
     hi[i] = h;
     if (lo) lo[i] = from_f32<T>(v - to_f32(h));
 }
+// Four consecutive values at once (i a multiple of 4): one 8- or 16-byte store per buffer.
+__device__ __forceinline__ void store_two_term_x4(float* hi, float*, size_t i, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(hi + i) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store_two_term_x4(bf16* hi, bf16* lo, size_t i, float a, float b, float c, float d) {
+    const __nv_bfloat162 h0 = __floats2bfloat162_rn(a, b), h1 = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t*>(&h0);
+    u.y = *reinterpret_cast<const uint32_t*>(&h1);
+    *reinterpret_cast<uint2*>(hi + i) = u;
+    if (lo) {
+        const __nv_bfloat162 l0 = __floats2bfloat162_rn(a - __low2float(h0), b - __high2float(h0));
+        const __nv_bfloat162 l1 = __floats2bfloat162_rn(c - __low2float(h1), d - __high2float(h1));
+        u.x = *reinterpret_cast<const uint32_t*>(&l0);
+        u.y = *reinterpret_cast<const uint32_t*>(&l1);
+        *reinterpret_cast<uint2*>(lo + i) = u;
+    }
+}
 // out[i, :] = rmsnorm(h[rows ? rows[i] : i, :]) * gain, written as TO (out_lo: low halves, may be null).
 template <typename TO>
 __global__ void rmsnorm_kernel(const float* __restrict__ h, const int* __restrict__ rows, const float* __restrict__ gain,
@@ -47,14 +65,29 @@ __global__ void rmsnorm_kernel(const float* __restrict__ h, const int* __restric
     __shared__ float sh[32];
     int i = blockIdx.x;
     const float* x = h + (size_t)(rows ? rows[i] : i) * d;
+    const bool vec = (d & 3) == 0;
     float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) ss += x[c] * x[c];
+    if (vec) {
+        for (int c = threadIdx.x; c < d / 4; c += blockDim.x) {
+            const float4 v = reinterpret_cast<const float4*>(x)[c];
+            ss += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) ss += x[c] * x[c];
+    }
     ss = block_sum(ss, sh);
     float inv = rsqrtf(ss / (float)d + eps);
     // rsqrtf is approximate (2 ulp); refine once so the fp32 model stays within 1e-4 relative
     float m = ss / (float)d + eps;
     inv = inv * (1.5f - 0.5f * m * inv * inv);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) store_two_term(out, out_lo, (size_t)i * d + c, x[c] * inv * gain[c]);
+    if (vec) {
+        for (int c = threadIdx.x; c < d / 4; c += blockDim.x) {
+            const float4 v = reinterpret_cast<const float4*>(x)[c], g = reinterpret_cast<const float4*>(gain)[c];
+            store_two_term_x4(out, out_lo, (size_t)i * d + 4 * c, v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) store_two_term(out, out_lo, (size_t)i * d + c, x[c] * inv * gain[c]);
+    }
 }
 
 // Y[m, n] (+)= scale * sum_k X[m, k] * W[n, k].  One warp per output column and
@@ -200,6 +233,14 @@ __global__ void attention_simt_kernel(const TA* __restrict__ q, const TKV* __res
 template <typename TA>
 __global__ void swiglu_kernel(const float* __restrict__ gu, TA* __restrict__ act, TA* __restrict__ act_lo, int M, int f) {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((f & 3) == 0) {       // four consecutive columns per thread; the grid has a thread per element, the rest leave
+        if (idx >= (size_t)M * (f / 4)) return;
+        const size_t m = idx / (f / 4), i = (idx % (f / 4)) * 4;
+        const float4 g = *reinterpret_cast<const float4*>(gu + m * 2 * f + i), u = *reinterpret_cast<const float4*>(gu + m * 2 * f + f + i);
+        store_two_term_x4(act, act_lo, m * f + i, g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                          g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+        return;
+    }
     if (idx >= (size_t)M * f) return;
     size_t m = idx / f, i = idx % f;
     float g = gu[m * 2 * f + i], u = gu[m * 2 * f + f + i];

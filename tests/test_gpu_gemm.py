@@ -20,7 +20,8 @@ def engine():
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (4, 256, 256), (8, 384, 128), (16, 128, 4096), (16, 6144, 4096),
                                    (5, 200, 192), (33, 1000, 512), (64, 4096, 1024), (100, 640, 2048), (257, 300, 320),
-                                   (512, 1024, 512), (16, 151936, 256), (3, 64, 704)])
+                                   (512, 1024, 512), (16, 151936, 256), (3, 64, 704),
+                                   (342, 6144, 1024), (200, 384, 512), (160, 4096, 12288)])   # two weight sub-tiles per CTA
 def test_gemm_matches_float64(engine, M, N, K):
     rng = np.random.default_rng(M * 1000003 + N * 101 + K)
     x = f32_to_bf16_bits(rng.standard_normal((M, K)).astype(np.float32))
