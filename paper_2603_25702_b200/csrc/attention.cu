@@ -20,6 +20,7 @@ struct AttnState {
     float* part_o = nullptr;
     float* part_ml = nullptr;
     size_t cap_items = 0;
+    bool umma_ok = false;        // tcgen05 work items (head_dim 128, 64-token pages)
     int n_sms = 148;
 };
 AttnState* state(s2d2_ctx* c) { return (AttnState*)c->attn_state; }
@@ -83,6 +84,10 @@ int attention_init(s2d2_ctx* c) {
     if (e == cudaSuccess)
         e = m.head_dim == 128 ? cudaFuncSetAttribute(att::attn_tc_kernel<128, false>, attr, smem)
                               : cudaFuncSetAttribute(att::attn_tc_kernel<64, false>, attr, smem);
+    if (e == cudaSuccess && m.head_dim == 128 && c->page_tokens == 64) {
+        e = cudaFuncSetAttribute(att::attn_umma_kernel, attr, (int)att::attn_umma_smem_bytes());
+        a->umma_ok = e == cudaSuccess;
+    }
     if (e != cudaSuccess) return S2D2_ERR_CUDA;
     a->tc_ok = true;
     return S2D2_OK;
@@ -156,7 +161,10 @@ int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_r
     dim3 grid(p.n_cache_splits + 1, p.n_qtiles, pv.n_seqs * m.n_kv_heads);
     const size_t smem = att::attn_smem_bytes(m.head_dim);
     // two-term queries and probabilities whenever the low halves of q exist (always on this path)
-    if (m.head_dim == 128) {
+    if (a->umma_ok && p.q_lo) {
+        att::attn_umma_kernel<<<grid, att::THREADS, att::attn_umma_smem_bytes(), c->stream>>>(a->map_kv, p);
+        att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);
+    } else if (m.head_dim == 128) {
         if (p.q_lo) att::attn_tc_kernel<128, true><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
         else att::attn_tc_kernel<128, false><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
         att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);

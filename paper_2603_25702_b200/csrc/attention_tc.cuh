@@ -373,6 +373,351 @@ __device__ __forceinline__ bool attn_item(const CUtensorMap* map_kv_ptr, const A
     return true;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same work item on the 5th-generation tensor cores (head_dim 128, 64-token pages, two-term q
+// and probabilities).  The shared-memory tiles are the ones above: 128-byte rows with the
+// 128-byte swizzle, which is the canonical K-major operand layout of tcgen05.mma (and, for V,
+// whose rows are keys, the MN-major one).  Per 64-key tile:
+//   S[q, key]  = (Q_hi + Q_lo) K^T   16 MMAs (M = 128, N = 64, K = 16) into 64 TMEM columns;
+//   one thread per query row (warps 0 and 1 of the group: TMEM lane = row) reads its 64 scores,
+//   masks, updates the running maximum and sum, and writes its probabilities as two bf16 terms
+//   into a K-major tile; if a maximum moved, the rows rescale their accumulator in TMEM;
+//   O[q, :]   += (P_hi + P_lo) V     8 MMAs (N = 128, K = 16) into 128 TMEM columns.
+// The MMA tile has 128 rows and a group has 64 query vectors: rows 64..127 read whatever follows
+// the 64-row tile in shared memory and their results are never looked at.  Every wait is bounded.
+// Shared memory (1024-byte aligned): Q_hi | Q_lo (16 KB each) | STAGES x (K, V).  The probabilities
+// (P_hi | P_lo, 8 KB each) take the place of the stage's K tile, which is dead once S is complete;
+// with 96 KB per CTA two CTAs share an SM.
+__host__ __device__ inline size_t attn_umma_tiles_bytes() { return (size_t)2 * QT * 128 * 2 + (size_t)STAGES * 2 * 64 * 128 * 2; }
+
+// Shared-memory descriptor of an MN-major operand tile stored as rows of 128 bytes (64 bf16 along
+// MN) with the 128-byte swizzle, the rows being consecutive K indices: 8-row groups are 1024 bytes
+// apart (stride byte offset), the next 64 MN elements start `mn_chunk_bytes` further (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t smem_addr, uint32_t mn_chunk_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((mn_chunk_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128_k(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// D fp32, A and B bf16, A K-major, M = 128; B K-major (b_mn = 0) or MN-major (b_mn = 1)
+__device__ __forceinline__ uint32_t umma_idesc(int n, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// `bars`: STAGES "tile landed" barriers, then the "scores ready" and "output ready" barriers;
+// ring_pos / s_cnt / o_cnt carry their phases from one item to the next.  tmem: 64 columns of
+// scores followed by 128 columns of output, lanes 0..127.
+__device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
+                                               uint8_t* base, uint64_t* bars, uint32_t tmem, uint32_t& ring_pos, uint32_t& s_cnt,
+                                               uint32_t& o_cnt, int tid, int bar_id) {
+    constexpr int HD = 128, CH = HD / 8, PT = 64;
+    constexpr int tile_bytes = 64 * HD * 2;
+    uint8_t* q_s = base;                                   // Q_hi, Q_lo: [QT][HD] each
+    uint8_t* kv_s = q_s + 2 * QT * HD * 2;                 // STAGES x (K tile, V tile)
+    uint64_t* full = bars;
+    uint64_t* bar_s = bars + STAGES;
+    uint64_t* bar_o = bars + STAGES + 1;
+    const uint32_t tmem_s = tmem, tmem_o = tmem + 64;
+
+    const int seq = z / p.Hkv, kvh = z % p.Hkv;
+    const int nrows = p.pv.seq_nrows[seq], row0 = p.pv.seq_row0[seq];
+    const int nq = nrows * p.group;
+    const int q0 = qt * QT;
+    if (q0 >= nq) return true;
+    const int n_ctx = p.pv.seq_nctx[seq];
+    const bool in_pass = split == p.n_cache_splits;
+    const int n_pages = (n_ctx + PT - 1) >> p.page_shift;
+    const int pg0 = split * p.pages_per_split;
+    const int pg1 = in_pass ? 0 : min(n_pages, pg0 + p.pages_per_split);
+    const int n_tiles = in_pass ? 1 : max(0, pg1 - pg0);
+    const size_t item = ((size_t)z * p.n_qtiles + qt) * (p.n_cache_splits + 1) + split;
+    const int warp = tid >> 5;
+    const uint32_t ring0 = ring_pos;
+    if (!in_pass) ring_pos += (uint32_t)n_tiles;
+
+    const int* pages = p.pv.seq_pages + (size_t)seq * p.pv.max_pages;
+    auto issue = [&](int t) {   // thread 0: TMA of cache tile t of this split into stage t % STAGES
+        int s = (int)((ring0 + t) % STAGES);
+        int page = pages[pg0 + t];
+        uint8_t* kd = kv_s + (size_t)s * 2 * tile_bytes;
+        uint8_t* vd = kd + tile_bytes;
+        long long rk = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 0) * p.Hkv + kvh) * PT;
+        long long rv = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 1) * p.Hkv + kvh) * PT;
+        tc::mbar_expect_tx(&full[s], (uint32_t)(2 * PT * HD * 2));
+#pragma unroll
+        for (int h = 0; h < HD / 64; ++h) {
+            tc::tma_load_2d(kd + h * PT * 128, map_kv_ptr, h * 64, (int)rk, &full[s]);
+            tc::tma_load_2d(vd + h * PT * 128, map_kv_ptr, h * 64, (int)rv, &full[s]);
+        }
+    };
+    if (!in_pass && tid == 0)
+        for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
+
+    // ---- Q tiles (both terms): global -> swizzled shared ----
+    {
+        constexpr int NQ = QT * CH / THREADS;
+        uint4 hi[NQ], lo[NQ];
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH, qv = q0 + r;
+            hi[k] = make_uint4(0, 0, 0, 0);
+            lo[k] = hi[k];
+            if (qv < nq) {
+                const int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
+                hi[k] = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
+                lo[k] = ldcg16(p.q_lo + ((size_t)row * p.Hq + hq) * HD + c * 8);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < NQ; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            *reinterpret_cast<uint4*>(q_s + sw_off(r, c, QT)) = hi[k];
+            *reinterpret_cast<uint4*>(q_s + QT * HD * 2 + sw_off(r, c, QT)) = lo[k];
+        }
+    }
+    if (in_pass) {
+        // K and V of this pass's rows of the sequence into stage 0 (rows past nrows are zero)
+        uint8_t* kd = kv_s;
+        uint8_t* vd = kd + tile_bytes;
+        constexpr int NK = 64 * CH / THREADS;
+        uint4 kk[NK], vv[NK];
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            kk[k] = make_uint4(0, 0, 0, 0);
+            vv[k] = kk[k];
+            if (r < nrows) {
+                size_t o = ((size_t)(row0 + r) * p.Hkv + kvh) * HD + c * 8;
+                kk[k] = ldcg16(p.k_rows + o);
+                vv[k] = ldcg16(p.v_rows + o);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int i = tid + k * THREADS, r = i / CH, c = i % CH;
+            *reinterpret_cast<uint4*>(kd + sw_off(r, c, 64)) = kk[k];
+            *reinterpret_cast<uint4*>(vd + sw_off(r, c, 64)) = vv[k];
+        }
+    }
+    // the tiles written with plain stores are read by the tensor core through the async proxy
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    group_sync(bar_id, THREADS);
+
+    const bool row_thread = tid < QT;                       // warps 0 and 1: thread = query row = TMEM lane
+    const int qv = q0 + tid;
+    unsigned long long row_mask = 0;
+    if (in_pass && row_thread && qv < nq) row_mask = p.pv.row_mask[row0 + qv / p.group];
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool failed = false;
+    const uint32_t idesc_s = umma_idesc(64, 0), idesc_o = umma_idesc(HD, 1);
+
+    for (int t = 0; t < n_tiles; ++t) {
+        const int s = in_pass ? 0 : (int)((ring0 + t) % STAGES);
+        bool ok = in_pass || tc::mbar_wait(&full[s], ((ring0 + t) / STAGES) & 1);
+        if (group_or(bar_id, THREADS, !ok)) {
+            failed = true;
+            break;
+        }
+        const uint32_t kb = tc::smem_u32(kv_s + (size_t)s * 2 * tile_bytes);
+        const uint32_t vb = kb + tile_bytes;
+        if (tid == 0) {
+            // ---- S = (Q_hi + Q_lo) K^T: two terms x two 64-column halves of head_dim x four k-steps ----
+            tc::tc_fence_after();
+            const uint32_t qb = tc::smem_u32(q_s);
+#pragma unroll
+            for (int term = 0; term < 2; ++term)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint64_t a = smem_desc_sw128_k(qb + term * (QT * HD * 2) + h * (QT * 128));
+                    const uint64_t b = smem_desc_sw128_k(kb + h * (64 * 128));
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tc::umma_bf16(tmem_s, a + 2 * k, b + 2 * k, idesc_s, (term | h | k) ? 1u : 0u);
+                }
+            tc::umma_commit(bar_s);
+        }
+        ok = tc::mbar_wait(bar_s, s_cnt & 1);
+        ++s_cnt;
+        if (group_or(bar_id, THREADS, !ok)) {
+            failed = true;
+            break;
+        }
+        tc::tc_fence_after();
+        // The commit above also covers the previous tile's P V MMAs: P, the other stage and the
+        // output accumulator are free to be rewritten.
+        if (!in_pass && tid == 0 && t >= 1 && t + 1 < n_tiles) issue(t + 1);
+        float alpha = 1.f;
+        if (row_thread) {
+            // ---- this row's scores: mask, running maximum and sum (log2 domain), probabilities ----
+            const int key0 = in_pass ? 0 : (pg0 + t) * PT;
+            float sc[64];
+            tc::tmem_ld32(tmem_s + lane_base, sc);
+            tc::tmem_ld32(tmem_s + lane_base + 32, sc + 32);
+            // raw scores first: the scale is positive, so the maximum can be taken before it is applied
+            const bool whole = !in_pass && key0 + 64 <= n_ctx;          // every key of the tile counts (all but a sequence's last page)
+            if (!whole) {
+#pragma unroll
+                for (int j = 0; j < 64; ++j) {
+                    const bool keep = in_pass ? (j < nrows && ((row_mask >> j) & 1ull)) : (key0 + j < n_ctx);
+                    if (!keep) sc[j] = -INFINITY;
+                }
+            }
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+            // The reference point of the exponentials follows the running maximum lazily: it moves only when
+            // the maximum has grown by more than 2^8 (probabilities then stay below 256, exact in two bf16
+            // terms and harmless in the fp32 sums), so the accumulator in tensor memory is rarely rescaled.
+            float m_new = m_run;
+            if (t == 0 || mx > m_run + 8.f) m_new = fmaxf(m_run, mx);
+            const float ref = m_new == -INFINITY ? 0.f : m_new;
+            alpha = m_new == m_run ? 1.f : exp2f(m_run - ref);
+            m_run = m_new;
+            float sum = 0.f, sum1 = 0.f;
+            uint8_t* ph = kv_s + (size_t)s * 2 * tile_bytes + tid * 128;      // P_hi | P_lo over the K tile, which S no longer needs
+            const float neg_ref = -ref;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float p0, p1;      // 2^(s * scale - ref); a masked score (-inf) gives 0
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p0) : "f"(fmaf(sc[c * 8 + 2 * e], p.scale_log2, neg_ref)));
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p1) : "f"(fmaf(sc[c * 8 + 2 * e + 1], p.scale_log2, neg_ref)));
+                    sum += p0;
+                    sum1 += p1;
+                    hi[e] = pack_bf16(p0, p1);
+                    // the bits of a bf16 are the high half of the float with the same value
+                    lo[e] = pack_bf16(p0 - __uint_as_float(hi[e] << 16), p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                }
+                const uint32_t off = (uint32_t)((c ^ (tid & 7)) << 4);
+                *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(ph + QT * 128 + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            l_run = l_run * alpha + (sum + sum1);
+        }
+        // ---- rescale the accumulator where a maximum moved (never on the first tile: it is overwritten) ----
+        if (t > 0 && group_or(bar_id, THREADS, row_thread && alpha != 1.f)) {
+            if (row_thread) {
+#pragma unroll
+                for (int c = 0; c < HD; c += 16) {
+                    float o[16];
+                    tc::tmem_ld16(tmem_o + lane_base + c, o);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) o[j] *= alpha;
+                    tmem_st16(tmem_o + lane_base + c, o);
+                }
+                tmem_wait_st();
+            }
+        }
+        tc::tc_fence_before();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        group_sync(bar_id, THREADS);
+        if (tid == 0) {
+            // ---- O += (P_hi + P_lo) V: two terms x four k-steps of 16 keys ----
+            tc::tc_fence_after();
+            const uint32_t pb = kb;
+#pragma unroll
+            for (int term = 0; term < 2; ++term) {
+                const uint64_t a = smem_desc_sw128_k(pb + term * (QT * 128));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t b = smem_desc_sw128_mn(vb + k * 2048, 64 * 128);
+                    tc::umma_bf16(tmem_o, a + 2 * k, b, idesc_o, (t | term | k) ? 1u : 0u);
+                }
+            }
+            tc::umma_commit(bar_o);
+        }
+        ++o_cnt;
+    }
+    if (!failed && n_tiles > 0) {
+        bool ok = tc::mbar_wait(bar_o, (o_cnt - 1) & 1);
+        if (group_or(bar_id, THREADS, !ok)) failed = true;
+    }
+    if (failed) {   // uniform across the group
+        if (tid == 0) atomicExch(p.status, 2);
+        return false;
+    }
+    tc::tc_fence_after();
+    // ---- partial (max, sum, O) of this split ----
+    if (row_thread) {
+        float* po = p.part_o + (item * QT + tid) * HD;
+        float* pml = p.part_ml + (item * QT + tid) * 2;
+        pml[0] = m_run;
+        pml[1] = l_run;
+#pragma unroll
+        for (int c = 0; c < HD; c += 16) {
+            float o[16];
+            if (n_tiles > 0) {
+                tc::tmem_ld16(tmem_o + lane_base + c, o);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(po + c + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+        }
+    }
+    // the accumulators are read: the next item's MMAs may overwrite them; shared memory is reused too
+    tc::tc_fence_before();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    group_sync(bar_id, THREADS);
+    return true;
+}
+
+// One CTA per work item, tcgen05 path.  256 columns of tensor memory (64 scores + 128 output used).
+static __global__ void __launch_bounds__(THREADS) attn_umma_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = (uint64_t*)(base + attn_umma_tiles_bytes());
+    uint32_t* tmem_slot = (uint32_t*)(bars + STAGES + 2);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES + 2; ++s) tc::mbar_init(&bars[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < 32) {
+        tc::tmem_alloc(tmem_slot, 256);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    uint32_t ring_pos = 0, s_cnt = 0, o_cnt = 0;
+    bool ok = attn_item_umma(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, bars, tmem, ring_pos, s_cnt, o_cnt, threadIdx.x, 0);
+    if (!ok && threadIdx.x == 0) {
+        // copies already issued target this CTA's shared memory: give them one more bounded wait
+        for (int s = 0; s < STAGES; ++s) tc::mbar_wait(&bars[s], 0);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tc::tmem_dealloc(tmem, 256);
+}
+__host__ __device__ inline size_t attn_umma_smem_bytes() { return attn_umma_tiles_bytes() + 64 + 1024; }
+
 template <int HD, bool HL>
 __global__ void __launch_bounds__(THREADS) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
