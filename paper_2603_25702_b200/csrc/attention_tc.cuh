@@ -429,13 +429,19 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 // `bars`: STAGES "tile landed" barriers, then the "scores ready" and "output ready" barriers;
 // ring_pos / s_cnt / o_cnt carry their phases from one item to the next.  tmem: 64 columns of
 // scores followed by 128 columns of output, lanes 0..127.
+// SPLIT: the 80 KB variant for a kernel that cannot spare two stages: one K tile, one V tile and a
+// separate P tile (P_hi | P_lo | Q_hi | Q_lo | K | V: what an MMA reads past a 64-row tile is the next
+// tile of the same region), the two "tile landed" barriers being K's and
+// V's.  The next K is requested as soon as S is complete and the next V as soon as the previous
+// P V is, so both arrive behind the softmax of the tile in between.
+template <bool SPLIT>
 __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
                                                uint8_t* base, uint64_t* bars, uint32_t tmem, uint32_t& ring_pos, uint32_t& s_cnt,
                                                uint32_t& o_cnt, int tid, int bar_id) {
     constexpr int HD = 128, CH = HD / 8, PT = 64;
     constexpr int tile_bytes = 64 * HD * 2;
-    uint8_t* q_s = base;                                   // Q_hi, Q_lo: [QT][HD] each
-    uint8_t* kv_s = q_s + 2 * QT * HD * 2;                 // STAGES x (K tile, V tile)
+    uint8_t* q_s = base + (SPLIT ? 2 * QT * 128 : 0);      // Q_hi, Q_lo: [QT][HD] each
+    uint8_t* kv_s = q_s + 2 * QT * HD * 2;                 // STAGES x (K tile, V tile); SPLIT: one of each
     uint64_t* full = bars;
     uint64_t* bar_s = bars + STAGES;
     uint64_t* bar_o = bars + STAGES + 1;
@@ -458,22 +464,29 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     if (!in_pass) ring_pos += (uint32_t)n_tiles;
 
     const int* pages = p.pv.seq_pages + (size_t)seq * p.pv.max_pages;
-    auto issue = [&](int t) {   // thread 0: TMA of cache tile t of this split into stage t % STAGES
-        int s = (int)((ring0 + t) % STAGES);
-        int page = pages[pg0 + t];
+    // thread 0: TMA of cache tile t of this split.  which: bit 0 = K, bit 1 = V.  Two-stage layout: both into
+    // stage t % STAGES on that stage's barrier; SPLIT: K on barrier 0, V on barrier 1.
+    auto issue = [&](int t, int which) {
+        const int s = SPLIT ? 0 : (int)((ring0 + t) % STAGES);
+        const int page = pages[pg0 + t];
         uint8_t* kd = kv_s + (size_t)s * 2 * tile_bytes;
         uint8_t* vd = kd + tile_bytes;
-        long long rk = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 0) * p.Hkv + kvh) * PT;
-        long long rv = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 1) * p.Hkv + kvh) * PT;
-        tc::mbar_expect_tx(&full[s], (uint32_t)(2 * PT * HD * 2));
+        const long long rk = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 0) * p.Hkv + kvh) * PT;
+        const long long rv = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 1) * p.Hkv + kvh) * PT;
+        if (SPLIT) {
+            if (which & 1) tc::mbar_expect_tx(&full[0], (uint32_t)(PT * HD * 2));
+            if (which & 2) tc::mbar_expect_tx(&full[1], (uint32_t)(PT * HD * 2));
+        } else {
+            tc::mbar_expect_tx(&full[s], (uint32_t)(2 * PT * HD * 2));
+        }
 #pragma unroll
         for (int h = 0; h < HD / 64; ++h) {
-            tc::tma_load_2d(kd + h * PT * 128, map_kv_ptr, h * 64, (int)rk, &full[s]);
-            tc::tma_load_2d(vd + h * PT * 128, map_kv_ptr, h * 64, (int)rv, &full[s]);
+            if (which & 1) tc::tma_load_2d(kd + h * PT * 128, map_kv_ptr, h * 64, (int)rk, &full[SPLIT ? 0 : s]);
+            if (which & 2) tc::tma_load_2d(vd + h * PT * 128, map_kv_ptr, h * 64, (int)rv, &full[SPLIT ? 1 : s]);
         }
     };
     if (!in_pass && tid == 0)
-        for (int t = 0; t < min(n_tiles, STAGES); ++t) issue(t);
+        for (int t = 0; t < min(n_tiles, SPLIT ? 1 : STAGES); ++t) issue(t, 3);
 
     // ---- Q tiles (both terms): global -> swizzled shared ----
     {
@@ -535,14 +548,16 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     const uint32_t idesc_s = umma_idesc(64, 0), idesc_o = umma_idesc(HD, 1);
 
     for (int t = 0; t < n_tiles; ++t) {
-        const int s = in_pass ? 0 : (int)((ring0 + t) % STAGES);
-        bool ok = in_pass || tc::mbar_wait(&full[s], ((ring0 + t) / STAGES) & 1);
+        const int s = (in_pass || SPLIT) ? 0 : (int)((ring0 + t) % STAGES);
+        // the tile (SPLIT: its K) has landed
+        bool ok = in_pass || tc::mbar_wait(&full[s], SPLIT ? ((ring0 + t) & 1) : (((ring0 + t) / STAGES) & 1));
         if (group_or(bar_id, THREADS, !ok)) {
             failed = true;
             break;
         }
         const uint32_t kb = tc::smem_u32(kv_s + (size_t)s * 2 * tile_bytes);
         const uint32_t vb = kb + tile_bytes;
+        uint8_t* p_tile = SPLIT ? base : kv_s + (size_t)s * 2 * tile_bytes;   // P_hi | P_lo: own tile, or over the dead K tile
         if (tid == 0) {
             // ---- S = (Q_hi + Q_lo) K^T: two terms x two 64-column halves of head_dim x four k-steps ----
             tc::tc_fence_after();
@@ -567,7 +582,14 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         tc::tc_fence_after();
         // The commit above also covers the previous tile's P V MMAs: P, the other stage and the
         // output accumulator are free to be rewritten.
-        if (!in_pass && tid == 0 && t >= 1 && t + 1 < n_tiles) issue(t + 1);
+        if (!in_pass && tid == 0) {
+            if (SPLIT) {
+                if (t + 1 < n_tiles) issue(t + 1, 1);      // K is free: S is complete
+                if (t >= 1) issue(t, 2);                   // V is free: the previous P V is complete; this tile's V is needed after the softmax
+            } else if (t >= 1 && t + 1 < n_tiles) {
+                issue(t + 1, 3);
+            }
+        }
         float alpha = 1.f;
         if (row_thread) {
             // ---- this row's scores: mask, running maximum and sum (log2 domain), probabilities ----
@@ -597,7 +619,7 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
             alpha = m_new == m_run ? 1.f : exp2f(m_run - ref);
             m_run = m_new;
             float sum = 0.f, sum1 = 0.f;
-            uint8_t* ph = kv_s + (size_t)s * 2 * tile_bytes + tid * 128;      // P_hi | P_lo over the K tile, which S no longer needs
+            uint8_t* ph = p_tile + tid * 128;
             const float neg_ref = -ref;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -635,11 +657,19 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         }
         tc::tc_fence_before();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        group_sync(bar_id, THREADS);
+        if (SPLIT && !in_pass) {       // this tile's V has landed (the barrier below makes the group agree)
+            ok = tc::mbar_wait(&full[1], (ring0 + t) & 1);
+            if (group_or(bar_id, THREADS, !ok)) {
+                failed = true;
+                break;
+            }
+        } else {
+            group_sync(bar_id, THREADS);
+        }
         if (tid == 0) {
             // ---- O += (P_hi + P_lo) V: two terms x four k-steps of 16 keys ----
             tc::tc_fence_after();
-            const uint32_t pb = kb;
+            const uint32_t pb = tc::smem_u32(p_tile);
 #pragma unroll
             for (int term = 0; term < 2; ++term) {
                 const uint64_t a = smem_desc_sw128_k(pb + term * (QT * 128));
@@ -707,7 +737,7 @@ static __global__ void __launch_bounds__(THREADS) attn_umma_kernel(const __grid_
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     uint32_t ring_pos = 0, s_cnt = 0, o_cnt = 0;
-    bool ok = attn_item_umma(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, bars, tmem, ring_pos, s_cnt, o_cnt, threadIdx.x, 0);
+    bool ok = attn_item_umma<false>(&map_kv, p, blockIdx.x, blockIdx.y, blockIdx.z, base, bars, tmem, ring_pos, s_cnt, o_cnt, threadIdx.x, 0);
     if (!ok && threadIdx.x == 0) {
         // copies already issued target this CTA's shared memory: give them one more bounded wait
         for (int s = 0; s < STAGES; ++s) tc::mbar_wait(&bars[s], 0);

@@ -43,6 +43,7 @@ constexpr int THREADS = 256;
 constexpr int CTHREADS = 128;        // compute warps 4..7
 constexpr int BAR_COMPUTE = 1;       // named barrier of the compute warps
 constexpr int ACC_STRIDE = 128;      // tensor-memory columns per accumulator buffer (2 T: high and low halves)
+constexpr int TMEM_COLS = 512;       // two accumulator buffers, then 64 columns of attention scores and 128 of attention output
 constexpr int MAX_T = 64;            // most token rows of a pass
 constexpr int W_TILE_BYTES = tc::BLOCK_N * 128;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
@@ -459,7 +460,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     uint64_t* acc_full = empty + S;
     uint64_t* acc_empty = acc_full + 2;
     uint64_t* kv_full = acc_empty + 2;
-    uint32_t* tmem_slot = (uint32_t*)(kv_full + att::STAGES);
+    uint32_t* tmem_slot = (uint32_t*)(kv_full + att::STAGES + 2);     // + the "scores ready" and "output ready" barriers of the tcgen05 attention items
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     volatile int* w_issued = abort_flag + 1;
     volatile int* x_issued = w_issued + 1;
@@ -478,7 +479,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             tc::mbar_init(&acc_full[b], 1);
             tc::mbar_init(&acc_empty[b], 4);
         }
-        for (int s = 0; s < att::STAGES; ++s) tc::mbar_init(&kv_full[s], 1);
+        for (int s = 0; s < att::STAGES + 2; ++s) tc::mbar_init(&kv_full[s], 1);
         *abort_flag = 0;
         *w_issued = 0;
         *x_issued = 0;
@@ -488,7 +489,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 2) {
-        tc::tmem_alloc(tmem_slot, 2 * ACC_STRIDE);
+        tc::tmem_alloc(tmem_slot, TMEM_COLS);
         tc::tmem_relinquish();
     }
     tc::tc_fence_before();
@@ -649,7 +650,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // ---------------- compute warps ----------------
         const int tid = threadIdx.x - (THREADS - CTHREADS), cw = tid >> 5;
         unsigned epoch = 0;
-        uint32_t seg = 0, kv_ring = 0;
+        uint32_t seg = 0, kv_ring = 0, attn_s_cnt = 0, attn_o_cnt = 0;
         bool ok = true;
         const int M = p.M, d = p.d;
         const int d_tiles = d / tc::BLOCK_N;
@@ -874,8 +875,19 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 for (int i = ap.sched_off ? __ldg(ap.sched_off + cta) : cta; i < i_end && ok; i += ap.sched_off ? 1 : G) {
                     const int idx = ap.sched_off ? __ldg(ap.sched_items + i) : i;
                     const int split = idx % n_splits, r = idx / n_splits;
-                    if (!att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
-                                            kv_ring, tid, BAR_COMPUTE)) {
+                    bool fine;
+                    if constexpr (HD == 128) {
+                        // 64-token pages: the work item runs on tcgen05 (scores and output in tensor memory)
+                        fine = ap.page_tokens == 64
+                                   ? att::attn_item_umma<true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
+                                                               tmem_base + 2 * ACC_STRIDE, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE)
+                                   : att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
+                                                              kv_ring, tid, BAR_COMPUTE);
+                    } else {
+                        fine = att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full, kv_ring,
+                                                        tid, BAR_COMPUTE);
+                    }
+                    if (!fine) {
                         ok = false;
                         *abort_flag = 1;
                     }
@@ -1292,7 +1304,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         for (int k = 0; k < 1000; ++k) __nanosleep(1000);   // copies whose partner never came have no barrier to wait on
     }
     __syncthreads();
-    if (warp == 2) tc::tmem_dealloc(tmem_base, 2 * ACC_STRIDE);
+    if (warp == 2) tc::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 }  // namespace pp
