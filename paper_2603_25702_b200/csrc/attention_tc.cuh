@@ -90,6 +90,15 @@ __device__ __forceinline__ bool group_or(int id, int n, bool pred) {
     return r != 0;
 }
 __device__ __forceinline__ uint4 ldcg16(const void* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
+// x / d for 0 <= x < 2^20 and a small run-time d by one multiplication (an integer division is about 40
+// dependent instructions, which a thread that has its scheduler to itself pays in full)
+__device__ __forceinline__ int fast_div(int x, int d, float inv_d) {
+    int q = (int)(((float)x + 0.5f) * inv_d);
+    const int r = x - q * d;
+    if (r < 0) --q;
+    else if (r >= d) ++q;
+    return q;
+}
 
 // One work item (sequence z / Hkv, kv head z % Hkv, query tile qt, key split) of the attention
 // step, run by a group of 128 threads (`tid` 0..127, barrier `bar_id`).  `base` is 1024-byte
@@ -434,10 +443,41 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 // tile of the same region), the two "tile landed" barriers being K's and
 // V's.  The next K is requested as soon as S is complete and the next V as soon as the previous
 // P V is, so both arrive behind the softmax of the tile in between.
+// SPLIT layout: the K and V tiles of a cache-split item's first page do not depend on anything the
+// current pass computes, so a kernel that knows its next item can request them long before it
+// reaches the item (the tiles must be free: the previous item of the group has ended).  Every thread
+// of the group evaluates the same condition, thread 0 issues the copies.  Returns whether the
+// request was made; the item is then entered with first_requested = true.
+__device__ __forceinline__ bool attn_umma_request_first(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
+                                                        uint8_t* base, uint64_t* bars, uint32_t ring_pos, int tid) {
+    constexpr int HD = 128, PT = 64, tile_bytes = 64 * HD * 2;
+    const int seq = z / p.Hkv, kvh = z % p.Hkv;
+    if (qt * QT >= p.pv.seq_nrows[seq] * p.group || split == p.n_cache_splits) return false;
+    const int n_pages = (p.pv.seq_nctx[seq] + PT - 1) >> p.page_shift;
+    const int pg0 = split * p.pages_per_split;
+    if (pg0 >= n_pages) return false;
+    if (tid == 0) {
+        uint8_t* kd = base + 2 * QT * 128 + 2 * QT * HD * 2;      // behind P and Q
+        uint8_t* vd = kd + tile_bytes;
+        const int page = p.pv.seq_pages[(size_t)seq * p.pv.max_pages + pg0];
+        const long long rk = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 0) * p.Hkv + kvh) * PT;
+        const long long rv = ((((long long)p.layer * p.n_pages_pool + page) * 2 + 1) * p.Hkv + kvh) * PT;
+        tc::mbar_expect_tx(&bars[0], (uint32_t)(PT * HD * 2));
+        tc::mbar_expect_tx(&bars[1], (uint32_t)(PT * HD * 2));
+#pragma unroll
+        for (int h = 0; h < HD / 64; ++h) {
+            tc::tma_load_2d(kd + h * PT * 128, map_kv_ptr, h * 64, (int)rk, &bars[0]);
+            tc::tma_load_2d(vd + h * PT * 128, map_kv_ptr, h * 64, (int)rv, &bars[1]);
+        }
+    }
+    (void)ring_pos;
+    return true;
+}
+// first_requested: tile 0 of this item was already requested by attn_umma_request_first.
 template <bool SPLIT>
 __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
                                                uint8_t* base, uint64_t* bars, uint32_t tmem, uint32_t& ring_pos, uint32_t& s_cnt,
-                                               uint32_t& o_cnt, int tid, int bar_id) {
+                                               uint32_t& o_cnt, int tid, int bar_id, bool first_requested = false) {
     constexpr int HD = 128, CH = HD / 8, PT = 64;
     constexpr int tile_bytes = 64 * HD * 2;
     uint8_t* q_s = base + (SPLIT ? 2 * QT * 128 : 0);      // Q_hi, Q_lo: [QT][HD] each
@@ -447,7 +487,8 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     uint64_t* bar_o = bars + STAGES + 1;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 64;
 
-    const int seq = z / p.Hkv, kvh = z % p.Hkv;
+    const int seq = fast_div(z, p.Hkv, 1.0f / (float)p.Hkv), kvh = z - seq * p.Hkv;
+    const float inv_group = 1.0f / (float)p.group;
     const int nrows = p.pv.seq_nrows[seq], row0 = p.pv.seq_row0[seq];
     const int nq = nrows * p.group;
     const int q0 = qt * QT;
@@ -486,7 +527,7 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         }
     };
     if (!in_pass && tid == 0)
-        for (int t = 0; t < min(n_tiles, SPLIT ? 1 : STAGES); ++t) issue(t, 3);
+        for (int t = first_requested ? 1 : 0; t < min(n_tiles, SPLIT ? 1 : STAGES); ++t) issue(t, 3);
 
     // ---- Q tiles (both terms): global -> swizzled shared ----
     {
@@ -498,7 +539,8 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
             hi[k] = make_uint4(0, 0, 0, 0);
             lo[k] = hi[k];
             if (qv < nq) {
-                const int row = row0 + qv / p.group, hq = kvh * p.group + qv % p.group;
+                const int qr = fast_div(qv, p.group, inv_group);
+                const int row = row0 + qr, hq = kvh * p.group + (qv - qr * p.group);
                 hi[k] = ldcg16(p.q + ((size_t)row * p.Hq + hq) * HD + c * 8);
                 lo[k] = ldcg16(p.q_lo + ((size_t)row * p.Hq + hq) * HD + c * 8);
             }
@@ -541,7 +583,7 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     const bool row_thread = tid < QT;                       // warps 0 and 1: thread = query row = TMEM lane
     const int qv = q0 + tid;
     unsigned long long row_mask = 0;
-    if (in_pass && row_thread && qv < nq) row_mask = p.pv.row_mask[row0 + qv / p.group];
+    if (in_pass && row_thread && qv < nq) row_mask = p.pv.row_mask[row0 + fast_div(qv, p.group, inv_group)];
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     float m_run = -INFINITY, l_run = 0.f;
     bool failed = false;
@@ -699,16 +741,16 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         pml[0] = m_run;
         pml[1] = l_run;
 #pragma unroll
-        for (int c = 0; c < HD; c += 16) {
-            float o[16];
+        for (int c = 0; c < HD; c += 32) {
+            float o[32];
             if (n_tiles > 0) {
-                tc::tmem_ld16(tmem_o + lane_base + c, o);
+                tc::tmem_ld32(tmem_o + lane_base + c, o);
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[j] = 0.f;
+                for (int j = 0; j < 32; ++j) o[j] = 0.f;
             }
 #pragma unroll
-            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(po + c + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4*>(po + c + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
         }
     }
     // the accumulators are read: the next item's MMAs may overwrite them; shared memory is reused too

@@ -777,6 +777,29 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
 
         for (int l = 0; l < p.n_layers && ok; ++l) {
             const LayerGains lg = p.gains[l];
+            // First attention item of this CTA in this layer: its first K/V page is in the cache already, so the
+            // copies are started now and land behind the QKV GEMM (tcgen05 items only).
+            bool attn_first_requested = false;
+            int attn_first = -1;
+            if constexpr (HD == 128) {
+                if (p.ap.page_tokens == 64) {
+                    att::AttnParams ap0 = p.ap;
+                    ap0.layer = l;
+                    const int n_splits0 = ap0.n_cache_splits + 1;
+                    const int total0 = ap0.pv.n_seqs * ap0.Hkv * ap0.n_qtiles * n_splits0;
+                    if (ap0.sched_off) {
+                        const int i0 = __ldg(ap0.sched_off + cta);
+                        if (i0 < __ldg(ap0.sched_off + cta + 1)) attn_first = __ldg(ap0.sched_items + i0);
+                    } else if (cta < total0) {
+                        attn_first = cta;
+                    }
+                    if (attn_first >= 0) {
+                        const int r0 = attn_first / n_splits0;
+                        attn_first_requested = att::attn_umma_request_first(p.maps + p.map_kv, ap0, attn_first % n_splits0, r0 % ap0.n_qtiles,
+                                                                            r0 / ap0.n_qtiles, attn_s, kv_full, kv_ring, tid);
+                    }
+                }
+            }
             // ---- QKV GEMM ----
             drain(l, K_QKV);
             if (!ok) break;
@@ -869,22 +892,26 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 ap.layer = l;
                 const int n_splits = ap.n_cache_splits + 1;
                 const int total = ap.pv.n_seqs * ap.Hkv * ap.n_qtiles * n_splits;
+                const FastDiv by_splits(n_splits), by_qtiles(ap.n_qtiles);
                 // Items of this CTA: a host-made list when the pass has several sequences (their context
                 // lengths differ, so items are dealt out by cost), else every G-th item.
                 const int i_end = ap.sched_off ? __ldg(ap.sched_off + cta + 1) : total;
                 for (int i = ap.sched_off ? __ldg(ap.sched_off + cta) : cta; i < i_end && ok; i += ap.sched_off ? 1 : G) {
                     const int idx = ap.sched_off ? __ldg(ap.sched_items + i) : i;
-                    const int split = idx % n_splits, r = idx / n_splits;
+                    int r, split, z_i, qt_i;
+                    by_splits.divmod(idx, r, split);
+                    by_qtiles.divmod(r, z_i, qt_i);
                     bool fine;
                     if constexpr (HD == 128) {
                         // 64-token pages: the work item runs on tcgen05 (scores and output in tensor memory)
                         fine = ap.page_tokens == 64
-                                   ? att::attn_item_umma<true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
-                                                               tmem_base + 2 * ACC_STRIDE, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE)
-                                   : att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full,
+                                   ? att::attn_item_umma<true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
+                                                               tmem_base + 2 * ACC_STRIDE, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE,
+                                                               attn_first_requested && idx == attn_first)
+                                   : att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
                                                               kv_ring, tid, BAR_COMPUTE);
                     } else {
-                        fine = att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, r % ap.n_qtiles, r / ap.n_qtiles, attn_s, kv_full, kv_ring,
+                        fine = att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full, kv_ring,
                                                         tid, BAR_COMPUTE);
                     }
                     if (!fine) {
