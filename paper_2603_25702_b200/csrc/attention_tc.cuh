@@ -474,10 +474,14 @@ __device__ __forceinline__ bool attn_umma_request_first(const CUtensorMap* map_k
     return true;
 }
 // first_requested: tile 0 of this item was already requested by attn_umma_request_first.
+// map_q (may be null): two 3D tensor maps of q's high and low halves viewed as [row, head, head_dim] with
+// boxes of (64 / group) rows x group heads x 64 columns; the Q tiles then arrive by TMA in query order (one more
+// barrier behind the two above, its phase in *q_cnt) instead of passing through registers.
 template <bool SPLIT>
 __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
                                                uint8_t* base, uint64_t* bars, uint32_t tmem, uint32_t& ring_pos, uint32_t& s_cnt,
-                                               uint32_t& o_cnt, int tid, int bar_id, bool first_requested = false) {
+                                               uint32_t& o_cnt, int tid, int bar_id, bool first_requested = false,
+                                               const CUtensorMap* map_q = nullptr, uint32_t* q_cnt = nullptr) {
     constexpr int HD = 128, CH = HD / 8, PT = 64;
     constexpr int tile_bytes = 64 * HD * 2;
     uint8_t* q_s = base + (SPLIT ? 2 * QT * 128 : 0);      // Q_hi, Q_lo: [QT][HD] each
@@ -529,8 +533,20 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     if (!in_pass && tid == 0)
         for (int t = first_requested ? 1 : 0; t < min(n_tiles, SPLIT ? 1 : STAGES); ++t) issue(t, 3);
 
-    // ---- Q tiles (both terms): global -> swizzled shared ----
-    {
+    // ---- Q tiles (both terms): by TMA, or global -> registers -> swizzled shared ----
+    const bool q_tma = map_q != nullptr && n_tiles > 0;
+    if (q_tma) {
+        if (tid == 0) {
+            uint64_t* bar_q = bars + STAGES + 2;
+            tc::mbar_expect_tx(bar_q, (uint32_t)(2 * QT * HD * 2));
+            const int r_first = row0 + qt * (QT / p.group);
+#pragma unroll
+            for (int term = 0; term < 2; ++term)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    tc::tma_load_3d(q_s + term * (QT * HD * 2) + h * (QT * 128), map_q + term, h * 64, kvh * p.group, r_first, bar_q);
+        }
+    } else {
         constexpr int NQ = QT * CH / THREADS;
         uint4 hi[NQ], lo[NQ];
 #pragma unroll
@@ -593,6 +609,10 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         const int s = (in_pass || SPLIT) ? 0 : (int)((ring0 + t) % STAGES);
         // the tile (SPLIT: its K) has landed
         bool ok = in_pass || tc::mbar_wait(&full[s], SPLIT ? ((ring0 + t) & 1) : (((ring0 + t) / STAGES) & 1));
+        if (q_tma && t == 0) {      // the Q tiles have landed
+            ok = tc::mbar_wait(bars + STAGES + 2, *q_cnt & 1) && ok;
+            ++*q_cnt;
+        }
         if (group_or(bar_id, THREADS, !ok)) {
             failed = true;
             break;

@@ -203,6 +203,19 @@ int gemm_encode_map(s2d2_ctx* c, void* out, const void* ptr, unsigned long long 
     return r == CUDA_SUCCESS ? 0 : (int)r;
 }
 
+int gemm_encode_map3(s2d2_ctx* c, void* out, const void* ptr, int cols, int mid, unsigned long long rows, int box_mid, int box_rows) {
+    GemmState* g = state(c);
+    if (!g || !g->encode) return -1;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)mid, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)mid};
+    cuuint32_t box[3] = {64u, (cuuint32_t)box_mid, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g->encode((CUtensorMap*)out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : (int)r;
+}
+
 void gemm_forget(s2d2_ctx* c, const void* ptr) {
     GemmState* g = state(c);
     if (!g) return;

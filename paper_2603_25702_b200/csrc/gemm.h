@@ -16,4 +16,6 @@ void gemm_forget(s2d2_ctx* c, const void* ptr);
 // 2D bf16 tensor map [rows, cols] with boxes of box_rows x 64 columns and the 128-byte swizzle.
 // `out` points to a CUtensorMap (128 bytes). Returns 0 on success.
 int gemm_encode_map(s2d2_ctx* c, void* out, const void* ptr, unsigned long long rows, int cols, int box_rows);
+// 3D bf16 tensor map [rows, mid, cols] (cols contiguous) with boxes of box_rows x box_mid x 64 columns, 128-byte swizzle.
+int gemm_encode_map3(s2d2_ctx* c, void* out, const void* ptr, int cols, int mid, unsigned long long rows, int box_mid, int box_rows);
 bool gemm_tc_available(s2d2_ctx* c);

@@ -29,6 +29,7 @@ struct PassState {
     int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act; then their low halves
     int map_act_e = 0;           // per T: experts' SwiGLU output, high halves then low halves
     int map_kv = 0;
+    bool q_by_tma = false;       // maps map_kv + 1 / + 2: q high and low halves as 3D boxes
     CUtensorMap* d_maps = nullptr;
     pp::LayerGains* d_gains = nullptr;
     float* ws = nullptr;
@@ -185,7 +186,7 @@ int pass_init(s2d2_ctx* c) {
     s->map_x0 = L * s->maps_per_layer + 1;
     s->map_act_e = s->map_x0 + 24;
     s->map_kv = s->map_act_e + 8;
-    std::vector<CUtensorMap> maps(s->map_kv + 1);
+    std::vector<CUtensorMap> maps(s->map_kv + 3);      // KV pool, then q (high and low halves) as [row, head, head_dim] for the attention items
     auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
         return gemm_encode_map(c, &maps[idx], ptr, rows, cols, box_rows) == 0;
     };
@@ -249,6 +250,14 @@ int pass_init(s2d2_ctx* c) {
         const void* mk = nullptr;
         if (!attention_plan(c, dummy, 1, 1, 0, &ap, &mk) || !mk) return S2D2_OK;
         maps[s->map_kv] = *(const CUtensorMap*)mk;
+    }
+    {
+        // A tile of 64 query vectors of one kv head is a box of (64 / group) rows x group heads: TMA writes it in query order
+        const int group = m.n_q_heads / m.n_kv_heads;
+        s->q_by_tma = m.head_dim == 128 && att::QT % group == 0 && group <= att::QT;
+        if (s->q_by_tma)
+            s->q_by_tma = gemm_encode_map3(c, &maps[s->map_kv + 1], c->q, m.head_dim, m.n_q_heads, c->max_rows, group, att::QT / group) == 0 &&
+                          gemm_encode_map3(c, &maps[s->map_kv + 2], s->q_lo, m.head_dim, m.n_q_heads, c->max_rows, group, att::QT / group) == 0;
     }
     // ---- per GEMM kind: shape, split-K workspace region, publish counters, part tables ----
     // N < 0 marks a kind this model does not run; for the two routed-expert GEMMs N is the largest (all experts touched).
@@ -332,6 +341,7 @@ int pass_init(s2d2_ctx* c) {
     size_t es = 2;
     cudaMemset(c->xn, 0, (size_t)c->max_rows * d * es);
     cudaMemset(c->attn, 0, (size_t)c->max_rows * nq * es);
+    cudaMemset(c->q, 0, (size_t)c->max_rows * nq * es);       // a Q tile fetched by TMA covers 64 / group rows, also past the sequence's own
     cudaMemset(c->act, 0, (size_t)c->max_rows * f * es);
     s->ok = true;
     return S2D2_OK;
@@ -445,6 +455,7 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.map_act = s->map_x0 + 8 + ti;
     p.map_act_e = s->map_act_e + ti;
     p.map_kv = s->map_kv;
+    p.map_q = s->q_by_tma ? s->map_kv + 1 : -1;
     p.barrier = s->barrier;
     p.status = c->d_status;
     p.S = stages_for(s, p.T, m.head_dim);

@@ -89,6 +89,7 @@ struct PassParams {
     KvPool<bf16> pool;
     const CUtensorMap* maps;  // device array: weights [n_layers*4 + 1], then the entries below
     int map_xn, map_attn, map_act, map_kv;
+    int map_q;                  // first of the two 3D maps of q (high, low halves) for the attention items, or -1
     att::AttnParams ap;       // attention geometry of this pass (layer filled in per layer)
     unsigned* barrier;        // grid barrier counter, zero at launch
     unsigned* tile_cnt[N_KINDS];    // per GEMM kind and weight tile: partials published so far (zero at launch)
@@ -460,7 +461,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     uint64_t* acc_full = empty + S;
     uint64_t* acc_empty = acc_full + 2;
     uint64_t* kv_full = acc_empty + 2;
-    uint32_t* tmem_slot = (uint32_t*)(kv_full + att::STAGES + 2);     // + the "scores ready" and "output ready" barriers of the tcgen05 attention items
+    uint32_t* tmem_slot = (uint32_t*)(kv_full + att::STAGES + 3);     // + the "scores ready" and "output ready" barriers of the tcgen05 attention items
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     volatile int* w_issued = abort_flag + 1;
     volatile int* x_issued = w_issued + 1;
@@ -479,7 +480,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             tc::mbar_init(&acc_full[b], 1);
             tc::mbar_init(&acc_empty[b], 4);
         }
-        for (int s = 0; s < att::STAGES + 2; ++s) tc::mbar_init(&kv_full[s], 1);
+        for (int s = 0; s < att::STAGES + 3; ++s) tc::mbar_init(&kv_full[s], 1);
         *abort_flag = 0;
         *w_issued = 0;
         *x_issued = 0;
@@ -650,7 +651,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // ---------------- compute warps ----------------
         const int tid = threadIdx.x - (THREADS - CTHREADS), cw = tid >> 5;
         unsigned epoch = 0;
-        uint32_t seg = 0, kv_ring = 0, attn_s_cnt = 0, attn_o_cnt = 0;
+        uint32_t seg = 0, kv_ring = 0, attn_s_cnt = 0, attn_o_cnt = 0, attn_q_cnt = 0;
         bool ok = true;
         const int M = p.M, d = p.d;
         const int d_tiles = d / tc::BLOCK_N;
@@ -907,7 +908,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         fine = ap.page_tokens == 64
                                    ? att::attn_item_umma<true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
                                                                tmem_base + 2 * ACC_STRIDE, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE,
-                                                               attn_first_requested && idx == attn_first)
+                                                               attn_first_requested && idx == attn_first,
+                                                               p.map_q >= 0 ? p.maps + p.map_q : nullptr, &attn_q_cnt)
                                    : att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
                                                               kv_ring, tid, BAR_COMPUTE);
                     } else {
