@@ -476,7 +476,9 @@ __device__ __forceinline__ bool attn_umma_request_first(const CUtensorMap* map_k
 // first_requested: tile 0 of this item was already requested by attn_umma_request_first.
 // map_q (may be null): two 3D tensor maps of q's high and low halves viewed as [row, head, head_dim] with
 // boxes of (64 / group) rows x group heads x 64 columns; the Q tiles then arrive by TMA in query order (one more
-// barrier behind the two above, its phase in *q_cnt) instead of passing through registers.
+// barrier behind the two above, its phase in *q_cnt) instead of passing through registers.  In the SPLIT layout
+// map_q[2] and map_q[3] are the same views of this pass's K and V rows (boxes of 64 rows x 1 head): the in-pass
+// tile is then fetched like a page.
 template <bool SPLIT>
 __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, const AttnParams& p, int split, int qt, int z,
                                                uint8_t* base, uint64_t* bars, uint32_t tmem, uint32_t& ring_pos, uint32_t& s_cnt,
@@ -505,8 +507,9 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     const int n_tiles = in_pass ? 1 : max(0, pg1 - pg0);
     const size_t item = ((size_t)z * p.n_qtiles + qt) * (p.n_cache_splits + 1) + split;
     const int warp = tid >> 5;
+    const bool kv_tma = SPLIT && in_pass && map_q != nullptr;      // the in-pass tile arrives by TMA on the K and V barriers
     const uint32_t ring0 = ring_pos;
-    if (!in_pass) ring_pos += (uint32_t)n_tiles;
+    if (!in_pass || kv_tma) ring_pos += (uint32_t)n_tiles;
 
     const int* pages = p.pv.seq_pages + (size_t)seq * p.pv.max_pages;
     // thread 0: TMA of cache tile t of this split.  which: bit 0 = K, bit 1 = V.  Two-stage layout: both into
@@ -568,7 +571,18 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
             *reinterpret_cast<uint4*>(q_s + QT * HD * 2 + sw_off(r, c, QT)) = lo[k];
         }
     }
-    if (in_pass) {
+    if (kv_tma) {
+        // rows past the sequence's own are other rows of the pass: their keys are masked below
+        if (tid == 0) {
+            tc::mbar_expect_tx(&full[0], (uint32_t)(PT * HD * 2));
+            tc::mbar_expect_tx(&full[1], (uint32_t)(PT * HD * 2));
+#pragma unroll
+            for (int h = 0; h < HD / 64; ++h) {
+                tc::tma_load_3d(kv_s + h * PT * 128, map_q + 2, h * 64, kvh, row0, &full[0]);
+                tc::tma_load_3d(kv_s + tile_bytes + h * PT * 128, map_q + 3, h * 64, kvh, row0, &full[1]);
+            }
+        }
+    } else if (in_pass) {
         // K and V of this pass's rows of the sequence into stage 0 (rows past nrows are zero)
         uint8_t* kd = kv_s;
         uint8_t* vd = kd + tile_bytes;
@@ -608,7 +622,7 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
     for (int t = 0; t < n_tiles; ++t) {
         const int s = (in_pass || SPLIT) ? 0 : (int)((ring0 + t) % STAGES);
         // the tile (SPLIT: its K) has landed
-        bool ok = in_pass || tc::mbar_wait(&full[s], SPLIT ? ((ring0 + t) & 1) : (((ring0 + t) / STAGES) & 1));
+        bool ok = (in_pass && !kv_tma) || tc::mbar_wait(&full[s], SPLIT ? ((ring0 + t) & 1) : (((ring0 + t) / STAGES) & 1));
         if (q_tma && t == 0) {      // the Q tiles have landed
             ok = tc::mbar_wait(bars + STAGES + 2, *q_cnt & 1) && ok;
             ++*q_cnt;
@@ -719,7 +733,7 @@ __device__ __forceinline__ bool attn_item_umma(const CUtensorMap* map_kv_ptr, co
         }
         tc::tc_fence_before();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (SPLIT && !in_pass) {       // this tile's V has landed (the barrier below makes the group agree)
+        if (SPLIT && (!in_pass || kv_tma)) {       // this tile's V has landed (the barrier below makes the group agree)
             ok = tc::mbar_wait(&full[1], (ring0 + t) & 1);
             if (group_or(bar_id, THREADS, !ok)) {
                 failed = true;

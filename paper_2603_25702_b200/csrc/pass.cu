@@ -186,7 +186,7 @@ int pass_init(s2d2_ctx* c) {
     s->map_x0 = L * s->maps_per_layer + 1;
     s->map_act_e = s->map_x0 + 24;
     s->map_kv = s->map_act_e + 8;
-    std::vector<CUtensorMap> maps(s->map_kv + 3);      // KV pool, then q (high and low halves) as [row, head, head_dim] for the attention items
+    std::vector<CUtensorMap> maps(s->map_kv + 5);      // KV pool, then q (high and low halves) and this pass's K and V rows as [row, head, head_dim] for the attention items
     auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
         return gemm_encode_map(c, &maps[idx], ptr, rows, cols, box_rows) == 0;
     };
@@ -257,7 +257,9 @@ int pass_init(s2d2_ctx* c) {
         s->q_by_tma = m.head_dim == 128 && att::QT % group == 0 && group <= att::QT;
         if (s->q_by_tma)
             s->q_by_tma = gemm_encode_map3(c, &maps[s->map_kv + 1], c->q, m.head_dim, m.n_q_heads, c->max_rows, group, att::QT / group) == 0 &&
-                          gemm_encode_map3(c, &maps[s->map_kv + 2], s->q_lo, m.head_dim, m.n_q_heads, c->max_rows, group, att::QT / group) == 0;
+                          gemm_encode_map3(c, &maps[s->map_kv + 2], s->q_lo, m.head_dim, m.n_q_heads, c->max_rows, group, att::QT / group) == 0 &&
+                          gemm_encode_map3(c, &maps[s->map_kv + 3], c->k_rows, m.head_dim, m.n_kv_heads, c->max_rows, 1, 64) == 0 &&
+                          gemm_encode_map3(c, &maps[s->map_kv + 4], c->v_rows, m.head_dim, m.n_kv_heads, c->max_rows, 1, 64) == 0;
     }
     // ---- per GEMM kind: shape, split-K workspace region, publish counters, part tables ----
     // N < 0 marks a kind this model does not run; for the two routed-expert GEMMs N is the largest (all experts touched).
@@ -342,6 +344,8 @@ int pass_init(s2d2_ctx* c) {
     cudaMemset(c->xn, 0, (size_t)c->max_rows * d * es);
     cudaMemset(c->attn, 0, (size_t)c->max_rows * nq * es);
     cudaMemset(c->q, 0, (size_t)c->max_rows * nq * es);       // a Q tile fetched by TMA covers 64 / group rows, also past the sequence's own
+    cudaMemset(c->k_rows, 0, (size_t)c->max_rows * m.n_kv_heads * m.head_dim * es);      // likewise the 64 in-pass key rows
+    cudaMemset(c->v_rows, 0, (size_t)c->max_rows * m.n_kv_heads * m.head_dim * es);
     cudaMemset(c->act, 0, (size_t)c->max_rows * f * es);
     s->ok = true;
     return S2D2_OK;
