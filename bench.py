@@ -155,7 +155,7 @@ def model_pass_bytes(m):
 # capture summarised in profiles/pass_kernel_c2.md, as a ratio to the launch's algorithmic bytes; the
 # capture is of the 1.7B-class shape (a few GB on the device) and is scaled by algorithmic bytes, which
 # the traffic follows (weights dominate both).  Set to None when the kernel changes until it is re-captured.
-PASS_TRAFFIC_RATIO = 1.015
+PASS_TRAFFIC_RATIO = 1.011
 
 
 def pass_traffic_bytes(m, algorithmic_bytes_per_launch):
