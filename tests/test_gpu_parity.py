@@ -246,3 +246,26 @@ def test_accept_override_replaces_only_the_accept_probability():
         assert [(r.n_accepted, r.first_reject, r.resampled_id) for r in ra] == [(r.n_accepted, r.first_reject, r.resampled_id) for r in rb]
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("tc", [1, 2])
+def test_attention_items_that_span_several_pages(tc):
+    """Eight sequences with 1100-1300 cached tokens on the head_dim-128 test model: with 16 (sequence, kv head)
+    pairs and about 20 pages each the key splits hold two 64-token pages, so every cache item of the tcgen05
+    attention runs its tile loop more than once (next K requested when the scores are complete, next V when the
+    previous P V is, lazily rescaled accumulator), and the items are dealt out by cost.  tc = 1: the persistent
+    kernel's 80 KB layout; tc = 2: the two-stage layout of the per-operation kernel."""
+    from tests.parity_util import run_steps
+    wl = get_config("t_bf16_128", batch=8, prompt_len=(1100, 1300), gen_tokens=16, block_size=4)      # 8 x 2 x 4 = 64 verifier rows
+    assert wl.kv_page_tokens == 64 and wl.model.head_dim == 128
+    W = generate_weights(wl.model, seed=2, gain_jitter=0.1)
+    e, ids, prompts = _start(wl, W, use_tensor_cores=tc)
+    e.reset_counters()
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=2, logit_atol=2e-2,
+                    stage_b_seqs={ids[0], ids[3], ids[7]})
+    print("pages", tc, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps == 2 * len(ids) and rep.stage_b_passes >= 6
+    launches = e.get_counters().n_kernel_launches
+    assert (launches < 40) if tc == 1 else (launches > 40)       # persistent passes, or one kernel per operation
+    e.close()
