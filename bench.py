@@ -331,7 +331,7 @@ def main():
                        "near_boundary": int(cnt.n_near_boundary),
                        "accepted_len_hist": [int(x) for x in list(cnt.accepted_len_hist)[:B + 1]]},
         "shaped": shaped,
-        "setup_s": setup_s, "prefill_ms": c0.ms_prefill,
+        "setup_s": setup_s, "prefill_ms": c0.ms_prefill, "prefill_launches": int(c0.n_kernel_launches),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
