@@ -61,11 +61,12 @@ class OracleShadow:
 
 def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: int = 1, seed: Optional[int] = None,
               gamma: float = 1.0, tau_conf: float = 0.9, logit_atol: float = 2e-2, logit_rtol: float = 0.0,
-              route=None, shadows=None, stage_b_seqs=None) -> ParityReport:
+              route=None, shadows=None, stage_b_seqs=None, resample: bool = True) -> ParityReport:
     """Run up to ``n_steps`` decode steps on all sequences (stops when every one has
     generated wl.gen_tokens) and check both parity stages.  ``stage_b_seqs``: restrict the
     oracle's forward (stage B) to these sequence ids (large batches at full model size); stage A
-    always covers every sequence."""
+    always covers every sequence.  ``resample=False``: the reject-only variant (the first rejected position stays
+    masked and is drafted again in the next step)."""
     cfg, B = wl.model, wl.block_size
     MASK = cfg.mask_id
     seed = wl.philox_seed if seed is None else seed
@@ -125,7 +126,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
                 stream, stp = rng_streams[sid], bf["step"]
                 u = [philox.uniform(seed, s0 + j + i, stream, stp, philox.STREAM_ACCEPT) for i in range(L)]
                 u2 = [philox.uniform(seed, s0 + j + i, stream, stp, philox.STREAM_RESAMPLE) for i in range(L)]
-                o = A.accept_scan(my_d[:L], my_v, xhat[:L], u, u2, gamma)
+                o = A.accept_scan(my_d[:L], my_v, xhat[:L], u, u2, gamma, resample=resample)
                 near = sum(1 for m_ in o.margin_u if m_ < 1e-4)
                 rep.near_boundary += near
                 exempt = near > 0
@@ -139,7 +140,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
                             rep.mismatches.append(f"{tag}: a/u at {i}: {o.a[i]} {rs.a[i]} {u[i]} {rs.u[i]}")
                 for i in range(rs.n_accepted):
                     committed[j + i] = int(st.xhat[i])
-                if rs.first_reject >= 0:
+                if rs.first_reject >= 0 and resample:
                     committed[j + rs.first_reject] = rs.resampled_id
                 rep.verified_steps += 1
                 rep.n_accepted += rs.n_accepted

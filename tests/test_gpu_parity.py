@@ -269,3 +269,25 @@ def test_attention_items_that_span_several_pages(tc):
     launches = e.get_counters().n_kernel_launches
     assert (launches < 40) if tc == 1 else (launches > 40)       # persistent passes, or one kernel per operation
     e.close()
+
+
+@pytest.mark.parametrize("kw", [dict(ratio_gamma=0.5), dict(ratio_gamma=2.0), dict(resample=False)])
+def test_accept_variants_match_oracle(kw):
+    """Ratio tempering (accept iff u < min(1, (v/d)^gamma), Appendix "ratio tempering") and the reject-only
+    variant of the paper's failure-case study (no residual resampling: the rejected position stays masked and
+    is drafted again) against the oracle's acceptance arithmetic and forward, on the workload whose peaked
+    logits (scale 4) make rejections frequent."""
+    from tests.parity_util import run_steps
+    wl = get_config("c1")
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.0)
+    e, ids, prompts = _start(wl, W, **kw)
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=80, logit_atol=0.0, logit_rtol=1e-4,
+                    gamma=kw.get("ratio_gamma", 1.0), resample=kw.get("resample", True))
+    print(kw, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps > 0 and rep.n_committed > 0
+    assert rep.n_resampled > 0                                  # steps that ended in a rejection
+    if not kw.get("resample", True):
+        assert e.get_counters().n_resampled == 0
+        assert rep.n_committed == rep.n_accepted            # only accepted drafts are ever committed
+    e.close()
