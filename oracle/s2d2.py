@@ -89,12 +89,16 @@ class SequenceOracle:
 
     def __init__(self, W, cfg, block_size: int, seed: int, seq_stream: int,
                  route: Callable[[StepTrace], bool] = None, tau_conf: float = 0.9,
-                 draft_mode: str = "greedy", gamma: float = 1.0, keep_logits: bool = False):
+                 draft_mode: str = "greedy", gamma: float = 1.0, keep_logits: bool = False,
+                 resample: bool = True):
         self.W, self.cfg, self.B = W, cfg, block_size
         self.seed, self.seq_stream = seed, seq_stream
         self.route = route or (lambda st: len(st.span) >= 1)      # minimum-span policy, tau_span = 1
         self.tau_conf, self.draft_mode, self.gamma = tau_conf, draft_mode, gamma
         self.keep_logits = keep_logits
+        # False: the reject-only variant of the paper's failure-case study (Appendix, D2F LLaDA table): no residual
+        # resampling, the first rejected position stays masked and is drafted again in the next step
+        self.resample = resample
         self.tokens: List[int] = []       # finalised tokens before the current block
         self.cache: Optional[M.KV] = None
         self.n_c = 0                      # tokens whose K/V is cached
@@ -159,7 +163,7 @@ class SequenceOracle:
             self.n_verify_passes += 1
             st.u_accept = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_ACCEPT) for i in span]
             st.u_resample = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_RESAMPLE) for i in span]
-            res = A.accept_scan(logits[:L], vlogits, xhat, st.u_accept, st.u_resample, self.gamma)
+            res = A.accept_scan(logits[:L], vlogits, xhat, st.u_accept, st.u_resample, self.gamma, resample=self.resample)
             st.result = res
             if self.keep_logits:
                 st.verify_logits = vlogits
@@ -170,7 +174,7 @@ class SequenceOracle:
             if res.n_accepted:
                 self.cache = M.append_kv(self.cache, vkv, np.arange(res.n_accepted))
                 self.n_c += res.n_accepted
-            if res.first_reject >= 0:
+            if res.first_reject >= 0 and self.resample:
                 self.xb[j + res.first_reject] = int(res.resampled)
                 st.committed.append(j + res.first_reject)
                 st.committed_tokens.append(int(res.resampled))

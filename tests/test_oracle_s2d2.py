@@ -147,3 +147,36 @@ def test_sequences_are_independent_of_their_stream_only_through_uniforms(tiny_f3
     a = S.SequenceOracle(W, cfg, 4, seed=1, seq_stream=0).generate([1, 2, 3], 8)
     b = S.SequenceOracle(W, cfg, 4, seed=1, seq_stream=0).generate([1, 2, 3], 8)
     assert a == b
+
+
+def test_reject_only_commits_nothing_but_accepted_drafts(tiny_f32):
+    """Reject-only variant (no residual resampling): a step commits exactly its accepted prefix, the rejected
+    position stays masked and is drafted again with the same proposal (the context has not changed unless a
+    prefix was accepted) but fresh uniforms; the run still ends, and it agrees with the resampling run up to
+    the first rejection of either."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=5)[1][:6]
+    ro = S.SequenceOracle(W, cfg, block_size=8, seed=1, seq_stream=4, keep_logits=True, resample=False)
+    out = ro.generate(prompt, 24)
+    assert len(out) == 24
+    n_rej = n_empty = 0
+    for k, st in enumerate(ro.trace):
+        r = st.result
+        assert r.resampled == -1
+        assert st.committed == list(range(st.j, st.j + r.n_accepted))
+        assert st.committed_tokens == [int(x) for x in st.xhat[:r.n_accepted]]
+        if r.first_reject >= 0:
+            n_rej += 1
+            nxt = ro.trace[k + 1]
+            assert nxt.j == st.j + r.n_accepted                 # the rejected position is the next first masked one
+            if r.n_accepted == 0:
+                n_empty += 1
+                assert nxt.xhat == st.xhat and nxt.u_accept != st.u_accept
+    assert n_rej >= 1 and n_empty >= 1
+    ref = S.SequenceOracle(W, cfg, block_size=8, seed=1, seq_stream=4, keep_logits=True)
+    ref.generate(prompt, 24)
+    for a, b in zip(ro.trace, ref.trace):                       # identical until one of them rejects
+        assert a.xhat == b.xhat and a.result.n_accepted == b.result.n_accepted
+        if a.result.first_reject >= 0:
+            break
