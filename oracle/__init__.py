@@ -12,10 +12,14 @@ Pins (what each part is checked against, see tests/test_oracle_*.py):
   model.py    a separately written composition of torch fp64 library ops for a
               plain causal pass; RoPE shift invariance; cached == recomputed;
               MoE top-k == dense evaluation with zeroed gates; K/V of bf16 models held
-              as bfloat16 (the cache's storage format) == torch's bfloat16 conversion.
+              as bfloat16 (the cache's storage format): nearest bfloat16 of the fp64 value,
+              ties to even, == torch's bfloat16 conversion on fp32 inputs.
   accept.py   scipy logsumexp; closed forms of speculative sampling (exact
               enumeration on tiny vocabularies); brute-force inverse CDF.
-  s2d2.py     verifier rows of the 2L pass == L literal single-row passes;
+  s2d2.py     draft rows == Eq. (draft_mask) block by block for every first masked position and
+              every cached prefix, and draft logits on a cache == one literal pass over
+              prompt ++ block under the composed mask (three wrong masks fail both);
+              verifier rows of the 2L pass == L literal single-row passes;
               block size 1 == greedy autoregressive decoding; committed K/V ==
               K/V of a final causal pass over the finished block.
   routing.py  hand-computed values of the expected accepted prefix length.

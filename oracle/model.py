@@ -34,13 +34,23 @@ def widen(w: np.ndarray) -> np.ndarray:
 def as_stored_kv(x: np.ndarray, cfg) -> np.ndarray:
     """K and V as the cache holds them.  The cache of a bf16 model stores bfloat16 (the
     workloads name a "paged bf16 KV cache"), so for such a model K and V are bfloat16 values
-    wherever they are used: rounded once, to nearest even, where they are produced (after
-    RoPE for K).  fp32 models keep them unrounded in the oracle.  Returned widened to fp64."""
+    wherever they are used: rounded once, fp64 to the nearest bfloat16 with ties to even, where
+    they are produced (after RoPE for K).  The rounding works on the fp64 bit pattern (bfloat16
+    keeps 7 of the 52 fraction bits; a carry moves into the exponent by itself), so no fp32
+    value lies in between; below bfloat16's normal range the spacing is the fixed 2^-133.
+    fp32 models keep them unrounded in the oracle.  Returned as fp64."""
     if cfg.dtype != "bf16":
         return x
-    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
-    r = (u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))) & np.uint32(0xFFFF0000)
-    return r.view(np.float32).astype(np.float64)
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    u = x.view(np.uint64)
+    drop = np.uint64(45)
+    r = (u + (((u >> drop) & np.uint64(1)) + np.uint64((1 << 44) - 1))) & ~np.uint64((1 << 45) - 1)
+    out = r.view(np.float64).copy()
+    tiny = np.abs(x) < 2.0 ** -126
+    if tiny.any():
+        q = 2.0 ** -133
+        out[tiny] = np.rint(x[tiny] / q) * q
+    return out
 
 
 def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
@@ -113,13 +123,15 @@ def moe_ffn(x: np.ndarray, W: Dict[str, np.ndarray], prefix: str, cfg,
 def forward(W: Dict[str, np.ndarray], cfg, tokens, positions, inblock_mask,
             kv_prefix: Optional[KV] = None, need_logits=None,
             forced_expert_ids: Optional[List[np.ndarray]] = None,
-            trace: Optional[dict] = None):
+            trace: Optional[dict] = None, kv_storage: bool = True):
     """One pass of the network over R rows.
 
     tokens [R] (cfg.mask_id = MASK), positions [R], inblock_mask [R, R] bool
     (row r attends row c of this pass iff mask[r, c]); every row attends all of
     kv_prefix.  Returns (logits [R or len(need_logits), V], kv_rows) where
     kv_rows[l] = (K [R, Hkv, hd], V [R, Hkv, hd]) are this pass's own K/V.
+    kv_storage=False keeps K and V in fp64 even for a bf16 model (used only to measure how much
+    of a logit difference is the cache's storage format).
     """
     tokens = np.asarray(tokens, dtype=np.int64)
     positions = np.asarray(positions, dtype=np.int64)
@@ -139,8 +151,9 @@ def forward(W: Dict[str, np.ndarray], cfg, tokens, positions, inblock_mask,
             q = rmsnorm(q, widen(W[p + "q_norm"]), cfg.rms_eps)
             k = rmsnorm(k, widen(W[p + "k_norm"]), cfg.rms_eps)
         q = rope(q, positions, cfg.rope_base)
-        k = as_stored_kv(rope(k, positions, cfg.rope_base), cfg)
-        v = as_stored_kv(v, cfg)
+        k = rope(k, positions, cfg.rope_base)
+        if kv_storage:
+            k, v = as_stored_kv(k, cfg), as_stored_kv(v, cfg)
         kv_rows.append((k, v))
         if kv_prefix is not None and kv_prefix[l][0].shape[0] > 0:
             K_all = np.concatenate([kv_prefix[l][0], k], axis=0)

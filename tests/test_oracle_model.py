@@ -148,17 +148,30 @@ def test_moe_model_forward_runs_and_is_finite(tiny_moe):
 
 def test_kv_is_held_as_the_cache_stores_it():
     """bf16 models: every K/V value the oracle hands out is a bfloat16 number (low 16 bits of
-    its fp32 pattern are zero) and equals torch's rounding of the unrounded value; fp32 models
-    keep fp64 K/V."""
+    its fp32 pattern are zero), is the bfloat16 nearest to the fp64 value (ties to even, one
+    rounding), and equals torch's conversion wherever that is a single rounding too (inputs that
+    are fp32 numbers); fp32 models keep fp64 K/V."""
     class Cfg:
         dtype = "bf16"
     x = np.random.default_rng(5).standard_normal(4096) * np.logspace(-6, 3, 4096)
     got = M.as_stored_kv(x, Cfg)
-    assert (got.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all()
-    want = torch.from_numpy(x).float().bfloat16().double().numpy()
-    assert (got == want).all()
+    assert (got.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all() and (got.astype(np.float32) == got).all()
+    # nearest: within half a unit in the last place of the result's binade (8 significant bits)
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(got))) - 7)
+    assert (np.abs(x - got) <= ulp / 2).all()
+    # torch converts fp64 through fp32; on fp32 inputs that is one rounding and must agree exactly
+    x32 = x.astype(np.float32).astype(np.float64)
+    assert (M.as_stored_kv(x32, Cfg) == torch.from_numpy(x32).float().bfloat16().double().numpy()).all()
+    # where the two-step conversion differs on fp64 inputs, the single rounding is strictly closer
+    two_step = torch.from_numpy(x).float().bfloat16().double().numpy()
+    differ = got != two_step
+    assert (np.abs(x - got)[differ] < np.abs(x - two_step)[differ]).all()
     ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8])      # exactly between two bfloat16 neighbours: to even
     assert M.as_stored_kv(ties, Cfg).tolist() == [1.0, 1.0 + 2.0 ** -6]
+    # a value that the fp32 detour rounds the wrong way: just above a tie in fp64, exactly the tie in fp32
+    sneaky = np.array([1.0 + 2.0 ** -8 + 2.0 ** -40])
+    assert M.as_stored_kv(sneaky, Cfg).tolist() == [1.0 + 2.0 ** -7]
+    assert M.as_stored_kv(np.array([0.0, -0.0, 2.0 ** -130, 1e-45]), Cfg).tolist() == [0.0, -0.0, 2.0 ** -130, 0.0]
     Cfg.dtype = "fp32"
     assert M.as_stored_kv(x, Cfg) is x
     wl = get_config("t_bf16")

@@ -180,3 +180,90 @@ def test_reject_only_commits_nothing_but_accepted_drafts(tiny_f32):
         assert a.xhat == b.xhat and a.result.n_accepted == b.result.n_accepted
         if a.result.first_reject >= 0:
             break
+
+
+# ---- the drafting mask of Eq. (draft_mask): the block-row half of a draft pass ---------------------
+def _eq_draft_mask(B: int, j: int) -> np.ndarray:
+    """M_draft^(j) typed out from its four blocks: [[A_j, 0], [1, 1]] with row sizes j and B - j."""
+    m = np.zeros((B, B), dtype=bool)
+    for r in range(B):
+        for c in range(B):
+            m[r, c] = (c <= r) if r < j else True
+    return m
+
+
+def _check_rows_against_eq_draft_mask(rows_fn, B: int = 8):
+    for j in range(B):                       # first masked position
+        want = _eq_draft_mask(B, j)
+        for cached in range(j + 1):          # block positions whose K/V is already in the cache
+            pend_pos = list(range(40 + cached, 40 + j))
+            blk_pos = list(range(40 + j, 40 + B))
+            toks, pos, mask = rows_fn([900 + p for p in pend_pos], pend_pos, [7000 + p for p in blk_pos], blk_pos)
+            assert pos.tolist() == list(range(40 + cached, 40 + B))
+            assert toks.tolist() == [900 + p for p in pend_pos] + [7000 + p for p in blk_pos]
+            # the rows of the pass are rows cached.. of the block; what they see of each other is the lower-right part
+            assert mask.shape == (B - cached, B - cached)
+            assert (mask == want[cached:, cached:]).all(), (j, cached)
+            # and the lower-left part is all ones: every row of the pass sees every cached block token,
+            # which is what "each row attends the whole cache" relies on
+            assert want[cached:, :cached].all()
+
+
+def _check_draft_logits_against_one_literal_pass(rows_fn, wl, W):
+    """Draft logits of a step that starts from a cache == one pass over prompt ++ block without any
+    cache under the composed mask: causal on the prompt, Eq. (draft_mask) on the block, block rows see
+    the whole prompt."""
+    cfg = wl.model
+    MASK = cfg.mask_id
+    prompt = [5, 9, 2, 44, 17, 3]
+    n, B, j, cached = len(prompt), 8, 3, 1
+    block = [11, 4, 30, MASK, MASK, 21, MASK, MASK]       # committed prefix of 3; position 5 known out of order
+    pre = prompt + block[:cached]
+    _, kv = M.forward(W, cfg, pre, np.arange(len(pre)), M.causal_mask(len(pre)), need_logits=[])
+    cache = M.append_kv(None, kv, np.arange(len(pre)))
+    pend_pos = list(range(n + cached, n + j))
+    toks, pos, mask = rows_fn([block[p - n] for p in pend_pos], pend_pos, block[j:], list(range(n + j, n + B)))
+    got, _ = M.forward(W, cfg, toks, pos, mask, cache)
+    full = np.zeros((n + B, n + B), dtype=bool)
+    full[:n, :n] = M.causal_mask(n)
+    full[n:, :n] = True
+    full[n:, n:] = _eq_draft_mask(B, j)
+    lit, _ = M.forward(W, cfg, prompt + block, np.arange(n + B), full)
+    np.testing.assert_allclose(got, lit[n + cached:], rtol=1e-9, atol=1e-11)
+    # the block rows really use what the mask gives them: a MASK row's logits move when a later block token changes
+    block2 = list(block)
+    block2[5] = 22
+    lit2, _ = M.forward(W, cfg, prompt + block2, np.arange(n + B), full)
+    assert np.abs(lit2[n + 3] - lit[n + 3]).max() > 1e-6
+
+
+def test_draft_pass_rows_are_eq_draft_mask():
+    _check_rows_against_eq_draft_mask(S.draft_pass_rows)
+
+
+def test_draft_logits_equal_one_literal_pass_under_eq_draft_mask(tiny_f32):
+    wl, W = tiny_f32
+    _check_draft_logits_against_one_literal_pass(S.draft_pass_rows, wl, W)
+
+
+@pytest.mark.parametrize("mutation", ["causal_block_rows", "block_rows_blind_to_pending", "pending_sees_block"])
+def test_draft_mask_pins_catch_a_wrong_mask(tiny_f32, mutation):
+    """The two pins above fail for plausible mistakes in the block-row half of the mask."""
+    wl, W = tiny_f32
+
+    def mutated(pending_tokens, pending_pos, block_tokens, block_pos):
+        toks, pos, mask = S.draft_pass_rows(pending_tokens, pending_pos, block_tokens, block_pos)
+        P = len(pending_tokens)
+        mask = mask.copy()
+        if mutation == "causal_block_rows":
+            mask[P:, :] = np.tril(np.ones_like(mask))[P:, :]
+        elif mutation == "block_rows_blind_to_pending":
+            mask[P:, :P] = False
+        else:
+            mask[:P, P:] = True
+        return toks, pos, mask
+
+    with pytest.raises(AssertionError):
+        _check_rows_against_eq_draft_mask(mutated)
+    with pytest.raises(AssertionError):
+        _check_draft_logits_against_one_literal_pass(mutated, wl, W)
