@@ -151,17 +151,108 @@ def model_pass_bytes(m):
     return total
 
 
-# DRAM traffic of one pass_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu
-# capture summarised in profiles/pass_kernel_c2.md, as a ratio to the launch's algorithmic bytes; the
-# capture is of the 1.7B-class shape (a few GB on the device) and is scaled by algorithmic bytes, which
-# the traffic follows (weights dominate both).  Set to None when the kernel changes until it is re-captured.
-PASS_TRAFFIC_RATIO = 1.011
+# DRAM traffic of one pass_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) comes from the ncu capture
+# summarised in profiles/pass_kernel_c2.md, as a ratio to the launch's algorithmic bytes; the capture is of the
+# 1.7B-class shape (a few GB on the device) and is scaled by algorithmic bytes, which the traffic follows (weights
+# dominate both).  The summary names the sources the captured kernel was built from by their SHA-256; when those
+# files have changed since, the figure no longer describes the kernel that runs and `traffic` is null.
+PASS_KERNEL_SOURCES = ("paper_2603_25702_b200/csrc/pass_kernel.cuh", "paper_2603_25702_b200/csrc/attention_tc.cuh",
+                       "paper_2603_25702_b200/csrc/tc_ptx.cuh")
 
 
-def pass_traffic_bytes(m, algorithmic_bytes_per_launch):
-    if PASS_TRAFFIC_RATIO is None:
-        return None
-    return PASS_TRAFFIC_RATIO * algorithmic_bytes_per_launch
+def kernel_sources_sha() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for rel in PASS_KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def pass_traffic_ratio():
+    """(ratio or None, note) read from the committed profile summary."""
+    path = os.path.join(ROOT, "profiles", "pass_kernel_c2.md")
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, "no profile summary"
+    import re
+    m_ratio = re.search(r"^traffic_ratio:\s*([0-9.]+)", text, flags=re.M)
+    m_sha = re.search(r"^kernel_sources_sha256_16:\s*([0-9a-f]+)", text, flags=re.M)
+    if not m_ratio or not m_sha:
+        return None, "profile summary carries no traffic ratio"
+    if m_sha.group(1) != kernel_sources_sha():
+        return None, "kernel sources changed since the capture in profiles/pass_kernel_c2.md"
+    return float(m_ratio.group(1)), "profiles/pass_kernel_c2.md (1.7B-class capture, scaled by algorithmic bytes)"
+
+
+def measured_bf16_sustained():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1400.0, "fallback"
+
+
+def batch32_point(W, n_steps: int, stream: int):
+    """The batch-32 half of the metric: a few decode steps of the 8B-class workload at batch 32 (workload c4b32) on
+    one GPU.  More than 64 rows per pass, so the passes run one kernel per operation; the GEMM launches are
+    bracketed by events and set against the tensor-pipe roofline (useful flops = 2 x rows x weights, against
+    the sustained bf16 peak)."""
+    import torch
+    from paper_2603_25702_b200 import Engine
+    wl = get_config("c4b32")
+    m, B = wl.model, wl.block_size
+    eng = Engine(m, block_size=B, max_batch=wl.batch, max_seq_len=wl.prompt_len[1] + (n_steps + 8) * B, kv_page_tokens=wl.kv_page_tokens,
+                 seed=wl.philox_seed, tau_conf=wl.tau_conf, stream=stream)
+    eng.load_weights(W)
+    ids = eng.prefill(generate_prompts(wl))
+    c0 = eng.get_counters()
+
+    def step():
+        st = eng.draft_block(ids)
+        fl = eng.route(st)
+        eng.verify_block(ids, fl)
+        return eng.accept_and_commit(ids, fl)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    eng.reset_counters()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    committed = 0
+    for _ in range(n_steps):
+        committed += sum(r.n_committed for r in step())
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    cnt = eng.get_counters()
+    # the same steps again with every GEMM launch bracketed (their sum is the GEMM share of a step)
+    eng.set_profiling(1)
+    r0 = eng.get_counters()
+    for _ in range(2):
+        step()
+    prof = eng.get_gemm_profile()
+    r1 = eng.get_counters()
+    eng.set_profiling(0)
+    rows = (r1.n_rows_draft + r1.n_rows_verify) - (r0.n_rows_draft + r0.n_rows_verify)
+    n_ctx = eng.debug_seq_state(ids[0])["n_cached"]
+    eng.close()
+    weights = model_pass_bytes(m) / 2                    # bf16 parameters one pass multiplies
+    flops = 2.0 * rows * weights
+    peak, kind = measured_bf16_sustained()
+    gemm_ms_per_step = prof["ms"] / 2
+    return {"workload": "c4b32", "batch": wl.batch, "steps": n_steps, "ms_per_step": ms / n_steps,
+            "value": committed / (ms * 1e-3), "unit": "tokens/s", "context": n_ctx,
+            "verify_us": 1e3 * cnt.ms_verify / max(1, cnt.n_verify_passes), "draft_us": 1e3 * cnt.ms_draft / max(1, cnt.n_draft_passes),
+            "accept_us": 1e3 * cnt.ms_accept / n_steps,
+            "rows_per_step": rows / 2, "gemm_launches_per_step": prof["launches"] / 2, "gemm_ms_per_step": gemm_ms_per_step,
+            "gemm_share": gemm_ms_per_step / (ms / n_steps),
+            "roofline": {"bound": "tensor", "achieved": flops / (prof["ms"] * 1e-3) / 1e12 if prof["ms"] > 0 else 0.0, "peak": peak,
+                         "unit": "TFLOP/s", "frac": (flops / (prof["ms"] * 1e-3) / 1e12 / peak) if prof["ms"] > 0 else 0.0,
+                         "peak_kind": f"of {kind} (sustained bf16)", "note": "useful flops: two-term operands double the issued work"},
+            "prefill_ms": c0.ms_prefill, "prefill_launches": int(c0.n_kernel_launches)}
 
 
 def main():
@@ -176,7 +267,11 @@ def main():
     ap.add_argument("--shaped-steps", type=int, default=20,
                     help="extra timed steps with the accept test overridden by u < 0.77 (the paper's per-token acceptance), reported under 'shaped'; 0: skip")
     ap.add_argument("--warmup-seconds", type=float, default=0.6,
-                    help="keep stepping after the --warmup steps until the clock sampler has had this long to deliver (0: exactly --warmup steps, for profiler runs)")
+                    help="untimed load phase before the timed repeats, long enough for the clock sampler to deliver (0: none, for profiler runs)")
+    ap.add_argument("--repeats", type=int, default=3,
+                    help="timed repeats of the --steps region, each from freshly prefilled sequences and --warmup steps; the median one is reported")
+    ap.add_argument("--batch32-steps", type=int, default=4,
+                    help="decode steps of the batch-32 point of the metric (workload c4b32), reported under 'batch32' by the default c4 run at one GPU; 0: skip")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = get_config(args.workload)
@@ -221,39 +316,56 @@ def main():
         eng.verify_block(ids, fl)
         return eng.accept_and_commit(ids, fl)
 
+    # Load phase for the clock sampler (nvidia-smi needs a few hundred ms to deliver): the same decode steps on
+    # these sequences, untimed.  Every timed repeat then starts from freshly prefilled sequences, so the context
+    # length of the timed region does not depend on how long this phase ran.
     sampler = ClockSampler(local_rank)
     sampler.start()
     t_w = time.perf_counter()
-    for _ in range(args.warmup):
-        step()
     n_extra = 0
-    while time.perf_counter() - t_w < args.warmup_seconds and n_extra < 390:      # same load until the clock sampler delivers
+    while time.perf_counter() - t_w < args.warmup_seconds and n_extra < 390:
         step()
         n_extra += 1
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    eng.reset_counters()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    sampler.mark_begin()
-    t0 = time.perf_counter()
-    ev0.record()
-    committed = 0
-    ctx_lens = []
-    for _ in range(args.steps):
-        res = step()
-        committed += sum(r.n_committed for r in res)
-    ev1.record()
-    torch.cuda.synchronize()
-    wall = time.perf_counter() - t0
-    sampler.mark_end()
-    dev_ms = ev0.elapsed_time(ev1)
-    cnt = eng.get_counters()
+
+    repeats = []
+    for rep in range(max(1, args.repeats)):
+        for sid in ids:
+            eng.release_seq(sid)
+        ids = eng.prefill(prompts)
+        for _ in range(args.warmup):
+            step()
+        ctx_begin = eng.debug_seq_state(ids[0])["n_cached"]
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        eng.reset_counters()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        if rep == 0:
+            sampler.mark_begin()
+        t0 = time.perf_counter()
+        ev0.record()
+        committed = 0
+        for _ in range(args.steps):
+            res = step()
+            committed += sum(r.n_committed for r in res)
+        ev1.record()
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        sampler.mark_end()
+        dev_ms = ev0.elapsed_time(ev1)
+        cnt = eng.get_counters()
+        if world > 1:
+            dist.barrier()
+        dev_ms, wall, committed = aggregate_over_ranks(dev_ms, wall, committed)
+        repeats.append({"dev_ms": dev_ms, "wall": wall, "committed": committed, "cnt": cnt, "context_at_begin": ctx_begin,
+                        "context_at_end": eng.debug_seq_state(ids[0])["n_cached"]})
     clocks = sampler.stop()
-    if world > 1:
-        dist.barrier()
-    dev_ms, wall, committed = aggregate_over_ranks(dev_ms, wall, committed)
+    # the reported repeat is the median one by device time
+    order = sorted(range(len(repeats)), key=lambda k: repeats[k]["dev_ms"])
+    med = repeats[order[len(order) // 2]]
+    dev_ms, wall, committed, cnt = med["dev_ms"], med["wall"], med["committed"], med["cnt"]
 
     # roofline of the dominant kernel: its launches are bracketed by CUDA event pairs on the library's
     # own stream (the persistent pass kernel, one launch per draft or verifier pass; on shapes it does
@@ -291,6 +403,7 @@ def main():
                   "mean_accepted_per_verify": sc.n_accepted_tokens / max(1, sc.n_verify_passes * wl.batch),
                   "tokens_per_step": s_committed / args.shaped_steps,
                   "accepted_len_hist": [int(x) for x in list(sc.accepted_len_hist)[:B + 1]]}
+    traffic_ratio, traffic_note = pass_traffic_ratio()
     achieved = prof["bytes"] / (prof["ms"] * 1e-3) / 1e9 if prof["ms"] > 0 else 0.0
     persistent = prof["launches"] <= 2 * args.profile_steps + 1
 
@@ -301,7 +414,8 @@ def main():
     accept_ms = cnt.ms_accept / steps_done
     draft_ms = cnt.ms_draft / max(1, cnt.n_draft_passes)
     kv_bytes_tok = 2 * m.n_layers * m.n_kv_heads * m.head_dim * (2 if m.dtype == "bf16" else 4)
-    verify_step_bytes = pass_bytes + wl.batch * n_ctx * kv_bytes_tok
+    n_ctx_mid = 0.5 * (med["context_at_begin"] + med["context_at_end"])      # cached tokens a verifier pass of the timed region reads, on average
+    verify_step_bytes = pass_bytes + wl.batch * n_ctx_mid * kv_bytes_tok
     line = {
         "metric": "committed_tokens_per_s", "value": committed / (dev_ms * 1e-3), "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dev_ms / args.steps,
@@ -309,18 +423,22 @@ def main():
         "dtype": "bf16" if m.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": wl.name, "model": m.name, "batch": wl.batch, "prompt_len": list(wl.prompt_len),
                    "block_size": B, "kv_page_tokens": wl.kv_page_tokens, "route": wl.route,
-                   "context_at_end": n_ctx, "l2": "inputs larger than L2 (weights streamed every pass)",
+                   "context_at_begin": med["context_at_begin"], "context_at_end": med["context_at_end"],
+                   "l2": "inputs larger than L2 (weights streamed every pass)",
                    "parallelism": "replicas" if world > 1 else "single"},
         "e2e": {"value": committed / wall, "unit": "tokens/s",
                 "h2d_bytes_per_step": cnt.h2d_bytes / args.steps, "d2h_bytes_per_step": cnt.d2h_bytes / args.steps},
         "gpu_launches": int(cnt.n_kernel_launches),
+        "repeats": [{"ms_per_step": r["dev_ms"] / args.steps, "value": r["committed"] / (r["dev_ms"] * 1e-3),
+                     "context_at_begin": r["context_at_begin"], "context_at_end": r["context_at_end"]} for r in repeats],
         "clocks": clocks,
         "roofline": {"bound": "hbm",
                      "kernel": "pass_kernel (persistent draft/verifier pass: weight stream + attention + element-wise phases)"
                      if persistent else "gemm_tc_kernel launches of the per-operation path",
                      "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": pass_traffic_bytes(m, prof["bytes"] / max(1, prof["launches"])) if persistent else None,
+                     "traffic": traffic_ratio * prof["bytes"] / max(1, prof["launches"]) if (persistent and traffic_ratio) else None,
+                     "traffic_source": traffic_note,
                      "launches": prof["launches"], "avg_launch_us": 1e3 * prof["ms"] / max(1, prof["launches"])},
         "verify_step": {"verify_us": 1e3 * verify_ms, "accept_us": 1e3 * accept_ms, "draft_us": 1e3 * draft_ms,
                         "algorithmic_bytes": verify_step_bytes,
@@ -340,9 +458,11 @@ def main():
                                 "kind": "oracle",
                                 "sample": f"1 decode step (draft+verify+accept, block {B}) of one sequence after an 8-token "
                                           f"prompt on the full model shape, x batch {wl.batch}; {sum(times):.1f} s"}
+    eng.close()
+    if rank == 0 and world == 1 and args.workload == "c4" and args.batch32_steps > 0:
+        line["batch32"] = batch32_point(W, args.batch32_steps, torch.cuda.current_stream().cuda_stream)
     if rank == 0:
         print(json.dumps(line))
-    eng.close()
     if world > 1:
         dist.destroy_process_group()
 

@@ -47,7 +47,19 @@ typedef enum {
 } s2d2_status;
 
 enum { S2D2_DTYPE_F32 = 0, S2D2_DTYPE_BF16 = 1 };
-enum { S2D2_DRAFT_GREEDY = 0 };
+/* SampleFromLogits: GREEDY proposes the argmax (ties -> lowest id); SAMPLE draws the proposal from pi_d by
+ * inverse CDF in vocabulary order with one uniform of the draft-sampling Philox stream (only then is the
+ * output law of the speculative step exactly the verifier's: Section "Background", speculative decoding).
+ * In both modes the confidence is pi_d(proposal); margin and entropy describe pi_d itself. */
+enum { S2D2_DRAFT_GREEDY = 0, S2D2_DRAFT_SAMPLE = 1 };
+/* How the verifier pass is laid out (Section "Self-Verification Mode").
+ * ALIGNED_2L: position-aligned models; 2L rows [drafted span ; L MASK copies] under Eq. (ver_mask), the logits
+ *   of the row at position i score position i.
+ * RIGHT_SHIFTED: models whose logits at position i - 1 score the token at position i; "the standard causal
+ *   mask already provides the verifier view": L causal rows [last committed token, drafted tokens but the
+ *   last], row k scores drafted token k + 1.  The draft pass reads its logits one row to the left in the same
+ *   way, and every pass starts with the row of the last committed token. */
+enum { S2D2_VERIFIER_ALIGNED_2L = 0, S2D2_VERIFIER_RIGHT_SHIFTED = 1 };
 
 /* The network (the paper treats x_theta as given; these fields describe the
  * decoder shapes of the synthetic workloads). Matrices are [out, in], y = x W^T. */
@@ -69,13 +81,17 @@ typedef struct {
     int32_t max_seq_len;        /* prompt + generated tokens per sequence        */
     int32_t kv_page_tokens;     /* tokens per KV page (power of two, <= 64)      */
     int32_t n_kv_pages;         /* pool size; 0 = max_batch*ceil(max_seq_len/page) */
-    int32_t draft_mode;         /* S2D2_DRAFT_GREEDY                             */
+    int32_t draft_mode;         /* S2D2_DRAFT_GREEDY | S2D2_DRAFT_SAMPLE         */
     int32_t resample;           /* 1: draw from the residual at a rejection      */
     float tau_conf;             /* threshold of the confidence branch            */
     float ratio_gamma;          /* accept iff u < min(1, (v/d)^gamma)            */
     uint32_t seed;              /* Philox key                                    */
     int32_t use_tensor_cores;   /* 1: default. 0: portable SIMT kernels only (debug).
-                                   2: tensor-core kernels, one per operation (no persistent pass kernel) */
+                                   2: tensor-core kernels, one per operation (no persistent pass kernel).
+                                   3: as 1, with every GEMM of the persistent pass kernel cut into sub-GEMMs wherever
+                                   its tile counts allow (test setting: a small model then runs the same
+                                   tile-by-tile hand-overs between GEMMs that a large one runs by default) */
+    int32_t verifier_layout;    /* S2D2_VERIFIER_*                               */
 } s2d2_decode_config;
 
 typedef struct {
@@ -130,6 +146,7 @@ typedef struct {
     int64_t kv_pages_in_use, kv_pages_total;
     int64_t moe_expert_tiles_touched;                   /* (layer, expert) pairs streamed */
     int64_t h2d_bytes, d2h_bytes;                       /* host<->device copies made by the calls */
+    int64_t n_rows_draft, n_rows_verify, n_rows_prefill; /* token rows the passes of each kind carried, summed */
 } s2d2_counters;
 
 typedef struct s2d2_ctx s2d2_ctx;
@@ -162,7 +179,14 @@ int s2d2_seq_set_rng_stream(s2d2_ctx* ctx, int32_t seq_id, uint32_t stream);
  * for a sequence that has none.  Rows per sequence: committed tokens not yet in
  * the cache (causal; their K/V is appended) followed by the block from its
  * first masked position (these see the whole pass).  Fills stats_out[n_seqs].
- * Synchronous (routing needs the stats on the host). */
+ * Synchronous (routing needs the stats on the host).  With S2D2_VERIFIER_RIGHT_SHIFTED the logits
+ * that score in-block position i are those of the row at position i - 1, so the pass always carries
+ * the last committed token as its first row (run again if its K/V is cached already).
+ * The logits of a draft pass and of a verifier pass live in per-context buffers, so one step uses one id
+ * list: every draft_block overwrites the previous one's rows.  A sequence drafted by an earlier call that has
+ * not been through accept_and_commit since is refused by verify_block and accept_and_commit (S2D2_ERR_STATE)
+ * and has to be drafted again, which is allowed (the repeated draft uses the same uniforms).  Likewise a
+ * second verify_block with a flagged sequence before accept_and_commit is refused. */
 int s2d2_draft_block(s2d2_ctx* ctx, int32_t n_seqs, const int32_t* seq_ids, s2d2_draft_stats* stats_out);
 
 /* Routing hook (Algorithm "DoVerify"): return non-zero to verify the span. */
@@ -172,7 +196,16 @@ enum {
     S2D2_ROUTE_SCORE = 1,         /* K_hat - c[*N_hi] >= tau_score                              */
     S2D2_ROUTE_HYSTERESIS = 2,    /* on/off thresholds on the same score, state per sequence    */
     S2D2_ROUTE_MEAN_CONF = 3,     /* mean draft confidence over M_t < p0                        */
-    S2D2_ROUTE_NEVER = 4
+    S2D2_ROUTE_NEVER = 4,
+    S2D2_ROUTE_UCB = 5            /* contextual bandit (Appendix "Contextual-bandit routing policy", Eq. (ucb)):
+                                     p0 = beta, p1 = bins per context dimension (0: the paper's default, 2).  Context
+                                     bucket = (span-length bin over 1..B, fraction of the block already unmasked,
+                                     mean over the span of H_i / log V); per bucket and action the mean reward
+                                     (tokens committed by the step / cost, cost 2 for a verified step, 1 otherwise)
+                                     and the count; the action maximises mean + beta * sqrt(log t / count), an
+                                     action not yet taken in the bucket goes first, ties verify.  One table per
+                                     context; s2d2_accept_and_commit feeds the rewards back (with the flags it is
+                                     given as the action taken).  s2d2_set_route_policy clears the table. */
 };
 typedef struct {
     int32_t policy;
@@ -191,7 +224,9 @@ int s2d2_route(s2d2_ctx* ctx, int32_t n_seqs, const s2d2_draft_stats* stats, uin
 /* Verifier pass (Section "Self-Verification Mode", the 2L construction and
  * Eq. (ver_mask)): for every flagged sequence 2L rows [drafted span ; L MASK
  * copies at the same positions]; K/V of the drafted rows is appended
- * speculatively to the cache pages. Asynchronous. */
+ * speculatively to the cache pages.  With S2D2_VERIFIER_RIGHT_SHIFTED: L causal rows
+ * [last committed token ; drafted tokens but the last], K/V of the drafted rows appended
+ * speculatively (the last drafted token gets its K/V in the next draft pass). Asynchronous. */
 int s2d2_verify_block(s2d2_ctx* ctx, int32_t n_seqs, const int32_t* seq_ids, const uint8_t* verify_flags);
 
 /* Acceptance and commit (Algorithm "SampleBlock for S2D2", the left-to-right
@@ -245,6 +280,16 @@ int s2d2_accept_logits(s2d2_ctx* ctx, const float* d_draft_logits, const float* 
                        const int32_t* position0, const uint32_t* rng_stream, const int32_t* step,
                        s2d2_step_result* res_out);
 
+/* Stand-alone entry to the SampleFromLogits kernels on caller-supplied device logits (Algorithm
+ * "SampleBlock for S2D2", SampleFromLogits; Section "Verification Routing Policies" for margin and
+ * entropy).  d_logits: fp32 [n_rows, vocab]; draft_mode S2D2_DRAFT_*; position[r], rng_stream[r], step[r]:
+ * Philox counter words of row r (read in SAMPLE mode only, may be NULL for GREEDY).  Host outputs, each
+ * [n_rows]: proposal, its probability, top-1 minus top-2 probability, entropy in nats.  n_rows is at most
+ * max_batch * block_size of the context.  Synchronous. */
+int s2d2_sample_logits(s2d2_ctx* ctx, const float* d_logits, int32_t n_rows, int32_t draft_mode,
+                       const int32_t* position, const uint32_t* rng_stream, const int32_t* step,
+                       int32_t* xhat_out, float* conf_out, float* margin_out, float* entropy_out);
+
 /* Test taps. which: 0 = logits of the last draft pass (rows = masked positions
  * of the listed sequences in call order), 1 = last verify pass (rows = span
  * positions of the verified sequences in call order). */
@@ -263,16 +308,20 @@ int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int3
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);
 
-/* Phase timeline of the last pass that ran as the persistent kernel: for every CTA, a row of
- * n_marks + 1 values: for each of its grid barriers b the GPU global timer (ns) at entry
- * (out[cta * (n_marks + 1) + 3*b]), at exit (.. + 3*b + 1) and at the moment the CTA had drained
- * its last accumulator of the phase that ends at the barrier (.. + 3*b + 2; 0 for phases without
- * a GEMM), then the id of the SM the CTA ran on.  Barrier 0 follows the embedding; per layer the barriers follow, in order,
- * QKV GEMM + q/k-norm + RoPE + K/V write, attention, its combine, O GEMM + residual add,
- * gate/up GEMM + SwiGLU, down GEMM + residual add (nine per layer for mixture-of-experts models).  One
- * more triple closes the row for the LM-head phase, which ends without a barrier: entry and exit both
- * hold the time the CTA finished its logits.  Marks are recorded only while
- * s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */
+/* Phase timeline of the last pass that ran as the persistent kernel: for every CTA a row of n_marks + 1
+ * values, GPU global-timer readings (ns) at named points of the pass followed by the id of the SM the CTA
+ * ran on.  Slots 0, 1: entry to and exit from the grid barrier behind the embedding (slot 2 unused).  Then
+ * per layer, for dense models 12 slots: QKV accumulators drained; entry, exit of the barrier behind q/k-norm +
+ * RoPE + K/V write; entry, exit of the barrier behind the attention items; key splits combined; O accumulators
+ * drained; residual add done; gate/up accumulators drained; SwiGLU done; down accumulators drained; residual
+ * add done (from the combine on, the GEMMs of a dense layer follow each other without a grid barrier).  For
+ * mixture-of-experts models 27 slots: (entry, exit, last accumulator drained before it or 0) for each of the
+ * layer's nine grid barriers.  Then two slots: LM-head accumulators drained, logits written.  Then, for every
+ * sub-GEMM of the pass in execution order (a GEMM may run as up to four), two slots: the CTA's first unit of it
+ * ready to be multiplied, its last unit issued (0, 0 if the CTA has no unit of it); then, again per sub-GEMM,
+ * four slots of the two producers: first weight tile requested, token-row producer arrived at the sub-GEMM,
+ * its input counted complete, first token-row slice about to be requested.  Marks are
+ * recorded only while s2d2_set_profiling is at level 2.  S2D2_ERR_STATE if no such pass has run. */
 int s2d2_debug_pass_trace(s2d2_ctx* ctx, uint64_t* out, int64_t cap, int32_t* n_ctas, int32_t* n_marks);
 
 /* Failure-path tap: runs the kernels' bounded-wait pattern on a word that nothing sets.  With
@@ -298,7 +347,8 @@ int s2d2_debug_wait_timeout(s2d2_ctx* ctx, uint32_t target, uint32_t limit_polls
  * The call is synchronous on `cuda_stream` (it reads back the status word) and calls
  * no cudaMalloc, cudaFree or allocating library routine.  The first call on a device
  * looks up the address of the scratch region and raises the kernel's shared-memory
- * limit; make that first call before any stream capture begins.  All calls on a
+ * limit (host threads that arrive there together take their turn); make that first
+ * call before any stream capture begins.  All calls on a
  * device share the one scratch region, which keeps the previous call's contents (the
  * counters are cleared at the start of every call): two calls that overlap on the
  * GPU, from different streams or threads, race and give wrong results. */

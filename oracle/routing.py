@@ -60,3 +60,52 @@ class Hysteresis:
 def mean_conf(d_masked: Sequence[float], tau: float = 0.9) -> bool:
     """Verify iff the mean draft confidence over the masked positions is below tau."""
     return (sum(d_masked) / len(d_masked)) < tau
+
+
+class UCBRouter:
+    """Contextual-bandit router (Appendix "Contextual-bandit routing policy", Eq. (ucb)).
+
+    Two actions: 0 = confidence-threshold step without verification, 1 = verify the span.  At
+    decision t (counted from 1 over all decisions of the router) in context bucket b the action is
+    argmax_a mu_hat[a, b] + beta * sqrt(log t / n[a, b]); an action never taken in the bucket has an
+    unbounded bonus, and ties go to verification.  The reward of a step is decoded tokens / cost with
+    cost 2 for a verified step and 1 otherwise.  The bucket is the tuple (span-length bin, progress
+    bin, entropy bin), each with ``bins`` equal bins: the span length 1..B partitioned linearly, the
+    fraction of the block already unmasked, and the mean over the span of H_i / log V (the paper says
+    only "normalized token entropy"; the mean over the span is the reading taken here)."""
+
+    def __init__(self, beta: float, block_size: int, vocab: int, bins: int = 2):
+        self.beta, self.B, self.V, self.bins = beta, block_size, vocab, bins
+        self.t = 0
+        self.n = {}        # (action, bucket) -> count
+        self.sum = {}      # (action, bucket) -> summed reward
+        self.last = None   # (bucket, action) awaiting its reward
+
+    def bucket(self, span_len: int, n_masked: int, span_entropies: Sequence[float]):
+        nb = self.bins
+        b_span = min(nb - 1, (span_len - 1) * nb // self.B)
+        b_prog = min(nb - 1, int((self.B - n_masked) * nb // self.B))
+        h = sum(span_entropies) / (len(span_entropies) * math.log(self.V))
+        b_ent = min(nb - 1, max(0, int(math.floor(h * nb))))
+        return (b_span, b_prog, b_ent)
+
+    def index(self, action: int, bucket) -> float:
+        n = self.n.get((action, bucket), 0)
+        if n == 0:
+            return math.inf
+        return self.sum[(action, bucket)] / n + self.beta * math.sqrt(math.log(self.t) / n)
+
+    def decide(self, span_len: int, n_masked: int, span_entropies: Sequence[float]) -> bool:
+        self.t += 1
+        b = self.bucket(span_len, n_masked, span_entropies)
+        a = 1 if self.index(1, b) >= self.index(0, b) else 0
+        self.last = (b, a)
+        return bool(a)
+
+    def update(self, decoded: int, action: int = None):
+        b, a = self.last
+        a = a if action is None else int(action)
+        r = decoded / (2.0 if a else 1.0)
+        self.n[(a, b)] = self.n.get((a, b), 0) + 1
+        self.sum[(a, b)] = self.sum.get((a, b), 0.0) + r
+        self.last = None

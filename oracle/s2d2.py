@@ -63,6 +63,19 @@ def verify_pass_rows(xhat, positions, mask_id):
     return tokens, pos, mask
 
 
+def verify_pass_rows_shifted(prev_token, xhat, first_position):
+    """Rows and mask of the verifier pass of a right-shifted model (Section "Self-Verification
+    Mode", last sentence: there the plain causal mask already gives the verifier view).  In such a
+    model the logits at position i - 1 score the token at position i, so the drafted span
+    xhat_1..xhat_L at positions first_position.. is scored by L causal rows: the last committed
+    token (position first_position - 1), whose logits score xhat_1, followed by xhat_1..xhat_{L-1};
+    row k scores xhat_{k+1}.  xhat_L needs no row.  No MASK copies: L rows instead of 2L."""
+    L = len(xhat)
+    tokens = np.asarray([int(prev_token)] + [int(t) for t in xhat[:L - 1]], dtype=np.int64)
+    pos = np.arange(first_position - 1, first_position - 1 + L, dtype=np.int64)
+    return tokens, pos, M.causal_mask(L)
+
+
 @dataclass
 class StepTrace:
     block_start: int
@@ -90,7 +103,7 @@ class SequenceOracle:
     def __init__(self, W, cfg, block_size: int, seed: int, seq_stream: int,
                  route: Callable[[StepTrace], bool] = None, tau_conf: float = 0.9,
                  draft_mode: str = "greedy", gamma: float = 1.0, keep_logits: bool = False,
-                 resample: bool = True):
+                 resample: bool = True, layout: str = "aligned"):
         self.W, self.cfg, self.B = W, cfg, block_size
         self.seed, self.seq_stream = seed, seq_stream
         self.route = route or (lambda st: len(st.span) >= 1)      # minimum-span policy, tau_span = 1
@@ -99,6 +112,13 @@ class SequenceOracle:
         # False: the reject-only variant of the paper's failure-case study (Appendix, D2F LLaDA table): no residual
         # resampling, the first rejected position stays masked and is drafted again in the next step
         self.resample = resample
+        # "aligned": logits of the row at position i score position i (the 2L verifier, Eq. (ver_mask)).
+        # "shifted": right-shifted model, logits of the row at position i - 1 score position i, in the draft pass
+        # and in the verifier pass alike; the verifier is L plain causal rows (verify_pass_rows_shifted).  Every
+        # pass then starts with the row of the last committed token, whether its K/V is cached already or not:
+        # the cache visible to the pass ends before that position and the row's K/V is written (again).
+        assert layout in ("aligned", "shifted")
+        self.layout = layout
         self.tokens: List[int] = []       # finalised tokens before the current block
         self.cache: Optional[M.KV] = None
         self.n_c = 0                      # tokens whose K/V is cached
@@ -130,14 +150,20 @@ class SequenceOracle:
         s = len(self.tokens)
         j = self.xb.index(MASK)
         full = self._all_tokens()
-        pend_pos = list(range(self.n_c, s + j))
+        shifted = self.layout == "shifted"
+        q0 = min(self.n_c, s + j - 1) if shifted else self.n_c       # first row of the pass
+        if q0 < self.n_c:                                            # the last committed token is run again as a row
+            self.cache = [(k[:q0], v[:q0]) for k, v in self.cache]
+            self.n_c = q0
+        pend_pos = list(range(q0, s + j))
         pend_tok = [full[p] for p in pend_pos]
         blk_pos = list(range(s + j, s + B))
         blk_tok = self.xb[j:]
         tokens, pos, mask = draft_pass_rows(pend_tok, pend_pos, blk_tok, blk_pos)
         P = len(pend_pos)
         masked = [i for i in range(B) if self.xb[i] == MASK]
-        need = [P + (i - j) for i in masked]
+        # the row whose logits score in-block position i: its own row, or the row one position to the left
+        need = [P + (i - j) - (1 if shifted else 0) for i in masked]
         logits, kv = M.forward(self.W, cfg, tokens, pos, mask, self.cache, need_logits=need)
         self.n_draft_passes += 1
         if P:
@@ -158,8 +184,15 @@ class SequenceOracle:
         st.verified = bool(self.route(st))
         if st.verified:
             xhat = st.xhat[:L]                       # masked[0:L] is exactly the span
-            vt, vp, vm = verify_pass_rows(xhat, [s + i for i in span], MASK)
-            vlogits, vkv = M.forward(self.W, cfg, vt, vp, vm, self.cache, need_logits=list(range(L, 2 * L)))
+            if shifted:
+                vt, vp, vm = verify_pass_rows_shifted(full[s + j - 1], xhat, s + j)
+                visible = [(k[:s + j - 1], v[:s + j - 1]) for k, v in self.cache]
+                vlogits, vkv = M.forward(self.W, cfg, vt, vp, vm, visible, need_logits=list(range(L)))
+                # vkv row 0 is the last committed token again, rows 1.. are xhat_1..xhat_{L-1}
+                vkv = [(k[1:], v[1:]) for k, v in vkv]
+            else:
+                vt, vp, vm = verify_pass_rows(xhat, [s + i for i in span], MASK)
+                vlogits, vkv = M.forward(self.W, cfg, vt, vp, vm, self.cache, need_logits=list(range(L, 2 * L)))
             self.n_verify_passes += 1
             st.u_accept = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_ACCEPT) for i in span]
             st.u_resample = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_RESAMPLE) for i in span]
@@ -171,9 +204,11 @@ class SequenceOracle:
                 self.xb[j + k] = int(xhat[k])
                 st.committed.append(j + k)
                 st.committed_tokens.append(int(xhat[k]))
-            if res.n_accepted:
-                self.cache = M.append_kv(self.cache, vkv, np.arange(res.n_accepted))
-                self.n_c += res.n_accepted
+            # accepted drafted tokens keep the K/V their verifier rows produced (the shifted layout has no row for xhat_L)
+            n_keep = min(res.n_accepted, L - 1) if shifted else res.n_accepted
+            if n_keep:
+                self.cache = M.append_kv(self.cache, vkv, np.arange(n_keep))
+                self.n_c += n_keep
             if res.first_reject >= 0 and self.resample:
                 self.xb[j + res.first_reject] = int(res.resampled)
                 st.committed.append(j + res.first_reject)

@@ -33,7 +33,7 @@ class DecodeConfigC(C.Structure):
     _fields_ = [("block_size", C.c_int32), ("max_batch", C.c_int32), ("max_seq_len", C.c_int32),
                 ("kv_page_tokens", C.c_int32), ("n_kv_pages", C.c_int32), ("draft_mode", C.c_int32),
                 ("resample", C.c_int32), ("tau_conf", C.c_float), ("ratio_gamma", C.c_float), ("seed", C.c_uint32),
-                ("use_tensor_cores", C.c_int32)]
+                ("use_tensor_cores", C.c_int32), ("verifier_layout", C.c_int32)]
 
 
 class TensorDesc(C.Structure):
@@ -62,11 +62,12 @@ class Counters(C.Structure):
                                          "n_kernel_launches")] + \
                [("accepted_len_hist", C.c_int64 * (MAX_BLOCK + 1))] + \
                [(n, C.c_double) for n in ("ms_draft", "ms_verify", "ms_accept", "ms_prefill")] + \
-               [(n, C.c_int64) for n in ("kv_pages_in_use", "kv_pages_total", "moe_expert_tiles_touched", "h2d_bytes", "d2h_bytes")]
+               [(n, C.c_int64) for n in ("kv_pages_in_use", "kv_pages_total", "moe_expert_tiles_touched", "h2d_bytes", "d2h_bytes",
+                                         "n_rows_draft", "n_rows_verify", "n_rows_prefill")]
 
 
 class RoutePolicy(C.Structure):
-    MIN_SPAN, SCORE, HYSTERESIS, MEAN_CONF, NEVER = range(5)
+    MIN_SPAN, SCORE, HYSTERESIS, MEAN_CONF, NEVER, UCB = range(6)
     _fields_ = [("policy", C.c_int32), ("p0", C.c_float), ("p1", C.c_float), ("cost", C.c_float),
                 ("dynamic_cost", C.c_int32), ("alpha_entropy", C.c_int32), ("alpha_param", C.c_float)]
 
@@ -77,7 +78,7 @@ EXPORTS = [
     "s2d2_create", "s2d2_destroy", "s2d2_last_error", "s2d2_load_weights", "s2d2_prefill",
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
-    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_set_accept_override", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_debug_copy_logits",
+    "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_set_accept_override", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_sample_logits", "s2d2_debug_copy_logits",
     "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace", "s2d2_debug_wait_timeout",
     "s2d2_gemm_bf16_noalloc", "s2d2_noalloc_last_error",
 ]
@@ -127,6 +128,9 @@ def load_library() -> C.CDLL:
     lib.s2d2_accept_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
                                        C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_uint32),
                                        C.POINTER(C.c_int32), C.POINTER(StepResult)]
+    lib.s2d2_sample_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_uint32),
+                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_float),
+                                       C.POINTER(C.c_float)]
     lib.s2d2_debug_copy_logits.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
     lib.s2d2_debug_copy_kv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.s2d2_debug_seq_state.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -161,7 +165,8 @@ class Engine:
 
     def __init__(self, model, block_size: int, max_batch: int, max_seq_len: int, kv_page_tokens: int = 64,
                  n_kv_pages: int = 0, seed: int = 1, tau_conf: float = 0.9, ratio_gamma: float = 1.0,
-                 resample: bool = True, stream: int = 0, use_tensor_cores: bool = True):
+                 resample: bool = True, stream: int = 0, use_tensor_cores: int = 1, verifier_layout: str = "aligned",
+                 draft_mode: str = "greedy"):
         self.lib = load_library()
         self.model = model
         self.block_size = block_size
@@ -170,8 +175,9 @@ class Engine:
                           model.vocab, 1 if model.dtype == "bf16" else 0, int(model.qk_norm), model.n_experts,
                           model.top_k, model.expert_ffn, model.n_shared, model.rope_base, model.rms_eps,
                           model.logit_scale)
-        dc = DecodeConfigC(block_size, max_batch, max_seq_len, kv_page_tokens, n_kv_pages, 0, int(resample), tau_conf,
-                           ratio_gamma, seed, int(use_tensor_cores))
+        dc = DecodeConfigC(block_size, max_batch, max_seq_len, kv_page_tokens, n_kv_pages,
+                           {"greedy": 0, "sample": 1}[draft_mode], int(resample), tau_conf,
+                           ratio_gamma, seed, int(use_tensor_cores), {"aligned": 0, "shifted": 1}[verifier_layout])
         self._h = C.c_void_p()
         rc = self.lib.s2d2_create(C.byref(mc), C.byref(dc), C.c_void_p(stream), C.byref(self._h))
         if rc != 0:
@@ -313,6 +319,19 @@ class Engine:
                                                 l_max, sl_p, xh_p, p0_p, rs.ctypes.data_as(C.POINTER(C.c_uint32)), stp_p, out))
         return out
 
+    def sample_logits(self, d_logits: int, n_rows: int, draft_mode: str = "greedy", position=None, rng_stream=None, step=None):
+        """SampleFromLogits on device logits (pointer as int, fp32 [n_rows, vocab]): (xhat, conf, margin, entropy)."""
+        pos, pos_p = _i32(position if position is not None else [0] * n_rows)
+        rs = np.ascontiguousarray(rng_stream if rng_stream is not None else [0] * n_rows, dtype=np.uint32)
+        stp, stp_p = _i32(step if step is not None else [0] * n_rows)
+        xh = np.zeros(n_rows, dtype=np.int32)
+        cf, mg, en = (np.zeros(n_rows, dtype=np.float32) for _ in range(3))
+        fp = lambda a: a.ctypes.data_as(C.POINTER(C.c_float))
+        self._check(self.lib.s2d2_sample_logits(self._h, C.c_void_p(d_logits), n_rows, {"greedy": 0, "sample": 1}[draft_mode], pos_p,
+                                                rs.ctypes.data_as(C.POINTER(C.c_uint32)), stp_p,
+                                                xh.ctypes.data_as(C.POINTER(C.c_int32)), fp(cf), fp(mg), fp(en)))
+        return xh, cf, mg, en
+
     def debug_copy_logits(self, which: int, max_rows: int) -> np.ndarray:
         buf = np.empty((max_rows, self.vocab), dtype=np.float32)
         n = C.c_int64()
@@ -345,15 +364,20 @@ class Engine:
         """Runs the bounded-wait pattern on a word nothing sets; raises S2D2Error(-5) when target > 0."""
         self._check(self.lib.s2d2_debug_wait_timeout(self._h, target, limit_polls))
 
-    def debug_pass_trace(self) -> np.ndarray:
-        """(marks [n_ctas, n_barriers, 3], sm_ids [n_ctas]): global-timer ns at entry to / exit from every grid
-        barrier of the last persistent pass and at the end of the phase's accumulator drain (0 if none), and
-        the SM each CTA ran on.  The last triple is the LM-head phase (entry = exit = the CTA's logits are written)."""
-        buf = np.zeros(256 * (3 * (9 * self.model.n_layers + 2) + 1), dtype=np.uint64)
+    # names of the 12 marks a dense layer records, in slot order (see s2d2_debug_pass_trace)
+    TRACE_DENSE_MARKS = ("qkv_drained", "rope_barrier_entry", "rope_barrier_exit", "attn_barrier_entry", "attn_barrier_exit",
+                         "combine_done", "o_drained", "o_residual_done", "gu_drained", "swiglu_done", "down_drained",
+                         "down_residual_done")
+
+    def debug_pass_trace(self):
+        """(marks [n_ctas, n_marks], sm_ids [n_ctas]): global-timer ns of the named points of the last persistent pass
+        (slot layout in include/s2d2.h: 3 slots of the embedding barrier, 12 marks per dense layer or 9 barrier
+        triples per mixture-of-experts layer, 2 marks of the LM-head phase, 2 per sub-GEMM) and the SM each CTA ran on."""
+        buf = np.zeros(256 * (3 + (27 + 6 * 21) * self.model.n_layers + 2 + 6 + 1), dtype=np.uint64)
         nc, nm = C.c_int32(), C.c_int32()
         self._check(self.lib.s2d2_debug_pass_trace(self._h, buf.ctypes.data, buf.size, C.byref(nc), C.byref(nm)))
         rows = buf[: nc.value * (nm.value + 1)].reshape(nc.value, nm.value + 1)
-        return rows[:, :nm.value].reshape(nc.value, nm.value // 3, 3), rows[:, nm.value].astype(np.int64)
+        return rows[:, :nm.value].astype(np.int64), rows[:, nm.value].astype(np.int64)
 
     def debug_copy_expert_ids(self, max_rows: int) -> np.ndarray:
         k, nl = self.model.top_k, self.model.n_layers

@@ -47,6 +47,9 @@ struct SeqState {
     bool verify_in_flight = false;
     int verify_row0 = 0;        // first row in the verifier-logit buffer
     bool hyst_on = true;
+    // which draft / verifier pass of the context produced the logit rows this sequence refers to
+    unsigned long long draft_stamp = 0, verify_stamp = 0;
+    int ucb_bucket = -1;        // context bucket of the bandit router's last decision for this sequence (-1: none pending)
 };
 
 // Fixed-layout staging area for the metadata of one pass (pinned host mirror and
@@ -115,12 +118,20 @@ struct s2d2_ctx {
     char *acc_h = nullptr, *acc_d = nullptr;      // staging for the acceptance kernel's inputs and outputs
     size_t acc_bytes = 0;
     char* stats_h = nullptr;                       // pinned mirror of the draft statistics
+    int *dsamp_h = nullptr, *dsamp_d = nullptr;    // draft sampling: per logit row position, Philox stream, step (pinned / device)
     int n_draft_logit_rows = 0, n_verify_logit_rows = 0;
+    // The logits of a pass live in per-context buffers that the next pass of the same kind overwrites; the passes
+    // are numbered so that a sequence whose rows have been overwritten is recognised (S2D2_ERR_STATE).
+    unsigned long long draft_gen = 0, verify_gen = 0;
 
     // routing
     s2d2_route_fn route_fn = nullptr;
     void* route_user = nullptr;
     s2d2_route_policy policy;
+    // contextual-bandit router: decisions so far, and per (bucket, action) the count and the summed reward
+    long long ucb_t = 0;
+    std::vector<long long> ucb_n;
+    std::vector<double> ucb_sum;
 
     // counters / timing
     s2d2_counters cnt;

@@ -6,7 +6,9 @@
 
 #include <cuda.h>
 
+#include <atomic>
 #include <map>
+#include <mutex>
 #include <tuple>
 
 #include "context.h"
@@ -287,7 +289,7 @@ static __device__ __align__(256) unsigned g_noalloc_tickets[NOALLOC_TICKETS];
 static __device__ __align__(256) int g_noalloc_status[4];
 
 struct NoallocDevice {
-    bool ready = false;
+    std::atomic<bool> ready{false};
     float* ws = nullptr;
     unsigned* tickets = nullptr;
     int* status = nullptr;
@@ -295,6 +297,7 @@ struct NoallocDevice {
 };
 NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
 EncodeTiledFn g_noalloc_encode = nullptr;
+std::mutex g_noalloc_setup;      // first calls from several host threads take their turn in the one-time set-up
 thread_local char g_noalloc_err[256] = "";
 
 int noalloc_fail(int code, const char* msg, cudaError_t e = cudaSuccess) {
@@ -331,8 +334,10 @@ extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d
     if (e != cudaSuccess) return noalloc_fail(S2D2_ERR_CUDA, "cudaGetDevice", e);
     if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return noalloc_fail(S2D2_ERR_UNSUPPORTED, "device index too large");
     NoallocDevice& nd = g_noalloc_dev[dev];
-    if (!nd.ready) {
-        // one-time set-up for this device (do this before any stream capture)
+    if (!nd.ready.load(std::memory_order_acquire)) {
+        // one-time set-up for this device (do this before any stream capture); host threads are serialised here
+        std::lock_guard<std::mutex> lock(g_noalloc_setup);
+        if (!nd.ready.load(std::memory_order_relaxed)) {
         int major = 0;
         if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
             return noalloc_fail(S2D2_ERR_CUDA, "cudaDeviceGetAttribute", e);
@@ -354,7 +359,8 @@ extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d
             return noalloc_fail(S2D2_ERR_CUDA, "cudaGetSymbolAddress(status)", e);
         if ((e = cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024)) != cudaSuccess)
             return noalloc_fail(S2D2_ERR_CUDA, "cudaFuncSetAttribute", e);
-        nd.ready = true;
+        nd.ready.store(true, std::memory_order_release);
+        }
     }
     tc::GemmParams p;
     p.Y = d_y;

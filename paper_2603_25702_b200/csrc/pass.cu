@@ -26,7 +26,7 @@ struct PassState {
     int grid = 0;
     int max_smem = 0;
     int maps_per_layer = 4;
-    int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act; then their low halves
+    int map_x0 = 0;              // xn maps for T = 16, 32, 48, 64; then attn; then act; then their low halves; then xn_b (+24) and its low halves (+36)
     int map_act_e = 0;           // per T: experts' SwiGLU output, high halves then low halves
     int map_kv = 0;
     bool q_by_tma = false;       // maps map_kv + 1 / + 2: q high and low halves as 3D boxes
@@ -34,15 +34,22 @@ struct PassState {
     pp::LayerGains* d_gains = nullptr;
     float* ws = nullptr;
     bf16 *xn_lo = nullptr, *attn_lo = nullptr, *act_lo = nullptr, *q_lo = nullptr, *act_e = nullptr, *act_e_lo = nullptr;
+    bf16 *xn_b = nullptr, *xn_b_lo = nullptr;
+    pp::SubDesc subs[pp::N_KINDS][pp::MAX_SUBS] = {};
+    int n_subs[pp::N_KINDS] = {};
     long long ws_off[pp::N_KINDS] = {};
     int max_segs[pp::N_KINDS] = {};
     float *ssq_a = nullptr, *ssq_b = nullptr;
     unsigned* barrier = nullptr;     // [64 | tile counters of the static GEMM kinds | x counters], zeroed before every launch
     size_t sync_bytes = 0;
     long long cnt_off[pp::N_KINDS] = {};     // -1: the kind publishes through a grid barrier
-    size_t xcnt_off[3] = {0, 0, 0};
+    size_t xcnt_off[4] = {0, 0, 0, 0};
     unsigned long long* trace = nullptr;
     int trace_cap = 0;
+    int trace_mma0 = 0, n_sub_gemms = 0;
+    int4* segs = nullptr;            // dense models: per CTA the list of its (weight tile, k-block range) segments, a layer's then the LM head's
+    int* seg_sub_begin = nullptr;    // per CTA: first segment of every sub-GEMM of the two lists, then the total
+    int seg_stride = 0, n_layer_subs = 0, n_lm_subs = 0;
     int last_marks = 0;
     int barriers_per_layer = 6;
     int* parts[pp::N_KINDS] = {};    // split-K part tables of the static GEMM kinds
@@ -156,7 +163,7 @@ int pass_init(s2d2_ctx* c) {
     PassState* s = new PassState();
     c->pass_state = s;
     const s2d2_model_config& m = c->m;
-    if (m.dtype != S2D2_DTYPE_BF16 || c->dc.use_tensor_cores != 1 || !gemm_tc_available(c)) return S2D2_OK;
+    if (m.dtype != S2D2_DTYPE_BF16 || (c->dc.use_tensor_cores != 1 && c->dc.use_tensor_cores != 3) || !gemm_tc_available(c)) return S2D2_OK;
     const bool moe = m.n_experts > 0;
     const int d = m.d_model, hd = m.head_dim, nq = m.n_q_heads * hd, nqkv = (m.n_q_heads + 2 * m.n_kv_heads) * hd;
     const int fe = m.expert_ffn, fs = moe ? m.expert_ffn * m.n_shared : 0, E = m.n_experts;
@@ -184,7 +191,7 @@ int pass_init(s2d2_ctx* c) {
     s->maps_per_layer = moe ? 8 : 4;
     s->barriers_per_layer = moe ? 9 : 6;
     s->map_x0 = L * s->maps_per_layer + 1;
-    s->map_act_e = s->map_x0 + 24;
+    s->map_act_e = s->map_x0 + 40;
     s->map_kv = s->map_act_e + 8;
     std::vector<CUtensorMap> maps(s->map_kv + 5);      // KV pool, then q (high and low halves) and this pass's K and V rows as [row, head, head_dim] for the attention items
     auto enc = [&](int idx, const void* ptr, unsigned long long rows, int cols, int box_rows) {
@@ -212,8 +219,11 @@ int pass_init(s2d2_ctx* c) {
     {
         size_t rows = c->max_rows;
         if (cudaMalloc((void**)&s->xn_lo, rows * d * 2) != cudaSuccess || cudaMalloc((void**)&s->attn_lo, rows * nq * 2) != cudaSuccess ||
-            cudaMalloc((void**)&s->act_lo, rows * f * 2) != cudaSuccess || cudaMalloc((void**)&s->q_lo, rows * nq * 2) != cudaSuccess)
+            cudaMalloc((void**)&s->act_lo, rows * f * 2) != cudaSuccess || cudaMalloc((void**)&s->q_lo, rows * nq * 2) != cudaSuccess ||
+            cudaMalloc((void**)&s->xn_b, rows * d * 2) != cudaSuccess || cudaMalloc((void**)&s->xn_b_lo, rows * d * 2) != cudaSuccess)
             return fail_alloc(c);
+        cudaMemset(s->xn_b, 0, rows * d * 2);
+        cudaMemset(s->xn_b_lo, 0, rows * d * 2);
         cudaMemset(s->xn_lo, 0, rows * d * 2);
         cudaMemset(s->attn_lo, 0, rows * nq * 2);
         cudaMemset(s->act_lo, 0, rows * f * 2);
@@ -234,7 +244,8 @@ int pass_init(s2d2_ctx* c) {
         const int T = 16 * (t + 1);
         good = enc(s->map_x0 + t, c->xn, c->max_rows, d, T) && enc(s->map_x0 + 4 + t, c->attn, c->max_rows, nq, T) &&
                enc(s->map_x0 + 8 + t, c->act, c->max_rows, f, T) && enc(s->map_x0 + 12 + t, s->xn_lo, c->max_rows, d, T) &&
-               enc(s->map_x0 + 16 + t, s->attn_lo, c->max_rows, nq, T) && enc(s->map_x0 + 20 + t, s->act_lo, c->max_rows, f, T);
+               enc(s->map_x0 + 16 + t, s->attn_lo, c->max_rows, nq, T) && enc(s->map_x0 + 20 + t, s->act_lo, c->max_rows, f, T) &&
+               enc(s->map_x0 + 24 + t, s->xn_b, c->max_rows, d, T) && enc(s->map_x0 + 36 + t, s->xn_b_lo, c->max_rows, d, T);
         if (moe && good)
             good = enc(s->map_act_e + t, s->act_e, (unsigned long long)E * pp::MAX_T, fe, T) &&
                    enc(s->map_act_e + 4 + t, s->act_e_lo, (unsigned long long)E * pp::MAX_T, fe, T);
@@ -278,45 +289,193 @@ int pass_init(s2d2_ctx* c) {
         NK[pp::K_SDOWN][0] = d, NK[pp::K_SDOWN][1] = fs;
         NK[pp::K_EDOWN][0] = (long long)d * E, NK[pp::K_EDOWN][1] = fe;
     }
+    // ---- sub-GEMMs of every kind (see pp::SubDesc) ----
+    // Dense layers: O finishes its first half of output tiles early; gate/up starts with the k-blocks that half
+    // feeds and finishes the first half of the SwiGLU columns early; down starts with those and finishes its first
+    // half of tiles early; the next layer's QKV starts with the k-blocks they feed.  A GEMM is only cut where every
+    // sub-GEMM still gives each CTA a few units; otherwise (small models, mixture-of-experts kinds) it stays whole.
+    {
+        const int MIN_UNITS = c->dc.use_tensor_cores == 3 ? 0 : 4;      // 3: cut wherever the tile counts allow (test setting)
+        auto whole = [&](int k) {
+            const int n_tiles = (int)((NK[k][0] + 127) / 128), kbt = (int)(NK[k][1] / 64);
+            s->n_subs[k] = 1;
+            s->subs[k][0] = pp::SubDesc{0, n_tiles, n_tiles, 0, 0, kbt, 0, 0, k == pp::K_GU || k == pp::K_SGU ? n_tiles / 2 : n_tiles};
+        };
+        for (int k = 0; k < pp::N_KINDS; ++k)
+            if (NK[k][0] >= 0) whole(k);
+        if (!moe) {
+            const int dt = d / 128, ft = f / 128, h = dt / 2;
+            auto enough = [&](long long units) { return units / G >= MIN_UNITS; };
+            const int kq = d / 64, ko = nq / 64, kd = f / 64, tq = nqkv / 128;
+            const bool o_split = h >= 1 && enough((long long)h * ko) && enough((long long)(dt - h) * ko);
+            if (o_split) {                                   // (H0, all K), (H1, all K)
+                s->n_subs[pp::K_O] = 2;
+                s->subs[pp::K_O][0] = pp::SubDesc{0, h, h, 0, 0, ko, 0, 0, h};
+                s->subs[pp::K_O][1] = pp::SubDesc{h, dt - h, dt - h, 0, 0, ko, 0, h, dt};
+            }
+            // gate/up: its SwiGLU columns in nh groups that complete one after the other, so that the element-wise
+            // chain behind a group (partials published, summed, activated, counted, fetched by the next GEMM) runs
+            // under the groups that follow; down: the k-blocks those groups feed, in the same order, its own output
+            // tiles in two groups during the last of them.  Three groups where every sub-GEMM keeps enough units.
+            const int k0 = o_split ? 2 * h : 0;              // gate/up k-blocks fed by O's first half run first, over all tiles
+            int nh = 1;
+            for (int cand = 3; cand >= 2 && nh == 1; --cand) {
+                if (ft < cand) continue;
+                bool fits = k0 == 0 || enough(2LL * ft * k0);
+                for (int i = 0; i < cand && fits; ++i) {
+                    const int a = ft * i / cand, b2 = ft * (i + 1) / cand;
+                    fits = enough(2LL * (b2 - a) * (kq - k0));
+                }
+                if (fits) nh = cand;
+            }
+            if (nh > 1) {
+                int n = 0;
+                if (k0 > 0) s->subs[pp::K_GU][n++] = pp::SubDesc{0, 2 * ft, 2 * ft, 0, 0, k0, 0, 0, 0};
+                for (int i = 0; i < nh; ++i) {
+                    const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
+                    s->subs[pp::K_GU][n++] = pp::SubDesc{a, 2 * (b2 - a), b2 - a, ft, k0, kq - k0, 0, a, b2};
+                }
+                s->n_subs[pp::K_GU] = n;
+                // down: k-blocks of group i = SwiGLU columns [128 a_i, 128 b_i)
+                bool three_way = h >= 1;                     // last group's k-blocks over two groups of output tiles
+                for (int i = 0; i < nh && three_way; ++i) {
+                    const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
+                    three_way = i + 1 < nh ? enough((long long)dt * 2 * (b2 - a)) : (enough((long long)h * 2 * (b2 - a)) && enough((long long)(dt - h) * 2 * (b2 - a)));
+                }
+                bool k_only = !three_way;
+                for (int i = 0; i < nh && k_only; ++i) k_only = enough((long long)dt * 2 * (ft * (i + 1) / nh - ft * i / nh));
+                if (three_way || k_only) {
+                    n = 0;
+                    for (int i = 0; i < nh; ++i) {
+                        const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
+                        if (i + 1 < nh || k_only) {
+                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{0, dt, dt, 0, 2 * a, 2 * (b2 - a), 0, 0, i + 1 < nh ? 0 : dt};
+                        } else {
+                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{0, h, h, 0, 2 * a, 2 * (b2 - a), 0, 0, h};
+                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{h, dt - h, dt - h, 0, 2 * a, 2 * (b2 - a), 0, h, dt};
+                        }
+                    }
+                    s->n_subs[pp::K_DOWN] = n;
+                }
+                if (three_way && enough((long long)tq * 2 * h) && enough((long long)tq * (kq - 2 * h))) {      // (all, K0), (all, K1): K0 = what down's first half feeds
+                    s->n_subs[pp::K_QKV] = 2;
+                    s->subs[pp::K_QKV][0] = pp::SubDesc{0, tq, tq, 0, 0, 2 * h, 0, 0, 0};
+                    s->subs[pp::K_QKV][1] = pp::SubDesc{0, tq, tq, 0, 2 * h, kq - 2 * h, 0, 0, tq};
+                }
+            }
+        }
+    }
+    // ---- per GEMM kind: split-K workspace region, publish counters, part tables ----
     long long ws_floats = 0;
     size_t sync_words = 64;
     for (int k = 0; k < pp::N_KINDS; ++k) {
         s->cnt_off[k] = -1;
         if (NK[k][0] < 0) continue;
         const bool dynamic = k == pp::K_EGU || k == pp::K_EDOWN;
-        const long long n_tiles = (NK[k][0] + 127) / 128, kbt = NK[k][1] / 64, U = n_tiles * kbt;
-        if (U * (long long)G >= (1LL << 40)) return S2D2_OK;
-        // the kernel shares a GEMM's units among Geff CTAs (pp::effective_ctas); for the routed-expert GEMMs the
-        // largest per-CTA share is that of the largest U, since Geff only grows with U
-        const int Geff = pp::effective_ctas(U, (int)kbt, G);
-        const long long per = (U + Geff - 1) / Geff;
-        s->max_segs[k] = (int)((per + kbt - 1) / kbt + 1);
+        const long long n_tiles_all = (NK[k][0] + 127) / 128;
+        int segs = 0;
+        for (int sb = 0; sb < s->n_subs[k]; ++sb) {
+            pp::SubDesc& sd = s->subs[k][sb];
+            const long long U = (long long)sd.nt * sd.nkb;
+            if (U * (long long)G >= (1LL << 40)) return S2D2_OK;
+            // the kernel shares a sub-GEMM's units among Geff CTAs (pp::effective_ctas); for the routed-expert GEMMs the
+            // largest per-CTA share is that of the largest U, since Geff only grows with U
+            const int Geff = pp::effective_ctas(U, sd.nkb, G);
+            const long long per = (U + Geff - 1) / Geff;
+            sd.seg_base = segs;
+            segs += (int)((per + sd.nkb - 1) / sd.nkb + 1);
+        }
+        s->max_segs[k] = segs;
         s->ws_off[k] = ws_floats;
         ws_floats += (long long)G * s->max_segs[k] * pp::MAX_T * 128;
         if (dynamic) continue;
         s->cnt_off[k] = (long long)sync_words;
-        sync_words += (size_t)n_tiles;
-        // per weight tile: the workspace slots of its split-K partials, in CTA order (the kernel cuts the
-        // tile-major (tile, k-block) units into G equal contiguous ranges)
-        std::vector<int> tab((size_t)n_tiles * (1 + pp::MAX_PARTS), 0);
-        for (int cta = 0; cta < Geff; ++cta) {
-            const long long u0 = U * cta / Geff, u1 = U * (cta + 1) / Geff;
-            if (u1 <= u0) continue;
-            const long long first = u0 / kbt, last = (u1 - 1) / kbt;
-            for (long long t = first; t <= last; ++t) {
-                int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
-                if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
-                tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs[k] + (int)(t - first);
-                ++cnt;
+        sync_words += (size_t)n_tiles_all;
+        // per weight tile: the workspace slots of its split-K partials, sub-GEMM by sub-GEMM and in CTA order inside
+        // each (the kernel cuts a sub-GEMM's tile-major (tile, k-block) units into Geff equal contiguous ranges)
+        std::vector<int> tab((size_t)n_tiles_all * (1 + pp::MAX_PARTS), 0);
+        for (int sb = 0; sb < s->n_subs[k]; ++sb) {
+            const pp::SubDesc& sd = s->subs[k][sb];
+            const long long U = (long long)sd.nt * sd.nkb;
+            const int Geff = pp::effective_ctas(U, sd.nkb, G);
+            for (int cta = 0; cta < Geff; ++cta) {
+                const long long u0 = U * cta / Geff, u1 = U * (cta + 1) / Geff;
+                if (u1 <= u0) continue;
+                const long long first = u0 / sd.nkb, last = (u1 - 1) / sd.nkb;
+                for (long long tl = first; tl <= last; ++tl) {
+                    const long long t = tl < sd.t_split ? sd.t0 + tl : sd.t0 + sd.t_jump + (tl - sd.t_split);
+                    int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
+                    if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
+                    tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs[k] + sd.seg_base + (int)(tl - first);
+                    ++cnt;
+                }
             }
         }
         if (cudaMalloc((void**)&s->parts[k], tab.size() * 4) != cudaSuccess ||
             cudaMemcpy(s->parts[k], tab.data(), tab.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
             return fail_alloc(c);
     }
+    if (!moe) {
+        // Static schedule of a dense model: what each CTA streams does not depend on the data, so the list of its
+        // segments (one weight tile times a range of k-blocks, in execution order) is made here once; the producer
+        // and MMA threads then walk a table instead of recomputing unit ranges with 64-bit divisions per GEMM.
+        const int order[4] = {pp::K_QKV, pp::K_O, pp::K_GU, pp::K_DOWN};
+        std::vector<std::vector<int4>> per_cta(G);
+        std::vector<std::vector<int>> begins(G);
+        auto add_kind = [&](int k) {
+            for (int sb = 0; sb < s->n_subs[k]; ++sb) {
+                const pp::SubDesc& sd = s->subs[k][sb];
+                const long long U = (long long)sd.nt * sd.nkb;
+                const int Geff = pp::effective_ctas(U, sd.nkb, G);
+                for (int cta = 0; cta < G; ++cta) {
+                    begins[cta].push_back((int)per_cta[cta].size());
+                    if (cta >= Geff) continue;
+                    long long u = U * cta / Geff;
+                    const long long u1 = U * (cta + 1) / Geff;
+                    const long long first = u / sd.nkb;
+                    while (u < u1) {
+                        const long long tl = u / sd.nkb;
+                        const int kb0 = (int)(u - tl * sd.nkb);
+                        const int kb1 = (int)std::min<long long>(sd.nkb, kb0 + (u1 - u));
+                        const long long t = tl < sd.t_split ? sd.t0 + tl : sd.t0 + sd.t_jump + (tl - sd.t_split);
+                        const int slot = sd.seg_base + (int)(tl - first);
+                        int4 e;
+                        e.x = k | (sb << 8) | (slot << 16);
+                        e.y = (int)(t * 128);
+                        e.z = (sd.kb0 + kb0) | ((kb1 - kb0) << 16);
+                        e.w = (int)t;
+                        per_cta[cta].push_back(e);
+                        u += kb1 - kb0;
+                    }
+                }
+            }
+        };
+        for (int k : order) add_kind(k);
+        s->n_layer_subs = s->n_subs[pp::K_QKV] + s->n_subs[pp::K_O] + s->n_subs[pp::K_GU] + s->n_subs[pp::K_DOWN];
+        add_kind(pp::K_LM);
+        s->n_lm_subs = s->n_subs[pp::K_LM];
+        size_t stride = 1;
+        for (int cta = 0; cta < G; ++cta) {
+            begins[cta].push_back((int)per_cta[cta].size());
+            stride = std::max(stride, per_cta[cta].size());
+        }
+        s->seg_stride = (int)stride;
+        const int nb = s->n_layer_subs + s->n_lm_subs + 1;
+        std::vector<int4> flat((size_t)G * stride, int4{0, 0, 0, 0});
+        std::vector<int> fb((size_t)G * nb);
+        for (int cta = 0; cta < G; ++cta) {
+            std::copy(per_cta[cta].begin(), per_cta[cta].end(), flat.begin() + (size_t)cta * stride);
+            std::copy(begins[cta].begin(), begins[cta].end(), fb.begin() + (size_t)cta * nb);
+        }
+        if (cudaMalloc((void**)&s->segs, flat.size() * sizeof(int4)) != cudaSuccess ||
+            cudaMalloc((void**)&s->seg_sub_begin, fb.size() * 4) != cudaSuccess ||
+            cudaMemcpy(s->segs, flat.data(), flat.size() * sizeof(int4), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(s->seg_sub_begin, fb.data(), fb.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+            return fail_alloc(c);
+    }
     {
-        const long long Xs[3] = {d, nq, f};       // columns of xn, attn, act
-        for (int k = 0; k < 3; ++k) {
+        const long long Xs[4] = {d, nq, f, d};       // columns of xn, attn, act, xn_b
+        for (int k = 0; k < 4; ++k) {
             s->xcnt_off[k] = sync_words;
             sync_words += (size_t)((Xs[k] + 127) / 128);
         }
@@ -326,7 +485,15 @@ int pass_init(s2d2_ctx* c) {
     std::vector<pp::LayerGains> gains(L);
     for (int l = 0; l < L; ++l) gains[l] = {c->layers[l].attn_norm, c->layers[l].ffn_norm, c->layers[l].q_norm, c->layers[l].k_norm};
     size_t ssq_bytes = (size_t)(d / 128) * pp::MAX_T * 4;
-    s->trace_cap = 3 * (s->barriers_per_layer * L + 2) + 1;      // three marks per grid barrier and for the LM-head phase + the SM id
+    {
+        int spl = 0;      // sub-GEMMs per layer, and the LM head's
+        const int dense_kinds[4] = {pp::K_QKV, pp::K_O, pp::K_GU, pp::K_DOWN};
+        const int moe_kinds[7] = {pp::K_QKV, pp::K_O, pp::K_ROUTER, pp::K_SGU, pp::K_EGU, pp::K_SDOWN, pp::K_EDOWN};
+        for (int j = 0; j < (moe ? 7 : 4); ++j) spl += s->n_subs[moe ? moe_kinds[j] : dense_kinds[j]];
+        s->n_sub_gemms = spl * L + s->n_subs[pp::K_LM];
+    }
+    s->trace_mma0 = 3 + (moe ? 27 : 12) * L + 2;
+    s->trace_cap = s->trace_mma0 + 6 * s->n_sub_gemms + 1;      // embedding barrier, per-layer marks, LM-head phase, two per sub-GEMM, the SM id
     if (cudaMalloc((void**)&s->trace, (size_t)G * s->trace_cap * 8) != cudaSuccess) return fail_alloc(c);
     if (cudaMalloc((void**)&s->d_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
         cudaMalloc((void**)&s->d_gains, gains.size() * sizeof(pp::LayerGains)) != cudaSuccess ||
@@ -360,7 +527,7 @@ void pass_destroy(s2d2_ctx* c) {
     PassState* s = state(c);
     if (!s) return;
     void* ptrs[] = {s->d_maps, s->d_gains, s->ws, s->ssq_a, s->ssq_b, s->barrier, s->trace, s->xn_lo, s->attn_lo, s->act_lo, s->q_lo,
-                    s->act_e, s->act_e_lo, s->n_touched};
+                    s->act_e, s->act_e_lo, s->n_touched, s->xn_b, s->xn_b_lo, s->segs, s->seg_sub_begin};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (int* p : s->parts)
@@ -421,6 +588,8 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.attn = (bf16*)c->attn;
     p.act = (bf16*)c->act;
     p.xn_lo = s->xn_lo;
+    p.xn_b = s->xn_b;
+    p.xn_b_lo = s->xn_b_lo;
     p.attn_lo = s->attn_lo;
     p.act_lo = s->act_lo;
     p.map_lo_off = 12;
@@ -432,7 +601,11 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
         p.max_segs[k] = s->max_segs[k];
         p.parts[k] = s->parts[k];
         p.tile_cnt[k] = s->cnt_off[k] >= 0 ? s->barrier + s->cnt_off[k] : nullptr;
+        p.n_subs[k] = s->n_subs[k];
+        for (int sb = 0; sb < pp::MAX_SUBS; ++sb) p.subs[k][sb] = s->subs[k][sb];
     }
+    p.acc_stride = p.T <= 16 ? 32 : (p.T <= 32 ? 64 : 128);
+    p.n_acc = pp::ACC_COLS / p.acc_stride;
     p.act_e = s->act_e;
     p.act_e_lo = s->act_e_lo;
     p.moe_ids = c->moe_ids;
@@ -455,6 +628,7 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.maps = s->d_maps;
     const int ti = p.T / 16 - 1;
     p.map_xn = s->map_x0 + ti;
+    p.map_xn_b = s->map_x0 + 24 + ti;
     p.map_attn = s->map_x0 + 4 + ti;
     p.map_act = s->map_x0 + 8 + ti;
     p.map_act_e = s->map_act_e + ti;
@@ -465,10 +639,20 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     p.S = stages_for(s, p.T, m.head_dim);
     p.trace = c->tracing ? s->trace : nullptr;
     p.trace_cap = s->trace_cap;
-    if (c->tracing) s->last_marks = 3 * (s->barriers_per_layer * m.n_layers + 2);
+    p.trace_mma0 = s->trace_mma0;
+    p.trace_n_sub = s->n_sub_gemms;
+    p.segs = s->segs;
+    p.seg_sub_begin = s->seg_sub_begin;
+    p.seg_stride = s->seg_stride;
+    p.n_layer_subs = s->n_layer_subs;
+    p.n_lm_subs = s->n_lm_subs;
+    if (c->tracing) {
+        s->last_marks = s->trace_cap - 1;
+        cudaMemsetAsync(s->trace, 0, (size_t)s->grid * s->trace_cap * 8, c->stream);
+    }
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
-    for (int k = 0; k < 3; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];
+    for (int k = 0; k < 4; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];
     void* args[] = {&p};
     gemm_prof_begin(c);
     cudaError_t e = m.head_dim == 128

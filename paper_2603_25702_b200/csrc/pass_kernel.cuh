@@ -21,8 +21,12 @@
 //
 // Work split of a GEMM (stream-K): its (weight tile, k-block) units, tile-major, are cut into
 // gridDim equal contiguous ranges; a CTA's range yields one partial accumulator per tile it
-// touches.  The phase after the barrier sums the partials of a tile in CTA order, so results do
-// not depend on timing.  RMSNorm is folded around the GEMM: the GEMM input is bf16(h * gain) and
+// touches.  The element-wise phase behind the GEMM sums the partials of a tile in a fixed order, so
+// results do not depend on timing.  A GEMM of a dense layer is cut into up to four sub-GEMMs (SubDesc)
+// so that consecutive GEMMs overlap: the first output tiles are complete, reduced and turned into
+// the next GEMM's input while the rest still streams, and the next GEMM begins with exactly those
+// k-blocks.  Between the attention block of one layer and the next, no grid barrier is left on
+// that path; every hand-over is a counted input tile or a counted partial.  RMSNorm is folded around the GEMM: the GEMM input is bf16(h * gain) and
 // the per-row 1/rms (from per-tile sums of squares written by the phase that produced h) scales
 // the summed output.
 //
@@ -42,16 +46,34 @@ namespace pp {
 constexpr int THREADS = 256;
 constexpr int CTHREADS = 128;        // compute warps 4..7
 constexpr int BAR_COMPUTE = 1;       // named barrier of the compute warps
-constexpr int ACC_STRIDE = 128;      // tensor-memory columns per accumulator buffer (2 T: high and low halves)
-constexpr int TMEM_COLS = 512;       // two accumulator buffers, then 64 columns of attention scores and 128 of attention output
+constexpr int ACC_COLS = 256;        // tensor-memory columns of the GEMM accumulators: a ring of 2..8 buffers of 2 T columns
+                                     // (high and low halves), rounded up to a power of two
+constexpr int MAX_ACC = 8;
+constexpr int TMEM_COLS = 512;       // the accumulator ring, then 64 columns of attention scores and 128 of attention output
 constexpr int MAX_T = 64;            // most token rows of a pass
 constexpr int W_TILE_BYTES = tc::BLOCK_N * 128;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;
-constexpr int MAX_PARTS = 16;        // most split-K partials of one weight tile
+constexpr int MAX_PARTS = 30;        // most split-K partials of one weight tile (the list of a tile is held one entry per lane)
+constexpr int MAX_SUBS = 4;          // most sub-GEMMs of one GEMM
 // GEMM kinds of a pass.  Dense layers run QKV, O, GU, DOWN; mixture-of-experts layers run QKV, O,
 // ROUTER, SGU (shared expert gate/up), EGU (gate/up of the touched routed experts), SDOWN, EDOWN.
 enum : int { K_QKV = 0, K_O = 1, K_GU = 2, K_DOWN = 3, K_LM = 4, K_ROUTER = 5, K_SGU = 6, K_EGU = 7, K_SDOWN = 8, K_EDOWN = 9, N_KINDS = 10 };
 constexpr int MAX_EXPERTS = 256;
+
+// A GEMM runs as one to four sub-GEMMs, each a set of weight tiles times a range of k-blocks with its
+// own stream-K split over the CTAs.  The order of the sub-GEMMs is what lets consecutive GEMMs overlap:
+// a GEMM whose output feeds the next one finishes a first group of tiles early (the element-wise work
+// on them then runs while the remaining tiles stream), and the next GEMM starts with the k-blocks that
+// this first group produces.
+struct SubDesc {
+    int t0, nt;          // first weight tile and number of tiles
+    int t_split, t_jump; // local tile i is global tile t0 + i for i < t_split, else t0 + t_jump + (i - t_split)
+                         // (the gate and the up rows that make the same columns of the SwiGLU output)
+    int kb0, nkb;        // k-block range
+    int seg_base;        // first workspace segment (per CTA) of this sub-GEMM
+    int ew_t0, ew_t1;    // output tiles that are complete once this sub-GEMM is drained everywhere: the
+                         // element-wise phase over them follows its drain (for gate/up: tiles of the SwiGLU output)
+};
 
 struct LayerGains {
     const float *attn_norm, *ffn_norm, *q_norm, *k_norm;
@@ -71,6 +93,8 @@ struct PassParams {
     float* h;                 // [M, d] residual stream
     bf16 *xn, *q, *k_rows, *v_rows, *attn, *act;
     bf16 *xn_lo, *attn_lo, *act_lo;   // low halves of the GEMM inputs: x = hi + lo, both bf16
+    bf16 *xn_b, *xn_b_lo;             // input of the GEMMs behind the attention block (gate/up, router): a buffer of its
+                                      // own, so that writing it never meets a late reader of the QKV input and vice versa
     bf16* q_lo;                       // low halves of q, same split, for the attention items
     int map_lo_off;                   // tensor map of a buffer's low half = that of its high half + this
     float* ws;                // split-K partials, one region per GEMM kind: [grid][max_segs][T][128]
@@ -88,18 +112,31 @@ struct PassParams {
     const float *rope_cos, *rope_sin;
     KvPool<bf16> pool;
     const CUtensorMap* maps;  // device array: weights [n_layers*4 + 1], then the entries below
-    int map_xn, map_attn, map_act, map_kv;
+    int map_xn, map_xn_b, map_attn, map_act, map_kv;
     int map_q;                  // first of the two 3D maps of q (high, low halves) for the attention items, or -1
     att::AttnParams ap;       // attention geometry of this pass (layer filled in per layer)
     unsigned* barrier;        // grid barrier counter, zero at launch
     unsigned* tile_cnt[N_KINDS];    // per GEMM kind and weight tile: partials published so far (zero at launch)
-    unsigned* x_cnt[3];       // per 128-column tile of xn / attn / act: (tile, row) pairs written so far (zero at launch)
+    unsigned* x_cnt[4];       // per 128-column tile of xn / attn / act / xn_b: (tile, row) pairs written so far (zero at launch)
+    SubDesc subs[N_KINDS][MAX_SUBS];
+    int n_subs[N_KINDS];
+    int acc_stride, n_acc;    // tensor-memory columns per accumulator buffer and buffers in the ring
     int* status;
     int S;                    // ring stages
     const int* parts[N_KINDS];      // per GEMM kind: [n_tiles][1 + MAX_PARTS] = count, then workspace slots in CTA order
     unsigned long long* trace;   // [grid][trace_cap] per grid barrier: globaltimer at entry, at exit, and when the
                                  // CTA's last accumulator of the phase had been drained (0 if the phase has no GEMM)
     int trace_cap;
+    int trace_mma0;              // first of the per-sub-GEMM slot pairs written by the MMA issuer
+    int trace_n_sub;             // sub-GEMMs of a pass with logits; behind the MMA issuer's pairs come four producer marks per sub-GEMM
+    // Dense models: host-made schedule.  segs[cta * seg_stride + i] = i-th segment of the CTA: x = kind | sub << 8 |
+    // workspace slot << 16, y = row coordinate of the weight tile, z = first k-block | k-blocks << 16, w = weight tile;
+    // a layer's segments first (the same list for every layer), then the LM head's.  seg_sub_begin[cta * (n_layer_subs +
+    // n_lm_subs + 1) + j] = first segment of sub-GEMM j in that order; the last entry is the total.  Null: the unit
+    // ranges are computed in the kernel (mixture-of-experts models, whose routed-expert GEMMs are sized at run time).
+    const int4* segs;
+    const int* seg_sub_begin;
+    int seg_stride, n_layer_subs, n_lm_subs;
 };
 
 __host__ __device__ inline size_t stage_bytes(int T) { return (size_t)W_TILE_BYTES + (size_t)2 * T * 128; }
@@ -109,53 +146,78 @@ __host__ __device__ inline size_t smem_bytes(int T, int S, int hd) {
 }
 
 struct GemmShape {
-    int n_tiles, kbt, map_w, map_x;
+    int n_tiles, kbt, map_w, map_x;      // tiles and k-blocks of this sub-GEMM (local numbering)
     int tpe;           // weight tiles per expert for the two routed-expert GEMMs, else 0
-    int Geff;          // CTAs that share the GEMM's units: all of them, or fewer for a small GEMM so that
+    int Geff;          // CTAs that share the sub-GEMM's units: all of them, or fewer for a small one so that
                        // no CTA gets less than an eighth of a tile's k-blocks and a tile has few parts
+    int t0, t_split, t_jump, kb0, seg_base;     // placement inside the whole GEMM (SubDesc)
     long long U;
+    __device__ __forceinline__ int tile_global(int i) const { return i < t_split ? t0 + i : t0 + t_jump + (i - t_split); }
 };
 __host__ __device__ inline int effective_ctas(long long U, int kbt, int G) {
     const long long min_units = kbt / 8 > 1 ? kbt / 8 : 1;
     const long long n = U / min_units;
     return (int)(n < 1 ? 1 : (n < G ? n : G));
 }
-// Shape of one GEMM of layer l; n_touched: touched routed experts of that layer (K_EGU, K_EDOWN).
-__device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int kind, int n_touched) {
-    int N, K, mx, mw;
+// Shape of sub-GEMM `sub` of one GEMM of layer l; n_touched: touched routed experts of that layer (K_EGU, K_EDOWN).
+__device__ __forceinline__ GemmShape gemm_shape(const PassParams& p, int l, int kind, int sub, int n_touched) {
+    int mx, mw;
     GemmShape g;
     g.tpe = 0;
     switch (kind) {
-        case K_QKV: N = (p.Hq + 2 * p.Hkv) * p.hd; K = p.d; mx = p.map_xn; mw = 0; break;
-        case K_O: N = p.d; K = p.Hq * p.hd; mx = p.map_attn; mw = 1; break;
-        case K_GU: N = 2 * p.f; K = p.d; mx = p.map_xn; mw = 2; break;
-        case K_DOWN: N = p.d; K = p.f; mx = p.map_act; mw = 3; break;
-        case K_ROUTER: N = p.n_experts; K = p.d; mx = p.map_xn; mw = 2; break;
-        case K_SGU: N = 2 * p.fs; K = p.d; mx = p.map_xn; mw = 3; break;
-        case K_EGU: g.tpe = 2 * p.fe / tc::BLOCK_N; N = n_touched * 2 * p.fe; K = p.d; mx = p.map_xn; mw = 4; break;   // gate map 4, up map 5
-        case K_SDOWN: N = p.d; K = p.fs; mx = p.map_act; mw = 6; break;
-        case K_EDOWN: g.tpe = p.d / tc::BLOCK_N; N = n_touched * p.d; K = p.fe; mx = p.map_act_e; mw = 7; break;
-        default: N = p.V; K = p.d; mx = p.map_xn; mw = 0; break;
+        case K_QKV: mx = p.map_xn; mw = 0; break;
+        case K_O: mx = p.map_attn; mw = 1; break;
+        case K_GU: mx = p.map_xn_b; mw = 2; break;
+        case K_DOWN: mx = p.map_act; mw = 3; break;
+        case K_ROUTER: mx = p.map_xn_b; mw = 2; break;
+        case K_SGU: mx = p.map_xn_b; mw = 3; break;
+        case K_EGU: g.tpe = 2 * p.fe / tc::BLOCK_N; mx = p.map_xn_b; mw = 4; break;   // gate map 4, up map 5
+        case K_SDOWN: mx = p.map_act; mw = 6; break;
+        case K_EDOWN: g.tpe = p.d / tc::BLOCK_N; mx = p.map_act_e; mw = 7; break;
+        default: mx = p.map_xn; mw = 0; break;
     }
-    g.n_tiles = (N + tc::BLOCK_N - 1) / tc::BLOCK_N;
-    g.kbt = K / tc::BLOCK_K;
+    const SubDesc& sd = p.subs[kind][sub];
+    g.n_tiles = sd.nt;
+    g.kbt = sd.nkb;
+    g.t0 = sd.t0;
+    g.t_split = sd.t_split;
+    g.t_jump = sd.t_jump;
+    g.kb0 = sd.kb0;
+    g.seg_base = sd.seg_base;
+    if (kind == K_EGU || kind == K_EDOWN) {      // tile count known at run time only; one sub-GEMM
+        g.n_tiles = n_touched * g.tpe;
+        g.t_split = g.n_tiles;
+    }
     g.map_w = kind == K_LM ? p.n_layers * p.maps_per_layer : l * p.maps_per_layer + mw;
     g.map_x = mx;
     g.U = (long long)g.n_tiles * g.kbt;
     g.Geff = effective_ctas(g.U, g.kbt, (int)gridDim.x);
     return g;
 }
-// The gi-th GEMM of the pass: its layer and kind.
-__device__ __forceinline__ void gemm_at(const PassParams& p, int gi, int& l, int& kind) {
-    const int gpl = p.moe ? 7 : 4;
-    if (gi >= p.n_layers * gpl) {
+// GEMM kinds of a layer in the order they run.
+__device__ __forceinline__ int layer_kind(const PassParams& p, int j) { return !p.moe ? j : (j < 2 ? j : K_ROUTER + (j - 2)); }
+// Sub-GEMMs of one layer.
+__device__ __forceinline__ int subs_per_layer(const PassParams& p) {
+    int n = 0;
+    for (int j = 0; j < (p.moe ? 7 : 4); ++j) n += p.n_subs[layer_kind(p, j)];
+    return n;
+}
+// The gi-th sub-GEMM of the pass: its layer, kind and index inside the GEMM.
+__device__ __forceinline__ void gemm_at(const PassParams& p, int gi, int spl, int& l, int& kind, int& sub) {
+    if (gi >= p.n_layers * spl) {
         l = p.n_layers;
         kind = K_LM;
+        sub = gi - p.n_layers * spl;
         return;
     }
-    l = gi / gpl;
-    const int j = gi - l * gpl;
-    kind = !p.moe ? j : (j < 2 ? j : K_ROUTER + (j - 2));
+    l = gi / spl;
+    int r = gi - l * spl;
+    for (int j = 0;; ++j) {
+        kind = layer_kind(p, j);
+        if (r < p.n_subs[kind]) break;
+        r -= p.n_subs[kind];
+    }
+    sub = r;
 }
 // What the routed-expert GEMMs of the current layer need to know; lives in shared memory, written by
 // the compute warps after the layer's routing, read by every role (layer_ready says for which layer).
@@ -174,7 +236,7 @@ __device__ __forceinline__ bool wait_routing(const PassParams& p, const Routing*
     }
     return false;
 }
-// Tensor map and row coordinate of weight tile `tile` of a GEMM.
+// Tensor map and row coordinate of (local) weight tile `tile` of a sub-GEMM.
 __device__ __forceinline__ void weight_tile_coord(const PassParams& p, const GemmShape& g, int kind, int tile, const Routing* r,
                                                   int& map_w, int& y) {
     map_w = g.map_w;
@@ -185,13 +247,13 @@ __device__ __forceinline__ void weight_tile_coord(const PassParams& p, const Gem
     } else if (kind == K_EDOWN) {
         y = r->list[tile / g.tpe] * p.d + (tile % g.tpe) * tc::BLOCK_N;
     } else {
-        y = tile * tc::BLOCK_N;
+        y = g.tile_global(tile) * tc::BLOCK_N;
     }
 }
 // First unit of CTA c: the units are cut into Geff equal contiguous ranges, CTAs past Geff get none.
 __device__ __forceinline__ long long unit_begin(const GemmShape& g, int c) { return c >= g.Geff ? g.U : g.U * c / g.Geff; }
 
-// Calls f(tile, kb0, kb1, local_segment) for the segments of this CTA's unit range.
+// Calls f(tile, kb0, kb1, local_segment) for the segments of this CTA's unit range (local tile and k-block numbers).
 template <class F>
 __device__ __forceinline__ void for_each_segment(const GemmShape& g, int cta, int G, F f) {
     long long u = unit_begin(g, cta), u1 = unit_begin(g, cta + 1);
@@ -233,14 +295,15 @@ __device__ __forceinline__ bool wait_counter(const PassParams& p, unsigned targe
 // per-unit step is two compares; divisions happen once per GEMM.  Before a layer's routed-expert
 // GEMMs the cursor waits for that layer's routing.
 struct UnitCursor {
-    int gi, n_gemms, cta, G;
+    int gi, n_gemms, cta, G, spl;
     int left, kb, tile, kind;
     GemmShape g;
     const Routing* routing;
     volatile int* abort_flag;
     bool failed, opened;
-    __device__ __forceinline__ void init(const PassParams&, int n_gemms_, int cta_, int G_, const Routing* r, volatile int* abort) {
+    __device__ __forceinline__ void init(const PassParams&, int n_gemms_, int spl_, int cta_, int G_, const Routing* r, volatile int* abort) {
         gi = 0;
+        spl = spl_;
         n_gemms = n_gemms_;
         cta = cta_;
         G = G_;
@@ -255,8 +318,8 @@ struct UnitCursor {
     __device__ __forceinline__ bool next(const PassParams& p, int& map_w_, int& kb_, int& y_) {
         while (!opened) {
             if (gi >= n_gemms) return false;
-            int l;
-            gemm_at(p, gi, l, kind);
+            int l, sub;
+            gemm_at(p, gi, spl, l, kind, sub);
             int n_touched = 0;
             if (kind == K_EGU || kind == K_EDOWN) {
                 if (!wait_routing(p, routing, l, abort_flag)) {
@@ -265,7 +328,7 @@ struct UnitCursor {
                 }
                 n_touched = routing->n_touched;
             }
-            g = gemm_shape(p, l, kind, n_touched);
+            g = gemm_shape(p, l, kind, sub, n_touched);
             const long long u = unit_begin(g, cta), u1 = unit_begin(g, cta + 1);
             if (u < u1) {
                 left = (int)(u1 - u);
@@ -277,7 +340,7 @@ struct UnitCursor {
             }
         }
         weight_tile_coord(p, g, kind, tile, routing, map_w_, y_);
-        kb_ = kb;
+        kb_ = g.kb0 + kb;
         if (--left == 0) {
             ++gi;
             opened = false;
@@ -325,10 +388,13 @@ __device__ __forceinline__ int dyn_tab(const GemmShape& g, int tile, int G, int 
 // drained them (round = layer + 1: the counters only grow).  Then the loads of up to PC parts of
 // every sum are issued together, and each sum is accumulated in part order.
 // published[s] == nullptr: no wait (a grid barrier already ordered the partials).
-template <int NS, int PC>
+// after(dep) runs once the counts have arrived and before the partials are requested: loads issued there whose
+// addresses include `dep` (always 0) are ordered behind the polls in the same way, which is how a phase reads
+// what the writers of the GEMM's input had stored before they counted (the sums of squares of the rows).
+template <int NS, int PC, class After>
 __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* ws, const int (&tab_lane)[NS], const int (&row)[NS],
                                               const unsigned* const (&published)[NS], unsigned round, int lane,
-                                              volatile int* abort_flag, float4 (&out)[NS]) {
+                                              volatile int* abort_flag, float4 (&out)[NS], After&& after) {
     int cnt[NS], max_cnt = 0;
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
@@ -369,6 +435,7 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* 
         }
         dep = low == 0u ? 1u : 0u;     // always 0, but only known once every poll has returned
     }
+    after(dep);
     for (int j0 = 0; j0 < max_cnt; j0 += PC) {
         float4 v[NS][PC];
 #pragma unroll
@@ -392,18 +459,24 @@ __device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* 
     }
     return true;
 }
+template <int NS, int PC>
+__device__ __forceinline__ bool tile_row_sums(const PassParams& p, const float* ws, const int (&tab_lane)[NS], const int (&row)[NS],
+                                              const unsigned* const (&published)[NS], unsigned round, int lane,
+                                              volatile int* abort_flag, float4 (&out)[NS]) {
+    return tile_row_sums<NS, PC>(p, ws, tab_lane, row, published, round, lane, abort_flag, out, [](unsigned) {});
+}
 // 1/rms of a row from the per-tile sums of squares of h, in two steps: the loads (lanes take
 // the tiles; nothing consumes them here, so they stay in flight with whatever the caller loads
 // next), and later the sum.  Up to 128 tiles (d <= 16384).
 struct SsqLane {
     float v[4];
 };
-__device__ __forceinline__ SsqLane row_ssq_lane(const float* ssq, int d_tiles, int row, int lane) {
+__device__ __forceinline__ SsqLane row_ssq_lane(const float* ssq, int d_tiles, int row, int lane, unsigned dep = 0u) {
     SsqLane r;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const int t = lane + 32 * k;
-        r.v[k] = t < d_tiles ? __ldcg(ssq + (size_t)t * MAX_T + row) : 0.f;
+        r.v[k] = t < d_tiles ? __ldcg(ssq + (size_t)t * MAX_T + row + dep) : 0.f;
     }
     return r;
 }
@@ -459,8 +532,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     uint64_t* full = (uint64_t*)misc;
     uint64_t* empty = full + S;
     uint64_t* acc_full = empty + S;
-    uint64_t* acc_empty = acc_full + 2;
-    uint64_t* kv_full = acc_empty + 2;
+    uint64_t* acc_empty = acc_full + MAX_ACC;
+    uint64_t* kv_full = acc_empty + MAX_ACC;
     uint32_t* tmem_slot = (uint32_t*)(kv_full + att::STAGES + 3);     // + the "scores ready" and "output ready" barriers of the tcgen05 attention items
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     volatile int* w_issued = abort_flag + 1;
@@ -469,14 +542,16 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     Routing* routing = (Routing*)(misc + 1024);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_gemms = p.n_layers * (p.moe ? 7 : 4) + (p.n_logit > 0 ? 1 : 0);
+    const int spl = subs_per_layer(p);
+    const int n_gemms = p.n_layers * spl + (p.n_logit > 0 ? p.n_subs[K_LM] : 0);
+    const int NACC = p.n_acc, ACC_STRIDE = p.acc_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             tc::mbar_init(&full[s], 2);
             tc::mbar_init(&empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < MAX_ACC; ++b) {
             tc::mbar_init(&acc_full[b], 1);
             tc::mbar_init(&acc_empty[b], 4);
         }
@@ -498,32 +573,92 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Dense models: this CTA's segments (one weight tile times a k-block range each) come from a host-made table,
+    // a layer's list (the same for every layer) and the LM head's; sb[j] is the first segment of sub-GEMM j.
+    const bool tabled = p.segs != nullptr;
+    const int4* my_segs = tabled ? p.segs + (size_t)cta * p.seg_stride : nullptr;
+    const int* sb = tabled ? p.seg_sub_begin + (size_t)cta * (p.n_layer_subs + p.n_lm_subs + 1) : nullptr;
+    // per-sub-GEMM trace slots (only while tracing): MMA issuer {first unit ready, last unit issued}; producers
+    // {first weight tile requested, token-row producer arrived, input counted complete, first slice about to be requested}
+    auto trace_slot = [&](int k) -> unsigned long long* {
+        return p.trace && k >= 0 && k + 3 < p.trace_cap - 1 ? p.trace + (size_t)cta * p.trace_cap + k : nullptr;
+    };
+    auto stamp = [](unsigned long long* dst) {
+        if (dst) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(*dst));
+    };
+
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- W producer: free-running over every GEMM of the pass ----------------
             uint64_t policy;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-            UnitCursor ld;
-            ld.init(p, n_gemms, cta, G, routing, abort_flag);
-            uint32_t i = 0;
             bool ok = true;
-            int mw, kb, y;
-            while (ld.next(p, mw, kb, y)) {
-                const int s = (int)(i % (uint32_t)S);
-                if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
-                    ok = false;
-                    break;
+            if (tabled) {
+                // One iteration per streamed unit is a wait for the stage, an expect and a copy: the stage index and
+                // its parity advance by increments, the coordinates come from the segment's table entry.
+                int s = 0;
+                uint32_t par = 0, issued = 0;      // par: parity of the stage's use count; the first use of a stage waits for nothing
+                bool first_round = true;
+                uint8_t* dst = ring;
+                auto run = [&](int seg_a, int seg_b, int map_base, int gi_base, int sub_a) {
+                    int sub = sub_a;
+                    int4 d = seg_a < seg_b ? __ldg(my_segs + seg_a) : make_int4(0, 0, 0, 0);
+                    for (int si = seg_a; si < seg_b && ok; ++si) {
+                        const int4 dn = si + 1 < seg_b ? __ldg(my_segs + si + 1) : d;      // next entry requested ahead of this segment's copies
+                        const int kind = d.x & 255;
+                        if (p.trace) {
+                            while (sb[sub + 1] <= si) ++sub;
+                            if (sb[sub] == si) stamp(trace_slot(p.trace_mma0 + 2 * p.trace_n_sub + 4 * (gi_base + sub - sub_a)));
+                        }
+                        const CUtensorMap* map = p.maps + map_base + (kind == K_LM ? 0 : kind);      // dense kinds 0..3 are the layer's map order
+                        int x = (d.z & 0xffff) * tc::BLOCK_K;
+                        const int y = d.y;
+                        for (int n = d.z >> 16; n > 0; --n, x += tc::BLOCK_K) {
+                            if (!first_round && !tc::mbar_wait(&empty[s], par ^ 1u, abort_flag)) {
+                                ok = false;
+                                break;
+                            }
+                            tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
+                            tc::tma_load_2d_hint(dst, map, x, y, &full[s], policy);
+                            ++issued;
+                            dst += sbytes;
+                            if (++s == S) {
+                                s = 0;
+                                dst = ring;
+                                par ^= 1u;
+                                first_round = false;
+                            }
+                        }
+                        *w_issued = (int)issued;
+                        d = dn;
+                    }
+                };
+                for (int l = 0; l < p.n_layers && ok; ++l) run(0, sb[p.n_layer_subs], l * p.maps_per_layer, l * p.n_layer_subs, 0);
+                if (ok && p.n_logit > 0)
+                    run(sb[p.n_layer_subs], sb[p.n_layer_subs + p.n_lm_subs], p.n_layers * p.maps_per_layer, p.n_layers * p.n_layer_subs, p.n_layer_subs);
+            } else {
+                UnitCursor ld;
+                ld.init(p, n_gemms, spl, cta, G, routing, abort_flag);
+                uint32_t i = 0;
+                int mw, kb, y;
+                while (ld.next(p, mw, kb, y)) {
+                    const int s = (int)(i % (uint32_t)S);
+                    if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    if (*abort_flag) {
+                        ok = false;
+                        break;
+                    }
+                    tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
+                    tc::tma_load_2d_hint(ring + s * sbytes, p.maps + mw, kb * tc::BLOCK_K, y, &full[s], policy);
+                    *w_issued = (int)i + 1;
+                    ++i;
                 }
-                if (*abort_flag) {
-                    ok = false;
-                    break;
-                }
-                tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
-                tc::tma_load_2d_hint(ring + s * sbytes, p.maps + mw, kb * tc::BLOCK_K, y, &full[s], policy);
-                *w_issued = (int)i + 1;
-                ++i;
+                if (ld.failed) ok = false;
             }
-            if (!ok || ld.failed) {
+            if (!ok) {
                 atomicCAS(p.status, 0, 7);
                 *abort_flag = 1;
             }
@@ -534,69 +669,150 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // tile; the lanes of this warp poll the tiles a segment needs in parallel, lane 0 issues the
         // copies.  The inputs are therefore fetched without waiting for the grid barrier, which only
         // guards buffer reuse.
-        uint32_t i = 0;
         bool ok = true;
-        for (int gi = 0; gi < n_gemms && ok; ++gi) {
-            int l, kind;
-            gemm_at(p, gi, l, kind);
-            int n_touched = 0;
-            if (kind == K_EGU || kind == K_EDOWN) {
-                if (!wait_routing(p, routing, l, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                n_touched = routing->n_touched;
-            }
-            const GemmShape g = gemm_shape(p, l, kind, n_touched);
-            const CUtensorMap* mx = p.maps + g.map_x;
-            // which counter set, and how many pairs make a tile complete for this GEMM
-            const unsigned* cnt = nullptr;
-            unsigned target = 0;
-            switch (kind) {
-                case K_QKV: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 1u); break;
-                case K_O: cnt = p.x_cnt[1]; target = (unsigned)p.M * (unsigned)(tc::BLOCK_N / HD) * (l + 1u); break;
-                case K_GU: case K_ROUTER: case K_SGU: case K_EGU: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * l + 2u); break;
-                case K_DOWN: case K_SDOWN: cnt = p.x_cnt[2]; target = (unsigned)p.M * (l + 1u); break;
-                case K_EDOWN: break;     // its input is published by the grid barrier that follows the experts' SwiGLU
-                default: cnt = p.x_cnt[0]; target = (unsigned)p.M * (2u * p.n_layers + 1u); break;
-            }
-            if (kind == K_EDOWN && unit_begin(g, cta + 1) > unit_begin(g, cta)) {
-                if (!wait_counter(p, (2u + 9u * l + 6u) * (unsigned)G, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-            }
-            for_each_segment(g, cta, G, [&](int tile, int kb0, int kb1, int) {
-                const int x_row = kind == K_EDOWN ? (tile / g.tpe) * T : 0;     // the expert slot's rows of act_e
-                // tiles of 128 columns = 2 k-blocks
-                for (int t0 = kb0 >> 1; cnt && t0 <= (kb1 - 1) >> 1; t0 += 32) {
-                    const int t = t0 + lane;
-                    bool ready = t > ((kb1 - 1) >> 1);
-                    for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
-                        ready = ld_acquire(cnt + t) >= target;
-                        if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
+        if (tabled) {
+            int s = 0;
+            uint32_t par = 0, issued = 0;
+            bool first_round = true;
+            uint8_t* dst = ring + W_TILE_BYTES;
+            auto run = [&](int seg_a, int seg_b, int l, int gi_base, int sub_a) {
+                int sub = sub_a;
+                int4 d = seg_a < seg_b ? __ldg(my_segs + seg_a) : make_int4(0, 0, 0, 0);
+                for (int si = seg_a; si < seg_b && ok; ++si) {
+                    const int4 dn = si + 1 < seg_b ? __ldg(my_segs + si + 1) : d;
+                    const int kind = d.x & 255;
+                    unsigned long long* tx = nullptr;
+                    if (p.trace) {
+                        while (sb[sub + 1] <= si) ++sub;
+                        if (sb[sub] == si && lane == 0) tx = trace_slot(p.trace_mma0 + 2 * p.trace_n_sub + 4 * (gi_base + sub - sub_a));
                     }
-                    if (!__all_sync(0xffffffffu, ready)) return ok = false;
-                }
-                asm volatile("fence.proxy.async;" ::: "memory");
-                for (int kb = kb0; kb < kb1; ++kb, ++i) {
-                    int s = (int)(i % (uint32_t)S);
-                    bool fine = true;
-                    if (lane == 0) {
-                        if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) fine = false;
-                        if (*abort_flag) fine = false;
-                        if (fine) {
-                            tc::mbar_expect_tx(&full[s], (uint32_t)T * 256u);
-                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, x_row, &full[s]);
-                            tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES + T * 128, mx + (kind == K_EDOWN ? 4 : p.map_lo_off), kb * tc::BLOCK_K,
-                                            x_row, &full[s]);
-                            *x_issued = (int)i + 1;
+                    stamp(tx ? tx + 1 : nullptr);
+                    // which counter set, and how many pairs make a tile complete for this GEMM
+                    const unsigned* cnt;
+                    unsigned target = (unsigned)p.M * (unsigned)(l + 1);
+                    int mx;
+                    switch (kind) {
+                        case K_QKV: cnt = p.x_cnt[0]; mx = p.map_xn; break;
+                        case K_O: cnt = p.x_cnt[1]; mx = p.map_attn; target *= (unsigned)(tc::BLOCK_N / HD); break;
+                        case K_GU: cnt = p.x_cnt[3]; mx = p.map_xn_b; break;
+                        case K_DOWN: cnt = p.x_cnt[2]; mx = p.map_act; break;
+                        default: cnt = p.x_cnt[0]; mx = p.map_xn; break;      // LM head: l == n_layers
+                    }
+                    const int kb0 = d.z & 0xffff, kb1 = kb0 + (d.z >> 16);
+                    // tiles of 128 columns = 2 k-blocks
+                    for (int t0 = kb0 >> 1; t0 <= (kb1 - 1) >> 1; t0 += 32) {
+                        const int t = t0 + lane;
+                        bool ready = t > ((kb1 - 1) >> 1);
+                        for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
+                            ready = ld_acquire(cnt + t) >= target;
+                            if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
                         }
+                        if (!__all_sync(0xffffffffu, ready)) ok = false;
                     }
-                    if (!__all_sync(0xffffffffu, fine)) return ok = false;
+                    if (!ok) break;
+                    stamp(tx ? tx + 2 : nullptr);
+                    if (lane == 0) {
+                        const CUtensorMap* m_hi = p.maps + mx;
+                        const CUtensorMap* m_lo = m_hi + p.map_lo_off;
+                        const uint32_t bytes = (uint32_t)T * 256u;
+                        bool fine = true;
+                        int x = kb0 * tc::BLOCK_K;
+                        for (int n = kb1 - kb0; n > 0; --n, x += tc::BLOCK_K) {
+                            if (!first_round && !tc::mbar_wait(&empty[s], par ^ 1u, abort_flag)) {
+                                fine = false;
+                                break;
+                            }
+                            if (tx) {
+                                stamp(tx + 3);
+                                tx = nullptr;
+                            }
+                            tc::mbar_expect_tx(&full[s], bytes);
+                            tc::tma_load_2d(dst, m_hi, x, 0, &full[s]);
+                            tc::tma_load_2d(dst + T * 128, m_lo, x, 0, &full[s]);
+                            ++issued;
+                            dst += sbytes;
+                            if (++s == S) {
+                                s = 0;
+                                dst = ring + W_TILE_BYTES;
+                                par ^= 1u;
+                                first_round = false;
+                            }
+                        }
+                        *x_issued = (int)issued;
+                        if (!fine) ok = false;
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    d = dn;
                 }
-                return true;
-            });
+            };
+            for (int l = 0; l < p.n_layers && ok; ++l) run(0, sb[p.n_layer_subs], l, l * p.n_layer_subs, 0);
+            if (ok && p.n_logit > 0) run(sb[p.n_layer_subs], sb[p.n_layer_subs + p.n_lm_subs], p.n_layers, p.n_layers * p.n_layer_subs, p.n_layer_subs);
+        } else {
+            uint32_t i = 0;
+            for (int gi = 0; gi < n_gemms && ok; ++gi) {
+                int l, kind, sub;
+                gemm_at(p, gi, spl, l, kind, sub);
+                int n_touched = 0;
+                if (kind == K_EGU || kind == K_EDOWN) {
+                    if (!wait_routing(p, routing, l, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    n_touched = routing->n_touched;
+                }
+                const GemmShape g = gemm_shape(p, l, kind, sub, n_touched);
+                const CUtensorMap* mx = p.maps + g.map_x;
+                // which counter set, and how many pairs make a tile complete for this GEMM
+                const unsigned* cnt = nullptr;
+                unsigned target = 0;
+                switch (kind) {
+                    case K_QKV: cnt = p.x_cnt[0]; target = (unsigned)p.M * (l + 1u); break;
+                    case K_O: cnt = p.x_cnt[1]; target = (unsigned)p.M * (unsigned)(tc::BLOCK_N / HD) * (l + 1u); break;
+                    case K_GU: case K_ROUTER: case K_SGU: case K_EGU: cnt = p.x_cnt[3]; target = (unsigned)p.M * (l + 1u); break;
+                    case K_DOWN: case K_SDOWN: cnt = p.x_cnt[2]; target = (unsigned)p.M * (l + 1u); break;
+                    case K_EDOWN: break;     // its input is published by the grid barrier that follows the experts' SwiGLU
+                    default: cnt = p.x_cnt[0]; target = (unsigned)p.M * (p.n_layers + 1u); break;
+                }
+                if (kind == K_EDOWN && unit_begin(g, cta + 1) > unit_begin(g, cta)) {
+                    if (!wait_counter(p, (2u + 9u * l + 6u) * (unsigned)G, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                }
+                for_each_segment(g, cta, G, [&](int tile, int kb0, int kb1, int) {
+                    const int x_row = kind == K_EDOWN ? (tile / g.tpe) * T : 0;     // the expert slot's rows of act_e
+                    kb0 += g.kb0;                                                    // k-blocks of the whole GEMM from here on
+                    kb1 += g.kb0;
+                    // tiles of 128 columns = 2 k-blocks
+                    for (int t0 = kb0 >> 1; cnt && t0 <= (kb1 - 1) >> 1; t0 += 32) {
+                        const int t = t0 + lane;
+                        bool ready = t > ((kb1 - 1) >> 1);
+                        for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
+                            ready = ld_acquire(cnt + t) >= target;
+                            if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
+                        }
+                        if (!__all_sync(0xffffffffu, ready)) return ok = false;
+                    }
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    for (int kb = kb0; kb < kb1; ++kb, ++i) {
+                        int s = (int)(i % (uint32_t)S);
+                        bool fine = true;
+                        if (lane == 0) {
+                            if (i >= (uint32_t)S && !tc::mbar_wait(&empty[s], ((i / S) - 1) & 1, abort_flag)) fine = false;
+                            if (*abort_flag) fine = false;
+                            if (fine) {
+                                tc::mbar_expect_tx(&full[s], (uint32_t)T * 256u);
+                                tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES, mx, kb * tc::BLOCK_K, x_row, &full[s]);
+                                tc::tma_load_2d(ring + s * sbytes + W_TILE_BYTES + T * 128, mx + (kind == K_EDOWN ? 4 : p.map_lo_off), kb * tc::BLOCK_K,
+                                                x_row, &full[s]);
+                                *x_issued = (int)i + 1;
+                            }
+                        }
+                        if (!__all_sync(0xffffffffu, fine)) return ok = false;
+                    }
+                    return true;
+                });
+            }
         }
         if (!ok && lane == 0) {
             atomicCAS(p.status, 0, 3);
@@ -606,41 +822,110 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
             const uint32_t idesc = tc::instr_desc_bf16(2 * T);     // token rows twice: high halves, then low halves
-            uint32_t i = 0, seg = 0;
+            uint32_t seg = 0;
             bool ok = true;
-            for (int gi = 0; gi < n_gemms && ok; ++gi) {
-                int l, kind;
-                gemm_at(p, gi, l, kind);
-                int n_touched = 0;
-                if (kind == K_EGU || kind == K_EDOWN) {
-                    if (!wait_routing(p, routing, l, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    n_touched = routing->n_touched;
-                }
-                const GemmShape g = gemm_shape(p, l, kind, n_touched);
-                for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
-                    const uint32_t b = seg & 1u;
-                    if (seg >= 2 && !tc::mbar_wait(&acc_empty[b], ((seg >> 1) - 1) & 1, abort_flag)) return ok = false;
-                    tc::tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + b * ACC_STRIDE;
-                    for (int kb = kb0; kb < kb1; ++kb, ++i) {
-                        int s = (int)(i % (uint32_t)S);
-                        if (!tc::mbar_wait(&full[s], (i / S) & 1, abort_flag)) return ok = false;
+            if (tabled) {
+                int s = 0;
+                uint32_t par = 0, done = 0;
+                uint32_t b = 0, use_par = 0;       // accumulator buffer of the segment and the parity of its use count
+                bool first_acc_round = true;
+                const uint64_t desc0 = tc::smem_desc_sw128(tc::smem_u32(ring));
+                const uint64_t desc_step = (uint64_t)(sbytes >> 4), desc_b = (uint64_t)(W_TILE_BYTES >> 4);      // descriptor addresses count 16-byte units
+                uint64_t a_desc = desc0;
+                auto run = [&](int seg_a, int seg_b, int gi_base, int sub_a) {
+                    int sub = sub_a;
+                    int4 d = seg_a < seg_b ? __ldg(my_segs + seg_a) : make_int4(0, 0, 0, 0);
+                    for (int si = seg_a; si < seg_b && ok; ++si) {
+                        const int4 dn = si + 1 < seg_b ? __ldg(my_segs + si + 1) : d;
+                        unsigned long long* tm = nullptr;
+                        bool last_of_sub = false;
+                        if (p.trace) {
+                            while (sb[sub + 1] <= si) ++sub;
+                            tm = trace_slot(p.trace_mma0 + 2 * (gi_base + sub - sub_a));
+                            last_of_sub = sb[sub + 1] == si + 1;
+                            if (sb[sub] != si) tm = last_of_sub ? tm : nullptr;
+                        }
+                        const bool first_of_sub = p.trace && sb[sub] == si;
+                        if (!first_acc_round && !tc::mbar_wait(&acc_empty[b], use_par ^ 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
                         tc::tc_fence_after();
-                        uint32_t a_addr = tc::smem_u32(ring + s * sbytes);
-                        uint64_t a_desc = tc::smem_desc_sw128(a_addr), b_desc = tc::smem_desc_sw128(a_addr + W_TILE_BYTES);
+                        const uint32_t d_tmem = tmem_base + b * ACC_STRIDE;
+                        uint32_t acc = 0;
+                        for (int n = d.z >> 16; n > 0; --n) {
+                            if (!tc::mbar_wait(&full[s], par, abort_flag)) {
+                                ok = false;
+                                break;
+                            }
+                            tc::tc_fence_after();
+                            if (first_of_sub && acc == 0) stamp(tm);
+                            const uint64_t b_desc = a_desc + desc_b;
 #pragma unroll
-                        for (int k = 0; k < tc::BLOCK_K / tc::UMMA_K; ++k)
-                            tc::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-                        tc::umma_commit(&empty[s]);
-                        *consumed = (int)i + 1;
+                            for (int k = 0; k < tc::BLOCK_K / tc::UMMA_K; ++k) {
+                                tc::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+                                acc = 1;
+                            }
+                            tc::umma_commit(&empty[s]);
+                            ++done;
+                            a_desc += desc_step;
+                            if (++s == S) {
+                                s = 0;
+                                a_desc = desc0;
+                                par ^= 1u;
+                            }
+                        }
+                        if (!ok) break;
+                        tc::umma_commit(&acc_full[b]);
+                        *consumed = (int)done;
+                        if (last_of_sub && tm) stamp(tm + 1);
+                        if (++b == (uint32_t)NACC) {
+                            b = 0;
+                            use_par ^= 1u;
+                            first_acc_round = false;
+                        }
+                        ++seg;
+                        d = dn;
                     }
-                    tc::umma_commit(&acc_full[b]);
-                    ++seg;
-                    return true;
-                });
+                };
+                for (int l = 0; l < p.n_layers && ok; ++l) run(0, sb[p.n_layer_subs], l * p.n_layer_subs, 0);
+                if (ok && p.n_logit > 0) run(sb[p.n_layer_subs], sb[p.n_layer_subs + p.n_lm_subs], p.n_layers * p.n_layer_subs, p.n_layer_subs);
+            } else {
+                uint32_t i = 0;
+                for (int gi = 0; gi < n_gemms && ok; ++gi) {
+                    int l, kind, sub;
+                    gemm_at(p, gi, spl, l, kind, sub);
+                    int n_touched = 0;
+                    if (kind == K_EGU || kind == K_EDOWN) {
+                        if (!wait_routing(p, routing, l, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        n_touched = routing->n_touched;
+                    }
+                    const GemmShape g = gemm_shape(p, l, kind, sub, n_touched);
+                    for_each_segment(g, cta, G, [&](int, int kb0, int kb1, int) {
+                        const uint32_t b = seg % (uint32_t)NACC, use = seg / (uint32_t)NACC;
+                        if (use >= 1 && !tc::mbar_wait(&acc_empty[b], (use - 1) & 1, abort_flag)) return ok = false;
+                        tc::tc_fence_after();
+                        const uint32_t d_tmem = tmem_base + b * ACC_STRIDE;
+                        for (int kb = kb0; kb < kb1; ++kb, ++i) {
+                            int s = (int)(i % (uint32_t)S);
+                            if (!tc::mbar_wait(&full[s], (i / S) & 1, abort_flag)) return ok = false;
+                            tc::tc_fence_after();
+                            uint32_t a_addr = tc::smem_u32(ring + s * sbytes);
+                            uint64_t a_desc = tc::smem_desc_sw128(a_addr), b_desc = tc::smem_desc_sw128(a_addr + W_TILE_BYTES);
+#pragma unroll
+                            for (int k = 0; k < tc::BLOCK_K / tc::UMMA_K; ++k)
+                                tc::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                            tc::umma_commit(&empty[s]);
+                            *consumed = (int)i + 1;
+                        }
+                        tc::umma_commit(&acc_full[b]);
+                        ++seg;
+                        return true;
+                    });
+                }
             }
             if (!ok) {
                 atomicCAS(p.status, 0, 4);
@@ -661,23 +946,29 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         // One thread publishes for the CTA: its release covers the writes the CTA barrier ordered
         // before it.
         unsigned long long t_drained = 0;
-        auto grid_sync = [&](bool tma_out) {
+        // Phase marks (only while tracing): the GPU timer at a named point of the pass, one slot each.
+        auto mark = [&](int k) {
+            if (p.trace && tid == 0 && k >= 0 && k < p.trace_cap - 1) {
+                unsigned long long t;
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                p.trace[(size_t)cta * p.trace_cap + k] = t;
+            }
+        };
+        // k: trace slot of the barrier's entry mark (exit at k + 1; with_drained: k + 2 gets the time the
+        // CTA's last accumulator before the barrier had been drained)
+        auto grid_sync = [&](bool tma_out, int k, bool with_drained) {
             ++epoch;
             if (tma_out) asm volatile("fence.proxy.async;" ::: "memory");
             att::group_sync(BAR_COMPUTE, CTHREADS);
             if (tid == 0) {
-                const int k = 3 * (int)epoch - 3;
-                unsigned long long t0 = 0, t1 = 0;
-                if (p.trace) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+                mark(k);
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
                 if (!wait_counter(p, epoch * (unsigned)G, abort_flag)) {
                     atomicCAS(p.status, 0, 5);
                     *abort_flag = 1;
                 }
-                if (p.trace && k + 2 < p.trace_cap - 1) {
-                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                    p.trace[(size_t)cta * p.trace_cap + k] = t0;
-                    p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
+                mark(k + 1);
+                if (with_drained && p.trace && k + 2 < p.trace_cap - 1) {
                     p.trace[(size_t)cta * p.trace_cap + k + 2] = t_drained;
                     t_drained = 0;
                 }
@@ -685,37 +976,57 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             att::group_sync(BAR_COMPUTE, CTHREADS);
             if (*abort_flag) ok = false;
         };
-        // accumulators of this CTA's segments of one GEMM -> split-K partials
-        auto drain = [&](int l, int kind) {
-            const GemmShape g = gemm_shape(p, l, kind, routing->n_touched);
-            for_each_segment(g, cta, G, [&](int tile, int, int, int local) {
-                const uint32_t b = seg & 1u;
-                if (!tc::mbar_wait(&acc_full[b], (seg >> 1) & 1, abort_flag)) return ok = false;
-                tc::tc_fence_after();
-                float* mine = p.ws + p.ws_off[kind] + ((size_t)cta * p.max_segs[kind] + local) * (size_t)T * tc::BLOCK_N + tid;
-                const uint32_t taddr = tmem_base + ((uint32_t)(cw * 32) << 16) + b * ACC_STRIDE;
-                for (int c0 = 0; c0 < T; c0 += 16) {
-                    float v[16], w[16];
-                    tc::tmem_ld16(taddr + c0, v);          // W x_hi
-                    tc::tmem_ld16(taddr + T + c0, w);      // W x_lo
+        // accumulators of this CTA's segments of one sub-GEMM -> split-K partials
+        uint32_t acc_b = 0, acc_par = 0;      // accumulator buffer of the next segment and the parity of its use count
+        auto drain_segment = [&](int kind, int slot, int tile_global) {
+            if (!tc::mbar_wait(&acc_full[acc_b], acc_par, abort_flag)) return ok = false;
+            tc::tc_fence_after();
+            float* mine = p.ws + p.ws_off[kind] + ((size_t)cta * p.max_segs[kind] + slot) * (size_t)T * tc::BLOCK_N + tid;
+            const uint32_t taddr = tmem_base + ((uint32_t)(cw * 32) << 16) + acc_b * ACC_STRIDE;
+            for (int c0 = 0; c0 < T; c0 += 16) {
+                float v[16], w[16];
+                tc::tmem_ld16(taddr + c0, v);          // W x_hi
+                tc::tmem_ld16(taddr + T + c0, w);      // W x_lo
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (c0 + j < M) mine[(size_t)(c0 + j) * tc::BLOCK_N] = v[j] + w[j];
+                for (int j = 0; j < 16; ++j)
+                    if (c0 + j < M) mine[(size_t)(c0 + j) * tc::BLOCK_N] = v[j] + w[j];
+            }
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc_b]);
+            // publish: every thread's part of the partial is stored, then one release for the CTA
+            att::group_sync(BAR_COMPUTE, CTHREADS);
+            if (tid == 0 && p.tile_cnt[kind])
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.tile_cnt[kind] + tile_global) : "memory");
+            if (++acc_b == (uint32_t)NACC) {
+                acc_b = 0;
+                acc_par ^= 1u;
+            }
+            ++seg;
+            return true;
+        };
+        // first sub-GEMM of each dense kind in the table's order
+        const int jb_o = p.n_subs[K_QKV], jb_gu = jb_o + p.n_subs[K_O], jb_down = jb_gu + p.n_subs[K_GU];
+        auto drain_sub = [&](int l, int kind, int sub) {
+            if (tabled) {
+                const int j = (kind == K_QKV ? 0 : kind == K_O ? jb_o : kind == K_GU ? jb_gu : kind == K_DOWN ? jb_down : p.n_layer_subs) + sub;
+                const int a = __ldg(sb + j), b = __ldg(sb + j + 1);
+                for (int si = a; si < b && ok; ++si) {
+                    const int4 d = __ldg(my_segs + si);
+                    drain_segment(kind, d.x >> 16, d.w);
                 }
-                tc::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[b]);
-                // publish: every thread's part of the partial is stored, then one release for the CTA
-                att::group_sync(BAR_COMPUTE, CTHREADS);
-                if (tid == 0 && p.tile_cnt[kind]) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.tile_cnt[kind] + tile) : "memory");
-                ++seg;
-                return true;
-            });
+            } else {
+                const GemmShape g = gemm_shape(p, l, kind, sub, routing->n_touched);
+                for_each_segment(g, cta, G, [&](int tile, int, int, int local) { return drain_segment(kind, g.seg_base + local, g.tile_global(tile)); });
+            }
             if (!ok) {
                 atomicCAS(p.status, 0, 6);
                 *abort_flag = 1;
             }
             if (p.trace && tid == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_drained));
+        };
+        auto drain = [&](int l, int kind) {
+            for (int sub = 0; sub < p.n_subs[kind] && ok; ++sub) drain_sub(l, kind, sub);
         };
         // The element-wise phases work warp by warp on (tile, row) pairs: 128 output columns of one
         // row, 4 per lane.  A pair's loads (its partials, its residual row, the sums of squares) are
@@ -723,37 +1034,46 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
         const int gw = cta * 4 + cw, GW = G * 4;
         const FastDiv by_M(M), by_Hq(p.Hq);
 
-        // h update shared by the embedding and the two residual phases: writes h, the next GEMM's
-        // input bf16(h * gain) and the (tile, row) sum of squares
-        // A (tile, row) pair of a GEMM input is written: count it.  The release orders the warp's stores
-        // before the count; the reader (the X producer) acquires the count and then crosses to the async
-        // proxy with its own fence before its TMA loads, which is the one proxy fence the chain needs.
+        // A (tile, row) pair of a GEMM input is written: count it.  Each writing thread first orders its
+        // generic-proxy stores before later async-proxy (TMA) reads of global memory, then the release orders the
+        // warp's stores before the count; the reader (the X producer) acquires the count and issues its TMA loads.
+        // The proxy fence sits with the writers because a writer has no copies in flight when it runs it, whereas
+        // the X producer always has: there the same fence waited for them, about two microseconds per segment.
         auto publish_x = [&](unsigned* counter) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
         };
-        auto h_phase = [&](const float* gain, float* ssq, auto&& value) {
-            for (int pair = gw; pair < d_tiles * M; pair += GW) {
+        // h update shared by the embedding and the residual phases, over the tiles [t_a, t_b) of the row: writes h,
+        // the next GEMM's input bf16(h * gain) (two terms) and the (tile, row) sum of squares.  The pair
+        // (t, m) always belongs to warp (t * M + m) mod GW, whatever the tile range, so the same warp reads
+        // and rewrites a given piece of h in every phase of the pass.
+        auto h_phase = [&](const float* gain, float* ssq, bf16* x_hi, bf16* x_lo, unsigned* x_counter, int t_a, int t_b, auto&& value) {
+            const int lo_pair = t_a * M;
+            int r0 = (gw - lo_pair) % GW;
+            if (r0 < 0) r0 += GW;
+            for (int pair = lo_pair + r0; pair < t_b * M; pair += GW) {
                 int t, m;
                 by_M.divmod(pair, t, m);
                 const int col = t * tc::BLOCK_N + 4 * lane;
                 const float4 gn = *reinterpret_cast<const float4*>(gain + col);
                 const float4 x = value(t, m, col);
                 *reinterpret_cast<float4*>(p.h + (size_t)m * d + col) = x;
-                store_hi_lo_x4(p.xn + (size_t)m * d + col, p.xn_lo + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
+                store_hi_lo_x4(x_hi + (size_t)m * d + col, x_lo + (size_t)m * d + col, x.x * gn.x, x.y * gn.y, x.z * gn.z, x.w * gn.w);
                 const float sq = warp_sum(x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w);
                 if (lane == 0) ssq[(size_t)t * MAX_T + m] = sq;
-                publish_x(p.x_cnt[0] + t);
+                publish_x(x_counter + t);
             }
         };
-        auto residual_phase = [&](int kind, unsigned round, const float* gain, float* ssq) {
-            h_phase(gain, ssq, [&](int t, int m, int col) {
+        // h += GEMM output over the output tiles [t_a, t_b); to_b: the result feeds the GEMMs behind the attention block
+        auto residual_phase = [&](int kind, unsigned round, const float* gain, float* ssq, bool to_b, int t_a, int t_b) {
+            h_phase(gain, ssq, to_b ? p.xn_b : p.xn, to_b ? p.xn_b_lo : p.xn_lo, p.x_cnt[to_b ? 3 : 0], t_a, t_b, [&](int t, int m, int col) {
                 const int tab = tile_row_tab(p, kind, t, lane);
                 const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
                 const int tabs[1] = {tab}, rows[1] = {m};
                 const unsigned* const pubs[1] = {p.tile_cnt[kind] + t};
                 float4 sums[1];
-                tile_row_sums<1, 8>(p, p.ws + p.ws_off[kind], tabs, rows, pubs, round, lane, abort_flag, sums);
+                tile_row_sums<1, 16>(p, p.ws + p.ws_off[kind], tabs, rows, pubs, round, lane, abort_flag, sums);
                 float4 x = sums[0];
                 x.x += hv.x;
                 x.y += hv.y;
@@ -769,15 +1089,19 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             p.trace[(size_t)cta * p.trace_cap + p.trace_cap - 1] = smid;
         }
         // ---- embedding ----
-        h_phase(p.gains[0].attn_norm, p.ssq_a, [&](int, int m, int col) {
+        h_phase(p.gains[0].attn_norm, p.ssq_a, p.xn, p.xn_lo, p.x_cnt[0], 0, d_tiles, [&](int, int m, int col) {
             const uint2 u = *reinterpret_cast<const uint2*>(p.embed + (size_t)p.pv.row_token[m] * d + col);
             const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&u.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&u.y);
             return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
         });
-        grid_sync(true);
+        grid_sync(true, 0, true);
+        // trace slots: 3 for the embedding barrier; then per dense layer 12 named marks, per mixture-of-experts
+        // layer 9 barrier triples; then two marks of the LM-head phase
+        const int marks_per_layer = p.moe ? 27 : 12;
 
         for (int l = 0; l < p.n_layers && ok; ++l) {
             const LayerGains lg = p.gains[l];
+            const int tb = 3 + marks_per_layer * l;        // this layer's first trace slot
             // First attention item of this CTA in this layer: its first K/V page is in the cache already, so the
             // copies are started now and land behind the QKV GEMM (tcgen05 items only).
             bool attn_first_requested = false;
@@ -804,6 +1128,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             // ---- QKV GEMM ----
             drain(l, K_QKV);
             if (!ok) break;
+            if (!p.moe) mark(tb);
             // ---- 1/rms, q/k norm, RoPE, K/V write: one warp per (128-column tile, row) ----
             {
                 constexpr int half = HD / 2, PART = half / 4;     // PART: lane distance of a RoPE pair
@@ -826,7 +1151,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
                         tabs[q] = on[q] ? tile_row_tab(p, 0, tt[q], lane) : 0;
                         pubs[q] = p.tile_cnt[0] + tt[q];
-                        sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, mm[q], lane);
                         pos[q] = __ldg(p.pv.row_pos + mm[q]);
                         flags[q] = __ldg(p.pv.row_flags + mm[q]);
                         const int sq = __ldg(p.pv.row_seq + mm[q]);
@@ -837,11 +1161,15 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         gq[q] = make_float4(1.f, 1.f, 1.f, 1.f);
                         if (p.qk_norm && (is_q || is_k)) gq[q] = __ldg(reinterpret_cast<const float4*>((is_q ? lg.q_norm : lg.k_norm) + ch));
                     }
-                    // 1/rms before the wait for the partials: it only needs what the last barrier ordered
-                    const float inv_q[2] = {inv_rms_from(sq_l[0], d, p.eps), inv_rms_from(sq_l[1], d, p.eps)};
+                    // The sums of squares of the rows were stored by the writers of this GEMM's input before they
+                    // counted it; no grid barrier lies in between, so they are read behind the polls of the partials.
                     float4 sums[2];
                     const unsigned* const pubs_c[2] = {pubs[0], pubs[1]};
-                    tile_row_sums<2, 8>(p, p.ws + p.ws_off[K_QKV], tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
+                    tile_row_sums<2, 8>(p, p.ws + p.ws_off[K_QKV], tabs, mm, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums, [&](unsigned dep) {
+                        sq_l[0] = row_ssq_lane(p.ssq_a, d_tiles, mm[0], lane, dep);
+                        sq_l[1] = row_ssq_lane(p.ssq_a, d_tiles, mm[1], lane, dep);
+                    });
+                    const float inv_q[2] = {inv_rms_from(sq_l[0], d, p.eps), inv_rms_from(sq_l[1], d, p.eps)};
 #pragma unroll
                     for (int q = 0; q < 2; ++q) {
                         const float inv = inv_q[q];
@@ -885,7 +1213,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                 }
             }
-            grid_sync(true);
+            grid_sync(true, p.moe ? tb : tb + 1, p.moe);
             if (!ok) break;
             // ---- attention items ----
             {
@@ -907,7 +1235,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         // 64-token pages: the work item runs on tcgen05 (scores and output in tensor memory)
                         fine = ap.page_tokens == 64
                                    ? att::attn_item_umma<true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
-                                                               tmem_base + 2 * ACC_STRIDE, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE,
+                                                               tmem_base + ACC_COLS, kv_ring, attn_s_cnt, attn_o_cnt, tid, BAR_COMPUTE,
                                                                attn_first_requested && idx == attn_first,
                                                                p.map_q >= 0 ? p.maps + p.map_q : nullptr, &attn_q_cnt)
                                    : att::attn_item<HD, true>(p.maps + p.map_kv, ap, split, qt_i, z_i, attn_s, kv_full,
@@ -922,16 +1250,26 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                 }
                 if (!ok) break;
-                grid_sync(false);
+                // the row table entries of this warp's first combine pair are fetched before the barrier, not behind it
+                int pre_seq = 0, pre_row0 = 0, pre_nctx = 0;
+                if (gw < M * p.Hq) {
+                    int r, hq;
+                    by_Hq.divmod(gw, r, hq);
+                    pre_seq = __ldg(p.pv.row_seq + r);
+                    pre_row0 = __ldg(p.pv.seq_row0 + pre_seq);
+                    pre_nctx = __ldg(p.pv.seq_nctx + pre_seq);
+                }
+                grid_sync(false, tb + 3, p.moe);
                 if (!ok) break;
                 // ---- combine the key splits of every (row, query head) ----
                 for (int pair = gw; pair < M * p.Hq; pair += GW) {
                     int r, hq;
                     by_Hq.divmod(pair, r, hq);
-                    const int seq = __ldg(p.pv.row_seq + r), kvh = hq / ap.group;
-                    const int qv = (r - __ldg(p.pv.seq_row0 + seq)) * ap.group + hq % ap.group;
+                    const bool first = pair == gw;
+                    const int seq = first ? pre_seq : __ldg(p.pv.row_seq + r), kvh = hq / ap.group;
+                    const int qv = (r - (first ? pre_row0 : __ldg(p.pv.seq_row0 + seq))) * ap.group + hq % ap.group;
                     const int qt = qv / att::QT, qi = qv % att::QT;
-                    const int n_ctx = __ldg(p.pv.seq_nctx + seq);
+                    const int n_ctx = first ? pre_nctx : __ldg(p.pv.seq_nctx + seq);
                     const int n_pages = (n_ctx + ap.page_tokens - 1) >> ap.page_shift;
                     const size_t item0 = ((size_t)(seq * ap.Hkv + kvh) * ap.n_qtiles + qt) * n_splits;
                     // Lanes take the splits for maxima and weights, and 4 output columns each (the
@@ -989,17 +1327,21 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     publish_x(p.x_cnt[1] + hq * HD / tc::BLOCK_N);
                 }
             }
-            grid_sync(true);
-            if (!ok) break;
-            // ---- O GEMM, residual ----
-            drain(l, K_O);
-            if (!ok) break;
-            residual_phase(K_O, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b);
-            grid_sync(true);
-            if (!ok) break;
+            // The O GEMM fetches the combined rows as their columns are counted, so dense layers need no
+            // barrier here; from this point to the next layer's q/k/v the GEMMs of a dense layer follow each
+            // other without one: every hand-over is a counted GEMM input or a counted partial, and every
+            // buffer is next written only behind the grid barrier that follows the next layer's q/k/v,
+            // which every CTA reaches after it has drained (hence read the inputs of) all of this layer's GEMMs.
+            if (p.moe) {
+                grid_sync(true, tb + 6, true);
+                if (!ok) break;
+            } else {
+                mark(tb + 5);
+            }
             // SwiGLU of a dense or shared-expert gate/up GEMM -> act (hi/lo), counted per tile
-            auto swiglu_phase = [&](int gu_kind) {
-                const int f_tiles = p.f / tc::BLOCK_N, n_pairs = f_tiles * M;
+            // over the tiles [t_a, t_b) of the SwiGLU output
+            auto swiglu_phase = [&](int gu_kind, int t_a, int t_b) {
+                const int f_tiles = p.f / tc::BLOCK_N, n_pairs = (t_b - t_a) * M;
                 // three (tile, row) pairs per step so that all their loads overlap
                 constexpr int NP = 3;
                 for (int pair = gw; pair < n_pairs; pair += NP * GW) {
@@ -1012,19 +1354,22 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const int pr = pair + q * GW;
                         on[q] = pr < n_pairs;
                         by_M.divmod(on[q] ? pr : 0, tt[q], mm[q]);
+                        tt[q] += t_a;
                         tabs[2 * q] = on[q] ? tile_row_tab(p, gu_kind, tt[q], lane) : 0;
                         tabs[2 * q + 1] = on[q] ? tile_row_tab(p, gu_kind, tt[q] + f_tiles, lane) : 0;
                         rows[2 * q] = rows[2 * q + 1] = mm[q];
                         pubs[2 * q] = p.tile_cnt[gu_kind] + tt[q];
                         pubs[2 * q + 1] = p.tile_cnt[gu_kind] + tt[q] + f_tiles;
-                        sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane);
                     }
-                    float inv_q[NP];      // before the wait for the partials: it only needs what the last barrier ordered
-#pragma unroll
-                    for (int q = 0; q < NP; ++q) inv_q[q] = inv_rms_from(sq_l[q], d, p.eps);
                     float4 sums[2 * NP];
                     const unsigned* const pubs_c[2 * NP] = {pubs[0], pubs[1], pubs[2], pubs[3], pubs[4], pubs[5]};
-                    tile_row_sums<2 * NP, 4>(p, p.ws + p.ws_off[gu_kind], tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums);
+                    tile_row_sums<2 * NP, 4>(p, p.ws + p.ws_off[gu_kind], tabs, rows, pubs_c, (unsigned)l + 1u, lane, abort_flag, sums, [&](unsigned dep) {
+#pragma unroll
+                        for (int q = 0; q < NP; ++q) sq_l[q] = row_ssq_lane(p.ssq_b, d_tiles, mm[q], lane, dep);
+                    });
+                    float inv_q[NP];
+#pragma unroll
+                    for (int q = 0; q < NP; ++q) inv_q[q] = inv_rms_from(sq_l[q], d, p.eps);
 #pragma unroll
                     for (int q = 0; q < NP; ++q) {
                         const float inv = inv_q[q];
@@ -1038,7 +1383,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         const size_t o = (size_t)mm[q] * p.f + tt[q] * tc::BLOCK_N + 4 * lane;
                         store_hi_lo_x4(p.act + o, p.act_lo + o, a[0], a[1], a[2], a[3]);
                     }
-                    // one release for the step's stores, then one count per finished pair (the proxy fence is the reader's)
+                    // the writers' proxy fence, one release for the step's stores, then one count per finished pair
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
                         asm volatile("fence.acq_rel.gpu;" ::: "memory");
@@ -1050,19 +1396,40 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             };
             const float* next_gain = l + 1 < p.n_layers ? p.gains[l + 1].attn_norm : p.final_norm;
             if (!p.moe) {
-                // ---- gate/up GEMM, SwiGLU ----
-                drain(l, K_GU);
-                if (!ok) break;
-                swiglu_phase(K_GU);
-                grid_sync(true);
-                if (!ok) break;
-                // ---- down GEMM, residual; prepares the next layer's (or the head's) input ----
-                drain(l, K_DOWN);
-                if (!ok) break;
-                residual_phase(K_DOWN, (unsigned)l + 1u, next_gain, p.ssq_a);
-                grid_sync(true);
+                // ---- O GEMM, residual; gate/up GEMM, SwiGLU; down GEMM, residual (prepares the next layer's or the
+                // head's input).  Each runs sub-GEMM by sub-GEMM: once a sub-GEMM that completes a group of output
+                // tiles is drained, the element-wise phase over that group follows, while the tensor pipe is already
+                // on the next sub-GEMM (the accumulator ring holds what it finishes meanwhile).
+                for (int sub = 0; sub < p.n_subs[K_O] && ok; ++sub) {
+                    drain_sub(l, K_O, sub);
+                    if (sub + 1 == p.n_subs[K_O]) mark(tb + 6);
+                    const SubDesc& sd = p.subs[K_O][sub];
+                    if (ok && sd.ew_t1 > sd.ew_t0) residual_phase(K_O, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b, true, sd.ew_t0, sd.ew_t1);
+                }
+                mark(tb + 7);
+                for (int sub = 0; sub < p.n_subs[K_GU] && ok; ++sub) {
+                    drain_sub(l, K_GU, sub);
+                    if (sub + 1 == p.n_subs[K_GU]) mark(tb + 8);
+                    const SubDesc& sd = p.subs[K_GU][sub];
+                    if (ok && sd.ew_t1 > sd.ew_t0) swiglu_phase(K_GU, sd.ew_t0, sd.ew_t1);
+                }
+                mark(tb + 9);
+                for (int sub = 0; sub < p.n_subs[K_DOWN] && ok; ++sub) {
+                    drain_sub(l, K_DOWN, sub);
+                    if (sub + 1 == p.n_subs[K_DOWN]) mark(tb + 10);
+                    const SubDesc& sd = p.subs[K_DOWN][sub];
+                    if (ok && sd.ew_t1 > sd.ew_t0) residual_phase(K_DOWN, (unsigned)l + 1u, next_gain, p.ssq_a, false, sd.ew_t0, sd.ew_t1);
+                }
+                mark(tb + 11);
+                if (*abort_flag) ok = false;
                 continue;
             }
+            // ---- O GEMM, residual ----
+            drain(l, K_O);
+            if (!ok) break;
+            residual_phase(K_O, (unsigned)l + 1u, lg.ffn_norm, p.ssq_b, true, 0, d_tiles);
+            grid_sync(true, tb + 9, true);
+            if (!ok) break;
             // ================= mixture of experts =================
             // ---- router GEMM; per row: softmax over the experts, top-k (ties -> lowest id), gates renormalised ----
             drain(l, K_ROUTER);
@@ -1138,7 +1505,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                 }
             }
-            grid_sync(false);
+            grid_sync(false, tb + 12, true);
             if (!ok) break;
             // ---- the touched experts of this layer, ascending; every CTA builds the same list ----
             {
@@ -1173,14 +1540,14 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
             // ---- shared expert gate/up, SwiGLU (its weights do not depend on the routing) ----
             drain(l, K_SGU);
             if (!ok) break;
-            swiglu_phase(K_SGU);
+            swiglu_phase(K_SGU, 0, p.f / tc::BLOCK_N);
             // ---- routed experts gate/up over all rows; SwiGLU only for the (row, expert) pairs that were routed ----
             drain(l, K_EGU);
             if (!ok) break;
-            grid_sync(true);
+            grid_sync(true, tb + 15, true);
             if (!ok) break;
             {
-                const GemmShape g = gemm_shape(p, l, K_EGU, n_touched);
+                const GemmShape g = gemm_shape(p, l, K_EGU, 0, n_touched);
                 const int fe_tiles = p.fe / tc::BLOCK_N;
                 const int n_items = M * p.top_k * fe_tiles;
                 const float* wsb = p.ws + p.ws_off[K_EGU];
@@ -1204,19 +1571,19 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     store_hi_lo_x4(p.act_e + o, p.act_e_lo + o, a[0], a[1], a[2], a[3]);
                 }
             }
-            grid_sync(true);
+            grid_sync(true, tb + 18, true);
             if (!ok) break;
             // ---- shared and routed down GEMMs; h += shared + sum_k gate_k * expert_k; next layer's input ----
             drain(l, K_SDOWN);
             if (!ok) break;
             drain(l, K_EDOWN);
             if (!ok) break;
-            grid_sync(false);
+            grid_sync(false, tb + 21, true);
             if (!ok) break;
             {
-                const GemmShape g = gemm_shape(p, l, K_EDOWN, n_touched);
+                const GemmShape g = gemm_shape(p, l, K_EDOWN, 0, n_touched);
                 const float* wsb = p.ws + p.ws_off[K_EDOWN];
-                h_phase(next_gain, p.ssq_a, [&](int t, int m, int col) {
+                h_phase(next_gain, p.ssq_a, p.xn, p.xn_lo, p.x_cnt[0], 0, d_tiles, [&](int t, int m, int col) {
                     const float4 hv = __ldcg(reinterpret_cast<const float4*>(p.h + (size_t)m * d + col));
                     float4 x;
                     {   // shared expert
@@ -1255,10 +1622,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     return x;
                 });
             }
-            grid_sync(true);
+            grid_sync(true, tb + 24, true);
         }
         if (ok && p.n_logit > 0) {
             // ---- LM head on the rows that need logits ----
+            t_drained = 0;
             drain(p.n_layers, K_LM);
             if (ok) {
                 const int n_tiles = (p.V + tc::BLOCK_N - 1) / tc::BLOCK_N;
@@ -1282,14 +1650,16 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         rows[q] = on ? __ldg(p.pv.logit_rows + lr0 + q) : 0;
                         tabs[q] = on ? tab : 0;
                         pubs[q] = p.tile_cnt[4] + t;
-                        sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, rows[q], lane);
                     }
+                    const unsigned* const pubs_c[NR] = {pubs[0], pubs[1], pubs[2], pubs[3]};
+                    float4 sums[NR];
+                    tile_row_sums<NR, 2>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs_c, 1u, lane, abort_flag, sums, [&](unsigned dep) {
+#pragma unroll
+                        for (int q = 0; q < NR; ++q) sq_l[q] = row_ssq_lane(p.ssq_a, d_tiles, rows[q], lane, dep);
+                    });
                     float sc_q[NR];
 #pragma unroll
                     for (int q = 0; q < NR; ++q) sc_q[q] = p.logit_scale * inv_rms_from(sq_l[q], d, p.eps);
-                    const unsigned* const pubs_c[NR] = {pubs[0], pubs[1], pubs[2], pubs[3]};
-                    float4 sums[NR];
-                    tile_row_sums<NR, 2>(p, p.ws + p.ws_off[K_LM], tabs, rows, pubs_c, 1u, lane, abort_flag, sums);
                     const int col = t * tc::BLOCK_N + 4 * lane;
 #pragma unroll
                     for (int q = 0; q < NR; ++q) {
@@ -1309,16 +1679,13 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 }
             }
         }
-        // the LM-head phase ends without a barrier: its marks are the time this CTA finished its
-        // logits (entry and exit) and the time it had drained its LM-head accumulators
+        // the LM-head phase ends without a barrier: its two marks are the time this CTA had drained its
+        // LM-head accumulators and the time it finished its logits
         if (p.trace && tid == 0) {
-            const int k = 3 * (int)epoch;
-            if (k + 2 < p.trace_cap - 1) {
-                unsigned long long t1;
-                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-                p.trace[(size_t)cta * p.trace_cap + k] = t1;
-                p.trace[(size_t)cta * p.trace_cap + k + 1] = t1;
-                p.trace[(size_t)cta * p.trace_cap + k + 2] = t_drained;
+            const int k = 3 + (p.moe ? 27 : 12) * p.n_layers;
+            if (k + 1 < p.trace_cap - 1) {
+                p.trace[(size_t)cta * p.trace_cap + k] = t_drained;
+                mark(k + 1);
             }
         }
     }

@@ -155,7 +155,8 @@ int validate(const s2d2_model_config& m, const s2d2_decode_config& dc, std::stri
     if (dc.max_batch < 1 || dc.max_seq_len < 1) return bad("decode: max_batch/max_seq_len");
     int p = dc.kv_page_tokens;
     if (p < 1 || p > 64 || (p & (p - 1))) return bad("decode: kv_page_tokens must be a power of two <= 64");
-    if (dc.draft_mode != S2D2_DRAFT_GREEDY) return bad("decode: draft_mode");
+    if (dc.draft_mode != S2D2_DRAFT_GREEDY && dc.draft_mode != S2D2_DRAFT_SAMPLE) return bad("decode: draft_mode");
+    if (dc.verifier_layout != S2D2_VERIFIER_ALIGNED_2L && dc.verifier_layout != S2D2_VERIFIER_RIGHT_SHIFTED) return bad("decode: verifier_layout");
     return S2D2_OK;
 }
 
@@ -305,6 +306,8 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
         if ((rc = dmalloc(c, &c->res_rsum, Sq * nch))) return rc;
         if ((rc = dmalloc(c, &c->res_vsum, Sq * nch))) return rc;
         CUDA_TRY(c, cudaMallocHost((void**)&c->stats_h, R * 16));
+        CUDA_TRY(c, cudaMallocHost((void**)&c->dsamp_h, std::max<size_t>(R, 1) * 12));
+        if ((rc = dmalloc(c, &c->dsamp_d, R * 3))) return rc;
         size_t S = dc->max_batch;
         c->acc_bytes = S * 4 * 12 + S * S2D2_MAX_BLOCK * 4 * 3 + 256;
         CUDA_TRY(c, cudaMallocHost((void**)&c->acc_h, c->acc_bytes));
@@ -333,11 +336,12 @@ extern "C" int s2d2_destroy(s2d2_ctx* c) {
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
                     c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
                     c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status, c->chunk_d, c->chunk_v, c->rej_info,
-                    c->res_rsum, c->res_vsum};
+                    c->res_rsum, c->res_vsum, c->dsamp_d};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->meta.h) cudaFreeHost(c->meta.h);
     if (c->stats_h) cudaFreeHost(c->stats_h);
+    if (c->dsamp_h) cudaFreeHost(c->dsamp_h);
     if (c->acc_h) cudaFreeHost(c->acc_h);
     if (c->h_status) cudaFreeHost(c->h_status);
     for (int i = 0; i < 8; ++i)
@@ -619,6 +623,7 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
         if (pb.n_rows == 0) break;
         if ((rc = run_pass(c, pb, nullptr))) return rc;
         c->cnt.n_prefill_passes++;
+        c->cnt.n_rows_prefill += pb.n_rows;
         // the metadata buffer is reused by the next chunk: wait for this pass to have consumed it
         CUDA_TRY(c, cudaStreamSynchronize(c->stream));
         for (size_t k = 0; k < ids.size(); ++k) c->seqs[ids[k]].n_c += took[k];
@@ -644,6 +649,27 @@ extern "C" int s2d2_seq_set_rng_stream(s2d2_ctx* c, int32_t id, uint32_t stream)
 // ---------------------------------------------------------------------------------------------
 // draft pass
 // ---------------------------------------------------------------------------------------------
+// SampleFromLogits over n_rows logit rows: per-chunk statistics, per-row merge (greedy proposal, confidence, margin,
+// entropy, log-sum-exp) and, in sampling mode, the inverse-CDF draw that replaces proposal and confidence.  The
+// Philox words of the rows are taken from dsamp_h (position | stream | step, n_rows each).
+static int launch_draft_stats(s2d2_ctx* c, const float* d_logits, int n_rows, int draft_mode) {
+    const int nch = vocab_chunks(c->m.vocab);
+    DraftStatsOut so{c->d_xhat, c->d_conf, c->d_margin, c->d_entropy, c->d_lse};
+    vocab_chunk_stats_kernel<<<dim3(nch, n_rows), VCHUNK_THREADS, 0, c->stream>>>(d_logits, c->m.vocab, (ChunkStats*)c->chunk_d);
+    LAUNCHED(c);
+    draft_finish_kernel<<<(n_rows + 3) / 4, 128, 0, c->stream>>>((const ChunkStats*)c->chunk_d, nch, n_rows, so);
+    LAUNCHED(c);
+    if (draft_mode == S2D2_DRAFT_SAMPLE) {
+        CUDA_TRY(c, cudaMemcpyAsync(c->dsamp_d, c->dsamp_h, (size_t)n_rows * 12, cudaMemcpyHostToDevice, c->stream));
+        c->cnt.h2d_bytes += (size_t)n_rows * 12;
+        DraftSampleIn in{d_logits, c->m.vocab, (const ChunkStats*)c->chunk_d, c->dsamp_d, (const unsigned*)(c->dsamp_d + n_rows),
+                         c->dsamp_d + 2 * n_rows, c->dc.seed};
+        draft_sample_kernel<<<n_rows, VCHUNK_THREADS, 0, c->stream>>>(in, nch, so);
+        LAUNCHED(c);
+    }
+    return S2D2_OK;
+}
+
 extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2_draft_stats* out) {
     if (!c || n < 1 || !ids || !out) return S2D2_ERR_INVALID;
     const int B = c->dc.block_size, MASK = c->m.vocab;
@@ -651,34 +677,44 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     for (int i = 0; i < n; ++i) {
         SeqState* s = get_seq(c, ids[i]);
         if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
-        if (s->drafted) FAIL(c, S2D2_ERR_STATE, "draft_block called twice without accept_and_commit");
+        // a sequence whose draft rows a later draft pass has overwritten may (and must) be drafted again
+        if (s->drafted && s->draft_stamp == c->draft_gen) FAIL(c, S2D2_ERR_STATE, "draft_block called twice without accept_and_commit");
         for (int k = 0; k < i; ++k)
             if (ids[k] == ids[i]) FAIL(c, S2D2_ERR_INVALID, "duplicate sequence id");
         if (!s->block_open && s->n_final + B > c->dc.max_seq_len) FAIL(c, S2D2_ERR_OOM, "max_seq_len reached");
     }
     PassBuild pb;
+    ++c->draft_gen;
     for (int i = 0; i < n; ++i) {
         SeqState& s = c->seqs[ids[i]];
+        s.draft_stamp = c->draft_gen;
+        s.verify_in_flight = false;       // a verifier pass made for an overwritten draft is void (its K/V rows lie past the cache length)
         if (!s.block_open) {
             s.tok.resize(s.n_final + B, MASK);
             s.block_open = true;
         }
         int st = s.n_final, j = 0;
         while (j < B && s.tok[st + j] != MASK) ++j;
-        int P = st + j - s.n_c;          // committed tokens without K/V
+        // Right-shifted layout: the logits that score in-block position i are those of the row at position i - 1, so the
+        // pass starts at the last committed token even when its K/V is cached already (the cache visible to the pass
+        // then ends before it, and the cached K/V is kept).
+        const bool shifted = c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED;
+        int q0 = shifted ? std::min(s.n_c, st + j - 1) : s.n_c;
+        int P = st + j - q0;             // committed tokens that run as causal rows (those without K/V get it appended)
         int rows = P + (B - j);
         if (rows > S2D2_MAX_ROWS_PER_SEQ) FAIL(c, S2D2_ERR_UNSUPPORTED, "too many rows for one sequence in a draft pass");
         if ((rc = ensure_pages(c, s, st + B))) return rc;
-        begin_seq(c, pb, s, s.n_c);
+        begin_seq(c, pb, s, q0);
         unsigned long long all = rows == 64 ? ~0ull : ((1ull << rows) - 1);
-        for (int p = 0; p < P; ++p)     // pending rows: causal among themselves, K/V appended
-            add_row(c, pb, s.tok[s.n_c + p], s.n_c + p, (1ull << (p + 1)) - 1, ROW_WRITE_KV, false);
         s.j = j;
         s.n_masked = 0;
         s.draft_row0 = pb.n_logit;
+        for (int p = 0; p < P; ++p)     // pending rows: causal among themselves, K/V appended
+            add_row(c, pb, s.tok[q0 + p], q0 + p, (1ull << (p + 1)) - 1, q0 + p >= s.n_c ? ROW_WRITE_KV : 0, shifted && p == P - 1);
         for (int i2 = j; i2 < B; ++i2) {  // block rows: see the whole pass
             bool masked = s.tok[st + i2] == MASK;
-            add_row(c, pb, s.tok[st + i2], st + i2, all, 0, masked);
+            bool scores_masked = shifted ? (i2 + 1 < B && s.tok[st + i2 + 1] == MASK) : masked;
+            add_row(c, pb, s.tok[st + i2], st + i2, all, 0, scores_masked);
             if (masked) s.masked_idx[s.n_masked++] = i2;
         }
         s.span_len = 1;
@@ -687,15 +723,18 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     if (pb.n_logit > c->max_logit_rows || pb.n_rows > c->max_rows) FAIL(c, S2D2_ERR_UNSUPPORTED, "pass too large");
     CUDA_TRY(c, cudaEventRecord(c->ev[0], c->stream));
     if ((rc = run_pass(c, pb, c->logits_draft))) return rc;
-    DraftStatsOut so{c->d_xhat, c->d_conf, c->d_margin, c->d_entropy, c->d_lse};
-    {
-        const int nch = vocab_chunks(c->m.vocab);
-        vocab_chunk_stats_kernel<<<dim3(nch, pb.n_logit), VCHUNK_THREADS, 0, c->stream>>>(c->logits_draft, c->m.vocab,
-                                                                                         (ChunkStats*)c->chunk_d);
-        LAUNCHED(c);
-        draft_finish_kernel<<<(pb.n_logit + 3) / 4, 128, 0, c->stream>>>((const ChunkStats*)c->chunk_d, nch, pb.n_logit, so);
-        LAUNCHED(c);
+    if (c->dc.draft_mode == S2D2_DRAFT_SAMPLE) {      // Philox words of the logit rows, in row order
+        int r = 0;
+        for (int i = 0; i < n; ++i) {
+            const SeqState& s = c->seqs[ids[i]];
+            for (int k = 0; k < s.n_masked; ++k, ++r) {
+                c->dsamp_h[r] = s.n_final + s.masked_idx[k];
+                c->dsamp_h[pb.n_logit + r] = (int)s.rng_stream;
+                c->dsamp_h[2 * pb.n_logit + r] = s.step;
+            }
+        }
     }
+    if ((rc = launch_draft_stats(c, c->logits_draft, pb.n_logit, c->dc.draft_mode))) return rc;
     size_t R = pb.n_logit;
     int* hx = (int*)c->stats_h;
     float* hc = (float*)(c->stats_h + R * 4);
@@ -714,6 +753,7 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
     cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]);
     c->cnt.ms_draft += ms;
     c->cnt.n_draft_passes++;
+    c->cnt.n_rows_draft += pb.n_rows;
     c->n_draft_logit_rows = pb.n_logit;
     for (int i = 0; i < n; ++i) {
         SeqState& s = c->seqs[ids[i]];
@@ -752,9 +792,16 @@ extern "C" int s2d2_set_router(s2d2_ctx* c, s2d2_route_fn fn, void* user) {
     return S2D2_OK;
 }
 extern "C" int s2d2_set_route_policy(s2d2_ctx* c, const s2d2_route_policy* p) {
-    if (!c || !p || p->policy < 0 || p->policy > S2D2_ROUTE_NEVER) return S2D2_ERR_INVALID;
+    if (!c || !p || p->policy < 0 || p->policy > S2D2_ROUTE_UCB) return S2D2_ERR_INVALID;
+    if (p->policy == S2D2_ROUTE_UCB && (p->p1 < 0.f || p->p1 > 16.f)) FAIL(c, S2D2_ERR_INVALID, "route policy: bins per context dimension must be 0..16");
     c->policy = *p;
-    for (auto& s : c->seqs) s.hyst_on = true;
+    for (auto& s : c->seqs) {
+        s.hyst_on = true;
+        s.ucb_bucket = -1;
+    }
+    c->ucb_t = 0;
+    c->ucb_n.clear();
+    c->ucb_sum.clear();
     return S2D2_OK;
 }
 
@@ -770,6 +817,24 @@ static double route_score(const s2d2_ctx* c, const s2d2_draft_stats* st) {
         khat += prod;
     }
     return p.dynamic_cost ? khat - (double)p.cost * st->n_hi : khat - (double)p.cost;
+}
+
+// Contextual-bandit router (Appendix "Contextual-bandit routing policy", Eq. (ucb)).
+static int ucb_bins(const s2d2_ctx* c) { return c->policy.p1 >= 1.f ? (int)c->policy.p1 : 2; }
+static int ucb_bucket_of(const s2d2_ctx* c, const s2d2_draft_stats* st) {
+    const int nb = ucb_bins(c), B = c->dc.block_size;
+    const int b_span = std::min(nb - 1, (st->span_len - 1) * nb / B);
+    const int b_prog = std::min(nb - 1, (B - st->n_masked) * nb / B);
+    double h = 0;
+    for (int i = 0; i < st->span_len; ++i) h += st->entropy[i];
+    h /= (double)st->span_len * log((double)c->m.vocab);
+    const int b_ent = std::min(nb - 1, std::max(0, (int)floor(h * nb)));
+    return (b_span * nb + b_prog) * nb + b_ent;
+}
+static double ucb_index(const s2d2_ctx* c, int action, int bucket) {
+    const long long n = c->ucb_n[2 * bucket + action];
+    if (n == 0) return INFINITY;
+    return c->ucb_sum[2 * bucket + action] / (double)n + (double)c->policy.p0 * sqrt(log((double)c->ucb_t) / (double)n);
 }
 
 extern "C" int s2d2_route(s2d2_ctx* c, int32_t n, const s2d2_draft_stats* st, uint8_t* flags) {
@@ -793,6 +858,22 @@ extern "C" int s2d2_route(s2d2_ctx* c, int32_t n, const s2d2_draft_stats* st, ui
                 break;
             }
             case S2D2_ROUTE_MEAN_CONF: flags[i] = st[i].mean_conf < p.p0; break;
+            case S2D2_ROUTE_UCB: {
+                SeqState* s = get_seq(c, st[i].seq_id);
+                if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id in stats");
+                if (st[i].span_len < 1 || st[i].span_len > c->dc.block_size || st[i].n_masked < st[i].span_len)
+                    FAIL(c, S2D2_ERR_INVALID, "draft stats: span");
+                const int nb = ucb_bins(c);
+                if (c->ucb_n.empty()) {
+                    c->ucb_n.assign((size_t)2 * nb * nb * nb, 0);
+                    c->ucb_sum.assign((size_t)2 * nb * nb * nb, 0.0);
+                }
+                ++c->ucb_t;
+                const int b = ucb_bucket_of(c, &st[i]);
+                flags[i] = ucb_index(c, 1, b) >= ucb_index(c, 0, b);
+                s->ucb_bucket = b;
+                break;
+            }
             default: flags[i] = 0;
         }
     }
@@ -811,13 +892,41 @@ extern "C" int s2d2_verify_block(s2d2_ctx* c, int32_t n, const int32_t* ids, con
         SeqState* s = get_seq(c, ids[i]);
         if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
         if (!s->drafted) FAIL(c, S2D2_ERR_STATE, "verify_block without a draft pass");
+        if (s->draft_stamp != c->draft_gen)
+            FAIL(c, S2D2_ERR_STATE, "the draft pass of this sequence was overwritten by a later draft_block: draft it again");
         if (s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "verify_block called twice");
+        for (int k = 0; k < i; ++k)
+            if (ids[k] == ids[i]) FAIL(c, S2D2_ERR_INVALID, "duplicate sequence id");
+    }
+    // one verifier pass per step: sequences verified by an earlier call of this step would lose their rows
+    for (auto& other : c->seqs)
+        if (other.active && other.verify_in_flight && other.verify_stamp == c->verify_gen && other.draft_stamp == c->draft_gen) {
+            bool flagged_now = false;
+            for (int i = 0; i < n; ++i) flagged_now = flagged_now || (flags[i] != 0);
+            if (flagged_now) FAIL(c, S2D2_ERR_STATE, "a second verify_block before accept_and_commit would overwrite the first one's logits");
+            break;
+        }
+    {
+        bool any = false;
+        for (int i = 0; i < n; ++i) any = any || flags[i];
+        if (any) ++c->verify_gen;
     }
     for (int i = 0; i < n; ++i) {
         if (!flags[i]) continue;
         SeqState& s = c->seqs[ids[i]];
         int L = s.span_len, p0 = s.n_final + s.j;
         if ((rc = ensure_pages(c, s, p0 + L))) return rc;
+        s.verify_stamp = c->verify_gen;
+        if (c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED) {
+            // L causal rows: the last committed token (its K/V is in the cache since the draft pass; the cache visible
+            // to this pass ends before it), then the drafted tokens but the last; row k scores drafted token k + 1
+            begin_seq(c, pb, s, p0 - 1);
+            s.verify_row0 = pb.n_logit;
+            add_row(c, pb, s.tok[p0 - 1], p0 - 1, 1ull, 0, true);
+            for (int k = 1; k < L; ++k) add_row(c, pb, s.xhat[k - 1], p0 + k - 1, (1ull << (k + 1)) - 1, ROW_WRITE_KV, true);
+            s.verify_in_flight = true;
+            continue;
+        }
         begin_seq(c, pb, s, s.n_c);
         s.verify_row0 = pb.n_logit;
         // drafted tokens: causal block A_L; their K/V goes to the cache speculatively
@@ -834,6 +943,7 @@ extern "C" int s2d2_verify_block(s2d2_ctx* c, int32_t n, const int32_t* ids, con
     CUDA_TRY(c, cudaEventRecord(c->ev[3], c->stream));
     c->verify_timing_pending = true;
     c->cnt.n_verify_passes++;
+    c->cnt.n_rows_verify += pb.n_rows;
     return S2D2_OK;
 }
 
@@ -928,6 +1038,10 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
         SeqState* s = get_seq(c, ids[i]);
         if (!s) FAIL(c, S2D2_ERR_INVALID, "bad sequence id");
         if (!s->drafted) FAIL(c, S2D2_ERR_STATE, "accept_and_commit without a draft pass");
+        if (s->draft_stamp != c->draft_gen)
+            FAIL(c, S2D2_ERR_STATE, "the draft pass of this sequence was overwritten by a later draft_block: draft it again");
+        if (flags[i] && s->verify_in_flight && s->verify_stamp != c->verify_gen)
+            FAIL(c, S2D2_ERR_STATE, "the verifier pass of this sequence was overwritten by a later verify_block");
         if (flags[i] && !s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "sequence flagged verified but verify_block did not run for it");
         if (!flags[i] && s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "verify flags differ from those given to verify_block");
     }
@@ -989,7 +1103,9 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
                 o.committed_idx[o.n_committed] = s.j + k;
                 o.committed_tok[o.n_committed++] = s.xhat[k];
             }
-            s.n_c += na;   // accepted drafted rows keep their K/V; rows past them are rolled back by length
+            // accepted drafted rows keep their K/V; rows past them are rolled back by length (the right-shifted
+            // verifier has no row for the last drafted token: it gets its K/V in the next draft pass)
+            s.n_c += c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED ? std::min(na, s.span_len - 1) : na;
             if (h_rej[i] >= 0 && c->dc.resample) {
                 s.tok[st + s.j + na] = h_res[i];
                 o.committed_idx[o.n_committed] = s.j + na;
@@ -1006,6 +1122,13 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
                     o.committed_idx[o.n_committed] = s.masked_idx[k];
                     o.committed_tok[o.n_committed++] = s.xhat[k];
                 }
+        }
+        if (c->policy.policy == S2D2_ROUTE_UCB && !c->route_fn && s.ucb_bucket >= 0 && !c->ucb_n.empty()) {
+            // reward of the step: tokens it committed / its cost (2 forward passes when verified, else 1)
+            const int a = flags[i] ? 1 : 0;
+            c->ucb_n[2 * s.ucb_bucket + a] += 1;
+            c->ucb_sum[2 * s.ucb_bucket + a] += (double)o.n_committed / (a ? 2.0 : 1.0);
+            s.ucb_bucket = -1;
         }
         c->cnt.n_committed_tokens += o.n_committed;
         c->cnt.n_steps++;
@@ -1064,6 +1187,31 @@ extern "C" int s2d2_accept_logits(s2d2_ctx* c, const float* d_draft, const float
             o.v[k] = ((const float*)(c->acc_h + a.o_v))[(size_t)i * S2D2_MAX_BLOCK + k];
         }
     }
+    return S2D2_OK;
+}
+
+extern "C" int s2d2_sample_logits(s2d2_ctx* c, const float* d_logits, int32_t n_rows, int32_t draft_mode, const int32_t* position,
+                                  const uint32_t* rng_stream, const int32_t* step, int32_t* xhat_out, float* conf_out,
+                                  float* margin_out, float* entropy_out) {
+    if (!c || !d_logits || n_rows < 1 || !xhat_out || !conf_out || !margin_out || !entropy_out) return S2D2_ERR_INVALID;
+    if (draft_mode != S2D2_DRAFT_GREEDY && draft_mode != S2D2_DRAFT_SAMPLE) FAIL(c, S2D2_ERR_INVALID, "sample_logits: draft_mode");
+    if (n_rows > c->max_logit_rows) FAIL(c, S2D2_ERR_INVALID, "sample_logits: more rows than the context holds");
+    if (draft_mode == S2D2_DRAFT_SAMPLE) {
+        if (!position || !rng_stream || !step) FAIL(c, S2D2_ERR_INVALID, "sample_logits: Philox words missing");
+        for (int r = 0; r < n_rows; ++r) {
+            c->dsamp_h[r] = position[r];
+            c->dsamp_h[n_rows + r] = (int)rng_stream[r];
+            c->dsamp_h[2 * n_rows + r] = step[r];
+        }
+    }
+    int rc = launch_draft_stats(c, d_logits, n_rows, draft_mode);
+    if (rc) return rc;
+    const size_t R = n_rows;
+    CUDA_TRY(c, cudaMemcpyAsync(xhat_out, c->d_xhat, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(conf_out, c->d_conf, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(margin_out, c->d_margin, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(entropy_out, c->d_entropy, R * 4, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     return S2D2_OK;
 }
 

@@ -359,6 +359,94 @@ __device__ __forceinline__ void load_chunk_contiguous(const float* row, int V, i
         }
     }
 }
+// SampleFromLogits, sampling mode: xhat ~ pi_d by inverse CDF in vocabulary order with one uniform of the
+// draft-sampling Philox stream; conf = pi_d(xhat).  One CTA per logit row, after stage 1 and the greedy stage 2
+// (which leave margin, entropy and the log-sum-exp of the row; this kernel replaces xhat and conf).  Thread 0 walks
+// the chunk masses s_c * exp(mx_c - mx) to the chunk that holds u * sum, the CTA then walks that chunk (prefix over
+// threads in vocabulary order, then the owning thread over its 16 entries), all in fp64.
+struct DraftSampleIn {
+    const float* logits;
+    int V;
+    const ChunkStats* chunks;
+    const int* row_pos;          // absolute position of the row's token
+    const unsigned* row_stream;  // Philox sequence stream
+    const int* row_step;         // Philox step word
+    unsigned seed;
+};
+static __global__ void __launch_bounds__(VCHUNK_THREADS) draft_sample_kernel(DraftSampleIn in, int n_chunks, DraftStatsOut o) {
+    __shared__ double sh_warp[VCHUNK_THREADS / 32];
+    __shared__ double sh_target, sh_mx;
+    __shared__ int sh_chunk, sh_pick;
+    const int r = blockIdx.x;
+    const ChunkStats* cs = in.chunks + (size_t)r * n_chunks;
+    const float* row = in.logits + (size_t)r * in.V;
+    if (threadIdx.x == 0) {
+        float mxf = -INFINITY;
+        for (int c = 0; c < n_chunks; ++c) mxf = fmaxf(mxf, cs[c].mx);
+        const double mx = (double)mxf;
+        double total = 0.0;
+        for (int c = 0; c < n_chunks; ++c) total += cs[c].s * exp((double)cs[c].mx - mx);
+        const double u = philox_uniform(in.seed, (unsigned)in.row_pos[r], in.row_stream[r], (unsigned)in.row_step[r], STREAM_DRAFT);
+        const double target = u * total;
+        double before = 0.0;
+        int pick_chunk = -1;
+        for (int c = 0; c < n_chunks; ++c) {
+            const double m = cs[c].s * exp((double)cs[c].mx - mx);
+            if (before + m > target) {
+                pick_chunk = c;
+                break;
+            }
+            before += m;
+        }
+        sh_chunk = pick_chunk;
+        sh_target = target - before;
+        sh_mx = mx;
+        sh_pick = in.V - 1;
+    }
+    __syncthreads();
+    const int chunk = sh_chunk;
+    if (chunk >= 0) {
+        const double target = sh_target, mx = sh_mx;
+        float x[VPER];
+        load_chunk_contiguous(row, in.V, chunk * VCHUNK, threadIdx.x, x);
+        double w[VPER], mine = 0.0;
+#pragma unroll
+        for (int k = 0; k < VPER; ++k) {
+            w[k] = x[k] == -INFINITY ? 0.0 : exp((double)x[k] - mx);
+            mine += w[k];
+        }
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        double incl = mine;
+#pragma unroll
+        for (int k = 1; k < 32; k <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, k);
+            if (lane >= k) incl += up;
+        }
+        if (lane == 31) sh_warp[warp] = incl;
+        __syncthreads();
+        double before = incl - mine;
+        for (int k = 0; k < warp; ++k) before += sh_warp[k];
+        if (before <= target && before + mine > target) {
+            int pick = VPER - 1;
+#pragma unroll
+            for (int k = VPER - 1; k >= 0; --k) {
+                double upto = before;
+#pragma unroll
+                for (int j = 0; j < VPER; ++j)
+                    if (j <= k) upto += w[j];
+                if (upto > target) pick = k;
+            }
+            atomicMin(&sh_pick, min(in.V - 1, chunk * VCHUNK + (int)threadIdx.x * VPER + pick));
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int tok = sh_pick;
+        o.xhat[r] = tok;
+        o.conf[r] = (float)exp((double)row[tok] - o.lse[r]);
+    }
+}
+
 static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_chunk_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
                                                                                double* __restrict__ rsum, double* __restrict__ vsum) {
     __shared__ double sh_d[32];

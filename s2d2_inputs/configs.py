@@ -75,6 +75,10 @@ _t_moe = ModelConfig("t-moe-bf16", 2, 256, 4, 2, 64, 0, 1000,
                      n_experts=16, top_k=4, expert_ffn=128, n_shared=1)
 _t_moe128 = ModelConfig("t-moe128-bf16", 2, 256, 4, 2, 64, 0, 1000,
                         n_experts=128, top_k=8, expert_ffn=128, n_shared=1)
+# the attention geometry of the 8B-/4B-class and of the MoE workloads (query / kv heads, head_dim, 64-token pages)
+# on a narrow two-layer body, so that the CPU side can afford contexts of one to two thousand tokens
+_t_geo32 = ModelConfig("t-geo-32q8kv", 2, 1024, 32, 8, 128, 2048, 2000)
+_t_geo16 = ModelConfig("t-geo-16q4kv", 2, 1024, 16, 4, 128, 2048, 2000)
 _t_f32 = ModelConfig("t-dense-fp32", 2, 64, 2, 1, 32, 96, 50, dtype="fp32",
                      rope_base=1.0e4, qk_norm=True, logit_scale=3.0)
 
@@ -84,12 +88,17 @@ CONFIGS = {
     "c3": WorkloadConfig("c3", _c3, 8, (128, 512), 4, 512, route="mean_conf"),
     "c4": WorkloadConfig("c4", _c4, 1, (1024, 1024), 8, 1024),
     "c4b32": WorkloadConfig("c4b32", _c4, 32, (1024, 1024), 8, 1024),
+    # the paper's batched runs on the 8B-class model use block size 16 and batch sizes up to 64 (its table of batched
+    # throughput): draft passes of 1024 rows, verifier passes of 2048 rows (the 2L construction)
+    "c4b64": WorkloadConfig("c4b64", _c4, 64, (1024, 1024), 16, 1024),
     "c5": WorkloadConfig("c5", _c5, 1, (512, 512), 32, 1024),
     "t_bf16": WorkloadConfig("t_bf16", _t_bf16, 3, (5, 70), 4, 16, kv_page_tokens=16),
     "t_bf16_128": WorkloadConfig("t_bf16_128", _t_bf16_128, 2, (60, 130), 8, 24),
     "t_moe": WorkloadConfig("t_moe", _t_moe, 2, (9, 40), 8, 16, kv_page_tokens=16),
     "t_moe128": WorkloadConfig("t_moe128", _t_moe128, 2, (9, 40), 8, 16, kv_page_tokens=16),
     "t_f32": WorkloadConfig("t_f32", _t_f32, 2, (3, 20), 4, 12, kv_page_tokens=8),
+    "t_geo32": WorkloadConfig("t_geo32", _t_geo32, 1, (1100, 1100), 8, 24),
+    "t_geo16": WorkloadConfig("t_geo16", _t_geo16, 1, (1100, 1100), 32, 64),
 }
 
 

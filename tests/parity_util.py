@@ -39,7 +39,9 @@ class ParityReport:
     n_accepted: int = 0
     n_resampled: int = 0
     n_committed: int = 0
-    moe_forced_rows: int = 0
+    moe_forced_rows: int = 0          # (row, layer) pairs whose expert set the oracle took from the engine (near ties)
+    moe_rows_checked: int = 0         # (row, layer) pairs compared
+    moe_max_forced_gap: float = 0.0   # largest distance of a swapped expert's router logit from the oracle's k-th
 
 
 class OracleShadow:
@@ -61,12 +63,17 @@ class OracleShadow:
 
 def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: int = 1, seed: Optional[int] = None,
               gamma: float = 1.0, tau_conf: float = 0.9, logit_atol: float = 2e-2, logit_rtol: float = 0.0,
-              route=None, shadows=None, stage_b_seqs=None, resample: bool = True) -> ParityReport:
+              route=None, shadows=None, stage_b_seqs=None, resample: bool = True, layout: str = "aligned",
+              stage_b_steps: Optional[int] = None, draft_mode: str = "greedy") -> ParityReport:
     """Run up to ``n_steps`` decode steps on all sequences (stops when every one has
     generated wl.gen_tokens) and check both parity stages.  ``stage_b_seqs``: restrict the
     oracle's forward (stage B) to these sequence ids (large batches at full model size); stage A
     always covers every sequence.  ``resample=False``: the reject-only variant (the first rejected position stays
-    masked and is drafted again in the next step)."""
+    masked and is drafted again in the next step).  ``layout="shifted"``: the right-shifted verifier layout (L causal
+    verifier rows, logits read one row to the left in both passes).  ``stage_b_steps``: run stage B on the first so many
+    steps only (long runs at full model size).  ``draft_mode="sample"``: proposals drawn from pi_d with the
+    draft-sampling uniforms."""
+    shifted = layout == "shifted"
     cfg, B = wl.model, wl.block_size
     MASK = cfg.mask_id
     seed = wl.philox_seed if seed is None else seed
@@ -89,7 +96,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
         eid_v = engine.debug_copy_expert_ids(64 * len(live)) if (cfg.is_moe and flags.any()) else None
         vlog = engine.debug_copy_logits(1, sum(s.span_len for s, f in zip(stats, flags) if f)) if flags.any() else None
         res = engine.accept_and_commit(live, flags)
-        do_b = stage_b_every > 0 and step_no % stage_b_every == 0
+        do_b = stage_b_every > 0 and step_no % stage_b_every == 0 and (stage_b_steps is None or step_no < stage_b_steps)
         drow = vrow = drow_all = vrow_all = 0
         for k, sid in enumerate(live):
             st, rs, bf = stats[k], res[k], before[sid]
@@ -104,7 +111,11 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
             my_d = dlog[drow:drow + nm]
             drow += nm
             # ---- stage A on the engine's logits ------------------------------------------------
-            o_stats = [A.sample_from_logits(my_d[r]) for r in range(nm)]
+            if draft_mode == "sample":
+                o_stats = [A.sample_from_logits(my_d[r], "sample", philox.uniform(seed, s0 + masked[r], rng_streams[sid], bf["step"], philox.STREAM_DRAFT))
+                           for r in range(nm)]
+            else:
+                o_stats = [A.sample_from_logits(my_d[r]) for r in range(nm)]
             xhat = [q.xhat for q in o_stats]
             exempt = False
             if xhat != list(st.xhat[:nm]):
@@ -162,20 +173,22 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
             rep.n_committed += rs.n_committed
             # ---- stage B: the oracle's own forward ------------------------------------------------
             n_c0 = bf["n_cached"]
-            n_draft_rows = (s0 + j - n_c0) + (B - j)
+            q0 = min(n_c0, s0 + j - 1) if shifted else n_c0       # first row of the draft pass
+            n_draft_rows = (s0 + j - q0) + (B - j)
             if do_b and (stage_b_seqs is None or sid in stage_b_seqs):
                 sh = shadows[sid]
                 if not cfg.is_moe:
                     sh.extend(full, n_c0)
                 assert sh.n == n_c0 or not cfg.is_moe
-                pend_pos = list(range(n_c0, s0 + j))
+                pend_pos = list(range(q0, s0 + j))
                 toks, pos, mask = S.draft_pass_rows([full[p] for p in pend_pos], pend_pos, blk[j:], list(range(s0 + j, s0 + B)))
-                need = [len(pend_pos) + (i - j) for i in masked]
+                need = [len(pend_pos) + (i - j) - (1 if shifted else 0) for i in masked]
                 forced, tr = None, None
+                visible = sh.cache if q0 == n_c0 else [(k_[:q0], v_[:q0]) for k_, v_ in sh.cache]
                 if cfg.is_moe:
                     forced = [eid_d[l][drow_all:drow_all + n_draft_rows] for l in range(cfg.n_layers)]
                     tr = {}
-                ol, kv = M.forward(W, cfg, toks, pos, mask, sh.cache, need_logits=need, forced_expert_ids=forced, trace=tr)
+                ol, kv = M.forward(W, cfg, toks, pos, mask, visible, need_logits=need, forced_expert_ids=forced, trace=tr)
                 if cfg.is_moe:
                     _check_expert_choice(rep, tag + " draft", tr, forced, cfg.top_k)
                     if pend_pos:                       # mirror the engine: pending rows enter the cache
@@ -186,12 +199,18 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
                 if flags[k]:
                     if not cfg.is_moe:
                         sh.extend(full, s0 + j)
-                    vt, vp, vm = S.verify_pass_rows(list(st.xhat[:L]), [s0 + j + i for i in range(L)], MASK)
-                    if cfg.is_moe:
-                        forced = [eid_v[l][vrow_all:vrow_all + 2 * L] for l in range(cfg.n_layers)]
-                        tr = {}
-                    ov, vkv = M.forward(W, cfg, vt, vp, vm, sh.cache, need_logits=list(range(L, 2 * L)),
-                                        forced_expert_ids=forced, trace=tr)
+                    if shifted:
+                        assert not cfg.is_moe
+                        vt, vp, vm = S.verify_pass_rows_shifted(full[s0 + j - 1], list(st.xhat[:L]), s0 + j)
+                        vis = [(k_[:s0 + j - 1], v_[:s0 + j - 1]) for k_, v_ in sh.cache]
+                        ov, vkv = M.forward(W, cfg, vt, vp, vm, vis, need_logits=list(range(L)))
+                    else:
+                        vt, vp, vm = S.verify_pass_rows(list(st.xhat[:L]), [s0 + j + i for i in range(L)], MASK)
+                        if cfg.is_moe:
+                            forced = [eid_v[l][vrow_all:vrow_all + 2 * L] for l in range(cfg.n_layers)]
+                            tr = {}
+                        ov, vkv = M.forward(W, cfg, vt, vp, vm, sh.cache, need_logits=list(range(L, 2 * L)),
+                                            forced_expert_ids=forced, trace=tr)
                     if cfg.is_moe:
                         _check_expert_choice(rep, tag + " verify", tr, forced, cfg.top_k)
                         if rs.n_accepted:              # accepted drafted rows keep their K/V
@@ -201,7 +220,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
                     rep.stage_b_passes += 1
             drow_all += n_draft_rows
             if flags[k]:
-                vrow_all += 2 * L
+                vrow_all += L if shifted else 2 * L
         rep.steps += 1
     return rep
 
@@ -260,13 +279,16 @@ def _check_expert_choice(rep: ParityReport, tag: str, trace: dict, forced, top_k
         for r in range(logits.shape[0]):
             mine = set(order[r, :top_k].tolist())
             theirs = set(int(e) for e in forced[l][r])
+            rep.moe_rows_checked += 1
             if len(theirs) != top_k:
                 rep.mismatches.append(f"{tag}: layer {l} row {r}: duplicate expert ids")
             if mine == theirs:
                 continue
             kth = logits[r, order[r, top_k - 1]]
-            if all(abs(logits[r, e] - kth) < tie_tol for e in mine ^ theirs):
+            gap = max(abs(logits[r, e] - kth) for e in mine ^ theirs)
+            if gap < tie_tol:
                 rep.moe_forced_rows += 1
+                rep.moe_max_forced_gap = max(rep.moe_max_forced_gap, float(gap))
             else:
                 rep.mismatches.append(f"{tag}: layer {l} row {r}: expert set {sorted(theirs)} vs {sorted(mine)}")
 

@@ -191,6 +191,26 @@ def test_error_paths_return_codes_not_faults():
     with pytest.raises(S2D2Error):
         e.draft_block([sid])
     e.close()
+    # one step uses one id list: a later draft pass overwrites the rows an earlier one produced
+    e = _engine(wl, W, max_batch=2)
+    a, b = e.prefill([[1, 2, 3], [4, 5, 6, 7]])
+    e.draft_block([a])
+    e.draft_block([b])
+    for call in (lambda: e.verify_block([a], [1]), lambda: e.accept_and_commit([a], [0])):
+        with pytest.raises(S2D2Error) as ei:
+            call()
+        assert ei.value.code == -4 and "draft it again" in str(ei.value)
+    e.verify_block([b], [1])
+    with pytest.raises(S2D2Error) as ei:                 # a second verifier pass would overwrite the first one's logits
+        e.verify_block([b], [1])
+    assert ei.value.code == -4
+    e.accept_and_commit([b], [1])
+    st = e.draft_block([a, b])                           # a is drafted again, together with b's next step
+    fl = e.route(st)
+    e.verify_block([a, b], fl)
+    res = e.accept_and_commit([a, b], fl)
+    assert all(r.n_committed >= 1 for r in res)
+    e.close()
 
 
 def test_bounded_wait_times_out_with_a_status_not_a_hang():
@@ -290,4 +310,97 @@ def test_accept_variants_match_oracle(kw):
     if not kw.get("resample", True):
         assert e.get_counters().n_resampled == 0
         assert rep.n_committed == rep.n_accepted            # only accepted drafts are ever committed
+    e.close()
+
+
+@pytest.mark.parametrize("name,atol,rtol", [("c1", 0.0, 1e-4), ("t_f32", 0.0, 1e-4), ("t_bf16", 2e-2, 0.0), ("t_bf16_128", 2e-2, 0.0)])
+def test_right_shifted_verifier_layout_matches_oracle(name, atol, rtol):
+    """S2D2_VERIFIER_RIGHT_SHIFTED (Section "Self-Verification Mode": for right-shifted models the plain causal
+    mask gives the verifier view): L causal verifier rows instead of 2L, logits read one row to the left in both
+    passes, every pass starting at the last committed token.  Both parity stages over the whole generation,
+    the cache against the oracle's causal pass, and for the fp32 workload the free-running token stream."""
+    from tests.parity_util import check_kv, run_steps
+    wl = get_config(name)
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.0 if name == "c1" else 0.1)
+    e, ids, prompts = _start(wl, W, verifier_layout="shifted")
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_atol=atol, logit_rtol=rtol,
+                    layout="shifted")
+    print(name, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps > 0 and rep.n_committed == wl.gen_tokens * len(ids)
+    for sid in ids:
+        check_kv(e, W, wl.model, sid, atol=1e-5 if wl.model.dtype == "fp32" else 4e-2)
+    e.close()
+    if name == "c1":
+        e, ids, prompts = _start(wl, W, verifier_layout="shifted")
+        e.generate(ids, wl.gen_tokens)
+        got = e.get_tokens(ids[0])[len(prompts[0]):].tolist()
+        orc = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0, layout="shifted")
+        assert got == orc.generate(prompts[0], wl.gen_tokens)
+        c = e.get_counters()
+        assert c.n_draft_passes == orc.n_draft_passes and c.n_verify_passes == orc.n_verify_passes
+        e.close()
+
+
+@pytest.mark.parametrize("V,n_rows", [(8, 6), (4096, 8), (1000, 32), (151936, 8), (157184, 16)])
+def test_sample_from_logits_kernels_on_synthetic_logits(V, n_rows):
+    """SampleFromLogits alone (s2d2_sample_logits): greedy proposals and, in sampling mode, inverse-CDF draws
+    from pi_d with the draft-sampling Philox stream, against the oracle on the same fp32 logits.  The draw is
+    an integer decided by a floating-point comparison; both sides take it in fp64, and a row whose target lies
+    within 1e-9 of a cumulative-sum boundary (summation order differs) is exempt and counted."""
+    from paper_2603_25702_b200 import Engine
+    wl = get_config("t_f32", model_vocab=V)
+    e = Engine(wl.model, block_size=min(n_rows, 32), max_batch=max(1, (n_rows + 31) // 32), max_seq_len=64, kv_page_tokens=8, seed=9,
+               stream=torch.cuda.current_stream().cuda_stream)
+    rng = np.random.default_rng(V + n_rows)
+    exempt = 0
+    for trial in range(3):
+        x = (rng.standard_normal((n_rows, V)) * (0.5 + 1.5 * trial)).astype(np.float32)
+        if trial == 2:
+            x[:, V // 3] += 6.0                 # a peaked row: most draws land on one token
+        pos = rng.integers(0, 5000, size=n_rows)
+        streams = rng.integers(0, 100, size=n_rows)
+        steps = rng.integers(0, 50, size=n_rows)
+        tx = torch.from_numpy(x).cuda()
+        gx, gc, gm, ge = e.sample_logits(tx.data_ptr(), n_rows, "greedy")
+        sx, sc, sm_, se = e.sample_logits(tx.data_ptr(), n_rows, "sample", pos, streams, steps)
+        for r in range(n_rows):
+            og = A.sample_from_logits(x[r])
+            assert og.xhat == gx[r] and abs(og.d - gc[r]) <= 1e-5 * og.d + 1e-9
+            assert abs(og.margin - gm[r]) <= 1e-5 and abs(og.entropy - ge[r]) <= 1e-4 * max(1.0, og.entropy)
+            u = philox.uniform(9, int(pos[r]), int(streams[r]), int(steps[r]), philox.STREAM_DRAFT)
+            os_ = A.sample_from_logits(x[r], "sample", u)
+            p = A.softmax(x[r])
+            c = np.cumsum(p)
+            near = np.abs(c - u * c[-1]).min() < 1e-9
+            exempt += int(near)
+            if not near:
+                assert os_.xhat == sx[r], (trial, r)
+                assert abs(os_.d - sc[r]) <= 1e-5 * os_.d + 1e-9
+            assert abs(os_.margin - sm_[r]) <= 1e-5 and abs(os_.entropy - se[r]) <= 1e-4 * max(1.0, os_.entropy)
+    assert exempt <= 1
+    e.close()
+
+
+def test_sampling_draft_mode_matches_oracle_end_to_end():
+    """S2D2_DRAFT_SAMPLE through the decode loop on the fp32 workload: stage A with sampled proposals on the engine's
+    logits, stage B, and the free-running token stream against the oracle in its sampling mode (the one
+    configuration in which the speculative output law equals the verifier's)."""
+    from tests.parity_util import run_steps
+    wl = get_config("c1")
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.0)
+    e, ids, prompts = _start(wl, W, draft_mode="sample")
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=80, logit_atol=0.0, logit_rtol=1e-4,
+                    draft_mode="sample")
+    print("sample", rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.n_committed == wl.gen_tokens
+    e.close()
+    e, ids, prompts = _start(wl, W, draft_mode="sample")
+    e.generate(ids, wl.gen_tokens)
+    got = e.get_tokens(ids[0])[len(prompts[0]):].tolist()
+    orc = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0, draft_mode="sample")
+    want = orc.generate(prompts[0], wl.gen_tokens)
+    greedy = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0).generate(prompts[0], wl.gen_tokens)
+    assert got == want and want != greedy          # and the sampled trajectory is a different one
     e.close()

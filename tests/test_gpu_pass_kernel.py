@@ -59,15 +59,22 @@ def test_pass_trace_is_monotone_and_complete():
     e.draft_block(ids)
     marks, sm = e.debug_pass_trace()
     e.set_profiling(0)
-    n_ctas, n_bar, _ = marks.shape
-    assert n_bar == 6 * wl.model.n_layers + 2 and n_ctas >= 1     # + the LM-head phase, which has no barrier
-    flat = marks[:, :, :2].reshape(n_ctas, -1).astype(np.int64)
-    assert (np.diff(flat, axis=1) >= 0).all()    # entry <= exit <= next entry for every CTA
-    drained = marks[:, :, 2].astype(np.int64)
-    has = drained > 0                            # phases with a GEMM: drained between the previous exit and the entry
-    assert has.any() and (drained[has] <= marks[:, :, 0].astype(np.int64)[has]).all()
-    # nobody leaves a barrier before everybody has entered it
-    assert (marks[:, :-1, 1].min(axis=0).astype(np.int64) >= marks[:, :-1, 0].max(axis=0).astype(np.int64) - 2000).all()
+    n_ctas, n_marks = marks.shape
+    L = wl.model.n_layers
+    n_named = 3 + 12 * L + 2                             # embedding barrier, 12 marks per dense layer, the LM-head phase
+    assert n_marks >= n_named + 6 * (4 * L + 1) and (n_marks - n_named) % 6 == 0 and n_ctas >= 1     # + two and four per sub-GEMM
+    n_sub = (n_marks - n_named) // 6
+    mma = marks[:, n_named:n_named + 2 * n_sub].reshape(n_ctas, n_sub, 2)
+    assert (mma[:, :, 0] <= mma[:, :, 1]).all() and (mma > 0).any()
+    names = Engine.TRACE_DENSE_MARKS
+    used = [0, 1] + list(range(3, n_named))                # slot 2 is unused
+    flat = marks[:, used]
+    assert (flat > 0).all() and (np.diff(flat, axis=1) >= 0).all()    # every CTA passes its marks in slot order
+    # nobody leaves a grid barrier before everybody has entered it
+    bars = [(0, 1)] + [(3 + 12 * l + names.index(n + "_entry"), 3 + 12 * l + names.index(n + "_exit"))
+                       for l in range(L) for n in ("rope_barrier", "attn_barrier")]
+    for ent, ex in bars:
+        assert marks[:, ex].min() >= marks[:, ent].max() - 2000
     assert len(set(sm.tolist())) == n_ctas       # one CTA per SM
     prof = e.get_gemm_profile()
     assert prof["launches"] >= 1 and prof["bytes"] > 0
@@ -88,3 +95,34 @@ def test_full_shape_passes_repeat_bit_for_bit():
     for step, (x, y) in enumerate(zip(a, b)):
         assert x[2] == y[2], step
         assert np.array_equal(x[0], y[0]) and np.array_equal(x[1], y[1]), step
+
+
+@pytest.mark.parametrize("name", ["t_bf16", "t_bf16_128"])
+def test_sub_gemm_cuts_match_oracle_on_small_models(name):
+    """use_tensor_cores = 3 cuts every GEMM of the persistent kernel into sub-GEMMs wherever the tile counts
+    allow, so a small model runs the hand-overs a large one runs by default: output tiles reduced and turned
+    into the next GEMM's input while the rest streams, the next GEMM starting on those k-blocks, and no grid
+    barrier between the attention block of one layer and the next.  Both parity stages over the whole
+    generation, then the cache against the oracle's causal pass."""
+    from paper_2603_25702_b200 import Engine
+    from tests.parity_util import check_kv, register_prompt_lens, run_steps
+    wl = get_config(name)
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.1)
+    e = Engine(wl.model, block_size=wl.block_size, max_batch=wl.batch, max_seq_len=wl.prompt_len[1] + wl.gen_tokens + wl.block_size,
+               kv_page_tokens=wl.kv_page_tokens, seed=wl.philox_seed, stream=torch.cuda.current_stream().cuda_stream,
+               use_tensor_cores=3)
+    e.load_weights(W)
+    prompts = generate_prompts(wl)
+    ids = e.prefill(prompts)
+    register_prompt_lens(ids, prompts)
+    for k, sid in enumerate(ids):
+        e.seq_set_rng_stream(sid, k)
+    e.reset_counters()
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_atol=2e-2)
+    print(name, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.n_committed == wl.gen_tokens * len(ids)
+    assert e.get_counters().n_kernel_launches < 12 * rep.steps     # persistent passes
+    for sid in ids:
+        check_kv(e, W, wl.model, sid, atol=4e-2)
+    e.close()

@@ -88,3 +88,33 @@ def test_builtin_policies_and_callback_match_the_oracle():
     assert seen == list(ids) and got == [int(arr[k].span_len >= 2) for k in range(2)]
     e.set_router(None)
     e.close()
+
+
+def test_ucb_router_follows_the_oracle_through_a_decode_run():
+    """S2D2_ROUTE_UCB on the tiny fp32 workload with peaked logits, against the oracle's bandit fed with the same
+    statistics and the same rewards: identical decisions at every step, and both actions occur."""
+    from paper_2603_25702_b200 import Engine, RoutePolicy
+    wl = get_config("t_f32", block_size=8, gen_tokens=64, model_logit_scale=12.0)
+    W = generate_weights(wl.model, seed=2, gain_jitter=0.1)
+    e = Engine(wl.model, block_size=8, max_batch=1, max_seq_len=128, kv_page_tokens=8, tau_conf=0.5,
+               stream=torch.cuda.current_stream().cuda_stream)
+    e.load_weights(W)
+    sid = e.prefill([[3, 1, 4, 1, 5]])[0]
+    beta = 0.7
+    e.set_route_policy(RoutePolicy(RoutePolicy.UCB, beta, 0, 0, 0, 0, 0))
+    orc = R.UCBRouter(beta, 8, wl.model.vocab, bins=2)
+    decisions = []
+    for step in range(60):
+        if e.debug_seq_state(sid)["block_start"] >= 5 + 64:
+            break
+        st = e.draft_block([sid])
+        fl = e.route(st)
+        s = st[0]
+        want = orc.decide(s.span_len, s.n_masked, [np.float32(s.entropy[i]) for i in range(s.span_len)])
+        assert bool(fl[0]) == want, step
+        e.verify_block([sid], fl)
+        res = e.accept_and_commit([sid], fl)
+        orc.update(res[0].n_committed)
+        decisions.append(int(fl[0]))
+    assert 0 in decisions and 1 in decisions and len(decisions) >= 8
+    e.close()

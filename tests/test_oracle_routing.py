@@ -34,3 +34,37 @@ def test_hysteresis_sequence():
 
 def test_mean_conf_rule():
     assert R.mean_conf([0.5, 0.95]) and not R.mean_conf([0.95, 0.95]) and not R.mean_conf([0.9, 0.9])
+
+
+def test_ucb_router_hand_computed_sequence():
+    """Eq. (ucb) on a short sequence worked out by hand (beta = 1, block 8, two bins per dimension)."""
+    r = R.UCBRouter(beta=1.0, block_size=8, vocab=100, bins=2)
+    lo = [0.1 * math.log(100)] * 3          # normalised entropy 0.1 -> entropy bin 0
+    # buckets: span 3 of 8 -> bin 0 ((3-1)*2//8 = 0); nothing unmasked yet -> progress bin 0
+    assert r.bucket(3, 8, lo) == (0, 0, 0)
+    assert r.bucket(5, 8, lo) == (1, 0, 0) and r.bucket(8, 8, lo) == (1, 0, 0) and r.bucket(4, 8, lo) == (0, 0, 0)
+    assert r.bucket(2, 4, lo) == (0, 1, 0) and r.bucket(2, 5, lo) == (0, 0, 0)      # 4 of 8 unmasked -> bin 1; 3 of 8 -> bin 0
+    assert r.bucket(3, 8, [0.7 * math.log(100)] * 3) == (0, 0, 1)
+    # t = 1: both actions untried, the tie goes to verification; the step decodes 3 tokens: reward 3 / 2
+    assert r.decide(3, 8, lo) is True
+    r.update(3)
+    # t = 2: action 0 is untried in this bucket -> taken; decodes 1 token: reward 1 / 1
+    assert r.decide(3, 8, lo) is False
+    r.update(1)
+    # t = 3: 1.5 + sqrt(ln 3 / 1) against 1.0 + sqrt(ln 3 / 1) -> verify; decodes 1 token: reward 0.5, mean of action 1 -> 1.0
+    assert abs(r.index(1, (0, 0, 0)) - (1.5 + math.sqrt(math.log(2)))) < 1e-12       # index() reads the current t = 2
+    assert r.decide(3, 8, lo) is True
+    r.update(1)
+    # t = 4: action 1: 1.0 + sqrt(ln 4 / 2) = 1.8326; action 0: 1.0 + sqrt(ln 4 / 1) = 2.1774 -> no verification
+    assert r.decide(3, 8, lo) is False
+    assert abs(r.index(1, (0, 0, 0)) - (1.0 + math.sqrt(math.log(4) / 2))) < 1e-12
+    assert abs(r.index(0, (0, 0, 0)) - (1.0 + math.sqrt(math.log(4)))) < 1e-12
+    r.update(2)
+    # another bucket starts from scratch (verify first), but t keeps counting
+    assert r.decide(8, 8, lo) is True and r.t == 5
+    r.update(8)
+    assert r.n[(1, (1, 0, 0))] == 1 and r.sum[(1, (1, 0, 0))] == 4.0
+    # the caller may override the action actually taken (flags given to the verifier differ from the decision)
+    r.decide(8, 8, lo)
+    r.update(2, action=0)
+    assert r.n[(0, (1, 0, 0))] == 1 and r.sum[(0, (1, 0, 0))] == 2.0

@@ -267,3 +267,75 @@ def test_draft_mask_pins_catch_a_wrong_mask(tiny_f32, mutation):
         _check_rows_against_eq_draft_mask(mutated)
     with pytest.raises(AssertionError):
         _check_draft_logits_against_one_literal_pass(mutated, wl, W)
+
+
+# ---- right-shifted verifier layout (Section "Self-Verification Mode", last sentence) -------------
+def test_shifted_verifier_rows_equal_literal_autoregressive_passes(tiny_f32):
+    """In a right-shifted model the logits at position i - 1 score token i, so verifier row k (the last
+    committed token, then the drafted tokens) must equal the last row of a plain causal pass over
+    prefix ++ xhat_1..xhat_k: the literal next-token distribution, with no MASK anywhere."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = [5, 9, 2, 44, 17, 3, 8]
+    n = len(prompt)
+    _, kv = M.forward(W, cfg, prompt[:-1], np.arange(n - 1), M.causal_mask(n - 1), need_logits=[])
+    cache = M.append_kv(None, kv, np.arange(n - 1))                 # everything before the last committed token
+    xhat = [11, 4, 30, 7]
+    L = len(xhat)
+    vt, vp, vm = S.verify_pass_rows_shifted(prompt[-1], xhat, n)
+    assert vt.tolist() == [prompt[-1]] + xhat[:-1] and vp.tolist() == list(range(n - 1, n - 1 + L))
+    assert vm.tolist() == np.tril(np.ones((L, L), bool)).tolist() and len(vt) == L      # L rows, not 2L
+    got, _ = M.forward(W, cfg, vt, vp, vm, cache)
+    for k in range(L):
+        seq = prompt + xhat[:k]
+        lit, _ = M.forward(W, cfg, seq, np.arange(len(seq)), M.causal_mask(len(seq)))
+        np.testing.assert_allclose(got[k], lit[-1], rtol=1e-9, atol=1e-11)
+
+
+def test_shifted_block_size_one_is_plain_next_token_greedy_decoding(tiny_f32):
+    """B = 1 in the shifted layout: the drafter's row and the verifier's row are the same causal row of
+    the last committed token, so nothing is ever rejected and the tokens are those of the textbook
+    greedy loop (full causal pass over everything so far, argmax of the last row)."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=4)[0][:9]
+    seq = S.SequenceOracle(W, cfg, block_size=1, seed=1, seq_stream=0, keep_logits=True, layout="shifted")
+    out = seq.generate(prompt, 8)
+    toks = [int(t) for t in prompt]
+    want = []
+    for _ in range(8):
+        lit, _ = M.forward(W, cfg, toks, np.arange(len(toks)), M.causal_mask(len(toks)))
+        want.append(int(np.argmax(lit[-1])))
+        toks.append(want[-1])
+    assert out == want
+    for st in seq.trace:
+        assert st.result.n_accepted == 1 and st.result.first_reject == -1 and abs(st.result.a[0] - 1.0) < 1e-9
+        np.testing.assert_allclose(st.verify_logits, st.draft_logits[:1], rtol=1e-9, atol=1e-11)
+
+
+@pytest.mark.parametrize("B", [4, 8])
+def test_shifted_loop_invariants_and_cache_is_causal(tiny_f32, B):
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=5)[1][:6]
+    seq = S.SequenceOracle(W, cfg, block_size=B, seed=1, seq_stream=2, keep_logits=True, layout="shifted")
+    out = seq.generate(prompt, 24)
+    assert len(out) == 24 and all(0 <= t < cfg.vocab for t in out)
+    n_rej = 0
+    for st in seq.trace:
+        assert st.verified and len(st.committed) >= 1
+        r = st.result
+        assert st.verify_logits.shape[0] == len(st.span)            # L verifier rows
+        # the first drafted position is scored by the same causal row in both passes: ratio 1, always accepted
+        assert abs(r.a[0] - 1.0) < 1e-9 and r.n_accepted >= 1
+        np.testing.assert_allclose(st.verify_logits[0], st.draft_logits[0], rtol=1e-9, atol=1e-11)
+        if r.first_reject >= 0:
+            n_rej += 1
+            assert r.resampled != st.xhat[r.first_reject]
+    assert n_rej >= 1
+    full = list(prompt) + out
+    _, kv = M.forward(W, cfg, full, np.arange(len(full)), M.causal_mask(len(full)), need_logits=[])
+    assert seq.n_c < len(full)                                       # the last committed token has no K/V of its own yet, or is re-run
+    for l in range(cfg.n_layers):
+        np.testing.assert_allclose(seq.cache[l][0], kv[l][0][: seq.n_c], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(seq.cache[l][1], kv[l][1][: seq.n_c], rtol=1e-9, atol=1e-12)
