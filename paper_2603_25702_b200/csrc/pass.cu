@@ -294,8 +294,15 @@ int pass_init(s2d2_ctx* c) {
     // feeds and finishes the first half of the SwiGLU columns early; down starts with those and finishes its first
     // half of tiles early; the next layer's QKV starts with the k-blocks they feed.  A GEMM is only cut where every
     // sub-GEMM still gives each CTA a few units; otherwise (small models, mixture-of-experts kinds) it stays whole.
+    // use_tensor_cores = 3 cuts wherever the tile counts allow (test setting); when a small model then ends up with more
+    // split-K parts per tile than the part lists hold, the next, more conservative threshold is taken
+    const int min_units_options[3] = {c->dc.use_tensor_cores == 3 ? 0 : 4, c->dc.use_tensor_cores == 3 ? 1 : 4, 1 << 30};
+    long long ws_floats = 0;
+    size_t sync_words = 64;
+    for (int attempt = 0; attempt < 3; ++attempt) {
+    bool parts_fit = true;
     {
-        const int MIN_UNITS = c->dc.use_tensor_cores == 3 ? 0 : 4;      // 3: cut wherever the tile counts allow (test setting)
+        const int MIN_UNITS = min_units_options[attempt];
         auto whole = [&](int k) {
             const int n_tiles = (int)((NK[k][0] + 127) / 128), kbt = (int)(NK[k][1] / 64);
             s->n_subs[k] = 1;
@@ -316,10 +323,12 @@ int pass_init(s2d2_ctx* c) {
             // gate/up: its SwiGLU columns in nh groups that complete one after the other, so that the element-wise
             // chain behind a group (partials published, summed, activated, counted, fetched by the next GEMM) runs
             // under the groups that follow; down: the k-blocks those groups feed, in the same order, its own output
-            // tiles in two groups during the last of them.  Three groups where every sub-GEMM keeps enough units.
+            // tiles in two groups during the last of them.  Two groups: every group boundary is a point where all
+            // CTAs wait for the slowest one's partials, and with three groups (measured on the 8B-class shape: 107 us per
+            // layer against 100) the added waits cost more than the shorter chains gain.
             const int k0 = o_split ? 2 * h : 0;              // gate/up k-blocks fed by O's first half run first, over all tiles
             int nh = 1;
-            for (int cand = 3; cand >= 2 && nh == 1; --cand) {
+            for (int cand = 2; cand >= 2 && nh == 1; --cand) {
                 if (ft < cand) continue;
                 bool fits = k0 == 0 || enough(2LL * ft * k0);
                 for (int i = 0; i < cand && fits; ++i) {
@@ -366,9 +375,9 @@ int pass_init(s2d2_ctx* c) {
         }
     }
     // ---- per GEMM kind: split-K workspace region, publish counters, part tables ----
-    long long ws_floats = 0;
-    size_t sync_words = 64;
-    for (int k = 0; k < pp::N_KINDS; ++k) {
+    ws_floats = 0;
+    sync_words = 64;
+    for (int k = 0; k < pp::N_KINDS && parts_fit; ++k) {
         s->cnt_off[k] = -1;
         if (NK[k][0] < 0) continue;
         const bool dynamic = k == pp::K_EGU || k == pp::K_EDOWN;
@@ -405,15 +414,24 @@ int pass_init(s2d2_ctx* c) {
                 for (long long tl = first; tl <= last; ++tl) {
                     const long long t = tl < sd.t_split ? sd.t0 + tl : sd.t0 + sd.t_jump + (tl - sd.t_split);
                     int& cnt = tab[(size_t)t * (1 + pp::MAX_PARTS)];
-                    if (cnt >= pp::MAX_PARTS) return S2D2_OK;       // too finely split for the tables: other path
+                    if (cnt >= pp::MAX_PARTS) {       // too finely split for the tables
+                        parts_fit = false;
+                        break;
+                    }
                     tab[(size_t)t * (1 + pp::MAX_PARTS) + 1 + cnt] = cta * s->max_segs[k] + sd.seg_base + (int)(tl - first);
                     ++cnt;
                 }
             }
         }
+        if (!parts_fit) break;
+        if (s->parts[k]) cudaFree(s->parts[k]);
+        s->parts[k] = nullptr;
         if (cudaMalloc((void**)&s->parts[k], tab.size() * 4) != cudaSuccess ||
             cudaMemcpy(s->parts[k], tab.data(), tab.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
             return fail_alloc(c);
+    }
+    if (parts_fit) break;
+    if (attempt == 2) return S2D2_OK;       // even whole GEMMs are split too finely for the tables: the per-operation path stays in charge
     }
     if (!moe) {
         // Static schedule of a dense model: what each CTA streams does not depend on the data, so the list of its

@@ -42,13 +42,14 @@ class ParityReport:
     moe_forced_rows: int = 0          # (row, layer) pairs whose expert set the oracle took from the engine (near ties)
     moe_rows_checked: int = 0         # (row, layer) pairs compared
     moe_max_forced_gap: float = 0.0   # largest distance of a swapped expert's router logit from the oracle's k-th
+    err_without_kv_storage: float = 0.0   # probe: engine's draft logits of step 0 against an oracle that keeps K/V in fp64
 
 
 class OracleShadow:
     """The oracle's own causal cache over the committed tokens of one sequence."""
 
-    def __init__(self, W, cfg):
-        self.W, self.cfg = W, cfg
+    def __init__(self, W, cfg, kv_storage: bool = True):
+        self.W, self.cfg, self.kv_storage = W, cfg, kv_storage
         self.cache: Optional[M.KV] = None
         self.n = 0
 
@@ -56,7 +57,8 @@ class OracleShadow:
         if upto <= self.n:
             return
         toks = [int(t) for t in all_tokens[self.n:upto]]
-        _, kv = M.forward(self.W, self.cfg, toks, np.arange(self.n, upto), M.causal_mask(len(toks)), self.cache, need_logits=[])
+        _, kv = M.forward(self.W, self.cfg, toks, np.arange(self.n, upto), M.causal_mask(len(toks)), self.cache, need_logits=[],
+                          kv_storage=self.kv_storage)
         self.cache = M.append_kv(self.cache, kv, np.arange(len(toks)))
         self.n = upto
 
@@ -64,7 +66,7 @@ class OracleShadow:
 def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: int = 1, seed: Optional[int] = None,
               gamma: float = 1.0, tau_conf: float = 0.9, logit_atol: float = 2e-2, logit_rtol: float = 0.0,
               route=None, shadows=None, stage_b_seqs=None, resample: bool = True, layout: str = "aligned",
-              stage_b_steps: Optional[int] = None, draft_mode: str = "greedy") -> ParityReport:
+              stage_b_steps: Optional[int] = None, draft_mode: str = "greedy", probe_kv_storage: bool = False) -> ParityReport:
     """Run up to ``n_steps`` decode steps on all sequences (stops when every one has
     generated wl.gen_tokens) and check both parity stages.  ``stage_b_seqs``: restrict the
     oracle's forward (stage B) to these sequence ids (large batches at full model size); stage A
@@ -196,6 +198,14 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
                         sh.n = s0 + j
                 _cmp(rep, "draft", tag, my_d, ol, logit_atol, logit_rtol)
                 rep.stage_b_passes += 1
+                if probe_kv_storage and step_no == 0 and not cfg.is_moe:
+                    # the same draft pass by an oracle that keeps K and V in fp64 (cache and in-pass rows): how much of the
+                    # engine's distance is the cache's storage format (recorded, not asserted)
+                    sh2 = OracleShadow(W, cfg, kv_storage=False)
+                    sh2.extend(full, n_c0)
+                    vis2 = sh2.cache if q0 == n_c0 else [(k_[:q0], v_[:q0]) for k_, v_ in sh2.cache]
+                    ol2, _ = M.forward(W, cfg, toks, pos, mask, vis2, need_logits=need, kv_storage=False)
+                    rep.err_without_kv_storage = max(rep.err_without_kv_storage, float(np.abs(my_d.astype(np.float64) - ol2).max()))
                 if flags[k]:
                     if not cfg.is_moe:
                         sh.extend(full, s0 + j)
