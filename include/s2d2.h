@@ -60,6 +60,15 @@ enum { S2D2_DRAFT_GREEDY = 0, S2D2_DRAFT_SAMPLE = 1 };
  *   last], row k scores drafted token k + 1.  The draft pass reads its logits one row to the left in the same
  *   way, and every pass starts with the row of the last committed token. */
 enum { S2D2_VERIFIER_ALIGNED_2L = 0, S2D2_VERIFIER_RIGHT_SHIFTED = 1 };
+/* When the K/V of a block enter the cache (Algorithm "Block-wise autoregressive decoding"; Section
+ * "Self-Verification Mode", Eq. (draft_mask)).
+ * AR: the partially causal drafting/caching mask: committed tokens are causal rows, their K/V is final and enters
+ *   the cache as they are committed (accepted drafted tokens keep the K/V of their verifier rows).
+ * BLOCK_END: the standard block-diffusion pattern: every row of the block sees the whole block in the draft
+ *   pass, nothing of the block is cached while it is decoded (the verifier pass carries the block's committed
+ *   prefix as causal rows), and when the block has no MASK left s2d2_accept_and_commit runs one more pass over
+ *   it, with full attention inside the block, whose K/V are appended.  Aligned verifier layout only. */
+enum { S2D2_CACHE_AR = 0, S2D2_CACHE_BLOCK_END = 1 };
 
 /* The network (the paper treats x_theta as given; these fields describe the
  * decoder shapes of the synthetic workloads). Matrices are [out, in], y = x W^T. */
@@ -92,6 +101,7 @@ typedef struct {
                                    its tile counts allow (test setting: a small model then runs the same
                                    tile-by-tile hand-overs between GEMMs that a large one runs by default) */
     int32_t verifier_layout;    /* S2D2_VERIFIER_*                               */
+    int32_t caching;            /* S2D2_CACHE_*                                  */
 } s2d2_decode_config;
 
 typedef struct {
@@ -147,6 +157,7 @@ typedef struct {
     int64_t moe_expert_tiles_touched;                   /* (layer, expert) pairs streamed */
     int64_t h2d_bytes, d2h_bytes;                       /* host<->device copies made by the calls */
     int64_t n_rows_draft, n_rows_verify, n_rows_prefill; /* token rows the passes of each kind carried, summed */
+    int64_t n_cache_passes;                             /* end-of-block cache passes (S2D2_CACHE_BLOCK_END) */
 } s2d2_counters;
 
 typedef struct s2d2_ctx s2d2_ctx;

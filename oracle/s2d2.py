@@ -63,6 +63,19 @@ def verify_pass_rows(xhat, positions, mask_id):
     return tokens, pos, mask
 
 
+def verify_pass_rows_with_prefix(prefix_tokens, xhat, block_start, mask_id):
+    """Verifier rows when the block's committed prefix x^b_{<j} has no K/V in the cache (block-end caching): the
+    block-size-1 view needs those tokens as causal context, so they ride along as rows.  Rows: the j prefix tokens
+    and the L drafted tokens (one causal run of j + L rows), then the L MASK copies of the span; the MASK copy of
+    span position i sees the token rows strictly to its left and itself: Eq. (ver_mask) over the first j + L
+    positions of the block, with the MASK copies of the prefix positions left out."""
+    j, L = len(prefix_tokens), len(xhat)
+    n = j + L
+    tokens, pos, mask = verify_pass_rows(list(prefix_tokens) + list(xhat), list(range(block_start, block_start + n)), mask_id)
+    keep = list(range(n)) + list(range(n + j, 2 * n))
+    return tokens[keep], pos[keep], mask[np.ix_(keep, keep)]
+
+
 def verify_pass_rows_shifted(prev_token, xhat, first_position):
     """Rows and mask of the verifier pass of a right-shifted model (Section "Self-Verification
     Mode", last sentence: there the plain causal mask already gives the verifier view).  In such a
@@ -103,7 +116,7 @@ class SequenceOracle:
     def __init__(self, W, cfg, block_size: int, seed: int, seq_stream: int,
                  route: Callable[[StepTrace], bool] = None, tau_conf: float = 0.9,
                  draft_mode: str = "greedy", gamma: float = 1.0, keep_logits: bool = False,
-                 resample: bool = True, layout: str = "aligned"):
+                 resample: bool = True, layout: str = "aligned", caching: str = "ar"):
         self.W, self.cfg, self.B = W, cfg, block_size
         self.seed, self.seq_stream = seed, seq_stream
         self.route = route or (lambda st: len(st.span) >= 1)      # minimum-span policy, tau_span = 1
@@ -119,6 +132,14 @@ class SequenceOracle:
         # the cache visible to the pass ends before that position and the row's K/V is written (again).
         assert layout in ("aligned", "shifted")
         self.layout = layout
+        # "ar": the partially causal drafting/caching mask of Eq. (draft_mask) (K/V of committed tokens are causal and
+        # enter the cache as they are committed).  "block": the standard block-diffusion pattern of Algorithm
+        # "Block-wise autoregressive decoding": every row of the block sees the whole block in the draft pass
+        # (Eq. (draft_mask) with j = 0), nothing of the block is cached while it is being decoded, and once it has no
+        # MASK left one more pass over it (full attention inside the block) yields K^b, V^b, which are appended.
+        assert caching in ("ar", "block") and not (caching == "block" and layout == "shifted")
+        self.caching = caching
+        self.n_cache_passes = 0
         self.tokens: List[int] = []       # finalised tokens before the current block
         self.cache: Optional[M.KV] = None
         self.n_c = 0                      # tokens whose K/V is cached
@@ -149,6 +170,8 @@ class SequenceOracle:
             self.xb = [MASK] * B                      # a new block of MASKs
         s = len(self.tokens)
         j = self.xb.index(MASK)
+        if self.caching == "block":
+            return self._step_block_caching(s, j)
         full = self._all_tokens()
         shifted = self.layout == "shifted"
         q0 = min(self.n_c, s + j - 1) if shifted else self.n_c       # first row of the pass
@@ -220,6 +243,65 @@ class SequenceOracle:
                 st.committed_tokens.append(self.xb[i])
         self.step_index += 1
         if MASK not in self.xb:
+            self.tokens = self.tokens + self.xb
+            self.xb = []
+        self.trace.append(st)
+        return st
+
+    # -- the same iteration under block-end caching ---------------------------------------------------
+    def _step_block_caching(self, s: int, j: int) -> StepTrace:
+        cfg, B = self.cfg, self.B
+        MASK = cfg.mask_id
+        assert self.n_c == s
+        blk_pos = list(range(s, s + B))
+        tokens, pos, mask = draft_pass_rows([], [], self.xb, blk_pos)          # j = 0: every row sees the whole block
+        masked = [i for i in range(B) if self.xb[i] == MASK]
+        logits, _ = M.forward(self.W, cfg, tokens, pos, mask, self.cache, need_logits=masked)
+        self.n_draft_passes += 1
+        stats = []
+        for r, i in enumerate(masked):
+            u = philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_DRAFT)
+            stats.append(A.sample_from_logits(logits[r], self.draft_mode, u))
+        L = 1
+        while j + L < B and self.xb[j + L] == MASK:
+            L += 1
+        span = list(range(j, j + L))
+        st = StepTrace(s, j, self.n_c, masked, span, [q.xhat for q in stats], [q.d for q in stats],
+                       [q.margin for q in stats], [q.entropy for q in stats], False)
+        if self.keep_logits:
+            st.draft_logits = logits
+        st.verified = bool(self.route(st))
+        if st.verified:
+            xhat = st.xhat[:L]
+            vt, vp, vm = verify_pass_rows_with_prefix(self.xb[:j], xhat, s, MASK)
+            vlogits, _ = M.forward(self.W, cfg, vt, vp, vm, self.cache, need_logits=list(range(j + L, j + 2 * L)))
+            self.n_verify_passes += 1
+            st.u_accept = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_ACCEPT) for i in span]
+            st.u_resample = [philox.uniform(self.seed, s + i, self.seq_stream, self.step_index, philox.STREAM_RESAMPLE) for i in span]
+            res = A.accept_scan(logits[:L], vlogits, xhat, st.u_accept, st.u_resample, self.gamma, resample=self.resample)
+            st.result = res
+            if self.keep_logits:
+                st.verify_logits = vlogits
+            for k in range(res.n_accepted):
+                self.xb[j + k] = int(xhat[k])
+                st.committed.append(j + k)
+                st.committed_tokens.append(int(xhat[k]))
+            if res.first_reject >= 0 and self.resample:
+                self.xb[j + res.first_reject] = int(res.resampled)
+                st.committed.append(j + res.first_reject)
+                st.committed_tokens.append(int(res.resampled))
+        else:
+            for i in A.threshold_select(st.d, masked, self.tau_conf):
+                self.xb[i] = int(st.xhat[masked.index(i)])
+                st.committed.append(i)
+                st.committed_tokens.append(self.xb[i])
+        self.step_index += 1
+        if MASK not in self.xb:
+            # K^b, V^b <- x_theta(x^b): one pass over the finished block, full attention inside it
+            _, kv = M.forward(self.W, cfg, self.xb, blk_pos, np.ones((B, B), dtype=bool), self.cache, need_logits=[])
+            self.cache = M.append_kv(self.cache, kv, np.arange(B))
+            self.n_c += B
+            self.n_cache_passes += 1
             self.tokens = self.tokens + self.xb
             self.xb = []
         self.trace.append(st)

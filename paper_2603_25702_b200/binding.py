@@ -33,7 +33,7 @@ class DecodeConfigC(C.Structure):
     _fields_ = [("block_size", C.c_int32), ("max_batch", C.c_int32), ("max_seq_len", C.c_int32),
                 ("kv_page_tokens", C.c_int32), ("n_kv_pages", C.c_int32), ("draft_mode", C.c_int32),
                 ("resample", C.c_int32), ("tau_conf", C.c_float), ("ratio_gamma", C.c_float), ("seed", C.c_uint32),
-                ("use_tensor_cores", C.c_int32), ("verifier_layout", C.c_int32)]
+                ("use_tensor_cores", C.c_int32), ("verifier_layout", C.c_int32), ("caching", C.c_int32)]
 
 
 class TensorDesc(C.Structure):
@@ -63,7 +63,7 @@ class Counters(C.Structure):
                [("accepted_len_hist", C.c_int64 * (MAX_BLOCK + 1))] + \
                [(n, C.c_double) for n in ("ms_draft", "ms_verify", "ms_accept", "ms_prefill")] + \
                [(n, C.c_int64) for n in ("kv_pages_in_use", "kv_pages_total", "moe_expert_tiles_touched", "h2d_bytes", "d2h_bytes",
-                                         "n_rows_draft", "n_rows_verify", "n_rows_prefill")]
+                                         "n_rows_draft", "n_rows_verify", "n_rows_prefill", "n_cache_passes")]
 
 
 class RoutePolicy(C.Structure):
@@ -166,7 +166,7 @@ class Engine:
     def __init__(self, model, block_size: int, max_batch: int, max_seq_len: int, kv_page_tokens: int = 64,
                  n_kv_pages: int = 0, seed: int = 1, tau_conf: float = 0.9, ratio_gamma: float = 1.0,
                  resample: bool = True, stream: int = 0, use_tensor_cores: int = 1, verifier_layout: str = "aligned",
-                 draft_mode: str = "greedy"):
+                 draft_mode: str = "greedy", caching: str = "ar"):
         self.lib = load_library()
         self.model = model
         self.block_size = block_size
@@ -177,7 +177,8 @@ class Engine:
                           model.logit_scale)
         dc = DecodeConfigC(block_size, max_batch, max_seq_len, kv_page_tokens, n_kv_pages,
                            {"greedy": 0, "sample": 1}[draft_mode], int(resample), tau_conf,
-                           ratio_gamma, seed, int(use_tensor_cores), {"aligned": 0, "shifted": 1}[verifier_layout])
+                           ratio_gamma, seed, int(use_tensor_cores), {"aligned": 0, "shifted": 1}[verifier_layout],
+                           {"ar": 0, "block": 1}[caching])
         self._h = C.c_void_p()
         rc = self.lib.s2d2_create(C.byref(mc), C.byref(dc), C.c_void_p(stream), C.byref(self._h))
         if rc != 0:

@@ -311,7 +311,13 @@ int pass_init(s2d2_ctx* c) {
         for (int k = 0; k < pp::N_KINDS; ++k)
             if (NK[k][0] >= 0) whole(k);
         if (!moe) {
-            const int dt = d / 128, ft = f / 128, h = dt / 2;
+            // TUNING (temporary): shares of the first group in eighths, from the environment
+            auto eighths = [](const char* name, int dflt) {
+                const char* v = getenv(name);
+                return v ? atoi(v) : dflt;
+            };
+            const int fr_o = eighths("S2D2_FR_O", 4), fr_gu = eighths("S2D2_FR_GU", 4), fr_dn = eighths("S2D2_FR_DN", 4);
+            const int dt = d / 128, ft = f / 128, h = std::max(1, dt * fr_o / 8), hd = std::max(1, dt * fr_dn / 8);
             auto enough = [&](long long units) { return units / G >= MIN_UNITS; };
             const int kq = d / 64, ko = nq / 64, kd = f / 64, tq = nqkv / 128;
             const bool o_split = h >= 1 && enough((long long)h * ko) && enough((long long)(dt - h) * ko);
@@ -332,7 +338,7 @@ int pass_init(s2d2_ctx* c) {
                 if (ft < cand) continue;
                 bool fits = k0 == 0 || enough(2LL * ft * k0);
                 for (int i = 0; i < cand && fits; ++i) {
-                    const int a = ft * i / cand, b2 = ft * (i + 1) / cand;
+                    const int a = i == 0 ? 0 : std::max(1, ft * fr_gu / 8), b2 = i == 0 ? std::max(1, ft * fr_gu / 8) : ft;
                     fits = enough(2LL * (b2 - a) * (kq - k0));
                 }
                 if (fits) nh = cand;
@@ -340,36 +346,38 @@ int pass_init(s2d2_ctx* c) {
             if (nh > 1) {
                 int n = 0;
                 if (k0 > 0) s->subs[pp::K_GU][n++] = pp::SubDesc{0, 2 * ft, 2 * ft, 0, 0, k0, 0, 0, 0};
+                auto gu_a = [&](int i) { return i == 0 ? 0 : std::max(1, ft * fr_gu / 8); };
+                auto gu_b = [&](int i) { return i == 0 ? std::max(1, ft * fr_gu / 8) : ft; };
                 for (int i = 0; i < nh; ++i) {
-                    const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
+                    const int a = gu_a(i), b2 = gu_b(i);
                     s->subs[pp::K_GU][n++] = pp::SubDesc{a, 2 * (b2 - a), b2 - a, ft, k0, kq - k0, 0, a, b2};
                 }
                 s->n_subs[pp::K_GU] = n;
                 // down: k-blocks of group i = SwiGLU columns [128 a_i, 128 b_i)
-                bool three_way = h >= 1;                     // last group's k-blocks over two groups of output tiles
+                bool three_way = hd >= 1 && hd < dt;         // last group's k-blocks over two groups of output tiles
                 for (int i = 0; i < nh && three_way; ++i) {
-                    const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
-                    three_way = i + 1 < nh ? enough((long long)dt * 2 * (b2 - a)) : (enough((long long)h * 2 * (b2 - a)) && enough((long long)(dt - h) * 2 * (b2 - a)));
+                    const int a = gu_a(i), b2 = gu_b(i);
+                    three_way = i + 1 < nh ? enough((long long)dt * 2 * (b2 - a)) : (enough((long long)hd * 2 * (b2 - a)) && enough((long long)(dt - hd) * 2 * (b2 - a)));
                 }
                 bool k_only = !three_way;
-                for (int i = 0; i < nh && k_only; ++i) k_only = enough((long long)dt * 2 * (ft * (i + 1) / nh - ft * i / nh));
+                for (int i = 0; i < nh && k_only; ++i) k_only = enough((long long)dt * 2 * (gu_b(i) - gu_a(i)));
                 if (three_way || k_only) {
                     n = 0;
                     for (int i = 0; i < nh; ++i) {
-                        const int a = ft * i / nh, b2 = ft * (i + 1) / nh;
+                        const int a = gu_a(i), b2 = gu_b(i);
                         if (i + 1 < nh || k_only) {
                             s->subs[pp::K_DOWN][n++] = pp::SubDesc{0, dt, dt, 0, 2 * a, 2 * (b2 - a), 0, 0, i + 1 < nh ? 0 : dt};
                         } else {
-                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{0, h, h, 0, 2 * a, 2 * (b2 - a), 0, 0, h};
-                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{h, dt - h, dt - h, 0, 2 * a, 2 * (b2 - a), 0, h, dt};
+                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{0, hd, hd, 0, 2 * a, 2 * (b2 - a), 0, 0, hd};
+                            s->subs[pp::K_DOWN][n++] = pp::SubDesc{hd, dt - hd, dt - hd, 0, 2 * a, 2 * (b2 - a), 0, hd, dt};
                         }
                     }
                     s->n_subs[pp::K_DOWN] = n;
                 }
-                if (three_way && enough((long long)tq * 2 * h) && enough((long long)tq * (kq - 2 * h))) {      // (all, K0), (all, K1): K0 = what down's first half feeds
+                if (three_way && enough((long long)tq * 2 * hd) && enough((long long)tq * (kq - 2 * hd))) {      // (all, K0), (all, K1): K0 = what down's first group feeds
                     s->n_subs[pp::K_QKV] = 2;
-                    s->subs[pp::K_QKV][0] = pp::SubDesc{0, tq, tq, 0, 0, 2 * h, 0, 0, 0};
-                    s->subs[pp::K_QKV][1] = pp::SubDesc{0, tq, tq, 0, 2 * h, kq - 2 * h, 0, 0, tq};
+                    s->subs[pp::K_QKV][0] = pp::SubDesc{0, tq, tq, 0, 0, 2 * hd, 0, 0, 0};
+                    s->subs[pp::K_QKV][1] = pp::SubDesc{0, tq, tq, 0, 2 * hd, kq - 2 * hd, 0, 0, tq};
                 }
             }
         }

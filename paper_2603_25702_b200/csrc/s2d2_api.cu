@@ -157,6 +157,8 @@ int validate(const s2d2_model_config& m, const s2d2_decode_config& dc, std::stri
     if (p < 1 || p > 64 || (p & (p - 1))) return bad("decode: kv_page_tokens must be a power of two <= 64");
     if (dc.draft_mode != S2D2_DRAFT_GREEDY && dc.draft_mode != S2D2_DRAFT_SAMPLE) return bad("decode: draft_mode");
     if (dc.verifier_layout != S2D2_VERIFIER_ALIGNED_2L && dc.verifier_layout != S2D2_VERIFIER_RIGHT_SHIFTED) return bad("decode: verifier_layout");
+    if (dc.caching != S2D2_CACHE_AR && dc.caching != S2D2_CACHE_BLOCK_END) return bad("decode: caching");
+    if (dc.caching == S2D2_CACHE_BLOCK_END && dc.verifier_layout != S2D2_VERIFIER_ALIGNED_2L) return bad("decode: block-end caching needs the aligned verifier layout");
     return S2D2_OK;
 }
 
@@ -699,6 +701,23 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
         // pass starts at the last committed token even when its K/V is cached already (the cache visible to the pass
         // then ends before it, and the cached K/V is kept).
         const bool shifted = c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED;
+        if (c->dc.caching == S2D2_CACHE_BLOCK_END) {
+            // block-end caching: the whole block, known tokens and MASKs, every row sees every row; nothing is cached
+            if ((rc = ensure_pages(c, s, st + B))) return rc;
+            begin_seq(c, pb, s, st);
+            s.j = j;
+            s.n_masked = 0;
+            s.draft_row0 = pb.n_logit;
+            const unsigned long long all_b = B == 64 ? ~0ull : ((1ull << B) - 1);
+            for (int i2 = 0; i2 < B; ++i2) {
+                bool masked = s.tok[st + i2] == MASK;
+                add_row(c, pb, s.tok[st + i2], st + i2, all_b, 0, masked);
+                if (masked) s.masked_idx[s.n_masked++] = i2;
+            }
+            s.span_len = 1;
+            while (j + s.span_len < B && s.tok[st + j + s.span_len] == MASK) ++s.span_len;
+            continue;
+        }
         int q0 = shifted ? std::min(s.n_c, st + j - 1) : s.n_c;
         int P = st + j - q0;             // committed tokens that run as causal rows (those without K/V get it appended)
         int rows = P + (B - j);
@@ -759,7 +778,7 @@ extern "C" int s2d2_draft_block(s2d2_ctx* c, int32_t n, const int32_t* ids, s2d2
         SeqState& s = c->seqs[ids[i]];
         s2d2_draft_stats& o = out[i];
         memset(&o, 0, sizeof(o));
-        s.n_c = s.n_final + s.j;         // pending rows are cached now
+        if (c->dc.caching == S2D2_CACHE_AR) s.n_c = s.n_final + s.j;         // pending rows are cached now
         o.seq_id = ids[i];
         o.block_start = s.n_final;
         o.first_masked = s.j;
@@ -924,6 +943,19 @@ extern "C" int s2d2_verify_block(s2d2_ctx* c, int32_t n, const int32_t* ids, con
             s.verify_row0 = pb.n_logit;
             add_row(c, pb, s.tok[p0 - 1], p0 - 1, 1ull, 0, true);
             for (int k = 1; k < L; ++k) add_row(c, pb, s.xhat[k - 1], p0 + k - 1, (1ull << (k + 1)) - 1, ROW_WRITE_KV, true);
+            s.verify_in_flight = true;
+            continue;
+        }
+        if (c->dc.caching == S2D2_CACHE_BLOCK_END) {
+            // the block's committed prefix has no K/V in the cache: it rides along as causal rows in front of the drafted
+            // tokens (one causal run of j + L rows, nothing written); MASK copy i sees the token rows to its left and itself
+            const int jj = s.j, st0 = s.n_final;
+            if (jj + 2 * L > S2D2_MAX_ROWS_PER_SEQ) FAIL(c, S2D2_ERR_UNSUPPORTED, "too many rows for one sequence in a verifier pass");
+            begin_seq(c, pb, s, st0);
+            s.verify_row0 = pb.n_logit;
+            for (int k = 0; k < jj; ++k) add_row(c, pb, s.tok[st0 + k], st0 + k, (1ull << (k + 1)) - 1, 0, false);
+            for (int k = 0; k < L; ++k) add_row(c, pb, s.xhat[k], p0 + k, (1ull << (jj + k + 1)) - 1, 0, false);
+            for (int k = 0; k < L; ++k) add_row(c, pb, MASK, p0 + k, ((1ull << (jj + k)) - 1) | (1ull << (jj + L + k)), 0, true);
             s.verify_in_flight = true;
             continue;
         }
@@ -1105,7 +1137,8 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
             }
             // accepted drafted rows keep their K/V; rows past them are rolled back by length (the right-shifted
             // verifier has no row for the last drafted token: it gets its K/V in the next draft pass)
-            s.n_c += c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED ? std::min(na, s.span_len - 1) : na;
+            if (c->dc.caching == S2D2_CACHE_AR)
+                s.n_c += c->dc.verifier_layout == S2D2_VERIFIER_RIGHT_SHIFTED ? std::min(na, s.span_len - 1) : na;
             if (h_rej[i] >= 0 && c->dc.resample) {
                 s.tok[st + s.j + na] = h_res[i];
                 o.committed_idx[o.n_committed] = s.j + na;
@@ -1143,6 +1176,32 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
             s.block_open = false;
         }
         o.block_done = done;
+    }
+    if (c->dc.caching == S2D2_CACHE_BLOCK_END) {
+        // K^b, V^b <- x_theta(x^b) (Algorithm "Block-wise autoregressive decoding"): one pass over every block that was
+        // finished by this step, full attention inside the block, K/V appended
+        PassBuild pb;
+        std::vector<int> finished;
+        for (int i = 0; i < n; ++i) {
+            SeqState& s = c->seqs[ids[i]];
+            if (!res[i].block_done) continue;
+            const int st = s.n_final - B;
+            int rc2;
+            if ((rc2 = ensure_pages(c, s, s.n_final))) return rc2;
+            begin_seq(c, pb, s, st);
+            const unsigned long long all_b = B == 64 ? ~0ull : ((1ull << B) - 1);
+            for (int k = 0; k < B; ++k) add_row(c, pb, s.tok[st + k], st + k, all_b, ROW_WRITE_KV, false);
+            finished.push_back(ids[i]);
+        }
+        if (pb.n_rows > 0) {
+            int rc2 = run_pass(c, pb, nullptr);
+            if (rc2) return rc2;
+            if ((rc2 = enqueue_status_read(c))) return rc2;
+            CUDA_TRY(c, cudaStreamSynchronize(c->stream));      // the row table is reused by the next pass
+            if ((rc2 = check_status(c))) return rc2;
+            c->cnt.n_cache_passes++;
+            for (int id : finished) c->seqs[id].n_c = c->seqs[id].n_final;
+        }
     }
     return S2D2_OK;
 }

@@ -62,11 +62,23 @@ class OracleShadow:
         self.cache = M.append_kv(self.cache, kv, np.arange(len(toks)))
         self.n = upto
 
+    def extend_blocks(self, all_tokens, upto: int, prompt_len: int, B: int):
+        """Block-end caching: causal over the prompt, then finished block by finished block with full attention
+        inside the block (``upto`` is a block boundary)."""
+        self.extend(all_tokens, min(upto, prompt_len))
+        while self.n < upto:
+            toks = [int(t) for t in all_tokens[self.n:self.n + B]]
+            _, kv = M.forward(self.W, self.cfg, toks, np.arange(self.n, self.n + B), np.ones((B, B), dtype=bool), self.cache, need_logits=[],
+                              kv_storage=self.kv_storage)
+            self.cache = M.append_kv(self.cache, kv, np.arange(B))
+            self.n += B
+
 
 def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: int = 1, seed: Optional[int] = None,
               gamma: float = 1.0, tau_conf: float = 0.9, logit_atol: float = 2e-2, logit_rtol: float = 0.0,
               route=None, shadows=None, stage_b_seqs=None, resample: bool = True, layout: str = "aligned",
-              stage_b_steps: Optional[int] = None, draft_mode: str = "greedy", probe_kv_storage: bool = False) -> ParityReport:
+              stage_b_steps: Optional[int] = None, draft_mode: str = "greedy", probe_kv_storage: bool = False,
+              caching: str = "ar") -> ParityReport:
     """Run up to ``n_steps`` decode steps on all sequences (stops when every one has
     generated wl.gen_tokens) and check both parity stages.  ``stage_b_seqs``: restrict the
     oracle's forward (stage B) to these sequence ids (large batches at full model size); stage A
@@ -76,6 +88,7 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
     steps only (long runs at full model size).  ``draft_mode="sample"``: proposals drawn from pi_d with the
     draft-sampling uniforms."""
     shifted = layout == "shifted"
+    block_cache = caching == "block"       # block-end caching: whole-block draft rows, verifier rows with the block's prefix
     cfg, B = wl.model, wl.block_size
     MASK = cfg.mask_id
     seed = wl.philox_seed if seed is None else seed
@@ -177,7 +190,20 @@ def run_steps(engine, W, wl, seq_ids, rng_streams, n_steps: int, stage_b_every: 
             n_c0 = bf["n_cached"]
             q0 = min(n_c0, s0 + j - 1) if shifted else n_c0       # first row of the draft pass
             n_draft_rows = (s0 + j - q0) + (B - j)
-            if do_b and (stage_b_seqs is None or sid in stage_b_seqs):
+            if block_cache and do_b and (stage_b_seqs is None or sid in stage_b_seqs):
+                assert n_c0 == s0 and not cfg.is_moe
+                sh = shadows[sid]
+                sh.extend_blocks(full, s0, _prompt_len(engine, sid), B)
+                toks, pos, mask = S.draft_pass_rows([], [], blk, list(range(s0, s0 + B)))
+                ol, _ = M.forward(W, cfg, toks, pos, mask, sh.cache, need_logits=masked)
+                _cmp(rep, "draft", tag, my_d, ol, logit_atol, logit_rtol)
+                rep.stage_b_passes += 1
+                if flags[k]:
+                    vt, vp, vm = S.verify_pass_rows_with_prefix(blk[:j], list(st.xhat[:L]), s0, MASK)
+                    ov, _ = M.forward(W, cfg, vt, vp, vm, sh.cache, need_logits=list(range(j + L, j + 2 * L)))
+                    _cmp(rep, "verify", tag, my_v, ov, logit_atol, logit_rtol)
+                    rep.stage_b_passes += 1
+            elif do_b and (stage_b_seqs is None or sid in stage_b_seqs):
                 sh = shadows[sid]
                 if not cfg.is_moe:
                     sh.extend(full, n_c0)
@@ -262,13 +288,17 @@ def _cmp(rep: ParityReport, which: str, tag: str, got: np.ndarray, want: np.ndar
         rep.mismatches.append(f"{tag}: {which} logits off by {mx:.3e} (bound {bound:.3e}, scale {scale:.2f})")
 
 
-def check_kv(engine, W, cfg, sid, atol: float) -> float:
-    """Cache contents of a sequence against the oracle's causal pass over the committed tokens."""
+def check_kv(engine, W, cfg, sid, atol: float, block_size: int = 0) -> float:
+    """Cache contents of a sequence against the oracle's causal pass over the committed tokens (``block_size`` > 0:
+    block-end caching, the oracle's block-causal passes)."""
     stt = engine.debug_seq_state(sid)
     n_c = stt["n_cached"]
     full = list(engine.get_tokens(sid)) + list(stt["block_tokens"])
     sh = OracleShadow(W, cfg)
-    sh.extend(full, n_c)
+    if block_size:
+        sh.extend_blocks(full, n_c, _prompt_len(engine, sid), block_size)
+    else:
+        sh.extend(full, n_c)
     worst = 0.0
     for l in range(cfg.n_layers):
         k, v = engine.debug_copy_kv(sid, l, n_c)

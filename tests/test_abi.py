@@ -28,10 +28,10 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_sizes_match_header():
     from paper_2603_25702_b200 import binding as b
     assert ctypes.sizeof(b.ModelConfigC) == 13 * 4 + 3 * 4
-    assert ctypes.sizeof(b.DecodeConfigC) == 12 * 4
+    assert ctypes.sizeof(b.DecodeConfigC) == 13 * 4
     assert ctypes.sizeof(b.DraftStats) == 7 * 4 + 5 * 32 * 4
     assert ctypes.sizeof(b.StepResult) == 8 * 4 + 5 * 32 * 4
-    assert ctypes.sizeof(b.Counters) == 9 * 8 + 33 * 8 + 4 * 8 + 8 * 8
+    assert ctypes.sizeof(b.Counters) == 9 * 8 + 33 * 8 + 4 * 8 + 9 * 8
     assert ctypes.sizeof(b.RoutePolicy) == 7 * 4
 
 

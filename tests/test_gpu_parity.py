@@ -404,3 +404,33 @@ def test_sampling_draft_mode_matches_oracle_end_to_end():
     greedy = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0).generate(prompts[0], wl.gen_tokens)
     assert got == want and want != greedy          # and the sampled trajectory is a different one
     e.close()
+
+
+@pytest.mark.parametrize("name,atol,rtol", [("c1", 0.0, 1e-4), ("t_f32", 0.0, 1e-4), ("t_bf16", 2e-2, 0.0), ("t_bf16_128", 2e-2, 0.0)])
+def test_block_end_caching_matches_oracle(name, atol, rtol):
+    """S2D2_CACHE_BLOCK_END (Algorithm "Block-wise autoregressive decoding", K^b, V^b <- x_theta(x^b)): whole-block draft
+    rows that see each other, verifier rows that carry the block's committed prefix, nothing cached until the block is
+    finished, then one pass over it with full attention inside the block.  Both parity stages over the whole generation,
+    the cache against the oracle's block-causal passes, and for the fp32 workload the free-running token stream."""
+    from tests.parity_util import check_kv, run_steps
+    wl = get_config(name)
+    W = generate_weights(wl.model, seed=wl.weight_seed, gain_jitter=0.0 if name == "c1" else 0.1)
+    e, ids, prompts = _start(wl, W, caching="block")
+    rep = run_steps(e, W, wl, ids, {sid: k for k, sid in enumerate(ids)}, n_steps=200, logit_atol=atol, logit_rtol=rtol, caching="block")
+    print(name, rep)
+    assert not rep.mismatches, rep.mismatches[:5]
+    assert rep.verified_steps > 0 and rep.n_committed == wl.gen_tokens * len(ids)
+    assert e.get_counters().n_cache_passes >= wl.gen_tokens // wl.block_size
+    for sid in ids:
+        assert e.debug_seq_state(sid)["n_cached"] == e.debug_seq_state(sid)["block_start"]
+        check_kv(e, W, wl.model, sid, atol=1e-5 if wl.model.dtype == "fp32" else 4e-2, block_size=wl.block_size)
+    e.close()
+    if name == "c1":
+        e, ids, prompts = _start(wl, W, caching="block")
+        e.generate(ids, wl.gen_tokens)
+        got = e.get_tokens(ids[0])[len(prompts[0]):].tolist()
+        orc = S.SequenceOracle(W, wl.model, wl.block_size, seed=wl.philox_seed, seq_stream=0, caching="block")
+        assert got == orc.generate(prompts[0], wl.gen_tokens)
+        c = e.get_counters()
+        assert c.n_draft_passes == orc.n_draft_passes and c.n_verify_passes == orc.n_verify_passes and c.n_cache_passes == orc.n_cache_passes
+        e.close()

@@ -339,3 +339,55 @@ def test_shifted_loop_invariants_and_cache_is_causal(tiny_f32, B):
     for l in range(cfg.n_layers):
         np.testing.assert_allclose(seq.cache[l][0], kv[l][0][: seq.n_c], rtol=1e-9, atol=1e-12)
         np.testing.assert_allclose(seq.cache[l][1], kv[l][1][: seq.n_c], rtol=1e-9, atol=1e-12)
+
+
+# ---- block-end caching (Algorithm "Block-wise autoregressive decoding", K^b, V^b <- x_theta(x^b)) -------------
+def test_block_caching_with_block_size_one_is_the_ar_cached_run(tiny_f32):
+    """A block of one token: full attention inside the block is the causal mask, so block-end caching and the AR-like
+    caching are the same computation, token for token and logit for logit."""
+    wl, W = tiny_f32
+    cfg = wl.model
+    prompt = generate_prompts(wl, seed=4)[0][:9]
+    a = S.SequenceOracle(W, cfg, block_size=1, seed=1, seq_stream=0, keep_logits=True, caching="block")
+    b = S.SequenceOracle(W, cfg, block_size=1, seed=1, seq_stream=0, keep_logits=True)
+    assert a.generate(prompt, 8) == b.generate(prompt, 8)
+    for x, y in zip(a.trace, b.trace):
+        np.testing.assert_allclose(x.draft_logits, y.draft_logits, rtol=1e-9, atol=1e-11)
+        np.testing.assert_allclose(x.verify_logits, y.verify_logits, rtol=1e-9, atol=1e-11)
+    assert a.n_cache_passes == 8
+
+
+def test_block_caching_cache_is_the_block_causal_pass_and_verifier_rows_are_literal(tiny_f32):
+    wl, W = tiny_f32
+    cfg = wl.model
+    MASK = cfg.mask_id
+    B = 4
+    prompt = [5, 9, 2, 44, 17, 3]
+    n = len(prompt)
+    seq = S.SequenceOracle(W, cfg, block_size=B, seed=1, seq_stream=2, keep_logits=True, caching="block")
+    out = seq.generate(prompt, 32)
+    assert seq.n_cache_passes == 8 and seq.n_c == n + 32
+    assert any(st.result.first_reject >= 0 for st in seq.trace)
+    # the cache is what ONE pass over everything gives under the block-causal pattern: causal prompt, then each block
+    # sees the prompt, the earlier blocks and all of itself
+    full = list(prompt) + out
+    T = len(full)
+    m = np.zeros((T, T), dtype=bool)
+    m[:n, :n] = M.causal_mask(n)
+    for b0 in range(n, T, B):
+        m[b0:b0 + B, :b0 + B] = True
+    _, kv = M.forward(W, cfg, full, np.arange(T), m, need_logits=[])
+    for l in range(cfg.n_layers):
+        np.testing.assert_allclose(seq.cache[l][0], kv[l][0], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(seq.cache[l][1], kv[l][1], rtol=1e-9, atol=1e-12)
+    # verifier rows with an uncached in-block prefix: MASK copy i == a literal pass of cache ++ prefix ++ xhat_<i ++ MASK,
+    # causal over the block part (the block-size-1 view), on top of the block-causal cache of the first block
+    cache1 = [(k[:n + B], v[:n + B]) for k, v in seq.cache]
+    prefix, xhat = [7, 3], [11, 30]
+    vt, vp, vm = S.verify_pass_rows_with_prefix(prefix, xhat, n + B, MASK)
+    assert len(vt) == 2 + 2 + 2 and vp.tolist() == [n + B, n + B + 1, n + B + 2, n + B + 3, n + B + 2, n + B + 3]
+    got, _ = M.forward(W, cfg, vt, vp, vm, cache1, need_logits=[4, 5])
+    for i in range(2):
+        toks = prefix + xhat[:i] + [MASK]
+        lit, _ = M.forward(W, cfg, toks, np.arange(n + B, n + B + len(toks)), M.causal_mask(len(toks)), cache1)
+        np.testing.assert_allclose(got[i], lit[-1], rtol=1e-9, atol=1e-11)
