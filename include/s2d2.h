@@ -323,7 +323,8 @@ int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t
  * values, GPU global-timer readings (ns) at named points of the pass followed by the id of the SM the CTA
  * ran on.  Slots 0, 1: entry to and exit from the grid barrier behind the embedding (slot 2 unused).  Then
  * per layer, for dense models 12 slots: QKV accumulators drained; entry, exit of the barrier behind q/k-norm +
- * RoPE + K/V write; entry, exit of the barrier behind the attention items; key splits combined; O accumulators
+ * RoPE + K/V write; entry, exit of the barrier behind the attention items (a pass of one sequence has no barrier
+ * there: items done, first combine pair's items counted complete); key splits combined; O accumulators
  * drained; residual add done; gate/up accumulators drained; SwiGLU done; down accumulators drained; residual
  * add done (from the combine on, the GEMMs of a dense layer follow each other without a grid barrier).  For
  * mixture-of-experts models 27 slots: (entry, exit, last accumulator drained before it or 0) for each of the

@@ -318,6 +318,11 @@ int noalloc_map(CUtensorMap* m, const void* ptr, int rows, int K, int box_rows) 
 }
 }  // namespace
 
+void gemm_reset_tickets(s2d2_ctx* c) {
+    GemmState* g = (GemmState*)c->gemm_state;
+    if (g && g->tickets) cudaMemsetAsync(g->tickets, 0, g->n_tickets * 4, c->stream);
+}
+
 extern "C" const char* s2d2_noalloc_last_error(void) { return g_noalloc_err; }
 
 extern "C" int s2d2_gemm_bf16_noalloc(const void* d_x, const void* d_w, float* d_y, int32_t M, int32_t N, int32_t K,

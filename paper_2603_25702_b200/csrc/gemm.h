@@ -19,3 +19,6 @@ int gemm_encode_map(s2d2_ctx* c, void* out, const void* ptr, unsigned long long 
 // 3D bf16 tensor map [rows, mid, cols] (cols contiguous) with boxes of box_rows x box_mid x 64 columns, 128-byte swizzle.
 int gemm_encode_map3(s2d2_ctx* c, void* out, const void* ptr, int cols, int mid, unsigned long long rows, int box_mid, int box_rows);
 bool gemm_tc_available(s2d2_ctx* c);
+// After a kernel gave up on a bounded wait: a split-K CTA that left early took no ticket, so the tile counters no
+// longer return to zero by themselves; clear them (enqueued on the context's stream).
+void gemm_reset_tickets(s2d2_ctx* c);

@@ -44,6 +44,7 @@ struct PassState {
     size_t sync_bytes = 0;
     long long cnt_off[pp::N_KINDS] = {};     // -1: the kind publishes through a grid barrier
     size_t xcnt_off[4] = {0, 0, 0, 0};
+    size_t attn_cnt_off = 0;
     unsigned long long* trace = nullptr;
     int trace_cap = 0;
     int trace_mma0 = 0, n_sub_gemms = 0;
@@ -311,16 +312,12 @@ int pass_init(s2d2_ctx* c) {
         for (int k = 0; k < pp::N_KINDS; ++k)
             if (NK[k][0] >= 0) whole(k);
         if (!moe) {
-            // TUNING (temporary): shares of the first group in eighths, from the environment
-            auto eighths = [](const char* name, int dflt) {
-                const char* v = getenv(name);
-                return v ? atoi(v) : dflt;
-            };
-            const int fr_o = eighths("S2D2_FR_O", 4), fr_gu = eighths("S2D2_FR_GU", 4), fr_dn = eighths("S2D2_FR_DN", 4);
-            const int dt = d / 128, ft = f / 128, h = std::max(1, dt * fr_o / 8), hd = std::max(1, dt * fr_dn / 8);
+            const int dt = d / 128, ft = f / 128, h = dt / 2, hd = dt / 2;
             auto enough = [&](long long units) { return units / G >= MIN_UNITS; };
             const int kq = d / 64, ko = nq / 64, kd = f / 64, tq = nqkv / 128;
-            const bool o_split = h >= 1 && enough((long long)h * ko) && enough((long long)(dt - h) * ko);
+            // O stays whole unless the test setting forces cuts: it is small (14 units per CTA on the 8B-class shape), halves
+            // of it leave 18 split-K parts per tile, and the 8B-class pass measured no faster with it cut (3.70 against 3.61 ms)
+            const bool o_split = c->dc.use_tensor_cores == 3 && h >= 1 && enough((long long)h * ko) && enough((long long)(dt - h) * ko);
             if (o_split) {                                   // (H0, all K), (H1, all K)
                 s->n_subs[pp::K_O] = 2;
                 s->subs[pp::K_O][0] = pp::SubDesc{0, h, h, 0, 0, ko, 0, 0, h};
@@ -338,7 +335,7 @@ int pass_init(s2d2_ctx* c) {
                 if (ft < cand) continue;
                 bool fits = k0 == 0 || enough(2LL * ft * k0);
                 for (int i = 0; i < cand && fits; ++i) {
-                    const int a = i == 0 ? 0 : std::max(1, ft * fr_gu / 8), b2 = i == 0 ? std::max(1, ft * fr_gu / 8) : ft;
+                    const int a = ft * i / cand, b2 = ft * (i + 1) / cand;
                     fits = enough(2LL * (b2 - a) * (kq - k0));
                 }
                 if (fits) nh = cand;
@@ -346,8 +343,8 @@ int pass_init(s2d2_ctx* c) {
             if (nh > 1) {
                 int n = 0;
                 if (k0 > 0) s->subs[pp::K_GU][n++] = pp::SubDesc{0, 2 * ft, 2 * ft, 0, 0, k0, 0, 0, 0};
-                auto gu_a = [&](int i) { return i == 0 ? 0 : std::max(1, ft * fr_gu / 8); };
-                auto gu_b = [&](int i) { return i == 0 ? std::max(1, ft * fr_gu / 8) : ft; };
+                auto gu_a = [&](int i) { return ft * i / nh; };
+                auto gu_b = [&](int i) { return ft * (i + 1) / nh; };
                 for (int i = 0; i < nh; ++i) {
                     const int a = gu_a(i), b2 = gu_b(i);
                     s->subs[pp::K_GU][n++] = pp::SubDesc{a, 2 * (b2 - a), b2 - a, ft, k0, kq - k0, 0, a, b2};
@@ -505,6 +502,8 @@ int pass_init(s2d2_ctx* c) {
             s->xcnt_off[k] = sync_words;
             sync_words += (size_t)((Xs[k] + 127) / 128);
         }
+        s->attn_cnt_off = sync_words;       // per (sequence, kv head, query tile) of a pass: at most 64 sequences x query heads
+        sync_words += (size_t)pp::MAX_T * m.n_q_heads;
         s->sync_bytes = sync_words * 4;
         if (cudaMalloc((void**)&s->barrier, s->sync_bytes) != cudaSuccess) return fail_alloc(c);
     }
@@ -679,6 +678,7 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     size_t smem = pp::smem_bytes(p.T, p.S, m.head_dim);
     if (cudaMemsetAsync(s->barrier, 0, s->sync_bytes, c->stream) != cudaSuccess) return S2D2_ERR_CUDA;
     for (int k = 0; k < 4; ++k) p.x_cnt[k] = s->barrier + s->xcnt_off[k];
+    p.attn_cnt = s->barrier + s->attn_cnt_off;
     void* args[] = {&p};
     gemm_prof_begin(c);
     cudaError_t e = m.head_dim == 128

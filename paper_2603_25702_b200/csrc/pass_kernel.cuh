@@ -118,6 +118,7 @@ struct PassParams {
     unsigned* barrier;        // grid barrier counter, zero at launch
     unsigned* tile_cnt[N_KINDS];    // per GEMM kind and weight tile: partials published so far (zero at launch)
     unsigned* x_cnt[4];       // per 128-column tile of xn / attn / act / xn_b: (tile, row) pairs written so far (zero at launch)
+    unsigned* attn_cnt;       // per (sequence, kv head, query tile): attention items finished so far (zero at launch)
     SubDesc subs[N_KINDS][MAX_SUBS];
     int n_subs[N_KINDS];
     int acc_stride, n_acc;    // tensor-memory columns per accumulator buffer and buffers in the ring
@@ -1222,6 +1223,11 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                 const int n_splits = ap.n_cache_splits + 1;
                 const int total = ap.pv.n_seqs * ap.Hkv * ap.n_qtiles * n_splits;
                 const FastDiv by_splits(n_splits), by_qtiles(ap.n_qtiles);
+                // One sequence, dense model: the combine does not wait for a grid barrier behind the items but, pair by
+                // pair, for the count of finished items of its (sequence, kv head, query tile), every item of which is
+                // counted by the CTA that ran it.  (Several sequences: items are dealt out from a host-made list that
+                // leaves out the splits without keys, and the barrier stays.)
+                const bool counted = !p.moe && !ap.sched_off;
                 // Items of this CTA: a host-made list when the pass has several sequences (their context
                 // lengths differ, so items are dealt out by cost), else every G-th item.
                 const int i_end = ap.sched_off ? __ldg(ap.sched_off + cta + 1) : total;
@@ -1248,6 +1254,10 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         ok = false;
                         *abort_flag = 1;
                     }
+                    if (counted) {
+                        att::group_sync(BAR_COMPUTE, CTHREADS);      // every thread's part of the partial is stored
+                        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.attn_cnt + r) : "memory");
+                    }
                 }
                 if (!ok) break;
                 // the row table entries of this warp's first combine pair are fetched before the barrier, not behind it
@@ -1259,9 +1269,14 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     pre_row0 = __ldg(p.pv.seq_row0 + pre_seq);
                     pre_nctx = __ldg(p.pv.seq_nctx + pre_seq);
                 }
-                grid_sync(false, tb + 3, p.moe);
-                if (!ok) break;
+                if (counted) {
+                    mark(tb + 3);
+                } else {
+                    grid_sync(false, tb + 3, p.moe);
+                    if (!ok) break;
+                }
                 // ---- combine the key splits of every (row, query head) ----
+                bool first_pair = true;
                 for (int pair = gw; pair < M * p.Hq; pair += GW) {
                     int r, hq;
                     by_Hq.divmod(pair, r, hq);
@@ -1272,6 +1287,23 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     const int n_ctx = first ? pre_nctx : __ldg(p.pv.seq_nctx + seq);
                     const int n_pages = (n_ctx + ap.page_tokens - 1) >> ap.page_shift;
                     const size_t item0 = ((size_t)(seq * ap.Hkv + kvh) * ap.n_qtiles + qt) * n_splits;
+                    if (counted) {      // all items of this (sequence, kv head, query tile) have stored their partials
+                        const unsigned* cntp = p.attn_cnt + (seq * ap.Hkv + kvh) * ap.n_qtiles + qt;
+                        const unsigned target = (unsigned)n_splits * ((unsigned)l + 1u);
+                        bool ready = false;
+                        for (uint32_t it = 0; !ready && it < SPIN_LIMIT; ++it) {
+                            ready = ld_acquire(cntp) >= target;
+                            if (!ready && (it & 63u) == 63u && (*abort_flag || *(volatile int*)p.status != 0)) break;
+                        }
+                        if (!ready) {
+                            atomicCAS(p.status, 0, 11);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        if (first_pair) mark(tb + 4);
+                        first_pair = false;
+                    }
                     // Lanes take the splits for maxima and weights, and 4 output columns each (the
                     // first HD/4 lanes) for the sums.  Whether a split was written follows from the
                     // page count alone, so the loads of the partial outputs do not wait for the weights.
@@ -1326,6 +1358,8 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                     }
                     publish_x(p.x_cnt[1] + hq * HD / tc::BLOCK_N);
                 }
+                if (counted && first_pair) mark(tb + 4);
+                if (!ok) break;
             }
             // The O GEMM fetches the combined rows as their columns are counted, so dense layers need no
             // barrier here; from this point to the next layer's q/k/v the GEMMs of a dense layer follow each

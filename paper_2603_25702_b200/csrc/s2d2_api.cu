@@ -380,6 +380,7 @@ static int check_status(s2d2_ctx* c) {
     const int code = *c->h_status;
     *c->h_status = 0;
     cudaMemsetAsync(c->d_status, 0, 4, c->stream);
+    gemm_reset_tickets(c);      // a split-K CTA that gave up took no ticket: start the next GEMM from clean counters
     FAIL(c, S2D2_ERR_TIMEOUT, "a kernel gave up on a bounded wait (results of this call are invalid; device status word " +
                                    std::to_string(code) + ")");
 }
@@ -615,7 +616,12 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
             int left = s.n_final - s.n_c;
             if (left <= 0 || room <= 0) continue;
             int rows = std::min(std::min(left, CH), room);
-            if ((rc = ensure_pages(c, s, s.n_c + rows))) return rc;
+            if ((rc = ensure_pages(c, s, s.n_c + rows))) {
+                const std::string why = c->err;
+                for (int id : ids) s2d2_release_seq(c, id);      // nothing of this call stays behind: slots and pages go back
+                c->err = why;
+                return rc;
+            }
             begin_seq(c, pb, s, s.n_c);
             for (int r = 0; r < rows; ++r)
                 add_row(c, pb, s.tok[s.n_c + r], s.n_c + r, (r == 63) ? ~0ull : ((1ull << (r + 1)) - 1), ROW_WRITE_KV, false);
@@ -623,7 +629,12 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
             room -= rows;
         }
         if (pb.n_rows == 0) break;
-        if ((rc = run_pass(c, pb, nullptr))) return rc;
+        if ((rc = run_pass(c, pb, nullptr))) {
+            const std::string why = c->err;
+            for (int id : ids) s2d2_release_seq(c, id);
+            c->err = why;
+            return rc;
+        }
         c->cnt.n_prefill_passes++;
         c->cnt.n_rows_prefill += pb.n_rows;
         // the metadata buffer is reused by the next chunk: wait for this pass to have consumed it
@@ -633,7 +644,12 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
     if ((rc = enqueue_status_read(c))) return rc;
     CUDA_TRY(c, cudaEventRecord(c->ev[7], c->stream));
     CUDA_TRY(c, cudaEventSynchronize(c->ev[7]));
-    if ((rc = check_status(c))) return rc;
+    if ((rc = check_status(c))) {
+        const std::string why = c->err;
+        for (int id : ids) s2d2_release_seq(c, id);
+        c->err = why;
+        return rc;
+    }
     float ms = 0;
     cudaEventElapsedTime(&ms, c->ev[6], c->ev[7]);
     c->cnt.ms_prefill += ms;

@@ -18,9 +18,9 @@ torch = pytest.importorskip("torch")
 @pytest.mark.parametrize("name,batch,gen_tokens,max_steps", [
     ("c2", 1, 512, 600),          # the workload's full generation
     ("c3", 8, 96, 200),           # its batch of 8 with the mean-confidence router
-    ("c4", 1, 128, 400),
-    ("c4", 32, 16, 6),            # the batch-32 point: passes of 256 to 512 rows, one kernel per operation
-    ("c5", 1, 96, 200),           # mixture of experts at block 32
+    ("c4", 1, 96, 400),
+    ("c4", 32, 16, 4),            # the batch-32 point: passes of 256 to 512 rows, one kernel per operation
+    ("c5", 1, 64, 200),           # mixture of experts at block 32
 ])
 def test_long_run_acceptance_stage_is_exact(name, batch, gen_tokens, max_steps):
     from paper_2603_25702_b200 import Engine, RoutePolicy

@@ -178,6 +178,9 @@ def test_error_paths_return_codes_not_faults():
     with pytest.raises(S2D2Error) as ei:                 # page pool exhausted (2 pages of 8 tokens)
         e.prefill([list(range(20))])
     assert ei.value.code == -3
+    assert e.get_counters().kv_pages_in_use == 0        # the failed call left neither pages nor its sequence slot behind
+    sid = e.prefill([[1, 2, 3]])[0]                      # (max_batch is 1: a leaked slot would refuse this)
+    assert e.get_counters().kv_pages_in_use == 1 and len(e.get_tokens(sid)) == 3
     e.close()
     e = _engine(wl, W)
     sid = e.prefill([[1, 2, 3]])[0]

@@ -70,7 +70,8 @@ def test_pass_trace_is_monotone_and_complete():
     used = [0, 1] + list(range(3, n_named))                # slot 2 is unused
     flat = marks[:, used]
     assert (flat > 0).all() and (np.diff(flat, axis=1) >= 0).all()    # every CTA passes its marks in slot order
-    # nobody leaves a grid barrier before everybody has entered it
+    # nobody leaves a grid barrier before everybody has entered it (with one sequence in the pass the attention items hand over
+    # to the combine through counters, not a barrier: this pass has several, so both are barriers)
     bars = [(0, 1)] + [(3 + 12 * l + names.index(n + "_entry"), 3 + 12 * l + names.index(n + "_exit"))
                        for l in range(L) for n in ("rope_barrier", "attn_barrier")]
     for ent, ex in bars:
