@@ -621,7 +621,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                             }
                             tc::mbar_expect_tx(&full[s], W_TILE_BYTES);
                             tc::tma_load_2d_hint(dst, map, x, y, &full[s], policy);
-                            ++issued;
+                            *w_issued = (int)++issued;
                             dst += sbytes;
                             if (++s == S) {
                                 s = 0;
@@ -630,7 +630,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                                 first_round = false;
                             }
                         }
-                        *w_issued = (int)issued;
                         d = dn;
                     }
                 };
@@ -868,7 +867,7 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                                 acc = 1;
                             }
                             tc::umma_commit(&empty[s]);
-                            ++done;
+                            *consumed = (int)++done;
                             a_desc += desc_step;
                             if (++s == S) {
                                 s = 0;
@@ -878,7 +877,6 @@ __global__ void __launch_bounds__(THREADS, 1) pass_kernel(const __grid_constant_
                         }
                         if (!ok) break;
                         tc::umma_commit(&acc_full[b]);
-                        *consumed = (int)done;
                         if (last_of_sub && tm) stamp(tm + 1);
                         if (++b == (uint32_t)NACC) {
                             b = 0;
