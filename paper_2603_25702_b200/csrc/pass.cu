@@ -572,7 +572,7 @@ int pass_run(s2d2_ctx* c, const PassView& pv, int max_ctx, int max_rows, long lo
     PassState* s = state(c);
     const s2d2_model_config& m = c->m;
     if (!s || !s->ok || pv.n_rows < 1 || pv.n_rows > pp::MAX_T) return S2D2_OK;
-    pp::PassParams p;
+    pp::PassParams p{};      // every field starts from zero; the ones a pass needs are set below
     // several sequences: finer key splits (about two items per CTA), dealt out by cost
     if (!attention_plan(c, pv, max_ctx, max_rows, pv.n_seqs > 1 ? 2 * s->grid : s->grid, &p.ap, nullptr)) return S2D2_OK;
     if (pv.n_seqs > 1) {
