@@ -73,7 +73,8 @@ int attention_init(s2d2_ctx* c) {
     if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return S2D2_ERR_CUDA;
     a->n_sms = prop.multiProcessorCount;
     int group = m.n_q_heads / m.n_kv_heads;
-    size_t base_items = (size_t)c->dc.max_batch * m.n_kv_heads * ((S2D2_MAX_ROWS_PER_SEQ * group + att::QT - 1) / att::QT);
+    // (a prefill pass lists every 64-row chunk of a prompt as a sequence of its own)
+    size_t base_items = (size_t)(c->dc.max_batch + c->max_rows / S2D2_MAX_ROWS_PER_SEQ) * m.n_kv_heads * ((S2D2_MAX_ROWS_PER_SEQ * group + att::QT - 1) / att::QT);
     a->cap_items = std::max<size_t>(2048, base_items * 2);
     if (cudaMalloc((void**)&a->part_o, a->cap_items * att::QT * m.head_dim * 4) != cudaSuccess) return S2D2_ERR_CUDA;
     if (cudaMalloc((void**)&a->part_ml, a->cap_items * att::QT * 2 * 4) != cudaSuccess) return S2D2_ERR_CUDA;

@@ -36,6 +36,9 @@ using namespace s2d2;
     } while (0)
 #define LAUNCHED(ctx) ((ctx)->cnt.n_kernel_launches++)
 
+// Rows of a wide prefill pass (the activation scratch of every context has at least this many rows).
+static constexpr int PREFILL_PASS_ROWS = 1024;
+
 static size_t esize(int dtype) { return dtype == S2D2_DTYPE_BF16 ? 2 : 4; }
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -217,7 +220,9 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
 
     // scratch
     int rows_per_seq = std::max(2 * dc->block_size, S2D2_MAX_ROWS_PER_SEQ);
-    c->max_rows = dc->max_batch * rows_per_seq;
+    // A prefill pass carries several 64-row chunks of one prompt (see s2d2_prefill), so even a context for one
+    // sequence gets room for a pass wide enough to be tensor-bound.
+    c->max_rows = std::max(dc->max_batch * rows_per_seq, (int)PREFILL_PASS_ROWS);
     c->max_logit_rows = dc->max_batch * dc->block_size;
     size_t M = c->max_rows, d = m->d_model, es = esize(m->dtype);
     size_t nqkv = (size_t)(m->n_q_heads + 2 * m->n_kv_heads) * m->head_dim, nq = (size_t)m->n_q_heads * m->head_dim;
@@ -270,7 +275,7 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
     {
         PassMeta& pm = c->meta;
         pm.cap_rows = c->max_rows;
-        pm.cap_seqs = dc->max_batch;
+        pm.cap_seqs = dc->max_batch + c->max_rows / S2D2_MAX_ROWS_PER_SEQ;     // sequences plus the chunks of a prefill pass
         pm.max_pages = c->max_pages_per_seq;
         size_t o = 0;
         auto take = [&](size_t b) {
@@ -602,29 +607,47 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
     }
     CUDA_TRY(c, cudaEventRecord(c->ev[6], c->stream));
     const int CH = S2D2_MAX_ROWS_PER_SEQ;
-    // Rows per pass: where the persistent pass kernel is available a chunk is cut to what that kernel
-    // takes (it is both faster and carries two-term operands); otherwise one chunk of every sequence.
-    // (a few sequences only: a large batch prefills faster as wide per-operation passes, which are tensor-bound)
-    const int budget = pass_max_rows(c) > 0 && ids.size() <= 4 ? pass_max_rows(c) : CH * (int)ids.size();
     std::vector<int> took(ids.size());
+    // A row's in-pass mask has 64 bits, so one prompt enters a pass as chunks of at most 64 rows.  The chunks of one
+    // prompt may share a pass: each is listed as a sequence of its own whose visible cache ends where the chunk
+    // begins and whose page list is the prompt's.  K/V of every row is in the cache before attention starts, so a
+    // chunk reads its predecessors of the same pass from the pages and only its own rows through the mask.
+    // Which passes: a prompt remainder that one persistent pass can take (and at most four of them) goes through the
+    // persistent kernel, which streams the weights once per 64 rows; everything longer goes through wide passes of
+    // the per-operation kernels, which are tensor-bound and stream the weights once per PREFILL_PASS_ROWS rows.
+    const int pr = pass_max_rows(c);
     for (;;) {
+        int n_short = 0, n_long = 0;
+        for (size_t k = 0; k < ids.size(); ++k) {
+            const SeqState& s = c->seqs[ids[k]];
+            const int left = s.n_final - s.n_c;
+            if (left > 0) ++(pr > 0 && left <= pr ? n_short : n_long);
+        }
+        const bool shorts_ride = pr == 0 || n_short > 4;
+        const bool wide = n_long > 0 || (n_short > 0 && shorts_ride);
         PassBuild pb;
-        int room = budget;
+        int room = wide ? c->max_rows : pr;
         for (size_t k = 0; k < ids.size(); ++k) {
             SeqState& s = c->seqs[ids[k]];
             took[k] = 0;
-            int left = s.n_final - s.n_c;
+            const int left = s.n_final - s.n_c;
             if (left <= 0 || room <= 0) continue;
-            int rows = std::min(std::min(left, CH), room);
+            if (wide && pr > 0 && left <= pr && !shorts_ride) continue;      // waits for the persistent pass
+            int rows = std::min(left, room);
+            if (rows < left) rows -= rows % CH;                               // whole chunks unless the prompt ends
+            if (rows <= 0) continue;
             if ((rc = ensure_pages(c, s, s.n_c + rows))) {
                 const std::string why = c->err;
                 for (int id : ids) s2d2_release_seq(c, id);      // nothing of this call stays behind: slots and pages go back
                 c->err = why;
                 return rc;
             }
-            begin_seq(c, pb, s, s.n_c);
-            for (int r = 0; r < rows; ++r)
-                add_row(c, pb, s.tok[s.n_c + r], s.n_c + r, (r == 63) ? ~0ull : ((1ull << (r + 1)) - 1), ROW_WRITE_KV, false);
+            for (int r0 = 0; r0 < rows; r0 += CH) {
+                const int n = std::min(CH, rows - r0), base = s.n_c + r0;
+                begin_seq(c, pb, s, base);
+                for (int r = 0; r < n; ++r)
+                    add_row(c, pb, s.tok[base + r], base + r, (r == 63) ? ~0ull : ((1ull << (r + 1)) - 1), ROW_WRITE_KV, false);
+            }
             took[k] = rows;
             room -= rows;
         }

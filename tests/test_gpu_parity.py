@@ -437,3 +437,29 @@ def test_block_end_caching_matches_oracle(name, atol, rtol):
         c = e.get_counters()
         assert c.n_draft_passes == orc.n_draft_passes and c.n_verify_passes == orc.n_verify_passes and c.n_cache_passes == orc.n_cache_passes
         e.close()
+
+
+@pytest.mark.parametrize("name,lens,passes", [
+    ("t_bf16_128", [300, 40, 129, 24], 2),      # two long prompts share one wide pass (5 + 3 chunks); the short ones take one persistent pass
+    ("t_bf16_128", [1500], 2),                  # 1024 rows (16 chunks of one prompt in one pass), then 476
+    ("t_bf16", [65, 5, 9, 70, 3, 11, 2], 1),    # more than four short prompts ride the wide pass; 16-token pages
+    ("t_f32", [150, 7], 1),                     # fp32 model: plain kernels, every prompt in wide passes
+])
+def test_prefill_in_wide_passes_matches_oracle(name, lens, passes):
+    """Prefill (first line of the block-wise decoding algorithm: the prompt's K/V under the causal mask).  A prompt
+    enters a pass as 64-row chunks, several chunks of one prompt in the same pass: chunk k reads chunks 0..k-1 of
+    that pass from the cache pages they were written to a kernel earlier.  The cache of every sequence must equal
+    the oracle's causal pass over its prompt."""
+    from tests.parity_util import check_kv
+    wl = get_config(name, batch=len(lens), prompt_len=(min(lens), max(lens)))
+    W = generate_weights(wl.model, seed=3)
+    rng = np.random.default_rng(11)
+    prompts = [rng.integers(0, wl.model.vocab, size=n).tolist() for n in lens]
+    e, ids, _ = _start(wl, W, prompts)
+    cnt = e.get_counters()
+    assert cnt.n_prefill_passes == passes and cnt.n_rows_prefill == sum(lens)
+    for sid, n in zip(ids, lens):
+        assert e.debug_seq_state(sid)["n_cached"] == n
+        worst = check_kv(e, W, wl.model, sid, atol=1e-5 if wl.model.dtype == "fp32" else 4e-2)
+        print(name, n, "KV off by", worst)
+    e.close()
