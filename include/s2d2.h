@@ -315,6 +315,10 @@ int s2d2_debug_seq_state(s2d2_ctx* ctx, int32_t seq_id, int32_t* n_cached, int32
  * x and w in the model's storage type (bf16 bit patterns or fp32), y fp32. Uses the
  * same kernel selection as the forward pass. Allocates temporaries. */
 int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int32_t N, int32_t K, float* y);
+/* The same with the token operand as two bf16 terms, x = x_hi + x_lo (x_lo may be NULL), an output scale and, with
+ * accumulate != 0, y_inout[M,N] += scale * x w^T (y_inout is read, then overwritten with the result). bf16 models only. */
+int s2d2_debug_gemm2(s2d2_ctx* ctx, const void* x_hi, const void* x_lo, const void* w, int32_t M, int32_t N, int32_t K,
+                     float scale, int32_t accumulate, float* y_inout);
 
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);

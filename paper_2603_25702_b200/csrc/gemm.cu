@@ -13,6 +13,7 @@
 
 #include "context.h"
 #include "gemm_tc.cuh"
+#include "gemm_wide.cuh"
 #include "kernels_simt.cuh"
 
 using namespace s2d2;
@@ -68,9 +69,87 @@ void gemm_simt(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N
     c->cnt.n_kernel_launches++;
 }
 
+// Wide passes (more than 64 token rows): gemm_wide_kernel.  One CTA per SM (its stage ring and its epilogue
+// buffers take most of the shared memory); the host picks weight sub-tiles per CTA and K splits so that the
+// CTAs cover the SMs: a GEMM with few weight tiles (QKV, O, down) would otherwise run on a third of the machine.
+// Cost model in microseconds: a k-block takes the slowest of the fill of one SM's shared memory (80 KB/us), the fill of
+// all streaming SMs together (10.5 MB/us) and its MMAs; a CTA adds WIDE_CTA_US of set-up and epilogue; a split adds the
+// round trip of its partial sub-tiles through the workspace.
+constexpr double WIDE_CTA_US = 7.0, WIDE_SPLIT_US = 3.0;
+int gemm_wide(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
+              int accumulate, const void* X_lo) {
+    GemmState* g = state(c);
+    tc::GemmParams p;
+    p.Y = Y;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.ldy = ldy;
+    p.scale = scale;
+    p.accumulate = accumulate;
+    p.kb_total = K / tc::BLOCK_K;
+    p.hilo = X_lo != nullptr;
+    const int t_max = 128;                        // an epilogue buffer is [T][128] fp32; three of them fit beside nothing else
+    p.m_tiles = (M + t_max - 1) / t_max;
+    const int per = (M + p.m_tiles - 1) / p.m_tiles;
+    p.T = std::min(t_max, (per + 15) / 16 * 16);
+    p.m_tiles = (M + p.T - 1) / p.T;
+    const int TN = p.hilo ? 2 * p.T : p.T;
+    const size_t smem_max = 225 * 1024;
+    int best = 0, best_wt = 0, best_stages = 0;
+    double best_cost = 1e30;
+    for (int wt = 1; wt <= 2; ++wt) {
+        if (wt == 2 && (2 * TN > 512 || N < 2 * tc::BLOCK_N)) break;
+        const size_t sb = tc::stage_bytes(TN, wt);
+        const int tiles = (N + wt * tc::BLOCK_N - 1) / (wt * tc::BLOCK_N) * p.m_tiles;
+        const double kb_kb = sb / 1024.0, mma_us = wt * TN * (0.276 / 256.0);
+        for (int s = 1; s <= 16 && (s == 1 || s <= p.kb_total / 4); ++s) {
+            int stages = (int)std::min<size_t>(8, (200 * 1024) / sb);
+            stages = std::min(stages, (p.kb_total + s - 1) / s);
+            if (stages < 2 && p.kb_total > 1) break;
+            stages = std::max(stages, 1);
+            if (tc::wide_smem_bytes(p.T, TN, stages, wt, s) > smem_max) continue;
+            if (s > 1 && ((size_t)tiles * s * wt * p.T * tc::BLOCK_N > g->ws_floats || (size_t)tiles > g->n_tickets)) break;
+            const int ctas = tiles * s, waves = (ctas + g->n_sms - 1) / g->n_sms, streaming = std::min(ctas, g->n_sms);
+            const double kb_us = std::max(std::max(kb_kb / 80.0, kb_kb * streaming / 10500.0), mma_us);
+            const double sub_kb = p.T * 0.5;
+            const double cost = waves * ((double)((p.kb_total + s - 1) / s) * kb_us + WIDE_CTA_US + wt * sub_kb / 80.0) +
+                                (s > 1 ? WIDE_SPLIT_US + wt * (s + 1) * sub_kb / 80.0 : 0.0);
+            if (cost < best_cost - 1e-9) {
+                best_cost = cost;
+                best = s;
+                best_wt = wt;
+                best_stages = stages;
+            }
+        }
+    }
+    if (!best) return -1;
+    p.splits = best;
+    p.wtiles = best_wt;
+    p.stages = best_stages;
+    p.n_tiles = (N + best_wt * tc::BLOCK_N - 1) / (best_wt * tc::BLOCK_N);
+    p.ws = g->ws;
+    p.tickets = g->tickets;
+    p.status = c->d_status;
+    p.evict_first = 0;
+    const CUtensorMap* mw = get_map(c, W, N, K, tc::BLOCK_N);
+    const CUtensorMap* mx = get_map(c, X, M, K, p.T);
+    const CUtensorMap* mx_lo = p.hilo ? get_map(c, X_lo, M, K, p.T) : mx;
+    if (!mw || !mx || !mx_lo) return S2D2_ERR_CUDA;
+    const int grid = p.n_tiles * p.m_tiles * p.splits;
+    tc::gemm_wide_kernel<<<grid, tc::THREADS, tc::wide_smem_bytes(p.T, TN, p.stages, p.wtiles, p.splits), c->stream>>>(*mw, *mx, *mx_lo, p);
+    c->cnt.n_kernel_launches++;
+    return S2D2_OK;
+}
+
 int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
             int accumulate, const void* X_lo) {
     GemmState* g = state(c);
+    // bulk copies want 16-byte rows: Y, its leading dimension and the width of the matrix in whole float4
+    if (M > 64 && ldy % 4 == 0 && N % 4 == 0 && ((uintptr_t)Y & 15) == 0) {
+        int rc = gemm_wide(c, X, W, Y, M, N, K, ldy, scale, accumulate, X_lo);
+        if (rc >= 0) return rc;
+    }
     tc::GemmParams p;
     p.Y = Y;
     p.M = M;
@@ -171,7 +250,8 @@ int gemm_init(s2d2_ctx* c) {
     if (cudaMalloc((void**)&g->ws, g->ws_floats * 4) != cudaSuccess) return S2D2_ERR_CUDA;
     if (cudaMalloc((void**)&g->tickets, g->n_tickets * 4) != cudaSuccess) return S2D2_ERR_CUDA;
     if (cudaMemset(g->tickets, 0, g->n_tickets * 4) != cudaSuccess) return S2D2_ERR_CUDA;
-    if (cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(tc::gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
         c->err = "cannot raise the dynamic shared memory limit";
         return S2D2_ERR_CUDA;
     }

@@ -1481,6 +1481,37 @@ extern "C" int s2d2_debug_gemm(s2d2_ctx* c, const void* x, const void* w, int32_
     return rc;
 }
 
+extern "C" int s2d2_debug_gemm2(s2d2_ctx* c, const void* x_hi, const void* x_lo, const void* w, int32_t M, int32_t N, int32_t K,
+                                float scale, int32_t accumulate, float* y) {
+    if (!c || !x_hi || !w || !y || M < 1 || N < 1 || K < 1) return S2D2_ERR_INVALID;
+    if (c->m.dtype != S2D2_DTYPE_BF16) FAIL(c, S2D2_ERR_UNSUPPORTED, "debug_gemm2: bf16 models only");
+    void *dx = nullptr, *dl = nullptr, *dw = nullptr;
+    float* dy = nullptr;
+    CUDA_TRY(c, cudaMalloc(&dx, (size_t)M * K * 2));
+    CUDA_TRY(c, cudaMalloc(&dl, (size_t)M * K * 2));
+    CUDA_TRY(c, cudaMalloc(&dw, (size_t)N * K * 2));
+    CUDA_TRY(c, cudaMalloc((void**)&dy, (size_t)M * N * 4));
+    CUDA_TRY(c, cudaMemcpyAsync(dx, x_hi, (size_t)M * K * 2, cudaMemcpyHostToDevice, c->stream));
+    if (x_lo) CUDA_TRY(c, cudaMemcpyAsync(dl, x_lo, (size_t)M * K * 2, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(dw, w, (size_t)N * K * 2, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(dy, y, (size_t)M * N * 4, cudaMemcpyHostToDevice, c->stream));
+    int rc = gemm(c, dx, dw, dy, M, N, K, N, scale, accumulate, x_lo ? dl : nullptr);
+    if (!rc) rc = enqueue_status_read(c);
+    if (!rc) {
+        CUDA_TRY(c, cudaMemcpyAsync(y, dy, (size_t)M * N * 4, cudaMemcpyDeviceToHost, c->stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        rc = check_status(c);
+    }
+    gemm_forget(c, dx);
+    gemm_forget(c, dl);
+    gemm_forget(c, dw);
+    cudaFree(dx);
+    cudaFree(dl);
+    cudaFree(dw);
+    cudaFree(dy);
+    return rc;
+}
+
 extern "C" int s2d2_debug_copy_expert_ids(s2d2_ctx* c, int32_t* out, int64_t cap, int32_t* n_rows) {
     if (!c || !out || !n_rows) return S2D2_ERR_INVALID;
     if (c->m.n_experts == 0) FAIL(c, S2D2_ERR_UNSUPPORTED, "not a MoE model");

@@ -35,3 +35,28 @@ def test_gemm_matches_float64(engine, M, N, K):
     # twice the same launch: bitwise identical (split-K partials are summed in a fixed order)
     again = engine.debug_gemm(x, w)
     assert np.array_equal(got, again)
+
+
+@pytest.mark.parametrize("M,N,K,acc,scale", [
+    (65, 256, 256, False, 1.0), (100, 640, 2048, True, 1.0), (181, 6144, 4096, False, 1.0), (265, 4096, 4096, True, 1.0),
+    (312, 4096, 12288, True, 1.0), (312, 24576, 4096, False, 1.0), (512, 6144, 4096, False, 0.5), (1024, 4096, 4096, True, 1.0),
+    (130, 300, 320, True, 2.0), (96, 151936, 256, False, 4.0), (700, 1000, 128, True, 1.0), (129, 128, 64, False, 1.0),
+])
+def test_wide_gemm_with_two_term_rows_matches_float64(engine, M, N, K, acc, scale):
+    """Passes of more than 64 rows (large batches, prefill): token operand x = hi + lo as two bf16 terms, results that
+    leave the CTA as bulk copies (plain, or added to the residual), K splits summed by the CTA that takes a tile's
+    last ticket.  Against float64 on the same inputs; the right and bottom edges of the matrix are ragged in some cases."""
+    rng = np.random.default_rng(M * 7919 + N * 31 + K)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    hi = f32_to_bf16_bits(x)
+    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi))
+    w = f32_to_bf16_bits((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
+    y0 = rng.standard_normal((M, N)).astype(np.float32)
+    got = engine.debug_gemm2(hi, lo, w, y0, scale=scale, accumulate=acc)
+    xs = bf16_bits_to_f32(hi).astype(np.float64) + bf16_bits_to_f32(lo).astype(np.float64)
+    want = scale * (xs @ bf16_bits_to_f32(w).astype(np.float64).T) + (y0.astype(np.float64) if acc else 0.0)
+    err = np.abs(got - want).max()
+    bound = 2e-6 * np.sqrt(K) * np.abs(want).max() + 1e-6
+    assert err <= bound, (err, bound)
+    again = engine.debug_gemm2(hi, lo, w, y0, scale=scale, accumulate=acc)
+    assert np.array_equal(got, again)
