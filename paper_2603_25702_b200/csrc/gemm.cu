@@ -142,6 +142,46 @@ int gemm_wide(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N,
     return S2D2_OK;
 }
 
+// gate/up GEMM of a wide pass with SwiGLU in its epilogue (see GemmParams::swiglu): two sub-tiles per CTA, no K split
+// (a layer's gate/up has weight tiles enough for every SM).
+int gemm_wide_swiglu(s2d2_ctx* c, const void* X, const void* X_lo, const void* W, int M, int f, int K, void* act, void* act_lo) {
+    tc::GemmParams p;
+    p.Y = nullptr;
+    p.M = M;
+    p.N = 2 * f;
+    p.K = K;
+    p.ldy = 0;
+    p.scale = 1.f;
+    p.accumulate = 0;
+    p.kb_total = K / tc::BLOCK_K;
+    p.hilo = X_lo != nullptr;
+    p.m_tiles = (M + 127) / 128;
+    const int per = (M + p.m_tiles - 1) / p.m_tiles;
+    p.T = std::min(128, (per + 15) / 16 * 16);
+    p.m_tiles = (M + p.T - 1) / p.T;
+    const int TN = p.hilo ? 2 * p.T : p.T;
+    p.wtiles = 2;
+    p.splits = 1;
+    p.stages = (int)std::min<size_t>(8, (200 * 1024) / tc::stage_bytes(TN, 2));
+    p.stages = std::max(1, std::min(p.stages, p.kb_total));
+    p.n_tiles = f / tc::BLOCK_N;
+    p.ws = nullptr;
+    p.tickets = nullptr;
+    p.status = c->d_status;
+    p.evict_first = 0;
+    p.swiglu = 1;
+    p.f = f;
+    p.act = (bf16*)act;
+    p.act_lo = (bf16*)act_lo;
+    const CUtensorMap* mw = get_map(c, W, 2 * f, K, tc::BLOCK_N);
+    const CUtensorMap* mx = get_map(c, X, M, K, p.T);
+    const CUtensorMap* mx_lo = p.hilo ? get_map(c, X_lo, M, K, p.T) : mx;
+    if (!mw || !mx || !mx_lo) return S2D2_ERR_CUDA;
+    tc::gemm_wide_kernel<<<p.n_tiles * p.m_tiles, tc::THREADS, tc::wide_smem_bytes(p.T, TN, p.stages, 2, 1), c->stream>>>(*mw, *mx, *mx_lo, p);
+    c->cnt.n_kernel_launches++;
+    return S2D2_OK;
+}
+
 int gemm_tc(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale,
             int accumulate, const void* X_lo) {
     GemmState* g = state(c);
@@ -351,6 +391,14 @@ int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int 
     gemm_simt<bf16, bf16>(c, X, W, Y, M, N, K, ldy, scale, accumulate);
     if (X_lo) gemm_simt<bf16, bf16>(c, X_lo, W, Y, M, N, K, ldy, scale, 1);
     return S2D2_OK;
+}
+
+int gemm_swiglu(s2d2_ctx* c, const void* X, const void* X_lo, const void* W, int M, int f, int K, void* act, void* act_lo) {
+    if (c->m.dtype != S2D2_DTYPE_BF16 || !state(c)->tc_ok || M <= 64 || K % tc::BLOCK_K || f % tc::BLOCK_N || !act_lo) return -1;
+    gemm_prof_begin(c);
+    int rc = gemm_wide_swiglu(c, X, X_lo, W, M, f, K, act, act_lo);
+    gemm_prof_end(c, 2.0 * f * K * 2 + (double)M * K * 2 * (X_lo ? 2 : 1) + (double)M * f * 4);
+    return rc;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -7,6 +7,9 @@ int gemm_init(s2d2_ctx* c);
 void gemm_destroy(s2d2_ctx* c);
 int gemm(s2d2_ctx* c, const void* X, const void* W, float* Y, int M, int N, int K, int ldy, float scale, int accumulate,
          const void* X_lo = nullptr);
+// act[M, f] = silu(X Wg^T) * (X Wu^T) with W = [Wg; Wu] ([2f, K]), written as two bf16 terms (act, act_lo), in one kernel.
+// Returns -1 when the shape or the model takes the separate GEMM and SwiGLU kernels instead (nothing was launched).
+int gemm_swiglu(s2d2_ctx* c, const void* X, const void* X_lo, const void* W, int M, int f, int K, void* act, void* act_lo);
 // Profiling helpers: bracket a launch with an event pair while profiling is on.
 void gemm_prof_begin(s2d2_ctx* c);
 void gemm_prof_end(s2d2_ctx* c, double algorithmic_bytes);

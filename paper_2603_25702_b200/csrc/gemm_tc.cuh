@@ -55,6 +55,12 @@ struct GemmParams {
     int evict_first;     // stream W with an evict-first L2 policy
     int wtiles;          // 128-row weight sub-tiles per CTA (1 or 2): two halve the re-reads of the token block
     int hilo;            // X arrives as two bf16 terms (X = X_hi + X_lo): both are token rows of one MMA (N = 2T, T <= 128)
+    // gemm_wide_kernel only: the GEMM is gate/up of a SwiGLU layer (W = [gate rows; up rows], f rows each).  A CTA takes the
+    // same 128 rows of both halves as its two sub-tiles and writes act = silu(gate) * up as two bf16 terms instead of Y.
+    int swiglu = 0;
+    int f = 0;
+    bf16* act = nullptr;
+    bf16* act_lo = nullptr;
 };
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes

@@ -141,7 +141,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             uint8_t* b = a + (size_t)WT * BLOCK_N * 128;
             mbar_expect_tx(&full[s], (uint32_t)sbytes);
             for (int h = 0; h < WT; ++h)       // a sub-tile past the matrix is zero-filled
-                tma_load_2d(a + h * BLOCK_N * 128, &map_w, kb * BLOCK_K, n0 + h * BLOCK_N, &full[s]);
+                tma_load_2d(a + h * BLOCK_N * 128, &map_w, kb * BLOCK_K, p.swiglu ? h * p.f + n_tile * BLOCK_N : n0 + h * BLOCK_N, &full[s]);
             tma_load_2d(b, &map_x, kb * BLOCK_K, m0, &full[s]);
             if (p.hilo) tma_load_2d(b + (size_t)T * 128, &map_x_lo, kb * BLOCK_K, m0, &full[s]);
             *issued = i + 1;
@@ -231,7 +231,35 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         bulk_commit();
     };
 
-    if (p.splits == 1) {
+    if (p.swiglu) {
+        // sub-tile 0 holds the gate columns, sub-tile 1 the up columns of the same 128 outputs: eight columns per thread and step
+        const float* g = (const float*)tiles;
+        const float* u = (const float*)(tiles + sub);
+        const int col0 = n_tile * BLOCK_N;
+        for (int idx = threadIdx.x; idx < m_hi * (BLOCK_N / 8); idx += THREADS) {
+            const int m = idx / (BLOCK_N / 8), c8 = (idx % (BLOCK_N / 8)) * 8;
+            float a[8];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const float4 gv = *(const float4*)(g + m * BLOCK_N + c8 + 4 * q), uv = *(const float4*)(u + m * BLOCK_N + c8 + 4 * q);
+                a[4 * q + 0] = gv.x / (1.f + expf(-gv.x)) * uv.x;
+                a[4 * q + 1] = gv.y / (1.f + expf(-gv.y)) * uv.y;
+                a[4 * q + 2] = gv.z / (1.f + expf(-gv.z)) * uv.z;
+                a[4 * q + 3] = gv.w / (1.f + expf(-gv.w)) * uv.w;
+            }
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bf16 h0 = __float2bfloat16_rn(a[2 * q]), h1 = __float2bfloat16_rn(a[2 * q + 1]);
+                const bf16 l0 = __float2bfloat16_rn(a[2 * q] - __bfloat162float(h0)), l1 = __float2bfloat16_rn(a[2 * q + 1] - __bfloat162float(h1));
+                hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                lo[q] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            }
+            const size_t o = (size_t)(m0 + m) * p.f + col0 + c8;
+            *(uint4*)(p.act + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *(uint4*)(p.act_lo + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+    } else if (p.splits == 1) {
         for (int h = 0; h < WT; ++h) rows_out(tiles + h * sub, h);
         bulk_wait_read();
     } else {

@@ -542,9 +542,13 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
             }
         } else {
             int f = m.ffn;
-            if ((rc = gemm(c, c->xn, L.wgu, c->gu, M, 2 * f, d, 2 * f, 1.f, 0, c->xn_lo))) return rc;
-            swiglu_kernel<TA><<<(unsigned)(((size_t)M * f + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, (TA*)c->act_lo, M, f);
-            LAUNCHED(c);
+            if ((rc = gemm_swiglu(c, c->xn, c->xn_lo, L.wgu, M, f, d, c->act, c->act_lo)) < 0) {      // wide passes: SwiGLU in the GEMM's epilogue
+                if ((rc = gemm(c, c->xn, L.wgu, c->gu, M, 2 * f, d, 2 * f, 1.f, 0, c->xn_lo))) return rc;
+                swiglu_kernel<TA><<<(unsigned)(((size_t)M * f + 255) / 256), 256, 0, st>>>(c->gu, (TA*)c->act, (TA*)c->act_lo, M, f);
+                LAUNCHED(c);
+            } else if (rc) {
+                return rc;
+            }
             if ((rc = gemm(c, c->act, L.wdown, c->h, M, d, f, d, 1.f, 1, c->act_lo))) return rc;
         }
     }
