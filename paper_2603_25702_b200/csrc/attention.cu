@@ -13,6 +13,61 @@
 
 using namespace s2d2;
 
+namespace s2d2 {
+namespace att {
+// The merge of attn_combine_kernel for wide passes: one block per row, a warp per query head at a time, four output columns per lane
+// (head_dim 128), so a pass of some hundred rows is a few hundred blocks instead of rows x heads small ones.
+static __global__ void __launch_bounds__(256) attn_combine_rows_kernel(AttnParams p) {
+    constexpr int HD = 128;
+    const int r = blockIdx.x, lane = threadIdx.x & 31;
+    const int seq = p.pv.row_seq[r];
+    const int n_splits = p.n_cache_splits + 1;
+    const int n_pages = (p.pv.seq_nctx[seq] + p.page_tokens - 1) >> p.page_shift;
+    const int qrow = (r - p.pv.seq_row0[seq]) * p.group;
+    for (int hq = threadIdx.x >> 5; hq < p.Hq; hq += 8) {
+        const int kvh = hq / p.group;
+        const int qv = qrow + hq % p.group;
+        const int qt = qv / QT, qi = qv % QT;
+        const size_t item0 = ((size_t)(seq * p.Hkv + kvh) * p.n_qtiles + qt) * n_splits;
+        float m = -INFINITY;
+        for (int s = 0; s < n_splits; ++s) {
+            const bool used = s == p.n_cache_splits || s * p.pages_per_split < n_pages;
+            if (used) m = fmaxf(m, __ldcg(p.part_ml + (item0 + s) * QT * 2 + qi * 2));
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
+        for (int s = 0; s < n_splits; ++s) {          // fixed split order
+            const bool used = s == p.n_cache_splits || s * p.pages_per_split < n_pages;
+            if (!used) continue;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (item0 + s) * QT * 2 + qi * 2));
+            if (ml.x == -INFINITY) continue;
+            const float w = exp2f(ml.x - m);
+            const float4 o = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((item0 + s) * QT + qi) * HD) + lane);
+            l += w * ml.y;
+            acc.x += w * o.x;
+            acc.y += w * o.y;
+            acc.z += w * o.z;
+            acc.w += w * o.w;
+        }
+        const float o0 = acc.x / l, o1 = acc.y / l, o2 = acc.z / l, o3 = acc.w / l;
+        const size_t off = ((size_t)r * p.Hq + hq) * HD + lane * 4;
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(o0, o1), h1 = __floats2bfloat162_rn(o2, o3);
+        uint2 u;
+        u.x = *reinterpret_cast<const uint32_t*>(&h0);
+        u.y = *reinterpret_cast<const uint32_t*>(&h1);
+        *reinterpret_cast<uint2*>(p.out + off) = u;
+        if (p.out_lo) {
+            const __nv_bfloat162 l0 = __floats2bfloat162_rn(o0 - __low2float(h0), o1 - __high2float(h0));
+            const __nv_bfloat162 l1 = __floats2bfloat162_rn(o2 - __low2float(h1), o3 - __high2float(h1));
+            u.x = *reinterpret_cast<const uint32_t*>(&l0);
+            u.y = *reinterpret_cast<const uint32_t*>(&l1);
+            *reinterpret_cast<uint2*>(p.out_lo + off) = u;
+        }
+    }
+}
+}  // namespace att
+}  // namespace s2d2
+
 namespace {
 struct AttnState {
     bool tc_ok = false;
@@ -164,7 +219,8 @@ int attention(s2d2_ctx* c, const PassView& pv, int layer, int max_ctx, int max_r
     // two-term queries and probabilities whenever the low halves of q exist (always on this path)
     if (a->umma_ok && p.q_lo) {
         att::attn_umma_kernel<<<grid, att::THREADS, att::attn_umma_smem_bytes(), c->stream>>>(a->map_kv, p);
-        att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);
+        if (pv.n_rows > 64) att::attn_combine_rows_kernel<<<pv.n_rows, 256, 0, c->stream>>>(p);
+        else att::attn_combine_kernel<128><<<dim3(pv.n_rows, m.n_q_heads), 128, 0, c->stream>>>(p);
     } else if (m.head_dim == 128) {
         if (p.q_lo) att::attn_tc_kernel<128, true><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);
         else att::attn_tc_kernel<128, false><<<grid, att::THREADS, smem, c->stream>>>(a->map_kv, p);

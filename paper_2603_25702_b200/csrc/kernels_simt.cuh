@@ -174,6 +174,90 @@ __global__ void qk_rope_kv_kernel(const float* __restrict__ qkv, PassView pv, co
     }
 }
 
+// The same for wide passes: a warp per (row, head), eight heads per block, the per-head sum of squares by warp
+// shuffles (head_dim up to 256: a lane holds up to four rotation pairs).
+template <typename TA, typename TKV>
+__global__ void __launch_bounds__(256) qk_rope_kv_rows_kernel(const float* __restrict__ qkv, PassView pv, const float* __restrict__ q_gain,
+                                       const float* __restrict__ k_gain, const float* __restrict__ rope_cos,
+                                       const float* __restrict__ rope_sin, TA* __restrict__ q_out, TA* __restrict__ q_lo,
+                                       TKV* __restrict__ k_rows, TKV* __restrict__ v_rows, KvPool<TKV> pool, int layer, int Hq,
+                                       int Hkv, int hd, float eps, int qk_norm) {
+    const int r = blockIdx.x, head = blockIdx.y * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (head >= Hq + 2 * Hkv) return;
+    const int half = hd >> 1;
+    const float* src = qkv + (size_t)r * (Hq + 2 * Hkv) * hd + (size_t)head * hd;
+    float x1[4], x2[4];
+    float ss = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i = lane + 32 * j;
+        x1[j] = x2[j] = 0.f;
+        if (i < half) {
+            x1[j] = src[i];
+            x2[j] = src[i + half];
+            ss += x1[j] * x1[j] + x2[j] * x2[j];
+        }
+    }
+    const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
+    const int pos = pv.row_pos[r];
+    if (is_q || is_k) {
+        float inv = 1.f;
+        if (qk_norm) {
+            ss = warp_sum(ss);
+            const float m = ss / (float)hd + eps;
+            inv = rsqrtf(m);
+            inv = inv * (1.5f - 0.5f * m * inv * inv);
+        }
+        const float* g = is_q ? q_gain : k_gain;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = lane + 32 * j;
+            if (i < half) {
+                float a = x1[j], b = x2[j];
+                if (qk_norm) {
+                    a = a * inv * g[i];
+                    b = b * inv * g[i + half];
+                }
+                const float c = rope_cos[(size_t)pos * half + i], s = rope_sin[(size_t)pos * half + i];
+                x1[j] = a * c - b * s;
+                x2[j] = b * c + a * s;
+            }
+        }
+    }
+    if (is_q) {
+        const size_t o = ((size_t)r * Hq + head) * hd;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = lane + 32 * j;
+            if (i < half) {
+                store_two_term(q_out, q_lo, o + i, x1[j]);
+                store_two_term(q_out, q_lo, o + i + half, x2[j]);
+            }
+        }
+        return;
+    }
+    const int kvh = is_k ? head - Hq : head - Hq - Hkv;
+    TKV* dst = (is_k ? k_rows : v_rows) + ((size_t)r * Hkv + kvh) * hd;
+    TKV* cache = nullptr;
+    if (pv.row_flags[r] & ROW_WRITE_KV) {
+        const int page = pv.seq_pages[(size_t)pv.row_seq[r] * pv.max_pages + (pos >> pool.page_shift)];
+        cache = pool.ptr(layer, page, is_k ? 0 : 1, kvh, pos & (pool.page_tokens - 1));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i = lane + 32 * j;
+        if (i < half) {
+            const TKV a = from_f32<TKV>(x1[j]), b = from_f32<TKV>(x2[j]);
+            dst[i] = a;
+            dst[i + half] = b;
+            if (cache) {
+                cache[i] = a;
+                cache[i + half] = b;
+            }
+        }
+    }
+}
+
 // Two-part attention, plain form: one warp per (row, query head).  Part 1: all
 // cached tokens [0, n_ctx) of the row's sequence, read from the pages.  Part 2:
 // the rows of this pass the row's bitmask allows, read from the pass's K/V rows.

@@ -506,9 +506,14 @@ int run_pass_t(s2d2_ctx* c, const PassBuild& pb, float* logits_out) {
         LAUNCHED(c);
         int rc = gemm(c, c->xn, L.wqkv, c->qkv, M, nqkv, d, nqkv, 1.f, 0, c->xn_lo);
         if (rc) return rc;
-        qk_rope_kv_kernel<TA, TKV><<<dim3(M, m.n_q_heads + 2 * m.n_kv_heads), hd / 2, 0, st>>>(
-            c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TA*)c->q_lo, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
-            l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
+        if (M > 64 && hd <= 256)      // wide passes: a warp per (row, head) instead of a block
+            qk_rope_kv_rows_kernel<TA, TKV><<<dim3(M, (m.n_q_heads + 2 * m.n_kv_heads + 7) / 8), 256, 0, st>>>(
+                c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TA*)c->q_lo, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
+                l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
+        else
+            qk_rope_kv_kernel<TA, TKV><<<dim3(M, m.n_q_heads + 2 * m.n_kv_heads), hd / 2, 0, st>>>(
+                c->qkv, pv, L.q_norm, L.k_norm, c->rope_cos, c->rope_sin, (TA*)c->q, (TA*)c->q_lo, (TKV*)c->k_rows, (TKV*)c->v_rows, pool,
+                l, m.n_q_heads, m.n_kv_heads, hd, m.rms_eps, m.qk_norm);
         LAUNCHED(c);
         if ((rc = attention(c, pv, l, pb.max_ctx, pb.max_rows))) return rc;
         if ((rc = gemm(c, c->attn, L.wo, c->h, M, d, nq, d, 1.f, 1, c->attn_lo))) return rc;
