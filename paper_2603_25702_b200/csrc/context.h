@@ -117,6 +117,7 @@ struct s2d2_ctx {
     double *res_rsum = nullptr, *res_vsum = nullptr;   // per (sequence, chunk) residual and pi_v mass
     char *acc_h = nullptr, *acc_d = nullptr;      // staging for the acceptance kernel's inputs and outputs
     size_t acc_bytes = 0;
+    unsigned* acc_tickets = nullptr;               // per sequence of an acceptance launch: CTAs done so far (zero between launches)
     char* stats_h = nullptr;                       // pinned mirror of the draft statistics
     int *dsamp_h = nullptr, *dsamp_d = nullptr;    // draft sampling: per logit row position, Philox stream, step (pinned / device)
     int n_draft_logit_rows = 0, n_verify_logit_rows = 0;

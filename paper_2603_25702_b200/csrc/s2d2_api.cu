@@ -316,7 +316,9 @@ extern "C" int s2d2_create(const s2d2_model_config* m, const s2d2_decode_config*
         CUDA_TRY(c, cudaMallocHost((void**)&c->dsamp_h, std::max<size_t>(R, 1) * 12));
         if ((rc = dmalloc(c, &c->dsamp_d, R * 3))) return rc;
         size_t S = dc->max_batch;
-        c->acc_bytes = S * 4 * 12 + S * S2D2_MAX_BLOCK * 4 * 3 + 256;
+        c->acc_bytes = S * 4 * 12 + R * 4 + S * S2D2_MAX_BLOCK * 4 * 3 + 256;      // per sequence, plus the row -> sequence table
+        if ((rc = dmalloc(c, &c->acc_tickets, S))) return rc;
+        CUDA_TRY(c, cudaMemset(c->acc_tickets, 0, S * 4));
         CUDA_TRY(c, cudaMallocHost((void**)&c->acc_h, c->acc_bytes));
         CUDA_TRY(c, cudaMalloc((void**)&c->acc_d, c->acc_bytes));
     }
@@ -343,7 +345,7 @@ extern "C" int s2d2_destroy(s2d2_ctx* c) {
                     c->logits_draft, c->logits_verify, c->rope_cos, c->rope_sin, c->router_logits, c->moe_gates,
                     c->moe_ids, c->moe_gu, c->moe_act, c->moe_out, c->moe_ids_trace, c->meta.d, c->d_xhat, c->d_conf,
                     c->d_margin, c->d_entropy, c->d_lse, c->acc_d, c->d_status, c->chunk_d, c->chunk_v, c->rej_info,
-                    c->res_rsum, c->res_vsum, c->dsamp_d};
+                    c->res_rsum, c->res_vsum, c->dsamp_d, c->acc_tickets};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->meta.h) cudaFreeHost(c->meta.h);
@@ -1033,14 +1035,14 @@ extern "C" int s2d2_verify_block(s2d2_ctx* c, int32_t n, const int32_t* ids, con
 namespace {
 struct AccStage {     // layout of acc_h / acc_d for S sequences
     size_t S;
-    size_t o_draft0, o_verify0, o_len, o_pos0, o_stream, o_step, o_mode;     // inputs
+    size_t o_draft0, o_verify0, o_len, o_pos0, o_stream, o_step, o_mode, o_row_seq;     // inputs (row_seq: per verifier logit row)
     size_t o_nacc, o_rej, o_res, o_near, o_bits, o_u, o_a, o_v;              // outputs
     size_t in_bytes, total;
-    explicit AccStage(size_t s) : S(s) {
+    AccStage(size_t s, size_t verify_rows) : S(s) {
         size_t o = 0;
         auto t = [&](size_t b) { size_t r = o; o += b; return r; };
         o_draft0 = t(S * 4); o_verify0 = t(S * 4); o_len = t(S * 4); o_pos0 = t(S * 4);
-        o_stream = t(S * 4); o_step = t(S * 4); o_mode = t(S * 4);
+        o_stream = t(S * 4); o_step = t(S * 4); o_mode = t(S * 4); o_row_seq = t(verify_rows * 4);
         in_bytes = o;
         o_nacc = t(S * 4); o_rej = t(S * 4); o_res = t(S * 4); o_near = t(S * 4); o_bits = t(S * 4);
         o_u = t(S * S2D2_MAX_BLOCK * 4); o_a = t(S * S2D2_MAX_BLOCK * 4); o_v = t(S * S2D2_MAX_BLOCK * 4);
@@ -1051,6 +1053,14 @@ struct AccStage {     // layout of acc_h / acc_d for S sequences
 // n_draft_rows / n_verify_rows: logit rows of the two buffers that the sequences refer to.
 int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, const float* d_verify, const int* d_xhat,
                   const double* d_lse, const float* d_conf, int n_draft_rows, int n_verify_rows) {
+    {   // verifier logit row -> index of its sequence in this call (-1: a row of a sequence that is not part of it)
+        int* row_seq = (int*)(c->acc_h + a.o_row_seq);
+        const int *v0 = (const int*)(c->acc_h + a.o_verify0), *len = (const int*)(c->acc_h + a.o_len), *mode = (const int*)(c->acc_h + a.o_mode);
+        for (int r = 0; r < n_verify_rows; ++r) row_seq[r] = -1;
+        for (int i = 0; i < n; ++i)
+            if (mode[i])
+                for (int k = 0; k < len[i] && v0[i] + k < n_verify_rows; ++k) row_seq[v0[i] + k] = i;
+    }
     CUDA_TRY(c, cudaMemcpyAsync(c->acc_d, c->acc_h, a.in_bytes, cudaMemcpyHostToDevice, c->stream));
     c->cnt.h2d_bytes += a.in_bytes;
     c->cnt.d2h_bytes += a.total - a.in_bytes;
@@ -1086,21 +1096,17 @@ int launch_accept(s2d2_ctx* c, const AccStage& a, int n, const float* d_draft, c
     const int nch = vocab_chunks(c->m.vocab);
     in.verify_chunks = (const ChunkStats*)c->chunk_v;
     in.draft_chunks = (const ChunkStats*)c->chunk_d;
-    if (n_verify_rows > 0) {
-        vocab_chunk_stats_kernel<<<dim3(nch, n_verify_rows), VCHUNK_THREADS, 0, c->stream>>>(d_verify, c->m.vocab, (ChunkStats*)c->chunk_v);
-        LAUNCHED(c);
-    }
-    if (!d_lse && n_draft_rows > 0) {
+    if (!d_lse && n_draft_rows > 0) {      // stand-alone entry without draft statistics: the drafter's chunk statistics first
         vocab_chunk_stats_kernel<<<dim3(nch, n_draft_rows), VCHUNK_THREADS, 0, c->stream>>>(d_draft, c->m.vocab, (ChunkStats*)c->chunk_d);
         LAUNCHED(c);
     }
-    RejectInfo* rej = (RejectInfo*)c->rej_info;
-    accept_scan_kernel<<<n, 128, 0, c->stream>>>(in, out, rej);
+    // chunk statistics + scan in one launch, the residual draw in a second (see accept_fused_kernel)
+    accept_fused_kernel<<<dim3(nch, n_verify_rows + n), VCHUNK_THREADS, 0, c->stream>>>(
+        in, out, (RejectInfo*)c->rej_info, (ChunkStats*)c->chunk_v, (const int*)(c->acc_d + a.o_row_seq), c->acc_tickets, n_verify_rows);
     LAUNCHED(c);
     if (c->dc.resample && n_verify_rows > 0) {
-        residual_chunk_kernel<<<dim3(nch, n), VCHUNK_THREADS, 0, c->stream>>>(in, rej, c->res_rsum, c->res_vsum);
-        LAUNCHED(c);
-        residual_pick_kernel<<<n, VCHUNK_THREADS, 0, c->stream>>>(in, rej, c->res_rsum, c->res_vsum, nch, out.resampled);
+        residual_fused_kernel<<<dim3(nch, n), VCHUNK_THREADS, 0, c->stream>>>(in, (const RejectInfo*)c->rej_info, c->res_rsum, c->res_vsum,
+                                                                              c->acc_tickets, out.resampled);
         LAUNCHED(c);
     }
     CUDA_TRY(c, cudaMemcpyAsync(c->acc_h + a.in_bytes, c->acc_d + a.in_bytes, a.total - a.in_bytes,
@@ -1125,7 +1131,7 @@ extern "C" int s2d2_accept_and_commit(s2d2_ctx* c, int32_t n, const int32_t* ids
         if (flags[i] && !s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "sequence flagged verified but verify_block did not run for it");
         if (!flags[i] && s->verify_in_flight) FAIL(c, S2D2_ERR_STATE, "verify flags differ from those given to verify_block");
     }
-    AccStage a(n);
+    AccStage a(n, c->n_verify_logit_rows);
     for (int i = 0; i < n; ++i) {
         SeqState& s = c->seqs[ids[i]];
         ((int*)(c->acc_h + a.o_draft0))[i] = s.draft_row0;
@@ -1261,7 +1267,7 @@ extern "C" int s2d2_accept_logits(s2d2_ctx* c, const float* d_draft, const float
         !rng_stream || !step || !res)
         return S2D2_ERR_INVALID;
     if (n > c->dc.max_batch || n * l_max > c->max_logit_rows) FAIL(c, S2D2_ERR_INVALID, "accept_logits: batch larger than the context");
-    AccStage a(n);
+    AccStage a(n, (size_t)n * l_max);
     for (int i = 0; i < n; ++i) {
         if (span_len[i] < 0 || span_len[i] > l_max) FAIL(c, S2D2_ERR_INVALID, "accept_logits: span_len");
         for (int k = 0; k < span_len[i]; ++k)

@@ -127,12 +127,9 @@ __device__ __forceinline__ void load_chunk_strided(const float* row, int V, int 
     }
 }
 
-static __global__ void __launch_bounds__(VCHUNK_THREADS) vocab_chunk_stats_kernel(const float* __restrict__ logits, int V,
-                                                                                  ChunkStats* __restrict__ out) {
-    __shared__ Top2 sh_t[32];
-    __shared__ double sh_d[32];
-    const int chunk = blockIdx.x, r = blockIdx.y, n_chunks = gridDim.x;
-    const float* row = logits + (size_t)r * V;
+// One (chunk, row) by the whole CTA of VCHUNK_THREADS threads; thread 0 writes *out.
+__device__ __forceinline__ void chunk_stats_block(const float* __restrict__ row, int V, int chunk, ChunkStats* __restrict__ out,
+                                                  Top2* sh_t, double* sh_d) {
     const int base = chunk * VCHUNK;
     float x[VPER];
     load_chunk_strided(row, V, base, threadIdx.x, x);
@@ -160,8 +157,15 @@ static __global__ void __launch_bounds__(VCHUNK_THREADS) vocab_chunk_stats_kerne
         o.pad = 0;
         o.s = s;
         o.sx = sx;
-        out[(size_t)r * n_chunks + chunk] = o;
+        *out = o;
     }
+}
+static __global__ void __launch_bounds__(VCHUNK_THREADS) vocab_chunk_stats_kernel(const float* __restrict__ logits, int V,
+                                                                                  ChunkStats* __restrict__ out) {
+    __shared__ Top2 sh_t[32];
+    __shared__ double sh_d[32];
+    const int chunk = blockIdx.x, r = blockIdx.y, n_chunks = gridDim.x;
+    chunk_stats_block(logits + (size_t)r * V, V, chunk, out + (size_t)r * n_chunks + chunk, sh_t, sh_d);
 }
 
 // Merge of a row's chunks by one warp: top-2 in chunk order, then the sums rescaled to the row
@@ -258,10 +262,13 @@ struct RejectInfo {
 // left-to-right loop; the else-branch for sequences that were not verified).  Warps merge the
 // verifier chunks of the span's rows, thread i evaluates position i (v_i, d_i, a_i, u_i), thread 0
 // scans left to right up to the first rejection.
-static __global__ void __launch_bounds__(128) accept_scan_kernel(AcceptIn in, AcceptOut out, RejectInfo* rej) {
-    __shared__ double sh_lse_v[32], sh_lse_d[32];
-    __shared__ double sh_a[32], sh_u[32], sh_v[32];
-    const int s = blockIdx.x, L = in.seq_len[s];
+struct ScanShared {
+    double lse_v[32], lse_d[32], a[32], u[32], v[32];
+};
+// Sequence s by the whole CTA (any number of warps).
+__device__ __forceinline__ void accept_scan_block(const AcceptIn& in, const AcceptOut& out, RejectInfo* rej, int s, ScanShared& sh) {
+    double *sh_lse_v = sh.lse_v, *sh_lse_d = sh.lse_d, *sh_a = sh.a, *sh_u = sh.u, *sh_v = sh.v;
+    const int L = in.seq_len[s];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_chunks = vocab_chunks(in.V);
     if (threadIdx.x == 0) rej[s].draft_row = -1;
@@ -284,7 +291,7 @@ static __global__ void __launch_bounds__(128) accept_scan_kernel(AcceptIn in, Ac
         return;
     }
     const int dr0 = in.seq_draft_row0[s], vr0 = in.seq_verify_row0[s];
-    for (int i = warp; i < L; i += 4) {
+    for (int i = warp; i < L; i += (int)(blockDim.x >> 5)) {
         const RowStats sv = warp_row_stats(in.verify_chunks + (size_t)(vr0 + i) * n_chunks, n_chunks, lane);
         if (lane == 0) sh_lse_v[i] = (double)sv.t.v1 + log(sv.s);
         if (in.draft_lse) {
@@ -447,12 +454,9 @@ static __global__ void __launch_bounds__(VCHUNK_THREADS) draft_sample_kernel(Dra
     }
 }
 
-static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_chunk_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
-                                                                               double* __restrict__ rsum, double* __restrict__ vsum) {
-    __shared__ double sh_d[32];
-    const int chunk = blockIdx.x, s = blockIdx.y, n_chunks = gridDim.x;
-    const RejectInfo r = rej[s];
-    if (r.draft_row < 0) return;
+// One chunk of the rejected position's residual by the whole CTA: thread 0 writes the chunk's residual mass and pi_v mass.
+__device__ __forceinline__ void residual_chunk_block(const AcceptIn& in, const RejectInfo& r, int chunk, double* rs_out, double* vs_out,
+                                                     double* sh_d) {
     float xv[VPER], xd[VPER];
     load_chunk_contiguous(in.verify_logits + (size_t)r.verify_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xv);
     load_chunk_contiguous(in.draft_logits + (size_t)r.draft_row * in.V, in.V, chunk * VCHUNK, threadIdx.x, xd);
@@ -467,8 +471,8 @@ static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_chunk_kernel(A
     rs = block_sum_d(rs, sh_d);
     vs = block_sum_d(vs, sh_d);
     if (threadIdx.x == 0) {
-        rsum[(size_t)s * n_chunks + chunk] = rs;
-        vsum[(size_t)s * n_chunks + chunk] = vs;
+        *rs_out = rs;
+        *vs_out = vs;
     }
 }
 
@@ -476,16 +480,17 @@ static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_chunk_kernel(A
 // the chunk that holds u * Z, the CTA then walks that chunk (prefix over threads, then the
 // owning thread over its 16 entries).  If the residual mass is zero (cannot follow a true
 // rejection in exact arithmetic) the draw is from pi_v.
-static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_pick_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
-                                                                              const double* __restrict__ rsum,
-                                                                              const double* __restrict__ vsum, int n_chunks,
-                                                                              int* __restrict__ resampled) {
-    __shared__ double sh_warp[VCHUNK_THREADS / 32];
-    __shared__ double sh_target;
-    __shared__ int sh_chunk, sh_use_res, sh_pick;
-    const int s = blockIdx.x;
-    const RejectInfo r = rej[s];
-    if (r.draft_row < 0) return;
+struct PickShared {
+    double warp[VCHUNK_THREADS / 32];
+    double target;
+    int chunk, use_res, pick;
+};
+__device__ __forceinline__ void residual_pick_block(const AcceptIn& in, const RejectInfo& r, int s, const double* __restrict__ rsum,
+                                                    const double* __restrict__ vsum, int n_chunks, int* __restrict__ resampled,
+                                                    PickShared& sh) {
+    double* sh_warp = sh.warp;
+    double& sh_target = sh.target;
+    int &sh_chunk = sh.chunk, &sh_use_res = sh.use_res, &sh_pick = sh.pick;
     if (threadIdx.x == 0) {
         double Z = 0.0;
         for (int c = 0; c < n_chunks; ++c) Z += rsum[(size_t)s * n_chunks + c];
@@ -557,6 +562,70 @@ static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_pick_kernel(Ac
     }
     __syncthreads();
     if (threadIdx.x == 0) resampled[s] = sh_pick;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The acceptance step in two launches that wait for nothing: verifier probabilities, ratio test against the Philox
+// uniforms and first rejection here, the residual draw in residual_fused_kernel (Algorithm "SampleBlock for S2D2", the
+// left-to-right loop and its resampling line).
+// Grid (vocabulary chunks, verifier logit rows + sequences).  CTA (chunk, row) computes the chunk statistics of its row
+// and takes a ticket of the row's sequence; the CTA that takes the sequence's last ticket (all chunks of all its rows
+// are then written) runs the scan for that sequence.  CTAs (0, n_verify_rows + s) serve the sequences that were not
+// verified (confidence branch).  row_seq[r] is the sequence of verifier logit row r (-1: none of this call's); tickets
+// are zero before and after the launch.  (The residual sums by that one CTA as well made a single launch, and a slow
+// one: 300 000 fp64 exponentials on one SM.)
+// ---------------------------------------------------------------------------------------------
+static __global__ void __launch_bounds__(VCHUNK_THREADS) accept_fused_kernel(AcceptIn in, AcceptOut out, RejectInfo* rej,
+                                                                             ChunkStats* __restrict__ chunk_v,
+                                                                             const int* __restrict__ row_seq, unsigned* tickets,
+                                                                             int n_verify_rows) {
+    __shared__ Top2 sh_t[32];
+    __shared__ double sh_d[32];
+    __shared__ ScanShared sh_scan;
+    __shared__ int sh_last;
+    const int chunk = blockIdx.x, n_chunks = gridDim.x;
+    if ((int)blockIdx.y >= n_verify_rows) {
+        const int s = blockIdx.y - n_verify_rows;
+        if (chunk == 0 && in.seq_mode && in.seq_mode[s] == 0) accept_scan_block(in, out, rej, s, sh_scan);
+        return;
+    }
+    const int r = blockIdx.y;
+    chunk_stats_block(in.verify_logits + (size_t)r * in.V, in.V, chunk, chunk_v + (size_t)r * n_chunks + chunk, sh_t, sh_d);
+    const int s = row_seq[r];
+    if (s < 0) return;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned t = atomicAdd(&tickets[s], 1u);
+        sh_last = t == (unsigned)(in.seq_len[s] * n_chunks) - 1u;
+    }
+    __syncthreads();
+    if (!sh_last) return;
+    if (threadIdx.x == 0) tickets[s] = 0;
+    __threadfence();
+    accept_scan_block(in, out, rej, s, sh_scan);
+}
+// The residual draw of the rejected positions as one launch, grid (vocabulary chunks, sequences): every CTA sums its chunk
+// of (pi_v - pi_d)_+ in fp64 (the sums are what is expensive, so they stay spread over the GPU), and the CTA that takes
+// the sequence's last ticket walks the inverse CDF.
+static __global__ void __launch_bounds__(VCHUNK_THREADS) residual_fused_kernel(AcceptIn in, const RejectInfo* __restrict__ rej,
+                                                                               double* rsum, double* vsum, unsigned* tickets,
+                                                                               int* __restrict__ resampled) {
+    __shared__ double sh_d[32];
+    __shared__ PickShared sh_pick;
+    __shared__ int sh_last;
+    const int chunk = blockIdx.x, s = blockIdx.y, n_chunks = gridDim.x;
+    const RejectInfo rj = rej[s];
+    if (rj.draft_row < 0) return;
+    residual_chunk_block(in, rj, chunk, rsum + (size_t)s * n_chunks + chunk, vsum + (size_t)s * n_chunks + chunk, sh_d);
+    if (threadIdx.x == 0) {
+        __threadfence();
+        sh_last = atomicAdd(&tickets[s], 1u) == (unsigned)n_chunks - 1u;
+    }
+    __syncthreads();
+    if (!sh_last) return;
+    if (threadIdx.x == 0) tickets[s] = 0;
+    __threadfence();
+    residual_pick_block(in, rj, s, rsum, vsum, n_chunks, resampled, sh_pick);
 }
 
 }  // namespace s2d2

@@ -309,7 +309,7 @@ def check_kv(engine, W, cfg, sid, atol: float, block_size: int = 0) -> float:
     return worst
 
 
-def _check_expert_choice(rep: ParityReport, tag: str, trace: dict, forced, top_k: int, tie_tol: float = 2e-2):
+def _check_expert_choice(rep: ParityReport, tag: str, trace: dict, forced, top_k: int, tie_tol: float = 5e-3):
     """Where the engine's expert set differs from the oracle's own top-k, every expert in
     the difference must sit within ``tie_tol`` of the oracle's k-th router logit (a near tie
     decided differently by the two precisions); anything else is a wrong selection."""
