@@ -627,12 +627,14 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
     // persistent kernel, which streams the weights once per 64 rows; everything longer goes through wide passes of
     // the per-operation kernels, which are tensor-bound and stream the weights once per PREFILL_PASS_ROWS rows.
     const int pr = pass_max_rows(c);
+    // (mixture-of-experts layers have no tensor-core form on the per-operation path: their prompts stay on persistent passes)
+    const bool wide_pays = c->m.n_experts == 0;
     for (;;) {
         int n_short = 0, n_long = 0;
         for (size_t k = 0; k < ids.size(); ++k) {
             const SeqState& s = c->seqs[ids[k]];
             const int left = s.n_final - s.n_c;
-            if (left > 0) ++(pr > 0 && left <= pr ? n_short : n_long);
+            if (left > 0) ++(pr > 0 && (left <= pr || !wide_pays) ? n_short : n_long);
         }
         const bool shorts_ride = pr == 0 || n_short > 4;
         const bool wide = n_long > 0 || (n_short > 0 && shorts_ride);
@@ -643,7 +645,7 @@ extern "C" int s2d2_prefill(s2d2_ctx* c, int32_t n, const int32_t* const* prompt
             took[k] = 0;
             const int left = s.n_final - s.n_c;
             if (left <= 0 || room <= 0) continue;
-            if (wide && pr > 0 && left <= pr && !shorts_ride) continue;      // waits for the persistent pass
+            if (wide && pr > 0 && (left <= pr || !wide_pays) && !shorts_ride) continue;      // waits for the persistent pass
             int rows = std::min(left, room);
             if (rows < left) rows -= rows % CH;                               // whole chunks unless the prompt ends
             if (rows <= 0) continue;
