@@ -319,6 +319,11 @@ int s2d2_debug_gemm(s2d2_ctx* ctx, const void* x, const void* w, int32_t M, int3
  * accumulate != 0, y_inout[M,N] += scale * x w^T (y_inout is read, then overwritten with the result). bf16 models only. */
 int s2d2_debug_gemm2(s2d2_ctx* ctx, const void* x_hi, const void* x_lo, const void* w, int32_t M, int32_t N, int32_t K,
                      float scale, int32_t accumulate, float* y_inout);
+/* The gate/up GEMM of a wide pass with SwiGLU in its epilogue (test tap): w is [2f, K] = gate rows then up rows,
+ * act = silu(x w_gate^T) * (x w_up^T) with x = x_hi + x_lo, returned as two bf16 terms (bit patterns, [M, f] each).
+ * S2D2_ERR_UNSUPPORTED for shapes the forward pass would not give to this kernel (M <= 64, f % 128, K % 64). */
+int s2d2_debug_gemm_swiglu(s2d2_ctx* ctx, const void* x_hi, const void* x_lo, const void* w, int32_t M, int32_t f, int32_t K,
+                           uint16_t* act_hi, uint16_t* act_lo);
 
 /* Expert ids chosen in the last pass, [n_layers, n_rows, top_k] (MoE models). */
 int s2d2_debug_copy_expert_ids(s2d2_ctx* ctx, int32_t* out, int64_t cap, int32_t* n_rows_out);

@@ -79,7 +79,7 @@ EXPORTS = [
     "s2d2_seq_set_rng_stream", "s2d2_draft_block", "s2d2_set_router", "s2d2_set_route_policy", "s2d2_route",
     "s2d2_verify_block", "s2d2_accept_and_commit", "s2d2_generate", "s2d2_get_tokens", "s2d2_release_seq",
     "s2d2_get_counters", "s2d2_reset_counters", "s2d2_set_profiling", "s2d2_set_accept_override", "s2d2_get_gemm_profile", "s2d2_accept_logits", "s2d2_sample_logits", "s2d2_debug_copy_logits",
-    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_gemm2", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace", "s2d2_debug_wait_timeout",
+    "s2d2_debug_copy_kv", "s2d2_debug_seq_state", "s2d2_debug_gemm", "s2d2_debug_gemm2", "s2d2_debug_gemm_swiglu", "s2d2_debug_copy_expert_ids", "s2d2_debug_pass_trace", "s2d2_debug_wait_timeout",
     "s2d2_gemm_bf16_noalloc", "s2d2_noalloc_last_error",
 ]
 
@@ -135,6 +135,7 @@ def load_library() -> C.CDLL:
     lib.s2d2_debug_copy_kv.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.s2d2_debug_seq_state.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.s2d2_debug_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+    lib.s2d2_debug_gemm_swiglu.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.s2d2_debug_gemm2.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_void_p]
     lib.s2d2_debug_copy_expert_ids.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_int64, C.POINTER(C.c_int32)]
     lib.s2d2_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32]
@@ -373,6 +374,17 @@ class Engine:
         self._check(self.lib.s2d2_debug_gemm2(self._h, x_hi.ctypes.data, None if x_lo is None else x_lo.ctypes.data, w.ctypes.data,
                                               M, N, K, C.c_float(scale), int(accumulate), y.ctypes.data))
         return y
+
+    def debug_gemm_swiglu(self, x_hi: np.ndarray, x_lo: np.ndarray, w: np.ndarray):
+        """w [2f, K] (gate rows, then up rows), bf16 bits: (act_hi, act_lo) of silu(x w_g^T) * (x w_u^T), bf16 bits [M, f]."""
+        x_hi, x_lo, w = np.ascontiguousarray(x_hi), np.ascontiguousarray(x_lo), np.ascontiguousarray(w)
+        M, K = x_hi.shape
+        f = w.shape[0] // 2
+        hi = np.empty((M, f), dtype=np.uint16)
+        lo = np.empty((M, f), dtype=np.uint16)
+        self._check(self.lib.s2d2_debug_gemm_swiglu(self._h, x_hi.ctypes.data, x_lo.ctypes.data, w.ctypes.data, M, f, K,
+                                                    hi.ctypes.data, lo.ctypes.data))
+        return hi, lo
 
     def debug_wait_timeout(self, target: int, limit_polls: int = 1000):
         """Runs the bounded-wait pattern on a word nothing sets; raises S2D2Error(-5) when target > 0."""

@@ -1529,6 +1529,42 @@ extern "C" int s2d2_debug_gemm2(s2d2_ctx* c, const void* x_hi, const void* x_lo,
     return rc;
 }
 
+extern "C" int s2d2_debug_gemm_swiglu(s2d2_ctx* c, const void* x_hi, const void* x_lo, const void* w, int32_t M, int32_t f, int32_t K,
+                                      uint16_t* act_hi, uint16_t* act_lo) {
+    if (!c || !x_hi || !x_lo || !w || !act_hi || !act_lo || M < 1 || f < 1 || K < 1) return S2D2_ERR_INVALID;
+    if (c->m.dtype != S2D2_DTYPE_BF16) FAIL(c, S2D2_ERR_UNSUPPORTED, "debug_gemm_swiglu: bf16 models only");
+    void *dx = nullptr, *dl = nullptr, *dw = nullptr, *dh = nullptr, *dlo = nullptr;
+    CUDA_TRY(c, cudaMalloc(&dx, (size_t)M * K * 2));
+    CUDA_TRY(c, cudaMalloc(&dl, (size_t)M * K * 2));
+    CUDA_TRY(c, cudaMalloc(&dw, (size_t)2 * f * K * 2));
+    CUDA_TRY(c, cudaMalloc(&dh, (size_t)M * f * 2));
+    CUDA_TRY(c, cudaMalloc(&dlo, (size_t)M * f * 2));
+    CUDA_TRY(c, cudaMemcpyAsync(dx, x_hi, (size_t)M * K * 2, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(dl, x_lo, (size_t)M * K * 2, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(dw, w, (size_t)2 * f * K * 2, cudaMemcpyHostToDevice, c->stream));
+    int rc = gemm_swiglu(c, dx, dl, dw, M, f, K, dh, dlo);
+    if (rc < 0) {
+        c->err = "debug_gemm_swiglu: this shape takes the separate GEMM and SwiGLU kernels (needs M > 64, f % 128 == 0, K % 64 == 0)";
+        rc = S2D2_ERR_UNSUPPORTED;
+    }
+    if (!rc) rc = enqueue_status_read(c);
+    if (!rc) {
+        CUDA_TRY(c, cudaMemcpyAsync(act_hi, dh, (size_t)M * f * 2, cudaMemcpyDeviceToHost, c->stream));
+        CUDA_TRY(c, cudaMemcpyAsync(act_lo, dlo, (size_t)M * f * 2, cudaMemcpyDeviceToHost, c->stream));
+        CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+        rc = check_status(c);
+    }
+    gemm_forget(c, dx);
+    gemm_forget(c, dl);
+    gemm_forget(c, dw);
+    cudaFree(dx);
+    cudaFree(dl);
+    cudaFree(dw);
+    cudaFree(dh);
+    cudaFree(dlo);
+    return rc;
+}
+
 extern "C" int s2d2_debug_copy_expert_ids(s2d2_ctx* c, int32_t* out, int64_t cap, int32_t* n_rows) {
     if (!c || !out || !n_rows) return S2D2_ERR_INVALID;
     if (c->m.n_experts == 0) FAIL(c, S2D2_ERR_UNSUPPORTED, "not a MoE model");

@@ -60,3 +60,26 @@ def test_wide_gemm_with_two_term_rows_matches_float64(engine, M, N, K, acc, scal
     assert err <= bound, (err, bound)
     again = engine.debug_gemm2(hi, lo, w, y0, scale=scale, accumulate=acc)
     assert np.array_equal(got, again)
+
+
+@pytest.mark.parametrize("M,f,K", [(65, 128, 64), (181, 768, 512), (312, 12288, 4096), (1024, 1024, 2048), (200, 384, 320)])
+def test_gate_up_gemm_with_swiglu_epilogue_matches_float64(engine, M, f, K):
+    """Wide passes compute act = silu(x Wg^T) * (x Wu^T) inside the gate/up GEMM (a CTA holds the same 128 rows of the gate
+    and of the up half) and write it as two bf16 terms.  Against float64 of the same inputs: the sum of the two terms is
+    within two-term bf16 rounding (2^-16 relative) plus the fp32 accumulation error of the GEMM."""
+    rng = np.random.default_rng(M * 131 + f * 7 + K)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    hi = f32_to_bf16_bits(x)
+    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi))
+    w = f32_to_bf16_bits((rng.standard_normal((2 * f, K)) * (1.0 / np.sqrt(K))).astype(np.float32))
+    a_hi, a_lo = engine.debug_gemm_swiglu(hi, lo, w)
+    got = bf16_bits_to_f32(a_hi).astype(np.float64) + bf16_bits_to_f32(a_lo).astype(np.float64)
+    xs = bf16_bits_to_f32(hi).astype(np.float64) + bf16_bits_to_f32(lo).astype(np.float64)
+    y = xs @ bf16_bits_to_f32(w).astype(np.float64).T
+    g, u = y[:, :f], y[:, f:]
+    want = g / (1.0 + np.exp(-g)) * u
+    err = np.abs(got - want).max()
+    bound = 2.0 ** -15 * np.abs(want).max() + 4e-6 * np.sqrt(K) * np.abs(y).max() ** 2 + 1e-6
+    assert err <= bound, (err, bound)
+    # the low term is the rounding remainder of the high one
+    assert np.all(np.abs(bf16_bits_to_f32(a_lo)) <= np.abs(bf16_bits_to_f32(a_hi)) * 2.0 ** -7 + 1e-30)
